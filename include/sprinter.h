@@ -1,0 +1,167 @@
+/*
+ * libsprinter - the verification-and-replacement step of SPRINTER (sequential
+ * approximate verification for speculative decoding) and, for comparison on
+ * the same inputs, standard speculative decoding's exact verification, as
+ * CUDA kernels for sm_100a behind a plain C ABI.
+ *
+ * Conventions shared by every entry point unless it says otherwise
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller; tensors are
+ *     dense, row-major, innermost dimension contiguous.  Element pointers must
+ *     be aligned to the element size; rows need no further alignment (16-byte
+ *     aligned rows take the fastest path).
+ *   - `dt` selects the element type of the "dt" tensors (logits, hidden
+ *     states, verifier weights): SPR_F32 or SPR_BF16.  Biases, uniforms,
+ *     scores and probabilities are float32; token ids and indices int32;
+ *     accept masks uint8.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL
+ *     is the default stream) and the call returns without synchronising.
+ *   - Arguments are validated on the host before anything is enqueued; on a
+ *     non-zero return nothing was launched.
+ *   - `ws` is caller-owned device scratch of at least spr_workspace_bytes()
+ *     bytes, 256-byte aligned, cleared once with spr_workspace_init() after
+ *     allocation.  A call leaves it ready for the next call.  Calls that may
+ *     overlap on the GPU (different streams) need separate workspaces.
+ *   - Problems a kernel detects (a draft token id outside [0,V), a row index
+ *     outside the logits tensor, a bounded wait that ran out) never trap: the
+ *     affected outputs are set to -1, a sticky status word in `ws` records the
+ *     first such code, and spr_device_status() returns and clears it.
+ *   - Outputs are fully overwritten and are bit-identical from run to run for
+ *     identical inputs (fixed reduction orders, no floating-point atomics).
+ *   - Logits must be finite or -inf; uniforms must lie in [0,1).
+ *   - The library runs only on compute capability 10.x devices; there is no
+ *     CPU or other fallback (SPR_ERR_UNSUPPORTED).
+ */
+#ifndef SPRINTER_H_
+#define SPRINTER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SPR_OK = 0,
+    SPR_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, ldv < V, misaligned pointer */
+    SPR_ERR_UNSUPPORTED = 2, /* unknown dtype / op, or not a compute-capability-10 device     */
+    SPR_ERR_WORKSPACE = 3,   /* ws is NULL, misaligned or smaller than spr_workspace_bytes()  */
+    SPR_ERR_CUDA = 4,        /* a CUDA runtime call failed (see spr_last_cuda_error)          */
+    SPR_ERR_TIMEOUT = 5,     /* device: a bounded wait inside a kernel expired                */
+    SPR_ERR_BAD_TOKEN = 6,   /* device: draft token id outside [0, V)                         */
+    SPR_ERR_BAD_ROW = 7      /* device: selected logits row outside [0, R)                    */
+} spr_status;
+
+typedef enum { SPR_F32 = 0, SPR_BF16 = 1 } spr_dtype;
+
+typedef enum { SPR_OP_SPRINTER_VERIFY = 0, SPR_OP_REPLACE_SAMPLE = 1, SPR_OP_SD_VERIFY = 2 } spr_op;
+
+/* Which verifier kernel sprinter_verify() uses.  AUTO picks the tensor-core
+ * kernel for bf16 MLPs whose shapes it supports and the SIMT kernel otherwise. */
+typedef enum { SPR_VERIFIER_AUTO = 0, SPR_VERIFIER_SIMT = 1, SPR_VERIFIER_TENSOR = 2 } spr_verifier_path;
+
+/* Bytes of device scratch one call of `op` needs.  For SPR_OP_REPLACE_SAMPLE,
+ * B is the number of draws n and K, d, h are ignored; for SPR_OP_SD_VERIFY d
+ * and h are ignored; for SPR_OP_SPRINTER_VERIFY V is ignored.  Returns 0 for
+ * invalid arguments.  A workspace sized for the largest op serves all three. */
+size_t spr_workspace_bytes(int op, int B, int K, int V, int d, int h, int dt);
+
+/* Clears a freshly allocated workspace (enqueues a memset on the stream). */
+int spr_workspace_init(void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * sprinter_verify - verifier score, threshold test and first rejection.
+ *
+ * Defined by: Algorithm 2 (detailed SPRINTER), the while-loop: a draft token is
+ * kept while V(s(x, prefix)) >= tau and generation stops at the first token
+ * that fails; Section 3.2 "Verifier architecture": V is one linear layer and a
+ * sigmoid on the draft model's last hidden state (tau = 0.5 in the experiments).
+ *
+ * hidden [B,K,d] dt : s(x, prefix) for the K draft positions of B sequences.
+ * MLP mode (h > 0)  : W1 [h,d] dt, b1 [h] f32, W2 [h] dt, b2 [1] f32
+ *                     score = sigmoid(b2 + W2 . relu(W1 hidden + b1))
+ * paper's verifier (h == 0): W1 is the weight vector [d] dt, b1 = W2 = NULL,
+ *                     score = sigmoid(b2 + W1 . hidden)
+ * accept[b,k]      = score[b,k] >= threshold            (uint8, 0/1)
+ * first_reject[b]  = min{k : accept[b,k] == 0}, K if every token passed
+ *                    (= the number of draft tokens kept)
+ * scores [B,K] f32 : optional (NULL to skip).
+ * path             : spr_verifier_path.
+ * Errors: SPR_ERR_INVALID_ARG (null / sizes), SPR_ERR_UNSUPPORTED (dtype, or
+ * SPR_VERIFIER_TENSOR forced on a shape it cannot take), SPR_ERR_WORKSPACE.
+ */
+int sprinter_verify(const void *hidden, const void *W1, const float *b1, const void *W2,
+                    const float *b2, float threshold, int B, int K, int d, int h, int dt, int path,
+                    float *scores, uint8_t *accept, int32_t *first_reject, void *ws, size_t ws_bytes,
+                    void *cuda_stream);
+
+/*
+ * replace_sample - the target model's replacement token for a rejected draft.
+ *
+ * Defined by: Algorithm 2, the lines after the loop ("Run M_p once"): p' <- p,
+ * t ~ p'.  The draw is an inverse CDF in vocabulary order driven by a
+ * caller-supplied uniform: with e_i = exp(l_i - max l),
+ *   t = min{ j : sum_{i<=j} e_i > u * sum_i e_i }
+ * (the last index with e_j > 0 if rounding leaves none).
+ *
+ * target_logits [R, ldv] dt, V <= ldv valid entries per row.
+ * Draw i (0 <= i < n) reads row
+ *   (rows ? rows[i] : i * seq_stride) + (first_reject ? first_reject[i] : 0)
+ * and is skipped - tokens[i] = -1, no memory traffic - when first_reject is
+ * given and first_reject[i] >= K (the verifier kept every draft token, so the
+ * target is not called).  Passing sprinter_verify's first_reject output here
+ * chains the two calls on one stream with no host synchronisation.
+ * uniforms [n] f32, tokens [n] int32.
+ * Device-detected: row outside [0,R) -> tokens[i] = -1, SPR_ERR_BAD_ROW.
+ */
+int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, const int32_t *rows,
+                   const int32_t *first_reject, int K, int seq_stride, int n, const float *uniforms,
+                   int dt, int32_t *tokens, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * sd_verify - exact verification of standard speculative decoding.
+ *
+ * Defined by: Section 2 (Preliminaries): draft token x is accepted with
+ * probability min(1, p(x)/q(x)); at the first rejection the target resamples
+ * from Eq. 1, p'(x) = norm(max(0, p(x) - q(x))).  With K = 1 on a token the
+ * verifier rejected this is also the keep-or-resample rule of Section 3
+ * ("Algorithm") that Theorem 1 analyses.
+ *
+ * p_logits [B,Kp,ldv] dt (Kp = K or K+1), q_logits [B,K,ldv] dt,
+ * draft_tokens [B,K] int32, uniforms [B,K+1] f32.
+ *   p(.), q(.)        = softmax of the rows (temperature 1)
+ *   accept[b,k]       = uniforms[b,k] <= min(1, p(x)/q(x)), x = draft_tokens[b,k]
+ *                       (every position is tested, also those after a rejection)
+ *   accepted_len[b]   = n_b = min{k : accept[b,k] == 0}, K if none
+ *   correction_token[b]:
+ *       n_b < K            inverse-CDF draw with uniforms[b,K] from
+ *                          norm(max(0, p - q)) at position n_b (from p itself
+ *                          in the degenerate case max(0, p - q) == 0)
+ *       n_b = K, Kp = K+1  draw with uniforms[b,K] from p at position K
+ *       n_b = K, Kp = K    -1
+ *   accept [B,K], p_tok [B,K] = p(x), q_tok [B,K] = q(x), residual_mass [B] =
+ *   sum_i max(0, p_i - q_i) at position n_b (0 when n_b = K): optional, NULL to skip.
+ * Device-detected: draft token outside [0,V) -> that sequence reports
+ * accepted_len = correction_token = -1, accept bits 0, p_tok = q_tok = -1 at that
+ * position, SPR_ERR_BAD_TOKEN.
+ */
+int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int32_t *draft_tokens,
+              const float *uniforms, int B, int K, int Kp, int V, int dt, int32_t *accepted_len,
+              int32_t *correction_token, uint8_t *accept, float *p_tok, float *q_tok,
+              float *residual_mass, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Synchronises the stream, returns the sticky device status word of `ws`
+ * (SPR_OK if nothing was detected) and clears it. */
+int spr_device_status(void *ws, void *cuda_stream);
+
+/* Text for a status code; the last CUDA runtime error string seen by this thread. */
+const char *spr_status_string(int status);
+const char *spr_last_cuda_error(void);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int spr_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPRINTER_H_ */

@@ -1,0 +1,141 @@
+// Shared device helpers and the workspace layout of libsprinter.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sprinter.h"
+
+namespace spr {
+
+// ---------------------------------------------------------------- constants
+constexpr int kThreads = 256;           // CTA size of the vocabulary kernels
+constexpr int kUnroll = 4;              // 16-byte vectors per thread per chunk and row
+constexpr int kWarps = kThreads / 32;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kHeaderBytes = 256;       // workspace header; word 0 is the sticky status
+
+__host__ __device__ constexpr int elem_size(int dt) { return dt == SPR_F32 ? 4 : 2; }
+__host__ __device__ constexpr int vec_elems(int dt) { return 16 / elem_size(dt); }
+// elements of one row that one CTA covers
+__host__ __device__ constexpr int chunk_elems(int dt) { return kThreads * kUnroll * vec_elems(dt); }
+// chunks per row; rows may start up to one vector minus one element past a 16-byte boundary
+__host__ __device__ inline int chunks_per_row(int V, int dt)
+{
+    return (V + vec_elems(dt) - 1 + chunk_elems(dt) - 1) / chunk_elems(dt);
+}
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---------------------------------------------------------------- workspace layouts
+// All offsets are multiples of 256 bytes from the start of the workspace.
+struct DrawWs {              // replace_sample, and the correction draw of sd_verify
+    size_t counters;         // int32 [n]      chunks finished per draw (0 between calls)
+    size_t part_m;           // float [n*C]    chunk maximum (softmax draws)
+    size_t part_s;           // double [n*C]   chunk weight sum
+    size_t end;
+};
+__host__ __device__ inline DrawWs draw_ws_layout(size_t base, int n, int C)
+{
+    DrawWs w;
+    w.counters = base;
+    w.part_m = align_up(w.counters + sizeof(int32_t) * (size_t)n, 256);
+    w.part_s = align_up(w.part_m + sizeof(float) * (size_t)n * C, 256);
+    w.end = align_up(w.part_s + sizeof(double) * (size_t)n * C, 256);
+    return w;
+}
+
+struct SdWs {
+    size_t row_counters;     // int32 [M]      chunks finished per row
+    size_t seq_counters;     // int32 [B]      rows finished per sequence
+    size_t acc;              // uint8 [M]      0 reject, 1 accept, 2 invalid token
+    size_t part;             // float4 [M*C]   (max_p, sum_p, max_q, sum_q) per chunk
+    size_t rowstats;         // float4 [M]     (max_p, ln Z_p, max_q, ln Z_q)
+    DrawWs draw;             // correction draw, n = B
+    size_t end;
+};
+__host__ __device__ inline SdWs sd_ws_layout(int B, int K, int C)
+{
+    const size_t M = (size_t)B * K;
+    SdWs w;
+    w.row_counters = kHeaderBytes;
+    w.seq_counters = align_up(w.row_counters + 4 * M, 256);
+    w.acc = align_up(w.seq_counters + 4 * (size_t)B, 256);
+    w.part = align_up(w.acc + M, 256);
+    w.rowstats = align_up(w.part + 16 * M * C, 256);
+    w.draw = draw_ws_layout(align_up(w.rowstats + 16 * M, 256), B, C);
+    w.end = w.draw.end;
+    return w;
+}
+
+struct VerifyWs {
+    size_t counter;          // int32 [1 + row tiles]   CTAs finished
+    size_t part_z;           // float [slices * M]      per-slice partial of W2 . relu(...)
+    size_t end;
+};
+__host__ __device__ inline VerifyWs verify_ws_layout(int M, int slices, int tiles)
+{
+    VerifyWs w;
+    w.counter = kHeaderBytes;
+    w.part_z = align_up(w.counter + 4 * (size_t)(1 + tiles), 256);
+    w.end = align_up(w.part_z + 4 * (size_t)slices * M, 256);
+    return w;
+}
+
+// ---------------------------------------------------------------- device helpers
+#ifdef __CUDACC__
+
+__device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
+
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// first error wins; the word stays set until the host clears it
+__device__ __forceinline__ void raise_status(int *status, int code) { atomicCAS(status, 0, code); }
+
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// (m, s): s = sum of exp(x - m) over some set.  Merge of two sets, safe for empty ones (m = -inf).
+struct MS {
+    float m, s;
+};
+__device__ __forceinline__ MS ms_merge(MS a, MS b)
+{
+    const float m = fmaxf(a.m, b.m);
+    const float ref = (m == neg_inf()) ? 0.f : m;
+    MS r;
+    r.m = m;
+    r.s = a.s * ex2((a.m - ref) * kLog2e) + b.s * ex2((b.m - ref) * kLog2e);
+    return r;
+}
+__device__ __forceinline__ MS warp_ms(MS v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        MS other;
+        other.m = __shfl_xor_sync(0xffffffffu, v.m, o);
+        other.s = __shfl_xor_sync(0xffffffffu, v.s, o);
+        v = ms_merge(v, other);
+    }
+    return v;
+}
+
+#endif  // __CUDACC__
+
+}  // namespace spr

@@ -1,0 +1,81 @@
+// Kernel parameter blocks and host-side launchers shared by the C-ABI layer.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace spr {
+
+struct SdParams {
+    const void *p;  // [B,Kp,ldv]
+    const void *q;  // [B,K,ldv]
+    int64_t ldv;
+    int V, K, Kp, chunks;
+    const int32_t *draft_tokens;  // [B,K]
+    const float *uniforms;        // [B,K+1]
+    // outputs
+    int32_t *accepted_len;  // [B]
+    uint8_t *accept;        // [B,K] or null
+    float *p_tok, *q_tok;   // [B,K] or null
+    // workspace
+    int *status;
+    int *row_counters;  // [B*K]
+    int *seq_counters;  // [B]
+    uint8_t *acc;       // [B*K]
+    float4 *part;       // [B*K*chunks]
+    float4 *rowstats;   // [B*K]
+};
+
+enum { DRAW_REPLACE = 0, DRAW_SD = 1 };
+
+struct DrawParams {
+    int kind;
+    const void *p;
+    const void *q;
+    int64_t ldv;
+    int V, chunks;
+    // replace_sample
+    int64_t R;
+    const int32_t *rows;
+    const int32_t *gate;
+    int seq_stride;
+    // sd_verify correction draw (K also bounds the gate of replace_sample)
+    int K, Kp;
+    const int32_t *accepted_len;
+    const float4 *rowstats;
+    const float *uniforms;
+    int32_t *tokens;
+    float *residual_mass;
+    // workspace
+    int *status;
+    int *counters;   // [n]
+    float *part_m;   // [n*chunks]
+    double *part_s;  // [n*chunks]
+};
+
+struct VerifyParams {
+    const void *hidden;  // [M,d]
+    const void *W1;      // [h,d] (or [d] when h == 0)
+    const float *b1;
+    const void *W2;
+    const float *b2;
+    float threshold;
+    int B, K, d, h;
+    float *scores;
+    uint8_t *accept;
+    int32_t *first_reject;
+    int *status;
+    int *counter;
+    float *part_z;  // [slices*M]
+    int slices;
+};
+
+cudaError_t launch_sd_verify(const SdParams &sp, const DrawParams &dp, int B, int K, int dt,
+                             cudaStream_t st);
+cudaError_t launch_draw(const DrawParams &dp, int n, int dt, cudaStream_t st);
+
+// SIMT verifier: any dtype and shape.  `slices` must equal verifier_simt_slices(h).
+int verifier_simt_slices(int h);
+cudaError_t launch_verifier_simt(const VerifyParams &vp, int dt, cudaStream_t st);
+
+}  // namespace spr

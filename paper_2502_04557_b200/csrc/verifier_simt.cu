@@ -1,0 +1,197 @@
+// SIMT verifier: score = sigmoid(b2 + W2 . relu(W1 s + b1)) (or sigmoid(b + w . s) for the
+// single linear layer of the paper), threshold test, first-rejection scan.  Takes any
+// element type and shape; it is the path for float32 inputs and for batches too small to
+// fill a tensor-core tile, where the work is a bandwidth-bound sweep over W1.
+#include "common.cuh"
+#include "launch.h"
+
+namespace spr {
+
+constexpr int kTokTile = 8;  // tokens processed per sweep over a W1 row
+
+template <typename T>
+__device__ __forceinline__ float to_f32(T v);
+template <>
+__device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T>
+__device__ __forceinline__ void unpack16(const uint4 &v, float (&f)[16 / sizeof(T)]);
+template <>
+__device__ __forceinline__ void unpack16<float>(const uint4 &v, float (&f)[4])
+{
+    f[0] = __uint_as_float(v.x);
+    f[1] = __uint_as_float(v.y);
+    f[2] = __uint_as_float(v.z);
+    f[3] = __uint_as_float(v.w);
+}
+template <>
+__device__ __forceinline__ void unpack16<__nv_bfloat16>(const uint4 &v, float (&f)[8])
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        f[2 * j] = __uint_as_float(w[j] << 16);
+        f[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+    }
+}
+
+// dot products of one weight row with up to kTokTile hidden rows, result in every lane
+template <typename T>
+__device__ __forceinline__ void warp_dots(const T *__restrict__ wrow, const T *__restrict__ hid, int d,
+                                          int m0, int M, bool vec_ok, float (&acc)[kTokTile])
+{
+    constexpr int N = 16 / sizeof(T);
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int t = 0; t < kTokTile; ++t) acc[t] = 0.f;
+    if (vec_ok) {
+        for (int i = lane * N; i < d; i += 32 * N) {
+            float w[N];
+            unpack16<T>(__ldg(reinterpret_cast<const uint4 *>(wrow + i)), w);
+#pragma unroll
+            for (int t = 0; t < kTokTile; ++t) {
+                if (m0 + t < M) {
+                    float x[N];
+                    unpack16<T>(__ldg(reinterpret_cast<const uint4 *>(hid + (int64_t)(m0 + t) * d + i)), x);
+#pragma unroll
+                    for (int e = 0; e < N; ++e) acc[t] = fmaf(w[e], x[e], acc[t]);
+                }
+            }
+        }
+    } else {
+        for (int i = lane; i < d; i += 32) {
+            const float w = to_f32<T>(wrow[i]);
+#pragma unroll
+            for (int t = 0; t < kTokTile; ++t)
+                if (m0 + t < M) acc[t] = fmaf(w, to_f32<T>(hid[(int64_t)(m0 + t) * d + i]), acc[t]);
+        }
+    }
+#pragma unroll
+    for (int t = 0; t < kTokTile; ++t) acc[t] = warp_sum(acc[t]);
+}
+
+// Last CTA: z = b2 + sum over slices (ascending), sigmoid, threshold, then the scan: one
+// warp per sequence, first rejection = lowest set bit of the reject ballot.
+__device__ void finalise_scores(const VerifyParams &prm)
+{
+    const int M = prm.B * prm.K;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const double tau = (double)prm.threshold;
+    const float b2 = prm.b2[0];
+    for (int m = tid; m < M; m += blockDim.x) {
+        float z = b2;
+        for (int s = 0; s < prm.slices; ++s) z += __ldcg(&prm.part_z[(int64_t)s * M + m]);
+        const double score = 1.0 / (1.0 + exp(-(double)z));
+        if (prm.scores) prm.scores[m] = (float)score;
+        prm.accept[m] = score >= tau ? 1 : 0;
+    }
+    __syncthreads();
+    if (!prm.first_reject) return;
+    const int nwarps = blockDim.x >> 5;
+    for (int b = warp; b < prm.B; b += nwarps) {
+        int first = prm.K;
+        for (int k0 = 0; k0 < prm.K; k0 += 32) {
+            const int k = k0 + lane;
+            const unsigned a = k < prm.K ? (unsigned)prm.accept[(int64_t)b * prm.K + k] : 1u;
+            const unsigned rej = __ballot_sync(0xffffffffu, a == 0u);
+            if (rej != 0u) {
+                first = k0 + __ffs(rej) - 1;
+                break;
+            }
+        }
+        if (lane == 0) prm.first_reject[b] = first;
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads) verifier_simt_kernel(const VerifyParams prm)
+{
+    __shared__ float s_z[kWarps][kTokTile];
+    __shared__ int s_last;
+    const int M = prm.B * prm.K;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const T *hid = static_cast<const T *>(prm.hidden);
+    const T *W1 = static_cast<const T *>(prm.W1);
+    constexpr int N = 16 / sizeof(T);
+    const bool vec_ok = (prm.d % N == 0) && ((reinterpret_cast<uintptr_t>(hid) & 15) == 0) &&
+                        ((reinterpret_cast<uintptr_t>(W1) & 15) == 0);
+
+    if (prm.h > 0) {
+        // slice = kWarps consecutive hidden units, one per warp
+        const int slice = blockIdx.x;
+        const int j = slice * kWarps + warp;
+        float b1j = 0.f, w2j = 0.f;
+        if (j < prm.h) {
+            b1j = prm.b1[j];
+            w2j = to_f32<T>(static_cast<const T *>(prm.W2)[j]);
+        }
+        for (int m0 = 0; m0 < M; m0 += kTokTile) {
+            float acc[kTokTile];
+            if (j < prm.h) {
+                warp_dots<T>(W1 + (int64_t)j * prm.d, hid, prm.d, m0, M, vec_ok, acc);
+            } else {
+#pragma unroll
+                for (int t = 0; t < kTokTile; ++t) acc[t] = 0.f;
+            }
+            if (lane == 0) {
+#pragma unroll
+                for (int t = 0; t < kTokTile; ++t)
+                    s_z[warp][t] = (j < prm.h) ? w2j * fmaxf(acc[t] + b1j, 0.f) : 0.f;
+            }
+            __syncthreads();
+            if (tid < kTokTile && m0 + tid < M) {
+                float z = 0.f;
+#pragma unroll
+                for (int w = 0; w < kWarps; ++w) z += s_z[w][tid];
+                prm.part_z[(int64_t)slice * M + m0 + tid] = z;
+            }
+            __syncthreads();
+        }
+    } else {
+        // single linear layer: one warp per token tile
+        const int m0 = (blockIdx.x * kWarps + warp) * kTokTile;
+        if (m0 < M) {
+            float acc[kTokTile];
+            warp_dots<T>(W1, hid, prm.d, m0, M, vec_ok, acc);
+            if (lane == 0) {
+#pragma unroll
+                for (int t = 0; t < kTokTile; ++t)
+                    if (m0 + t < M) prm.part_z[m0 + t] = acc[t];
+            }
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        s_last = (atomicAdd(prm.counter, 1) == (int)gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    finalise_scores(prm);
+    if (tid == 0) *prm.counter = 0;
+}
+
+int verifier_simt_slices(int h) { return h > 0 ? (h + kWarps - 1) / kWarps : 1; }
+
+static int simt_grid(const VerifyParams &vp)
+{
+    if (vp.h > 0) return verifier_simt_slices(vp.h);
+    const int M = vp.B * vp.K;
+    return (M + kWarps * kTokTile - 1) / (kWarps * kTokTile);
+}
+
+cudaError_t launch_verifier_simt(const VerifyParams &vp, int dt, cudaStream_t st)
+{
+    const int grid = simt_grid(vp);
+    if (grid <= 0) return cudaSuccess;
+    if (dt == SPR_F32)
+        verifier_simt_kernel<float><<<grid, kThreads, 0, st>>>(vp);
+    else
+        verifier_simt_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(vp);
+    return cudaGetLastError();
+}
+
+}  // namespace spr

@@ -1,0 +1,610 @@
+// Vocabulary-wide kernels: softmax statistics, the min(1, p/q) accept test, the
+// first-rejection scan, and inverse-CDF draws from softmax(l) or from the residual
+// norm(max(0, p - q)) of Eq. 1.  All of them stream each logits row from HBM once in
+// 16-byte vectors, keep probabilities in registers only, and hand per-chunk partial
+// results to the last CTA that finishes a row ("last block done" tickets: nothing ever
+// waits on another CTA).
+#include <limits.h>
+
+#include "common.cuh"
+#include "launch.h"
+
+namespace spr {
+
+// ---------------------------------------------------------------- 16-byte vectors
+template <typename T>
+struct Vec;
+
+template <>
+struct Vec<float> {
+    static constexpr int N = 4;
+    static __device__ __forceinline__ void unpack(const uint4 &v, float (&f)[N])
+    {
+        f[0] = __uint_as_float(v.x);
+        f[1] = __uint_as_float(v.y);
+        f[2] = __uint_as_float(v.z);
+        f[3] = __uint_as_float(v.w);
+    }
+    static __device__ __forceinline__ float vmax(const uint4 &v)
+    {
+        return fmaxf(fmaxf(__uint_as_float(v.x), __uint_as_float(v.y)),
+                     fmaxf(__uint_as_float(v.z), __uint_as_float(v.w)));
+    }
+    // elements i0 .. i0+3 of the row, -inf where the index falls outside [0, V)
+    static __device__ __forceinline__ uint4 gather(const float *row, int i0, int V)
+    {
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int i = i0 + e;
+            w[e] = (i >= 0 && i < V) ? __float_as_uint(row[i]) : 0xff800000u;
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+template <>
+struct Vec<__nv_bfloat16> {
+    static constexpr int N = 8;
+    static __device__ __forceinline__ void unpack(const uint4 &v, float (&f)[N])
+    {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            f[2 * j] = __uint_as_float(w[j] << 16);
+            f[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+        }
+    }
+    static __device__ __forceinline__ float vmax(const uint4 &v)
+    {
+        const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162 *>(&v.x);
+        const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162 *>(&v.y);
+        const __nv_bfloat162 c = *reinterpret_cast<const __nv_bfloat162 *>(&v.z);
+        const __nv_bfloat162 d = *reinterpret_cast<const __nv_bfloat162 *>(&v.w);
+        const __nv_bfloat162 m = __hmax2(__hmax2(a, b), __hmax2(c, d));
+        return fmaxf(__low2float(m), __high2float(m));
+    }
+    static __device__ __forceinline__ uint4 gather(const __nv_bfloat16 *row, int i0, int V)
+    {
+        const unsigned short *r = reinterpret_cast<const unsigned short *>(row);
+        uint32_t w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int a = i0 + 2 * j, b = a + 1;
+            const uint32_t lo = (a >= 0 && a < V) ? (uint32_t)r[a] : 0xff80u;
+            const uint32_t hi = (b >= 0 && b < V) ? (uint32_t)r[b] : 0xff80u;
+            w[j] = lo | (hi << 16);
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// Elements i0 .. i0+N-1 of a row as one vector.  One 16-byte load when the vector lies
+// inside the row and its address is 16-byte aligned, element loads with -inf fill otherwise.
+template <typename T>
+__device__ __forceinline__ uint4 load_vec(const T *__restrict__ row, int i0, int V)
+{
+    constexpr int N = Vec<T>::N;
+    if (i0 >= 0 && i0 + N <= V && (reinterpret_cast<uintptr_t>(row + i0) & 15) == 0)
+        return ld_stream(reinterpret_cast<const uint4 *>(row + i0));
+    if (i0 + N <= 0 || i0 >= V) {
+        const uint32_t f = sizeof(T) == 4 ? 0xff800000u : 0xff80ff80u;
+        return make_uint4(f, f, f, f);
+    }
+    return Vec<T>::gather(row, i0, V);
+}
+
+// Number of elements by which the row start lies past a 16-byte boundary.  Vector j of
+// thread t in chunk c starts at element (c*CH + (j*256 + t)*N) - pad of the row, which makes
+// every interior vector 16-byte aligned whatever the row's own alignment.
+template <typename T>
+__device__ __forceinline__ int row_pad(const T *row)
+{
+    return (int)((reinterpret_cast<uintptr_t>(row) & 15) / sizeof(T));
+}
+
+template <typename T>
+__device__ __forceinline__ int vec_start(int c, int j, int tid, int pad)
+{
+    constexpr int N = Vec<T>::N;
+    return c * (kThreads * kUnroll * N) + (j * kThreads + tid) * N - pad;
+}
+
+// (max, sum of exp(x - max)) over the kUnroll vectors a thread holds
+template <typename T>
+__device__ __forceinline__ MS thread_ms(const uint4 (&raw)[kUnroll])
+{
+    constexpr int N = Vec<T>::N;
+    float m = Vec<T>::vmax(raw[0]);
+#pragma unroll
+    for (int j = 1; j < kUnroll; ++j) m = fmaxf(m, Vec<T>::vmax(raw[j]));
+    const float ref = (m == neg_inf()) ? 0.f : m;
+    const float off = -ref * kLog2e;
+    float s = 0.f;
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) {
+        float f[N];
+        Vec<T>::unpack(raw[j], f);
+#pragma unroll
+        for (int e = 0; e < N; ++e) s += ex2(fmaf(f[e], kLog2e, off));
+    }
+    MS r;
+    r.m = m;
+    r.s = s;
+    return r;
+}
+
+// ================================================================ sd_verify, stage 1
+// One CTA per (row, chunk): chunk statistics of the p row and the q row.  The CTA that
+// finishes a row last merges the chunks, runs the accept test for that position, and the
+// row that finishes a sequence last runs the first-rejection scan.
+template <typename T>
+__global__ void __launch_bounds__(kThreads) sd_row_stats_kernel(const SdParams prm)
+{
+    __shared__ float4 s_part[kWarps];
+    __shared__ int s_last;
+
+    const int C = prm.chunks;
+    const int64_t row = blockIdx.x / C;  // = b*K + k
+    const int c = blockIdx.x % C;
+    const int b = (int)(row / prm.K), k = (int)(row % prm.K);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    const T *prow = static_cast<const T *>(prm.p) + ((int64_t)b * prm.Kp + k) * prm.ldv;
+    const T *qrow = static_cast<const T *>(prm.q) + row * prm.ldv;
+    const int pad_p = row_pad(prow), pad_q = row_pad(qrow);
+
+    uint4 rp[kUnroll], rq[kUnroll];
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) rp[j] = load_vec<T>(prow, vec_start<T>(c, j, tid, pad_p), prm.V);
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) rq[j] = load_vec<T>(qrow, vec_start<T>(c, j, tid, pad_q), prm.V);
+
+    MS mp = warp_ms(thread_ms<T>(rp));
+    MS mq = warp_ms(thread_ms<T>(rq));
+    if (lane == 0) s_part[warp] = make_float4(mp.m, mp.s, mq.m, mq.s);
+    __syncthreads();
+    if (warp == 0) {
+        float4 v = lane < kWarps ? s_part[lane] : make_float4(neg_inf(), 0.f, neg_inf(), 0.f);
+        mp = warp_ms(MS{v.x, v.y});
+        mq = warp_ms(MS{v.z, v.w});
+        if (lane == 0) {
+            prm.part[row * C + c] = make_float4(mp.m, mp.s, mq.m, mq.s);
+            __threadfence();
+            const int ticket = atomicAdd(&prm.row_counters[row], 1);
+            s_last = (ticket == C - 1);
+        }
+    }
+    __syncthreads();
+    if (!s_last || warp != 0) return;
+
+    // ---- this CTA saw the last chunk of the row: merge chunks in chunk order (warp 0)
+    __threadfence();
+    float m_p = neg_inf(), m_q = neg_inf();
+    for (int cc = lane; cc < C; cc += 32) {
+        const float4 v = __ldcg(&prm.part[row * C + cc]);
+        m_p = fmaxf(m_p, v.x);
+        m_q = fmaxf(m_q, v.z);
+    }
+    m_p = warp_max(m_p);
+    m_q = warp_max(m_q);
+    double z_p = 0.0, z_q = 0.0;
+    for (int c0 = 0; c0 < C; c0 += 32) {  // fixed order: chunk groups ascending, butterfly inside
+        const int cc = c0 + lane;
+        double a = 0.0, bq = 0.0;
+        if (cc < C) {
+            const float4 v = __ldcg(&prm.part[row * C + cc]);
+            a = v.y > 0.f ? (double)v.y * exp((double)v.x - (double)m_p) : 0.0;
+            bq = v.w > 0.f ? (double)v.w * exp((double)v.z - (double)m_q) : 0.0;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            a += __shfl_xor_sync(0xffffffffu, a, o);
+            bq += __shfl_xor_sync(0xffffffffu, bq, o);
+        }
+        z_p += a;
+        z_q += bq;
+    }
+    int last_row = 0;
+    if (lane == 0) {
+        const double lnz_p = log(z_p), lnz_q = log(z_q);
+        const int x = prm.draft_tokens[row];
+        unsigned char acc;
+        float P = -1.f, Q = -1.f;
+        if (x < 0 || x >= prm.V) {
+            raise_status(prm.status, SPR_ERR_BAD_TOKEN);
+            acc = 2;
+        } else {
+            float lpx, lqx;
+            if (sizeof(T) == 4) {
+                lpx = reinterpret_cast<const float *>(prow)[x];
+                lqx = reinterpret_cast<const float *>(qrow)[x];
+            } else {
+                lpx = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(prow)[x]);
+                lqx = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(qrow)[x]);
+            }
+            const double logP = (double)lpx - (double)m_p - lnz_p;
+            const double logQ = (double)lqx - (double)m_q - lnz_q;
+            const double ratio = exp(logP - logQ);
+            const double u = (double)prm.uniforms[(int64_t)b * (prm.K + 1) + k];
+            acc = (u <= fmin(1.0, ratio)) ? 1 : 0;
+            P = (float)exp(logP);
+            Q = (float)exp(logQ);
+        }
+        prm.acc[row] = acc;
+        if (prm.accept) prm.accept[row] = acc == 1 ? 1 : 0;
+        if (prm.p_tok) prm.p_tok[row] = P;
+        if (prm.q_tok) prm.q_tok[row] = Q;
+        prm.rowstats[row] = make_float4(m_p, (float)lnz_p, m_q, (float)lnz_q);
+        prm.row_counters[row] = 0;  // ready for the next call
+        __threadfence();
+        last_row = (atomicAdd(&prm.seq_counters[b], 1) == prm.K - 1);
+    }
+    last_row = __shfl_sync(0xffffffffu, last_row, 0);
+    if (!last_row) return;
+
+    // ---- last row of the sequence: first rejection = lowest set bit of the reject ballot
+    __threadfence();
+    int first = prm.K;
+    bool bad = false;
+    for (int k0 = 0; k0 < prm.K; k0 += 32) {
+        const int kk = k0 + lane;
+        const unsigned v = kk < prm.K ? (unsigned)__ldcg(&prm.acc[(int64_t)b * prm.K + kk]) : 1u;
+        const unsigned rej = __ballot_sync(0xffffffffu, v != 1u);
+        bad |= __ballot_sync(0xffffffffu, v == 2u) != 0u;
+        if (rej != 0u && first == prm.K) first = k0 + __ffs(rej) - 1;
+    }
+    if (lane == 0) {
+        prm.accepted_len[b] = bad ? -1 : first;
+        if (bad && prm.accept)
+            for (int kk = 0; kk < prm.K; ++kk) prm.accept[(int64_t)b * prm.K + kk] = 0;
+        prm.seq_counters[b] = 0;
+    }
+}
+
+// ================================================================ inverse-CDF draws
+enum { MODE_NONE = 0, MODE_SOFTMAX = 1, MODE_RESIDUAL = 2 };
+
+template <typename T>
+struct Job {
+    int mode;
+    const T *p_row;
+    const T *q_row;
+    float cp, cq;  // residual: (max + ln Z) * log2(e) of the p row and of the q row
+    float u;
+};
+
+template <typename T>
+__device__ __forceinline__ Job<T> resolve_job(const DrawParams &prm, int i)
+{
+    Job<T> job;
+    job.mode = MODE_NONE;
+    job.p_row = job.q_row = nullptr;
+    job.cp = job.cq = 0.f;
+    job.u = 0.f;
+    const T *p = static_cast<const T *>(prm.p);
+    if (prm.kind == DRAW_REPLACE) {
+        int off = 0;
+        if (prm.gate) {
+            off = prm.gate[i];
+            if (off >= prm.K) return job;  // verifier kept every token: the target is not called
+        }
+        const int64_t row = (prm.rows ? (int64_t)prm.rows[i] : (int64_t)i * prm.seq_stride) + off;
+        if (row < 0 || row >= prm.R) {
+            raise_status(prm.status, SPR_ERR_BAD_ROW);
+            return job;
+        }
+        job.mode = MODE_SOFTMAX;
+        job.p_row = p + row * prm.ldv;
+        job.u = prm.uniforms[i];
+    } else {
+        const int nb = prm.accepted_len[i];
+        if (nb < 0) return job;  // invalid draft token in this sequence
+        if (nb < prm.K) {
+            const float4 st = prm.rowstats[(int64_t)i * prm.K + nb];
+            job.mode = MODE_RESIDUAL;
+            job.p_row = p + ((int64_t)i * prm.Kp + nb) * prm.ldv;
+            job.q_row = static_cast<const T *>(prm.q) + ((int64_t)i * prm.K + nb) * prm.ldv;
+            job.cp = (st.x + st.y) * kLog2e;
+            job.cq = (st.z + st.w) * kLog2e;
+        } else if (prm.Kp == prm.K + 1) {
+            job.mode = MODE_SOFTMAX;
+            job.p_row = p + ((int64_t)i * prm.Kp + prm.K) * prm.ldv;
+        } else {
+            return job;
+        }
+        job.u = prm.uniforms[(int64_t)i * (prm.K + 1) + prm.K];
+    }
+    return job;
+}
+
+// residual weights max(0, p_i - q_i) of one vector (probabilities, already normalised)
+template <typename T>
+__device__ __forceinline__ void residual_weights(const uint4 &vp, const uint4 &vq, float cp, float cq,
+                                                 float (&w)[Vec<T>::N])
+{
+    constexpr int N = Vec<T>::N;
+    float fp[N], fq[N];
+    Vec<T>::unpack(vp, fp);
+    Vec<T>::unpack(vq, fq);
+#pragma unroll
+    for (int e = 0; e < N; ++e)
+        w[e] = fmaxf(0.f, ex2(fmaf(fp[e], kLog2e, -cp)) - ex2(fmaf(fq[e], kLog2e, -cq)));
+}
+
+struct DrawSmem {
+    float4 red[kWarps];
+    double scan[kWarps];
+    double base;
+    double t_in;
+    double total;
+    float ref;
+    int chunk;
+    int first;
+    int lastpos;
+    int token;
+    int last;
+};
+
+// (chunk max, chunk sum) of softmax weights, or (0, chunk sum) of residual weights; the
+// result is valid in thread 0.
+template <typename T>
+__device__ __forceinline__ MS block_chunk_stats(const Job<T> &job, int mode, int V, int c, DrawSmem &sm)
+{
+    constexpr int N = Vec<T>::N;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int pad = row_pad(job.p_row);
+    uint4 rp[kUnroll];
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) rp[j] = load_vec<T>(job.p_row, vec_start<T>(c, j, tid, pad), V);
+    MS v;
+    if (mode == MODE_SOFTMAX) {
+        v = warp_ms(thread_ms<T>(rp));
+    } else {
+        uint4 rq[kUnroll];
+#pragma unroll
+        for (int j = 0; j < kUnroll; ++j) rq[j] = load_vec<T>(job.q_row, vec_start<T>(c, j, tid, pad), V);
+        float s = 0.f;
+#pragma unroll
+        for (int j = 0; j < kUnroll; ++j) {
+            float w[N];
+            residual_weights<T>(rp[j], rq[j], job.cp, job.cq, w);
+#pragma unroll
+            for (int e = 0; e < N; ++e) s += w[e];
+        }
+        v.m = 0.f;
+        v.s = warp_sum(s);
+    }
+    __syncthreads();  // sm.red may still be read by the previous use
+    if (lane == 0) sm.red[warp] = make_float4(v.m, v.s, 0.f, 0.f);
+    __syncthreads();
+    if (warp == 0) {
+        const float4 r = lane < kWarps ? sm.red[lane] : make_float4(neg_inf(), 0.f, 0.f, 0.f);
+        if (mode == MODE_SOFTMAX) {
+            v = warp_ms(MS{r.x, r.y});
+        } else {
+            v.m = 0.f;
+            v.s = warp_sum(lane < kWarps ? r.y : 0.f);
+        }
+    }
+    return v;
+}
+
+// Finds, inside chunk c, the first element whose running weight sum exceeds t_in (weights
+// taken relative to `ref` for softmax draws).  Falls back to the last positive-weight
+// element of the chunk when rounding leaves no crossing; -1 if the chunk has no weight.
+template <typename T>
+__device__ int block_locate(const Job<T> &job, int mode, int V, int c, double t_in, float ref,
+                            DrawSmem &sm)
+{
+    constexpr int N = Vec<T>::N;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int pad = row_pad(job.p_row);
+    const float off = -ref * kLog2e;
+    if (tid == 0) {
+        sm.first = INT_MAX;
+        sm.lastpos = -1;
+        sm.base = 0.0;
+        sm.token = -1;
+    }
+    __syncthreads();
+    for (int j = 0; j < kUnroll; ++j) {
+        const int i0 = vec_start<T>(c, j, tid, pad);
+        float w[N];
+        const uint4 vp = load_vec<T>(job.p_row, i0, V);
+        if (mode == MODE_SOFTMAX) {
+            float f[N];
+            Vec<T>::unpack(vp, f);
+#pragma unroll
+            for (int e = 0; e < N; ++e) w[e] = ex2(fmaf(f[e], kLog2e, off));
+        } else {
+            const uint4 vq = load_vec<T>(job.q_row, i0, V);
+            residual_weights<T>(vp, vq, job.cp, job.cq, w);
+        }
+        double ts = 0.0;
+        int lp = -1;
+#pragma unroll
+        for (int e = 0; e < N; ++e) {
+            ts += (double)w[e];
+            if (w[e] > 0.f) lp = i0 + e;
+        }
+        // inclusive scan of ts in thread order
+        double incl = ts;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const double up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        if (lane == 31) sm.scan[warp] = incl;
+        __syncthreads();
+        double before = sm.base;
+        for (int ww = 0; ww < warp; ++ww) before += sm.scan[ww];
+        incl += before;
+        if (incl > t_in) atomicMin(&sm.first, tid);
+        if (lp >= 0) atomicMax(&sm.lastpos, lp);
+        __syncthreads();
+        if (sm.first != INT_MAX) {
+            if (tid == sm.first) {
+                double run = incl - ts;
+                int tok = -1;
+#pragma unroll
+                for (int e = 0; e < N; ++e) {
+                    run += (double)w[e];
+                    if (tok < 0 && run > t_in && w[e] > 0.f) tok = i0 + e;
+                }
+                sm.token = tok >= 0 ? tok : (lp >= 0 ? lp : sm.lastpos);
+            }
+            __syncthreads();
+            return sm.token;
+        }
+        if (tid == kThreads - 1) sm.base = incl;
+        __syncthreads();
+    }
+    return sm.lastpos;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads) draw_kernel(const DrawParams prm)
+{
+    __shared__ DrawSmem sm;
+    const int C = prm.chunks;
+    const int i = blockIdx.x / C;
+    const int c = blockIdx.x % C;
+    const int tid = threadIdx.x;
+
+    Job<T> job = resolve_job<T>(prm, i);
+    if (job.mode == MODE_NONE) {
+        if (c == 0 && tid == 0) {
+            prm.tokens[i] = -1;
+            if (prm.residual_mass) prm.residual_mass[i] = 0.f;
+        }
+        return;
+    }
+    int mode = job.mode;
+    float *part_m = prm.part_m + (int64_t)i * C;
+    double *part_s = prm.part_s + (int64_t)i * C;
+
+    const MS v = block_chunk_stats<T>(job, mode, prm.V, c, sm);
+    if (tid == 0) {
+        part_m[c] = v.m;
+        part_s[c] = (double)v.s;
+        __threadfence();
+        sm.last = (atomicAdd(&prm.counters[i], 1) == C - 1);
+    }
+    __syncthreads();
+    if (!sm.last) return;
+    __threadfence();
+
+    // ---- last CTA of this draw: total weight, crossing chunk, then the token inside it
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        if (tid == 0) {
+            float M = neg_inf();
+            for (int cc = 0; cc < C; ++cc) M = fmaxf(M, __ldcg(&part_m[cc]));
+            double total = 0.0;
+            for (int cc = 0; cc < C; ++cc) {
+                const double s = __ldcg(&part_s[cc]);
+                if (s > 0.0) total += s * exp((double)__ldcg(&part_m[cc]) - (double)M);
+            }
+            const double target = (double)job.u * total;
+            double prefix = 0.0, before = 0.0;
+            int chunk = -1, lastpos_chunk = -1;
+            for (int cc = 0; cc < C; ++cc) {
+                const double s = __ldcg(&part_s[cc]);
+                if (!(s > 0.0)) continue;
+                const double S = s * exp((double)__ldcg(&part_m[cc]) - (double)M);
+                if (S > 0.0) lastpos_chunk = cc;
+                if (prefix + S > target) {
+                    chunk = cc;
+                    before = prefix;
+                    break;
+                }
+                prefix += S;
+            }
+            sm.total = total;
+            if (chunk >= 0) {
+                const float mc = __ldcg(&part_m[chunk]);
+                sm.chunk = chunk;
+                sm.ref = mc;
+                sm.t_in = (target - before) * exp((double)M - (double)mc);
+            } else {  // u*total not below total (rounding, or u >= 1): last positive weight
+                sm.chunk = lastpos_chunk;
+                sm.ref = lastpos_chunk >= 0 ? __ldcg(&part_m[lastpos_chunk]) : 0.f;
+                sm.t_in = __longlong_as_double(0x7ff0000000000000LL);
+            }
+        }
+        __syncthreads();
+        if (attempt == 0 && prm.kind == DRAW_SD && tid == 0 && prm.residual_mass)
+            prm.residual_mass[i] = mode == MODE_RESIDUAL ? (float)sm.total : 0.f;
+        if (mode == MODE_RESIDUAL && !(sm.total > 0.0)) {
+            // max(0, p - q) vanished: Eq. 1 is undefined, draw from p itself (one CTA, rare)
+            mode = MODE_SOFTMAX;
+            for (int cc = 0; cc < C; ++cc) {
+                const MS r = block_chunk_stats<T>(job, mode, prm.V, cc, sm);
+                if (tid == 0) {
+                    part_m[cc] = r.m;
+                    part_s[cc] = (double)r.s;
+                }
+            }
+            __threadfence();
+            __syncthreads();
+            continue;
+        }
+        break;
+    }
+    int token = -1;
+    if (sm.chunk >= 0) {
+        const int chunk = sm.chunk;
+        const double t_in = sm.t_in;
+        const float ref = sm.ref;
+        token = block_locate<T>(job, mode, prm.V, chunk, t_in, ref, sm);
+    }
+    if (tid == 0) {
+        prm.tokens[i] = token;
+        prm.counters[i] = 0;  // ready for the next call
+    }
+}
+
+// ================================================================ host launchers
+template <typename T>
+static cudaError_t launch_sd_t(const SdParams &sp, const DrawParams &dp, int B, int K, cudaStream_t st)
+{
+    const int64_t grid_a = (int64_t)B * K * sp.chunks;
+    const int64_t grid_b = (int64_t)B * dp.chunks;
+    if (grid_a > 0x7fffffffLL || grid_b > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    if (grid_a == 0) return cudaSuccess;
+    sd_row_stats_kernel<T><<<(unsigned)grid_a, kThreads, 0, st>>>(sp);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    draw_kernel<T><<<(unsigned)grid_b, kThreads, 0, st>>>(dp);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_sd_verify(const SdParams &sp, const DrawParams &dp, int B, int K, int dt,
+                             cudaStream_t st)
+{
+    return dt == SPR_F32 ? launch_sd_t<float>(sp, dp, B, K, st)
+                         : launch_sd_t<__nv_bfloat16>(sp, dp, B, K, st);
+}
+
+cudaError_t launch_draw(const DrawParams &dp, int n, int dt, cudaStream_t st)
+{
+    const int64_t grid = (int64_t)n * dp.chunks;
+    if (grid > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    if (grid == 0) return cudaSuccess;
+    if (dt == SPR_F32)
+        draw_kernel<float><<<(unsigned)grid, kThreads, 0, st>>>(dp);
+    else
+        draw_kernel<__nv_bfloat16><<<(unsigned)grid, kThreads, 0, st>>>(dp);
+    return cudaGetLastError();
+}
+
+}  // namespace spr
