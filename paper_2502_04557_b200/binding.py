@@ -1,0 +1,221 @@
+"""Thin ctypes binding of libsprinter: argument marshalling only.
+
+Every function takes CUDA ``torch`` tensors (used here purely as device buffers), passes
+their pointers to the C ABI declared in ``include/sprinter.h`` and returns the output
+tensors.  All arithmetic happens in the CUDA kernels of the library; there is no fallback:
+if the library is missing or the device is not a compute-capability-10 GPU the call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from . import build as _build
+
+F32, BF16 = 0, 1
+OP_SPRINTER_VERIFY, OP_REPLACE_SAMPLE, OP_SD_VERIFY = 0, 1, 2
+PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
+
+EXPORTS = [
+    "spr_workspace_bytes", "spr_workspace_init", "sprinter_verify", "replace_sample", "sd_verify",
+    "spr_device_status", "spr_status_string", "spr_last_cuda_error", "spr_version",
+]
+
+
+class SprinterError(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        L = lib()
+        msg = L.spr_status_string(status).decode()
+        if status == 4:
+            msg += " (" + L.spr_last_cuda_error().decode() + ")"
+        super().__init__(f"{fn}: status {status}: {msg}")
+        self.status = status
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def lib():
+    """Loads libsprinter.so (never builds it implicitly on a machine without nvcc)."""
+    global _lib
+    if _lib is None:
+        path = lib_path()
+        if not os.path.exists(path):
+            raise ImportError(
+                f"{path} is missing: build it with `python -m paper_2502_04557_b200.build`")
+        L = C.CDLL(path)
+        vp, i32, i64, f32, sz = C.c_void_p, C.c_int, C.c_int64, C.c_float, C.c_size_t
+        L.spr_workspace_bytes.restype = sz
+        L.spr_workspace_bytes.argtypes = [i32] * 7
+        L.spr_workspace_init.restype = i32
+        L.spr_workspace_init.argtypes = [vp, sz, vp]
+        L.sprinter_verify.restype = i32
+        L.sprinter_verify.argtypes = [vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32,
+                                      vp, vp, vp, vp, sz, vp]
+        L.replace_sample.restype = i32
+        L.replace_sample.argtypes = [vp, i64, i32, i64, vp, vp, i32, i32, i32, vp, i32, vp, vp, sz, vp]
+        L.sd_verify.restype = i32
+        L.sd_verify.argtypes = [vp, vp, i64, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp,
+                                vp, sz, vp]
+        L.spr_device_status.restype = i32
+        L.spr_device_status.argtypes = [vp, vp]
+        L.spr_status_string.restype = C.c_char_p
+        L.spr_status_string.argtypes = [i32]
+        L.spr_last_cuda_error.restype = C.c_char_p
+        L.spr_last_cuda_error.argtypes = []
+        L.spr_version.restype = i32
+        L.spr_version.argtypes = []
+        _lib = L
+    return _lib
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported element type {t.dtype}")
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(fn: str, rc: int):
+    if rc != 0:
+        raise SprinterError(fn, rc)
+
+
+def _dev(t: torch.Tensor, dtype=None, name="tensor"):
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}")
+    return t
+
+
+def workspace_bytes(op: int, B: int, K: int = 1, V: int = 1, d: int = 1, h: int = 0, dt: int = BF16) -> int:
+    return int(lib().spr_workspace_bytes(op, B, K, V, d, h, dt))
+
+
+class Workspace:
+    """Device scratch for the library calls, cleared once at creation."""
+
+    def __init__(self, nbytes: int, device="cuda"):
+        nbytes = max(int(nbytes), 256)
+        self.buf = torch.empty((nbytes + 255) // 256 * 256, dtype=torch.uint8, device=device)
+        assert self.buf.data_ptr() % 256 == 0
+        _check("spr_workspace_init", lib().spr_workspace_init(_ptr(self.buf), self.buf.numel(), _stream()))
+
+    @property
+    def nbytes(self) -> int:
+        return self.buf.numel()
+
+    def device_status(self) -> int:
+        """Synchronises the current stream; returns and clears the sticky device status."""
+        return int(lib().spr_device_status(_ptr(self.buf), _stream()))
+
+    @classmethod
+    def for_problem(cls, B: int, K: int, V: int, d: int, h: int, dt: int, device="cuda"):
+        n = max(workspace_bytes(OP_SPRINTER_VERIFY, B, K, V, d, h, dt),
+                workspace_bytes(OP_REPLACE_SAMPLE, B, K, V, d, h, dt),
+                workspace_bytes(OP_SD_VERIFY, B, K, V, d, h, dt))
+        return cls(n, device)
+
+
+def sprinter_verify(hidden, W1, b1, W2, b2, threshold: float, ws: Workspace, path: int = PATH_AUTO,
+                    want_scores: bool = True, out=None):
+    """hidden [B,K,d]; W1 [h,d], b1 [h], W2 [h], b2 [1] (or W1 [d], b1 = W2 = None).
+
+    Returns (scores f32 [B,K] or None, accept u8 [B,K], first_reject i32 [B])."""
+    _dev(hidden, name="hidden")
+    B, K, d = hidden.shape
+    dt = _dt(hidden)
+    _dev(W1, hidden.dtype, "W1")
+    h = 0 if W1.dim() == 1 else W1.shape[0]
+    if W1.shape[-1] != d:
+        raise ValueError("W1 inner dimension must equal d")
+    _dev(b2, torch.float32, "b2")
+    if h:
+        _dev(b1, torch.float32, "b1")
+        _dev(W2, hidden.dtype, "W2")
+        if b1.numel() != h or W2.numel() != h:
+            raise ValueError("b1 and W2 must have h entries")
+    else:
+        b1 = W2 = None
+    if out is None:
+        scores = torch.empty((B, K), dtype=torch.float32, device=hidden.device) if want_scores else None
+        accept = torch.empty((B, K), dtype=torch.uint8, device=hidden.device)
+        first_reject = torch.empty((B,), dtype=torch.int32, device=hidden.device)
+    else:
+        scores, accept, first_reject = out
+    rc = lib().sprinter_verify(_ptr(hidden), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), float(threshold),
+                               B, K, d, h, dt, path, _ptr(scores), _ptr(accept), _ptr(first_reject),
+                               _ptr(ws.buf), ws.nbytes, _stream())
+    _check("sprinter_verify", rc)
+    return scores, accept, first_reject
+
+
+def replace_sample(target_logits, V: int, uniforms, ws: Workspace, rows=None, first_reject=None,
+                   K: int = 0, seq_stride: int = 1, out=None):
+    """target_logits [R, ldv] (any leading shape is flattened to rows); returns tokens i32 [n]."""
+    _dev(target_logits, name="target_logits")
+    ldv = target_logits.shape[-1]
+    R = target_logits.numel() // ldv
+    _dev(uniforms, torch.float32, "uniforms")
+    n = uniforms.numel()
+    if rows is not None:
+        _dev(rows, torch.int32, "rows")
+    if first_reject is not None:
+        _dev(first_reject, torch.int32, "first_reject")
+    tokens = torch.empty((n,), dtype=torch.int32, device=target_logits.device) if out is None else out
+    rc = lib().replace_sample(_ptr(target_logits), ldv, V, R, _ptr(rows), _ptr(first_reject), K,
+                              seq_stride, n, _ptr(uniforms), _dt(target_logits), _ptr(tokens),
+                              _ptr(ws.buf), ws.nbytes, _stream())
+    _check("replace_sample", rc)
+    return tokens
+
+
+def sd_verify(p_logits, q_logits, V: int, draft_tokens, uniforms, ws: Workspace, extras: bool = True,
+              out=None):
+    """p_logits [B,Kp,ldv], q_logits [B,K,ldv], draft_tokens i32 [B,K], uniforms f32 [B,K+1].
+
+    Returns dict(accepted_len, correction_token[, accept, p_tok, q_tok, residual_mass])."""
+    _dev(p_logits, name="p_logits")
+    _dev(q_logits, p_logits.dtype, "q_logits")
+    B, Kp, ldv = p_logits.shape
+    K = q_logits.shape[1]
+    if q_logits.shape[0] != B or q_logits.shape[2] != ldv:
+        raise ValueError("p_logits and q_logits disagree in batch or row stride")
+    _dev(draft_tokens, torch.int32, "draft_tokens")
+    _dev(uniforms, torch.float32, "uniforms")
+    if tuple(draft_tokens.shape) != (B, K) or tuple(uniforms.shape) != (B, K + 1):
+        raise ValueError("draft_tokens must be [B,K] and uniforms [B,K+1]")
+    dev = p_logits.device
+    if out is None:
+        out = dict(accepted_len=torch.empty((B,), dtype=torch.int32, device=dev),
+                   correction_token=torch.empty((B,), dtype=torch.int32, device=dev))
+        if extras:
+            out.update(accept=torch.empty((B, K), dtype=torch.uint8, device=dev),
+                       p_tok=torch.empty((B, K), dtype=torch.float32, device=dev),
+                       q_tok=torch.empty((B, K), dtype=torch.float32, device=dev),
+                       residual_mass=torch.empty((B,), dtype=torch.float32, device=dev))
+    rc = lib().sd_verify(_ptr(p_logits), _ptr(q_logits), ldv, _ptr(draft_tokens), _ptr(uniforms),
+                         B, K, Kp, V, _dt(p_logits), _ptr(out["accepted_len"]),
+                         _ptr(out["correction_token"]), _ptr(out.get("accept")), _ptr(out.get("p_tok")),
+                         _ptr(out.get("q_tok")), _ptr(out.get("residual_mass")),
+                         _ptr(ws.buf), ws.nbytes, _stream())
+    _check("sd_verify", rc)
+    return out

@@ -1,0 +1,277 @@
+// C ABI of libsprinter: host-side argument validation, workspace carving, launches.
+#include <stdio.h>
+#include <string.h>
+
+#include "common.cuh"
+#include "launch.h"
+
+using namespace spr;
+
+namespace {
+
+thread_local char g_cuda_error[256] = "";
+
+int cuda_fail(cudaError_t e)
+{
+    snprintf(g_cuda_error, sizeof g_cuda_error, "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
+    return SPR_ERR_CUDA;
+}
+
+// compute capability 10.x only; the answer is cached per device ordinal
+int check_device()
+{
+    static int cached[64];  // 0 unknown, 1 ok, 2 unsupported
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev >= 0 && dev < 64 && cached[dev]) return cached[dev] == 1 ? SPR_OK : SPR_ERR_UNSUPPORTED;
+    int major = 0;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev >= 0 && dev < 64) cached[dev] = major == 10 ? 1 : 2;
+    return major == 10 ? SPR_OK : SPR_ERR_UNSUPPORTED;
+}
+
+bool dtype_ok(int dt) { return dt == SPR_F32 || dt == SPR_BF16; }
+bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+template <typename T>
+T *at(void *ws, size_t off)
+{
+    return reinterpret_cast<T *>(static_cast<char *>(ws) + off);
+}
+
+size_t verify_ws_bytes(int B, int K, int h)
+{
+    const int M = B * K;
+    return verify_ws_layout(M, verifier_simt_slices(h), (M + 127) / 128).end;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t spr_workspace_bytes(int op, int B, int K, int V, int d, int h, int dt)
+{
+    if (!dtype_ok(dt) || B < 0) return 0;
+    switch (op) {
+    case SPR_OP_SPRINTER_VERIFY:
+        if (K <= 0 || d <= 0 || h < 0 || (int64_t)B * K > 0x7fffffff) return 0;
+        return verify_ws_bytes(B, K, h);
+    case SPR_OP_REPLACE_SAMPLE:
+        if (V <= 0) return 0;
+        return draw_ws_layout(kHeaderBytes, B, chunks_per_row(V, dt)).end;
+    case SPR_OP_SD_VERIFY:
+        if (K <= 0 || V <= 0 || (int64_t)B * K > 0x7fffffff) return 0;
+        return sd_ws_layout(B, K, chunks_per_row(V, dt)).end;
+    default:
+        return 0;
+    }
+}
+
+int spr_workspace_init(void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    if (!ws || !aligned(ws, 256) || ws_bytes < (size_t)kHeaderBytes) return SPR_ERR_WORKSPACE;
+    cudaError_t e = cudaMemsetAsync(ws, 0, ws_bytes, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? SPR_OK : cuda_fail(e);
+}
+
+int sprinter_verify(const void *hidden, const void *W1, const float *b1, const void *W2,
+                    const float *b2, float threshold, int B, int K, int d, int h, int dt, int path,
+                    float *scores, uint8_t *accept, int32_t *first_reject, void *ws, size_t ws_bytes,
+                    void *cuda_stream)
+{
+    if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
+    if (path != SPR_VERIFIER_AUTO && path != SPR_VERIFIER_SIMT && path != SPR_VERIFIER_TENSOR)
+        return SPR_ERR_UNSUPPORTED;
+    if (!hidden || !W1 || !b2 || !accept || !first_reject) return SPR_ERR_INVALID_ARG;
+    if (B < 0 || K <= 0 || d <= 0 || h < 0 || (int64_t)B * K > 0x7fffffff) return SPR_ERR_INVALID_ARG;
+    if (h > 0 && (!b1 || !W2)) return SPR_ERR_INVALID_ARG;
+    const size_t es = elem_size(dt);
+    if (!aligned(hidden, es) || !aligned(W1, es) || (W2 && !aligned(W2, es)) || !aligned(b2, 4) ||
+        (b1 && !aligned(b1, 4)) || (scores && !aligned(scores, 4)) || !aligned(first_reject, 4))
+        return SPR_ERR_INVALID_ARG;
+    if (!ws || !aligned(ws, 256) || ws_bytes < verify_ws_bytes(B, K, h)) return SPR_ERR_WORKSPACE;
+    int rc = check_device();
+    if (rc != SPR_OK) return rc;
+    if (B == 0) return SPR_OK;
+
+    const int M = B * K;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    VerifyParams vp;
+    memset(&vp, 0, sizeof vp);
+    vp.hidden = hidden;
+    vp.W1 = W1;
+    vp.b1 = b1;
+    vp.W2 = W2;
+    vp.b2 = b2;
+    vp.threshold = threshold;
+    vp.B = B;
+    vp.K = K;
+    vp.d = d;
+    vp.h = h;
+    vp.scores = scores;
+    vp.accept = accept;
+    vp.first_reject = first_reject;
+    vp.status = at<int>(ws, 0);
+    const VerifyWs lay = verify_ws_layout(M, verifier_simt_slices(h), (M + 127) / 128);
+    vp.counter = at<int>(ws, lay.counter);
+    vp.part_z = at<float>(ws, lay.part_z);
+
+    if (path != SPR_VERIFIER_SIMT) {
+        const int tensor_rc = launch_verifier_tensor(vp, dt, st);  // < 0: shape not taken
+        if (tensor_rc == 0) return SPR_OK;
+        if (tensor_rc > 0) return cuda_fail((cudaError_t)tensor_rc);
+        if (path == SPR_VERIFIER_TENSOR) return SPR_ERR_UNSUPPORTED;
+    }
+    vp.slices = verifier_simt_slices(h);
+    cudaError_t e = launch_verifier_simt(vp, dt, st);
+    return e == cudaSuccess ? SPR_OK : cuda_fail(e);
+}
+
+int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, const int32_t *rows,
+                   const int32_t *first_reject, int K, int seq_stride, int n, const float *uniforms,
+                   int dt, int32_t *tokens, void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
+    if (!target_logits || !uniforms || !tokens) return SPR_ERR_INVALID_ARG;
+    if (V <= 0 || ldv < V || R <= 0 || n < 0 || seq_stride < 0) return SPR_ERR_INVALID_ARG;
+    if (first_reject && K <= 0) return SPR_ERR_INVALID_ARG;
+    if (!aligned(target_logits, elem_size(dt)) || !aligned(uniforms, 4) || !aligned(tokens, 4) ||
+        (rows && !aligned(rows, 4)) || (first_reject && !aligned(first_reject, 4)))
+        return SPR_ERR_INVALID_ARG;
+    const int C = chunks_per_row(V, dt);
+    const DrawWs lay = draw_ws_layout(kHeaderBytes, n, C);
+    if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
+    int rc = check_device();
+    if (rc != SPR_OK) return rc;
+    if (n == 0) return SPR_OK;
+
+    DrawParams dp;
+    memset(&dp, 0, sizeof dp);
+    dp.kind = DRAW_REPLACE;
+    dp.p = target_logits;
+    dp.ldv = ldv;
+    dp.V = V;
+    dp.chunks = C;
+    dp.R = R;
+    dp.rows = rows;
+    dp.gate = first_reject;
+    dp.seq_stride = seq_stride;
+    dp.K = K;
+    dp.uniforms = uniforms;
+    dp.tokens = tokens;
+    dp.status = at<int>(ws, 0);
+    dp.counters = at<int>(ws, lay.counters);
+    dp.part_m = at<float>(ws, lay.part_m);
+    dp.part_s = at<double>(ws, lay.part_s);
+    cudaError_t e = launch_draw(dp, n, dt, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? SPR_OK : cuda_fail(e);
+}
+
+int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int32_t *draft_tokens,
+              const float *uniforms, int B, int K, int Kp, int V, int dt, int32_t *accepted_len,
+              int32_t *correction_token, uint8_t *accept, float *p_tok, float *q_tok,
+              float *residual_mass, void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
+    if (!p_logits || !q_logits || !draft_tokens || !uniforms || !accepted_len || !correction_token)
+        return SPR_ERR_INVALID_ARG;
+    if (B < 0 || K <= 0 || V <= 0 || ldv < V || (Kp != K && Kp != K + 1) ||
+        (int64_t)B * K > 0x7fffffff)
+        return SPR_ERR_INVALID_ARG;
+    const size_t es = elem_size(dt);
+    if (!aligned(p_logits, es) || !aligned(q_logits, es) || !aligned(draft_tokens, 4) ||
+        !aligned(uniforms, 4) || !aligned(accepted_len, 4) || !aligned(correction_token, 4) ||
+        (p_tok && !aligned(p_tok, 4)) || (q_tok && !aligned(q_tok, 4)) ||
+        (residual_mass && !aligned(residual_mass, 4)))
+        return SPR_ERR_INVALID_ARG;
+    const int C = chunks_per_row(V, dt);
+    const SdWs lay = sd_ws_layout(B, K, C);
+    if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
+    int rc = check_device();
+    if (rc != SPR_OK) return rc;
+    if (B == 0) return SPR_OK;
+
+    SdParams sp;
+    memset(&sp, 0, sizeof sp);
+    sp.p = p_logits;
+    sp.q = q_logits;
+    sp.ldv = ldv;
+    sp.V = V;
+    sp.K = K;
+    sp.Kp = Kp;
+    sp.chunks = C;
+    sp.draft_tokens = draft_tokens;
+    sp.uniforms = uniforms;
+    sp.accepted_len = accepted_len;
+    sp.accept = accept;
+    sp.p_tok = p_tok;
+    sp.q_tok = q_tok;
+    sp.status = at<int>(ws, 0);
+    sp.row_counters = at<int>(ws, lay.row_counters);
+    sp.seq_counters = at<int>(ws, lay.seq_counters);
+    sp.acc = at<uint8_t>(ws, lay.acc);
+    sp.part = at<float4>(ws, lay.part);
+    sp.rowstats = at<float4>(ws, lay.rowstats);
+
+    DrawParams dp;
+    memset(&dp, 0, sizeof dp);
+    dp.kind = DRAW_SD;
+    dp.p = p_logits;
+    dp.q = q_logits;
+    dp.ldv = ldv;
+    dp.V = V;
+    dp.chunks = C;
+    dp.K = K;
+    dp.Kp = Kp;
+    dp.accepted_len = accepted_len;
+    dp.rowstats = sp.rowstats;
+    dp.uniforms = uniforms;
+    dp.tokens = correction_token;
+    dp.residual_mass = residual_mass;
+    dp.status = sp.status;
+    dp.counters = at<int>(ws, lay.draw.counters);
+    dp.part_m = at<float>(ws, lay.draw.part_m);
+    dp.part_s = at<double>(ws, lay.draw.part_s);
+
+    cudaError_t e = launch_sd_verify(sp, dp, B, K, dt, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? SPR_OK : cuda_fail(e);
+}
+
+int spr_device_status(void *ws, void *cuda_stream)
+{
+    if (!ws) return SPR_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, ws, sizeof word, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (word != 0) {
+        e = cudaMemsetAsync(ws, 0, sizeof word, st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return word;
+}
+
+const char *spr_status_string(int status)
+{
+    switch (status) {
+    case SPR_OK: return "ok";
+    case SPR_ERR_INVALID_ARG: return "invalid argument";
+    case SPR_ERR_UNSUPPORTED: return "unsupported dtype, op, path or device";
+    case SPR_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case SPR_ERR_CUDA: return "CUDA runtime error";
+    case SPR_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
+    case SPR_ERR_BAD_TOKEN: return "draft token id outside the vocabulary";
+    case SPR_ERR_BAD_ROW: return "logits row index outside the tensor";
+    default: return "unknown status";
+    }
+}
+
+const char *spr_last_cuda_error(void) { return g_cuda_error; }
+
+int spr_version(void) { return 100; }
+
+}  // extern "C"

@@ -78,4 +78,9 @@ cudaError_t launch_draw(const DrawParams &dp, int n, int dt, cudaStream_t st);
 int verifier_simt_slices(int h);
 cudaError_t launch_verifier_simt(const VerifyParams &vp, int dt, cudaStream_t st);
 
+// Tensor-core (tcgen05) verifier for bf16 MLPs.  Returns 0 when launched, a negative
+// value when it does not take this shape or dtype (nothing launched), or a positive
+// cudaError_t.  It sets the slice count itself.
+int launch_verifier_tensor(const VerifyParams &vp, int dt, cudaStream_t st);
+
 }  // namespace spr

@@ -1,0 +1,107 @@
+"""CPU-side checks: the C-ABI library loads and exports what include/sprinter.h declares,
+rejects bad arguments before touching a device, and the workload generator is seeded."""
+import ctypes
+import os
+import re
+
+import pytest
+import torch
+
+import paper_2502_04557_b200 as spr
+from paper_2502_04557_b200 import binding, workloads
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    names = []
+    for fn in sorted(os.listdir(os.path.join(ROOT, "include"))):
+        if fn.endswith(".h"):
+            text = open(os.path.join(ROOT, "include", fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names += re.findall(r"^\s*(?:const\s+)?(?:int|size_t|char\s*\*|void)\s*\*?\s*(\w+)\s*\(", text, flags=re.M)
+    return sorted(set(names))
+
+
+def test_library_exports_every_declared_symbol():
+    L = spr.lib()
+    names = declared_functions()
+    assert {"sprinter_verify", "replace_sample", "sd_verify", "spr_workspace_bytes"} <= set(names)
+    for n in names:
+        assert hasattr(L, n), f"{n} declared in include/ but not exported"
+    assert set(binding.EXPORTS) <= set(names)
+    assert L.spr_version() >= 100
+
+
+def test_workspace_bytes():
+    wb = spr.workspace_bytes
+    assert wb(binding.OP_SD_VERIFY, 256, 16, 128256, 1, 0, spr.BF16) > 0
+    assert wb(binding.OP_SD_VERIFY, 256, 0, 128256, 1, 0, spr.BF16) == 0
+    assert wb(binding.OP_SD_VERIFY, 256, 16, 128256, 1, 0, 7) == 0
+    assert wb(9, 1, 1, 1, 1, 1, 0) == 0
+    a = wb(binding.OP_REPLACE_SAMPLE, 10, 0, 1000, 0, 0, spr.F32)
+    b = wb(binding.OP_REPLACE_SAMPLE, 1000, 0, 1000, 0, 0, spr.F32)
+    assert 0 < a < b and a % 256 == 0
+    assert wb(binding.OP_SPRINTER_VERIFY, 32, 8, 0, 768, 256, spr.BF16) > 0
+
+
+def test_argument_validation_happens_on_the_host():
+    L = spr.lib()
+    buf = (ctypes.c_char * 4096)()
+    addr = (ctypes.addressof(buf) + 255) // 256 * 256
+    p = ctypes.c_void_p(addr)           # a non-null, aligned stand-in: never dereferenced
+    odd = ctypes.c_void_p(addr + 1)
+    # null tensors
+    assert L.sd_verify(None, p, 8, p, p, 1, 1, 1, 8, 0, p, p, None, None, None, None, p, 4096, None) == 1
+    # ldv < V, Kp not in {K, K+1}, bad dtype
+    assert L.sd_verify(p, p, 4, p, p, 1, 1, 1, 8, 0, p, p, None, None, None, None, p, 4096, None) == 1
+    assert L.sd_verify(p, p, 8, p, p, 1, 1, 3, 8, 0, p, p, None, None, None, None, p, 4096, None) == 1
+    assert L.sd_verify(p, p, 8, p, p, 1, 1, 1, 8, 5, p, p, None, None, None, None, p, 4096, None) == 2
+    # misaligned pointer, workspace too small / missing
+    assert L.sd_verify(odd, p, 8, p, p, 1, 1, 1, 8, 0, p, p, None, None, None, None, p, 4096, None) == 1
+    assert L.sd_verify(p, p, 8, p, p, 1, 1, 1, 8, 0, p, p, None, None, None, None, p, 16, None) == 3
+    assert L.sd_verify(p, p, 8, p, p, 1, 1, 1, 8, 0, p, p, None, None, None, None, None, 4096, None) == 3
+    assert L.replace_sample(p, 8, 0, 1, None, None, 0, 1, 1, p, 0, p, p, 4096, None) == 1
+    assert L.replace_sample(p, 8, 8, 1, None, p, 0, 1, 1, p, 0, p, p, 4096, None) == 1      # gate needs K > 0
+    assert L.replace_sample(p, 8, 8, 1, None, None, 0, 1, 1, p, 0, p, p, 8, None) == 3
+    assert L.sprinter_verify(p, p, None, None, p, 0.5, 1, 1, 8, 4, 0, 0, None, p, p, p, 4096, None) == 1
+    assert L.sprinter_verify(p, p, p, p, p, 0.5, 1, 0, 8, 4, 0, 0, None, p, p, p, 4096, None) == 1
+    assert L.sprinter_verify(p, p, p, p, p, 0.5, 1, 1, 8, 4, 0, 9, None, p, p, p, 4096, None) == 2
+    assert L.spr_status_string(6).decode().startswith("draft token")
+
+
+def test_binding_rejects_host_tensors():
+    with pytest.raises(ValueError):
+        binding._dev(torch.zeros(4), name="x")
+    with pytest.raises(TypeError):
+        binding._dt(torch.zeros(4, dtype=torch.float16))
+
+
+def test_workloads_are_seeded_and_shaped():
+    a = workloads.make("tiny", "cpu")
+    b = workloads.make("tiny", "cpu")
+    c = workloads.make("tiny", "cpu", sweep=1)
+    assert torch.equal(a.q_logits, b.q_logits) and torch.equal(a.uniforms, b.uniforms)
+    assert not torch.equal(a.q_logits, c.q_logits)
+    assert a.hidden.shape == (1, 4, 256) and a.p_logits.shape == (1, 5, 1000)
+    assert a.draft_tokens.dtype == torch.int32 and a.hidden.dtype == torch.float32
+    assert float(a.uniforms.min()) >= 0 and float(a.uniforms.max()) < 1
+    s = workloads.make("sequential", "cpu", B=2, bonus_row=False)
+    assert s.hidden.shape == (2, 1, 4096) and s.W1.shape == (1024, 4096)
+    assert s.p_logits.shape == (2, 1, 128256) and s.q_logits.dtype == torch.bfloat16
+    g = workloads.make("gpt2", "cpu", B=2, ldv=50264)
+    assert g.q_logits.shape == (2, 8, 50264) and float(g.q_logits[0, 0, 50257]) == 60.0
+    assert int(g.draft_tokens.max()) < 50257
+    # target/draft correlation of the llama3-style law
+    cfg = workloads.CONFIGS["llama3"]
+    assert abs(cfg.rho ** 2 * cfg.q_std ** 2 + cfg.noise_std ** 2 - 9.0) < 1e-9
+
+
+def test_shard_batch_partitions():
+    for B in (1, 7, 256, 1000):
+        for world in (1, 2, 3, 8):
+            spans = [workloads.shard_batch(B, r, world) for r in range(world)]
+            assert spans[0][0] == 0 and sum(n for _, n in spans) == B
+            for (f0, n0), (f1, _) in zip(spans, spans[1:]):
+                assert f0 + n0 == f1
+            assert max(n for _, n in spans) - min(n for _, n in spans) <= 1
