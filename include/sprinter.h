@@ -19,8 +19,10 @@
  *     non-zero return nothing was launched.
  *   - `ws` is caller-owned device scratch of at least spr_workspace_bytes()
  *     bytes, 256-byte aligned, cleared once with spr_workspace_init() after
- *     allocation.  A call leaves it ready for the next call.  Calls that may
- *     overlap on the GPU (different streams) need separate workspaces.
+ *     allocation (this zeroes the status word).  Each call clears the counters
+ *     it needs on the stream before its kernels, so one workspace serves calls
+ *     of any op and shape it is large enough for, one after the other.  Calls
+ *     that may overlap on the GPU (different streams) need separate workspaces.
  *   - Problems a kernel detects (a draft token id outside [0,V), a row index
  *     outside the logits tensor, a bounded wait that ran out) never trap: the
  *     affected outputs are set to -1, a sticky status word in `ws` records the
@@ -149,6 +151,40 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
               const float *uniforms, int B, int K, int Kp, int V, int dt, int32_t *accepted_len,
               int32_t *correction_token, uint8_t *accept, float *p_tok, float *q_tok,
               float *residual_mass, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Host-buffer variants.  Same operations and arguments as the calls above, but every
+ * tensor pointer is a HOST pointer (pinned memory makes the copies asynchronous and
+ * fast).  Each call copies its inputs into `arena` - caller-owned device memory of at
+ * least spr_host_arena_bytes() bytes, 256-byte aligned - runs the device entry point,
+ * copies the outputs back, synchronises the stream and returns the device status
+ * (so SPR_ERR_BAD_TOKEN / SPR_ERR_BAD_ROW come back directly).  replace_sample_host
+ * resolves the row of every draw on the host and uploads only the rows that are
+ * drawn from.  For spr_host_arena_bytes, B is the number of draws n for
+ * SPR_OP_REPLACE_SAMPLE, and unused sizes may be 0.
+ */
+size_t spr_host_arena_bytes(int op, int B, int K, int Kp, int64_t ldv, int d, int h, int dt);
+
+int sprinter_verify_host(const void *hidden, const void *W1, const float *b1, const void *W2,
+                         const float *b2, float threshold, int B, int K, int d, int h, int dt, int path,
+                         float *scores, uint8_t *accept, int32_t *first_reject, void *arena,
+                         size_t arena_bytes, void *ws, size_t ws_bytes, void *cuda_stream);
+
+int replace_sample_host(const void *target_logits, int64_t ldv, int V, int64_t R, const int32_t *rows,
+                        const int32_t *first_reject, int K, int seq_stride, int n,
+                        const float *uniforms, int dt, int32_t *tokens, void *arena, size_t arena_bytes,
+                        void *ws, size_t ws_bytes, void *cuda_stream);
+
+int sd_verify_host(const void *p_logits, const void *q_logits, int64_t ldv, const int32_t *draft_tokens,
+                   const float *uniforms, int B, int K, int Kp, int V, int dt, int32_t *accepted_len,
+                   int32_t *correction_token, uint8_t *accept, float *p_tok, float *q_tok,
+                   float *residual_mass, void *arena, size_t arena_bytes, void *ws, size_t ws_bytes,
+                   void *cuda_stream);
+
+/* Timing aid: while set (non-NULL cudaEvent_t handles), sd_verify calls made by this
+ * host thread record `before` / `after` on their stream around the row-statistics
+ * kernel, the launch that reads the 2*B*K*V logits.  Pass NULL, NULL to stop. */
+void spr_set_stage_events(void *before, void *after);
 
 /* Synchronises the stream, returns the sticky device status word of `ws`
  * (SPR_OK if nothing was detected) and clears it. */

@@ -21,6 +21,8 @@ PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
 EXPORTS = [
     "spr_workspace_bytes", "spr_workspace_init", "sprinter_verify", "replace_sample", "sd_verify",
     "spr_device_status", "spr_status_string", "spr_last_cuda_error", "spr_version",
+    "spr_host_arena_bytes", "sprinter_verify_host", "replace_sample_host", "sd_verify_host",
+    "spr_set_stage_events",
 ]
 
 
@@ -63,6 +65,19 @@ def lib():
         L.sd_verify.restype = i32
         L.sd_verify.argtypes = [vp, vp, i64, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp,
                                 vp, sz, vp]
+        L.spr_host_arena_bytes.restype = sz
+        L.spr_host_arena_bytes.argtypes = [i32, i32, i32, i32, i64, i32, i32, i32]
+        L.sprinter_verify_host.restype = i32
+        L.sprinter_verify_host.argtypes = [vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32,
+                                           vp, vp, vp, vp, sz, vp, sz, vp]
+        L.replace_sample_host.restype = i32
+        L.replace_sample_host.argtypes = [vp, i64, i32, i64, vp, vp, i32, i32, i32, vp, i32, vp,
+                                          vp, sz, vp, sz, vp]
+        L.sd_verify_host.restype = i32
+        L.sd_verify_host.argtypes = [vp, vp, i64, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp,
+                                     vp, vp, sz, vp, sz, vp]
+        L.spr_set_stage_events.restype = None
+        L.spr_set_stage_events.argtypes = [vp, vp]
         L.spr_device_status.restype = i32
         L.spr_device_status.argtypes = [vp, vp]
         L.spr_status_string.restype = C.c_char_p
@@ -219,3 +234,111 @@ def sd_verify(p_logits, q_logits, V: int, draft_tokens, uniforms, ws: Workspace,
                          _ptr(ws.buf), ws.nbytes, _stream())
     _check("sd_verify", rc)
     return out
+
+
+# ---------------------------------------------------------------------------- host buffers
+
+
+def _host(t: torch.Tensor, dtype=None, name="tensor"):
+    if t.is_cuda:
+        raise ValueError(f"{name} must be a host tensor")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}")
+    return t
+
+
+def host_arena_bytes(op: int, B: int, K: int = 1, Kp: int = 1, ldv: int = 0, d: int = 0, h: int = 0,
+                     dt: int = BF16) -> int:
+    return int(lib().spr_host_arena_bytes(op, B, K, Kp, ldv, d, h, dt))
+
+
+class Arena:
+    """Device staging memory for the host-buffer calls."""
+
+    def __init__(self, nbytes: int, device="cuda"):
+        self.buf = torch.empty((max(int(nbytes), 256) + 255) // 256 * 256, dtype=torch.uint8, device=device)
+
+    @property
+    def nbytes(self) -> int:
+        return self.buf.numel()
+
+
+def sprinter_verify_host(hidden, W1, b1, W2, b2, threshold: float, arena: Arena, ws: Workspace,
+                         path: int = PATH_AUTO, want_scores: bool = True, out=None):
+    """Host tensors in, host tensors out (pinned memory recommended); synchronises."""
+    _host(hidden, name="hidden")
+    B, K, d = hidden.shape
+    h = 0 if W1.dim() == 1 else W1.shape[0]
+    _host(W1, hidden.dtype, "W1")
+    _host(b2, torch.float32, "b2")
+    if h:
+        _host(b1, torch.float32, "b1")
+        _host(W2, hidden.dtype, "W2")
+    else:
+        b1 = W2 = None
+    if out is None:
+        scores = torch.empty((B, K), dtype=torch.float32) if want_scores else None
+        accept = torch.empty((B, K), dtype=torch.uint8)
+        first_reject = torch.empty((B,), dtype=torch.int32)
+    else:
+        scores, accept, first_reject = out
+    rc = lib().sprinter_verify_host(_ptr(hidden), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2),
+                                    float(threshold), B, K, d, h, _dt(hidden), path, _ptr(scores),
+                                    _ptr(accept), _ptr(first_reject), _ptr(arena.buf), arena.nbytes,
+                                    _ptr(ws.buf), ws.nbytes, _stream())
+    _check("sprinter_verify_host", rc)
+    return scores, accept, first_reject
+
+
+def replace_sample_host(target_logits, V: int, uniforms, arena: Arena, ws: Workspace, rows=None,
+                        first_reject=None, K: int = 0, seq_stride: int = 1, out=None):
+    _host(target_logits, name="target_logits")
+    ldv = target_logits.shape[-1]
+    R = target_logits.numel() // ldv
+    _host(uniforms, torch.float32, "uniforms")
+    n = uniforms.numel()
+    if rows is not None:
+        _host(rows, torch.int32, "rows")
+    if first_reject is not None:
+        _host(first_reject, torch.int32, "first_reject")
+    tokens = torch.empty((n,), dtype=torch.int32) if out is None else out
+    rc = lib().replace_sample_host(_ptr(target_logits), ldv, V, R, _ptr(rows), _ptr(first_reject), K,
+                                   seq_stride, n, _ptr(uniforms), _dt(target_logits), _ptr(tokens),
+                                   _ptr(arena.buf), arena.nbytes, _ptr(ws.buf), ws.nbytes, _stream())
+    _check("replace_sample_host", rc)
+    return tokens
+
+
+def sd_verify_host(p_logits, q_logits, V: int, draft_tokens, uniforms, arena: Arena, ws: Workspace,
+                   extras: bool = False, out=None):
+    _host(p_logits, name="p_logits")
+    _host(q_logits, p_logits.dtype, "q_logits")
+    B, Kp, ldv = p_logits.shape
+    K = q_logits.shape[1]
+    _host(draft_tokens, torch.int32, "draft_tokens")
+    _host(uniforms, torch.float32, "uniforms")
+    if out is None:
+        out = dict(accepted_len=torch.empty((B,), dtype=torch.int32),
+                   correction_token=torch.empty((B,), dtype=torch.int32))
+        if extras:
+            out.update(accept=torch.empty((B, K), dtype=torch.uint8),
+                       p_tok=torch.empty((B, K), dtype=torch.float32),
+                       q_tok=torch.empty((B, K), dtype=torch.float32),
+                       residual_mass=torch.empty((B,), dtype=torch.float32))
+    rc = lib().sd_verify_host(_ptr(p_logits), _ptr(q_logits), ldv, _ptr(draft_tokens), _ptr(uniforms),
+                              B, K, Kp, V, _dt(p_logits), _ptr(out["accepted_len"]),
+                              _ptr(out["correction_token"]), _ptr(out.get("accept")),
+                              _ptr(out.get("p_tok")), _ptr(out.get("q_tok")),
+                              _ptr(out.get("residual_mass")), _ptr(arena.buf), arena.nbytes,
+                              _ptr(ws.buf), ws.nbytes, _stream())
+    _check("sd_verify_host", rc)
+    return out
+
+
+def set_stage_events(before=None, after=None):
+    """torch.cuda.Event pair (created with enable_timing=True and recorded once so that the
+    handles exist) that sd_verify records around its row-statistics kernel; None to stop."""
+    lib().spr_set_stage_events(None if before is None else C.c_void_p(before.cuda_event),
+                               None if after is None else C.c_void_p(after.cuda_event))

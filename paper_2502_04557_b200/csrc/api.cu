@@ -16,6 +16,13 @@ int cuda_fail(cudaError_t e)
     snprintf(g_cuda_error, sizeof g_cuda_error, "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
     return SPR_ERR_CUDA;
 }
+}  // namespace
+
+namespace spr {
+int report_cuda_error(cudaError_t e) { return cuda_fail(e); }
+}  // namespace spr
+
+namespace {
 
 // compute capability 10.x only; the answer is cached per device ordinal
 int check_device()
@@ -60,7 +67,7 @@ size_t spr_workspace_bytes(int op, int B, int K, int V, int d, int h, int dt)
         return verify_ws_bytes(B, K, h);
     case SPR_OP_REPLACE_SAMPLE:
         if (V <= 0) return 0;
-        return draw_ws_layout(kHeaderBytes, B, chunks_per_row(V, dt)).end;
+        return replace_ws_layout(B, chunks_per_row(V, dt)).end;
     case SPR_OP_SD_VERIFY:
         if (K <= 0 || V <= 0 || (int64_t)B * K > 0x7fffffff) return 0;
         return sd_ws_layout(B, K, chunks_per_row(V, dt)).end;
@@ -84,8 +91,9 @@ int sprinter_verify(const void *hidden, const void *W1, const float *b1, const v
     if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
     if (path != SPR_VERIFIER_AUTO && path != SPR_VERIFIER_SIMT && path != SPR_VERIFIER_TENSOR)
         return SPR_ERR_UNSUPPORTED;
-    if (!hidden || !W1 || !b2 || !accept || !first_reject) return SPR_ERR_INVALID_ARG;
     if (B < 0 || K <= 0 || d <= 0 || h < 0 || (int64_t)B * K > 0x7fffffff) return SPR_ERR_INVALID_ARG;
+    if (B == 0) return SPR_OK;  // empty batch: nothing to read or write, pointers may be null
+    if (!hidden || !W1 || !b2 || !accept || !first_reject) return SPR_ERR_INVALID_ARG;
     if (h > 0 && (!b1 || !W2)) return SPR_ERR_INVALID_ARG;
     const size_t es = elem_size(dt);
     if (!aligned(hidden, es) || !aligned(W1, es) || (W2 && !aligned(W2, es)) || !aligned(b2, 4) ||
@@ -117,6 +125,8 @@ int sprinter_verify(const void *hidden, const void *W1, const float *b1, const v
     const VerifyWs lay = verify_ws_layout(M, verifier_simt_slices(h), (M + 127) / 128);
     vp.counter = at<int>(ws, lay.counter);
     vp.part_z = at<float>(ws, lay.part_z);
+    cudaError_t ce = cudaMemsetAsync(vp.counter, 0, lay.counters_end - lay.counter, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
 
     if (path != SPR_VERIFIER_SIMT) {
         const int tensor_rc = launch_verifier_tensor(vp, dt, st);  // < 0: shape not taken
@@ -134,14 +144,15 @@ int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, con
                    int dt, int32_t *tokens, void *ws, size_t ws_bytes, void *cuda_stream)
 {
     if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
-    if (!target_logits || !uniforms || !tokens) return SPR_ERR_INVALID_ARG;
-    if (V <= 0 || ldv < V || R <= 0 || n < 0 || seq_stride < 0) return SPR_ERR_INVALID_ARG;
+    if (V <= 0 || ldv < V || R < 0 || n < 0 || seq_stride < 0) return SPR_ERR_INVALID_ARG;
+    if (n == 0) return SPR_OK;  // no draws: pointers may be null
+    if (!target_logits || !uniforms || !tokens || R == 0) return SPR_ERR_INVALID_ARG;
     if (first_reject && K <= 0) return SPR_ERR_INVALID_ARG;
     if (!aligned(target_logits, elem_size(dt)) || !aligned(uniforms, 4) || !aligned(tokens, 4) ||
         (rows && !aligned(rows, 4)) || (first_reject && !aligned(first_reject, 4)))
         return SPR_ERR_INVALID_ARG;
     const int C = chunks_per_row(V, dt);
-    const DrawWs lay = draw_ws_layout(kHeaderBytes, n, C);
+    const DrawWs lay = replace_ws_layout(n, C);
     if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
     int rc = check_device();
     if (rc != SPR_OK) return rc;
@@ -165,7 +176,9 @@ int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, con
     dp.counters = at<int>(ws, lay.counters);
     dp.part_m = at<float>(ws, lay.part_m);
     dp.part_s = at<double>(ws, lay.part_s);
-    cudaError_t e = launch_draw(dp, n, dt, static_cast<cudaStream_t>(cuda_stream));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaMemsetAsync(dp.counters, 0, sizeof(int) * (size_t)n, st);
+    if (e == cudaSuccess) e = launch_draw(dp, n, dt, st);
     return e == cudaSuccess ? SPR_OK : cuda_fail(e);
 }
 
@@ -175,10 +188,11 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
               float *residual_mass, void *ws, size_t ws_bytes, void *cuda_stream)
 {
     if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
-    if (!p_logits || !q_logits || !draft_tokens || !uniforms || !accepted_len || !correction_token)
-        return SPR_ERR_INVALID_ARG;
     if (B < 0 || K <= 0 || V <= 0 || ldv < V || (Kp != K && Kp != K + 1) ||
         (int64_t)B * K > 0x7fffffff)
+        return SPR_ERR_INVALID_ARG;
+    if (B == 0) return SPR_OK;  // empty batch: pointers may be null
+    if (!p_logits || !q_logits || !draft_tokens || !uniforms || !accepted_len || !correction_token)
         return SPR_ERR_INVALID_ARG;
     const size_t es = elem_size(dt);
     if (!aligned(p_logits, es) || !aligned(q_logits, es) || !aligned(draft_tokens, 4) ||
@@ -235,7 +249,9 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
     dp.part_m = at<float>(ws, lay.draw.part_m);
     dp.part_s = at<double>(ws, lay.draw.part_s);
 
-    cudaError_t e = launch_sd_verify(sp, dp, B, K, dt, static_cast<cudaStream_t>(cuda_stream));
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaMemsetAsync(sp.row_counters, 0, lay.counters_end - lay.row_counters, st);
+    if (e == cudaSuccess) e = launch_sd_verify(sp, dp, B, K, dt, st);
     return e == cudaSuccess ? SPR_OK : cuda_fail(e);
 }
 
@@ -271,6 +287,11 @@ const char *spr_status_string(int status)
 }
 
 const char *spr_last_cuda_error(void) { return g_cuda_error; }
+
+void spr_set_stage_events(void *before, void *after)
+{
+    set_stage_events(static_cast<cudaEvent_t>(before), static_cast<cudaEvent_t>(after));
+}
 
 int spr_version(void) { return 100; }
 

@@ -29,26 +29,35 @@ __host__ __device__ inline int chunks_per_row(int V, int dt)
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // ---------------------------------------------------------------- workspace layouts
-// All offsets are multiples of 256 bytes from the start of the workspace.
+// All offsets are multiples of 256 bytes from the start of the workspace.  Every layout
+// puts its ticket counters in one contiguous zone right after the header; the entry point
+// clears that zone on the stream before its first kernel, so a workspace may be shared by
+// calls of different ops and shapes.
 struct DrawWs {              // replace_sample, and the correction draw of sd_verify
-    size_t counters;         // int32 [n]      chunks finished per draw (0 between calls)
+    size_t counters;         // int32 [n]      chunks finished per draw
     size_t part_m;           // float [n*C]    chunk maximum (softmax draws)
     size_t part_s;           // double [n*C]   chunk weight sum
     size_t end;
 };
-__host__ __device__ inline DrawWs draw_ws_layout(size_t base, int n, int C)
+__host__ __device__ inline DrawWs draw_ws_layout(size_t counters, size_t scratch, int n, int C)
 {
     DrawWs w;
-    w.counters = base;
-    w.part_m = align_up(w.counters + sizeof(int32_t) * (size_t)n, 256);
+    w.counters = counters;
+    w.part_m = align_up(scratch, 256);
     w.part_s = align_up(w.part_m + sizeof(float) * (size_t)n * C, 256);
     w.end = align_up(w.part_s + sizeof(double) * (size_t)n * C, 256);
     return w;
+}
+// replace_sample alone: counters [n] directly after the header
+__host__ __device__ inline DrawWs replace_ws_layout(int n, int C)
+{
+    return draw_ws_layout(kHeaderBytes, kHeaderBytes + align_up(sizeof(int32_t) * (size_t)n, 256), n, C);
 }
 
 struct SdWs {
     size_t row_counters;     // int32 [M]      chunks finished per row
     size_t seq_counters;     // int32 [B]      rows finished per sequence
+    size_t counters_end;     // end of the zone cleared per call (includes the draw counters)
     size_t acc;              // uint8 [M]      0 reject, 1 accept, 2 invalid token
     size_t part;             // float4 [M*C]   (max_p, sum_p, max_q, sum_q) per chunk
     size_t rowstats;         // float4 [M]     (max_p, ln Z_p, max_q, ln Z_q)
@@ -60,17 +69,20 @@ __host__ __device__ inline SdWs sd_ws_layout(int B, int K, int C)
     const size_t M = (size_t)B * K;
     SdWs w;
     w.row_counters = kHeaderBytes;
-    w.seq_counters = align_up(w.row_counters + 4 * M, 256);
-    w.acc = align_up(w.seq_counters + 4 * (size_t)B, 256);
+    w.seq_counters = w.row_counters + 4 * M;
+    const size_t draw_counters = w.seq_counters + 4 * (size_t)B;
+    w.counters_end = align_up(draw_counters + 4 * (size_t)B, 256);
+    w.acc = w.counters_end;
     w.part = align_up(w.acc + M, 256);
     w.rowstats = align_up(w.part + 16 * M * C, 256);
-    w.draw = draw_ws_layout(align_up(w.rowstats + 16 * M, 256), B, C);
+    w.draw = draw_ws_layout(draw_counters, align_up(w.rowstats + 16 * M, 256), B, C);
     w.end = w.draw.end;
     return w;
 }
 
 struct VerifyWs {
     size_t counter;          // int32 [1 + row tiles]   CTAs finished
+    size_t counters_end;
     size_t part_z;           // float [slices * M]      per-slice partial of W2 . relu(...)
     size_t end;
 };
@@ -78,7 +90,8 @@ __host__ __device__ inline VerifyWs verify_ws_layout(int M, int slices, int tile
 {
     VerifyWs w;
     w.counter = kHeaderBytes;
-    w.part_z = align_up(w.counter + 4 * (size_t)(1 + tiles), 256);
+    w.counters_end = align_up(w.counter + 4 * (size_t)(1 + tiles), 256);
+    w.part_z = w.counters_end;
     w.end = align_up(w.part_z + 4 * (size_t)slices * M, 256);
     return w;
 }

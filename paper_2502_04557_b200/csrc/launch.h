@@ -72,6 +72,8 @@ struct VerifyParams {
 
 cudaError_t launch_sd_verify(const SdParams &sp, const DrawParams &dp, int B, int K, int dt,
                              cudaStream_t st);
+int report_cuda_error(cudaError_t e);  // records the text, returns SPR_ERR_CUDA
+void set_stage_events(cudaEvent_t before, cudaEvent_t after);
 cudaError_t launch_draw(const DrawParams &dp, int n, int dt, cudaStream_t st);
 
 // SIMT verifier: any dtype and shape.  `slices` must equal verifier_simt_slices(h).

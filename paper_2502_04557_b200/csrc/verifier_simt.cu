@@ -171,7 +171,6 @@ __global__ void __launch_bounds__(kThreads) verifier_simt_kernel(const VerifyPar
     if (!s_last) return;
     __threadfence();
     finalise_scores(prm);
-    if (tid == 0) *prm.counter = 0;
 }
 
 int verifier_simt_slices(int h) { return h > 0 ? (h + kWarps - 1) / kWarps : 1; }

@@ -245,7 +245,6 @@ __global__ void __launch_bounds__(kThreads) sd_row_stats_kernel(const SdParams p
         if (prm.p_tok) prm.p_tok[row] = P;
         if (prm.q_tok) prm.q_tok[row] = Q;
         prm.rowstats[row] = make_float4(m_p, (float)lnz_p, m_q, (float)lnz_q);
-        prm.row_counters[row] = 0;  // ready for the next call
         __threadfence();
         last_row = (atomicAdd(&prm.seq_counters[b], 1) == prm.K - 1);
     }
@@ -267,7 +266,6 @@ __global__ void __launch_bounds__(kThreads) sd_row_stats_kernel(const SdParams p
         prm.accepted_len[b] = bad ? -1 : first;
         if (bad && prm.accept)
             for (int kk = 0; kk < prm.K; ++kk) prm.accept[(int64_t)b * prm.K + kk] = 0;
-        prm.seq_counters[b] = 0;
     }
 }
 
@@ -569,11 +567,19 @@ __global__ void __launch_bounds__(kThreads) draw_kernel(const DrawParams prm)
     }
     if (tid == 0) {
         prm.tokens[i] = token;
-        prm.counters[i] = 0;  // ready for the next call
     }
 }
 
 // ================================================================ host launchers
+// Optional CUDA events recorded right before and after the row-statistics kernel (the
+// launch that moves almost all the bytes), so a caller can time it inside a longer step.
+static thread_local cudaEvent_t g_stage_before = nullptr, g_stage_after = nullptr;
+void set_stage_events(cudaEvent_t before, cudaEvent_t after)
+{
+    g_stage_before = before;
+    g_stage_after = after;
+}
+
 template <typename T>
 static cudaError_t launch_sd_t(const SdParams &sp, const DrawParams &dp, int B, int K, cudaStream_t st)
 {
@@ -581,9 +587,11 @@ static cudaError_t launch_sd_t(const SdParams &sp, const DrawParams &dp, int B, 
     const int64_t grid_b = (int64_t)B * dp.chunks;
     if (grid_a > 0x7fffffffLL || grid_b > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     if (grid_a == 0) return cudaSuccess;
+    if (g_stage_before) cudaEventRecord(g_stage_before, st);
     sd_row_stats_kernel<T><<<(unsigned)grid_a, kThreads, 0, st>>>(sp);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    if (g_stage_after) cudaEventRecord(g_stage_after, st);
     draw_kernel<T><<<(unsigned)grid_b, kThreads, 0, st>>>(dp);
     return cudaGetLastError();
 }

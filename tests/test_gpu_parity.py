@@ -329,6 +329,7 @@ def test_sd_equal_and_disjoint_distributions(spr):
     p2 = torch.full((B, K, V), ninf); p2[..., :100] = torch.randn((B, K, 100), generator=g)
     q2 = torch.full((B, K, V), ninf); q2[..., 100:] = torch.randn((B, K, V - 100), generator=g)
     x2 = torch.randint(100, V, (B, K), generator=g, dtype=torch.int32)
+    ws = spr.Workspace(spr.workspace_bytes(2, B, K, V, 1, 0, spr.F32))
     out = spr.sd_verify(p2.cuda(), q2.cuda(), V, x2.cuda(), u.clamp(min=1e-3).cuda(), ws)
     assert (out["accept"] == 0).all() and (out["accepted_len"] == 0).all()
     assert ((out["correction_token"] >= 0) & (out["correction_token"] < 100)).all()

@@ -66,6 +66,9 @@ def test_argument_validation_happens_on_the_host():
     assert L.replace_sample(p, 8, 8, 1, None, None, 0, 1, 1, p, 0, p, p, 8, None) == 3
     assert L.sprinter_verify(p, p, None, None, p, 0.5, 1, 1, 8, 4, 0, 0, None, p, p, p, 4096, None) == 1
     assert L.sprinter_verify(p, p, p, p, p, 0.5, 1, 0, 8, 4, 0, 0, None, p, p, p, 4096, None) == 1
+    # empty problems are fine and touch nothing
+    assert L.sd_verify(None, None, 8, None, None, 0, 1, 1, 8, 0, None, None, None, None, None, None, None, 0, None) == 0
+    assert L.replace_sample(None, 8, 8, 0, None, None, 0, 1, 0, None, 0, None, None, 0, None) == 0
     assert L.sprinter_verify(p, p, p, p, p, 0.5, 1, 1, 8, 4, 0, 9, None, p, p, p, 4096, None) == 2
     assert L.spr_status_string(6).decode().startswith("draft token")
 
