@@ -181,6 +181,38 @@ int sd_verify_host(const void *p_logits, const void *q_logits, int64_t ldv, cons
                    float *residual_mass, void *arena, size_t arena_bytes, void *ws, size_t ws_bytes,
                    void *cuda_stream);
 
+/*
+ * replace_sample_static - replace_sample without a caller workspace.
+ *
+ * The paper has no counterpart: this exists for callers of this library that are not
+ * allowed to allocate device memory around the call - code that runs inside someone
+ * else's memory budget (a serving engine that has handed all free HBM to its KV-cache
+ * pool, a plugin whose host forbids cudaMalloc), or that runs where cudaMalloc would
+ * stall everything (it synchronises the device).  They have nowhere to get a `ws` from.
+ * Same operation, arguments and results as replace_sample(), but the scratch is a fixed
+ * array inside the library image (about 200 KB on every GPU that loads the library, held
+ * until the process exits).  The call allocates and frees nothing.
+ *
+ * Limits: n <= SPR_STATIC_MAX_DRAWS and n * chunks <= SPR_STATIC_MAX_DRAW_CHUNKS, where
+ * chunks = ceil((V + 7) / 8192) for bf16 and ceil((V + 3) / 4096) for f32 (16 for
+ * V = 128256 bf16, so up to 1024 draws per call).  Larger requests return
+ * SPR_ERR_WORKSPACE and launch nothing; split them or use replace_sample().
+ *
+ * First call on a device: looks up the device address of the array (the device must be
+ * current).  Make that first call before starting any stream capture.
+ * Sharing: every call on a GPU uses the same array.  Calls that can overlap on that GPU
+ * (two streams, two host threads) race on it and give wrong tokens; issue them on one
+ * stream or serialise them.  The array keeps the previous call's contents; the call clears
+ * the part that must start at zero itself.
+ * Device-detected bad rows still give tokens[i] = -1, but there is no status word to read
+ * back.
+ */
+#define SPR_STATIC_MAX_DRAWS 1024
+#define SPR_STATIC_MAX_DRAW_CHUNKS 16384
+int replace_sample_static(const void *target_logits, int64_t ldv, int V, int64_t R, const int32_t *rows,
+                          const int32_t *first_reject, int K, int seq_stride, int n,
+                          const float *uniforms, int dt, int32_t *tokens, void *cuda_stream);
+
 /* Timing aid: while set (non-NULL cudaEvent_t handles), sd_verify calls made by this
  * host thread record `before` / `after` on their stream around the row-statistics
  * kernel, the launch that reads the 2*B*K*V logits.  Pass NULL, NULL to stop. */

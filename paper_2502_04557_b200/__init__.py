@@ -5,6 +5,6 @@ of ``libsprinter.so`` (CUDA kernels for sm_100a); ``workloads`` draws the synthe
 """
 from . import workloads  # noqa: F401
 from .binding import (Arena, host_arena_bytes, replace_sample_host, sd_verify_host,  # noqa: F401
-                      set_stage_events, sprinter_verify_host)
+                      replace_sample_static, set_stage_events, sprinter_verify_host)
 from .binding import (BF16, F32, PATH_AUTO, PATH_SIMT, PATH_TENSOR, SprinterError, Workspace,  # noqa: F401
                       lib, replace_sample, sd_verify, sprinter_verify, workspace_bytes)

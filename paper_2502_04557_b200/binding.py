@@ -22,7 +22,7 @@ EXPORTS = [
     "spr_workspace_bytes", "spr_workspace_init", "sprinter_verify", "replace_sample", "sd_verify",
     "spr_device_status", "spr_status_string", "spr_last_cuda_error", "spr_version",
     "spr_host_arena_bytes", "sprinter_verify_host", "replace_sample_host", "sd_verify_host",
-    "spr_set_stage_events",
+    "spr_set_stage_events", "replace_sample_static",
 ]
 
 
@@ -76,6 +76,8 @@ def lib():
         L.sd_verify_host.restype = i32
         L.sd_verify_host.argtypes = [vp, vp, i64, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp,
                                      vp, vp, sz, vp, sz, vp]
+        L.replace_sample_static.restype = i32
+        L.replace_sample_static.argtypes = [vp, i64, i32, i64, vp, vp, i32, i32, i32, vp, i32, vp, vp]
         L.spr_set_stage_events.restype = None
         L.spr_set_stage_events.argtypes = [vp, vp]
         L.spr_device_status.restype = i32
@@ -342,3 +344,25 @@ def set_stage_events(before=None, after=None):
     handles exist) that sd_verify records around its row-statistics kernel; None to stop."""
     lib().spr_set_stage_events(None if before is None else C.c_void_p(before.cuda_event),
                                None if after is None else C.c_void_p(after.cuda_event))
+
+
+def replace_sample_static(target_logits, V: int, uniforms, tokens, rows=None, first_reject=None,
+                          K: int = 0, seq_stride: int = 1):
+    """replace_sample on the library's built-in scratch: no workspace argument, and nothing is
+    allocated here either - the caller passes the output tensor `tokens` (int32 [n]).  For
+    code that must not allocate device memory around the call; limited to
+    n <= 1024 draws and n * chunks <= 16384 (see include/sprinter.h).  Calls that may overlap
+    on one GPU race on the shared scratch: keep them on one stream."""
+    _dev(target_logits, name="target_logits")
+    ldv = target_logits.shape[-1]
+    R = target_logits.numel() // ldv
+    _dev(uniforms, torch.float32, "uniforms")
+    _dev(tokens, torch.int32, "tokens")
+    n = uniforms.numel()
+    if tokens.numel() != n:
+        raise ValueError("tokens must have one entry per uniform")
+    rc = lib().replace_sample_static(_ptr(target_logits), ldv, V, R, _ptr(rows), _ptr(first_reject), K,
+                                     seq_stride, n, _ptr(uniforms), _dt(target_logits), _ptr(tokens),
+                                     _stream())
+    _check("replace_sample_static", rc)
+    return tokens
