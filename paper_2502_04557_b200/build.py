@@ -10,7 +10,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libsprinter.so")
 SOURCES = ["api.cu", "host_api.cu", "vocab_kernels.cu", "verifier_simt.cu", "verifier_tensor.cu", "no_alloc.cu"]
-HEADERS = ["common.cuh", "launch.h"]
+HEADERS = ["common.cuh", "launch.h", "verifier_common.cuh"]
 
 
 def _nvcc() -> str:

@@ -421,3 +421,46 @@ def test_verifier_threshold_equality(spr):
     tau = float(np.nextafter(np.float32(0.5), np.float32(1)))
     s, a, fr = spr.sprinter_verify(H, z(8, 64).cuda(), z(8).cuda(), z(8).cuda(), z(1).cuda(), tau, ws)
     assert (a == 0).all() and (fr == 0).all()
+
+
+@pytest.mark.parametrize("B,K,d,h", [(4, 8, 64, 16), (40, 8, 256, 96), (130, 3, 136, 20), (32, 8, 768, 256),
+                                      (64, 1, 4096, 1024), (100, 16, 2048, 512)])
+def test_verifier_tensor_core_path(spr, B, K, d, h):
+    """tcgen05 kernel forced (PATH_TENSOR) on shapes with ragged M, h and d tails."""
+    g = torch.Generator().manual_seed(B * 7 + K + d + h)
+    H = torch.randn((B, K, d), generator=g).to(torch.bfloat16)
+    W1 = (torch.randn((h, d), generator=g) / d ** 0.5).to(torch.bfloat16)
+    b1 = torch.randn(h, generator=g) / d ** 0.5
+    W2 = (torch.randn(h, generator=g) / h ** 0.5 * 3).to(torch.bfloat16)
+    b2 = torch.tensor([0.1])
+    tau = 0.5
+    for _ in range(20):
+        s_ref, a_ref, fr_ref = oracle.sprinter_verify(to_np(H), to_np(W1), to_np(b1), to_np(W2), to_np(b2), tau)
+        near = np.argwhere(np.abs(s_ref - tau) < MARGIN)
+        if not len(near):
+            break
+        for b, k in near:
+            H[b, k] = torch.randn(d, generator=g).to(torch.bfloat16)
+    ws = spr.Workspace(spr.workspace_bytes(0, B, K, 1, d, h, spr.BF16))
+    args = (H.cuda(), W1.cuda(), b1.cuda(), W2.cuda(), b2.cuda(), tau, ws)
+    scores, accept, fr = spr.sprinter_verify(*args, path=spr.PATH_TENSOR)
+    assert ws.device_status() == 0
+    eq(accept, a_ref, "accept")
+    eq(fr, fr_ref, "first_reject")
+    assert_close_rel(scores, s_ref, 1e-3, "scores")
+    # second call on the same workspace, and agreement with the SIMT kernel
+    scores2, accept2, fr2 = spr.sprinter_verify(*args, path=spr.PATH_TENSOR)
+    assert torch.equal(scores, scores2) and torch.equal(fr, fr2)
+    scores3, accept3, _ = spr.sprinter_verify(*args, path=spr.PATH_SIMT)
+    assert torch.equal(accept, accept3)
+    assert torch.allclose(scores, scores3, rtol=1e-4, atol=1e-6)
+
+
+def test_verifier_tensor_path_refuses_unsupported_shapes(spr):
+    H = torch.randn(2, 4, 64).cuda()          # fp32
+    z = torch.zeros
+    ws = spr.Workspace(spr.workspace_bytes(0, 2, 4, 1, 64, 8, spr.F32))
+    with pytest.raises(spr.SprinterError) as e:
+        spr.sprinter_verify(H, z(8, 64).cuda(), z(8).cuda(), z(8).cuda(), z(1).cuda(), 0.5, ws,
+                            path=spr.PATH_TENSOR)
+    assert e.value.status == 2
