@@ -70,7 +70,7 @@ size_t spr_workspace_bytes(int op, int B, int K, int V, int d, int h, int dt)
         return replace_ws_layout(B, chunks_per_row(V, dt)).end;
     case SPR_OP_SD_VERIFY:
         if (K <= 0 || V <= 0 || (int64_t)B * K > 0x7fffffff) return 0;
-        return sd_ws_layout(B, K, chunks_per_row(V, dt)).end;
+        return sd_ws_layout(B, K, stat_segments_per_row(V, dt), chunks_per_row(V, dt)).end;
     default:
         return 0;
     }
@@ -200,8 +200,8 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
         (p_tok && !aligned(p_tok, 4)) || (q_tok && !aligned(q_tok, 4)) ||
         (residual_mass && !aligned(residual_mass, 4)))
         return SPR_ERR_INVALID_ARG;
-    const int C = chunks_per_row(V, dt);
-    const SdWs lay = sd_ws_layout(B, K, C);
+    const int C = chunks_per_row(V, dt), S = stat_segments_per_row(V, dt);
+    const SdWs lay = sd_ws_layout(B, K, S, C);
     if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
     int rc = check_device();
     if (rc != SPR_OK) return rc;
@@ -215,7 +215,7 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
     sp.V = V;
     sp.K = K;
     sp.Kp = Kp;
-    sp.chunks = C;
+    sp.chunks = S;
     sp.draft_tokens = draft_tokens;
     sp.uniforms = uniforms;
     sp.accepted_len = accepted_len;

@@ -26,6 +26,16 @@ __host__ __device__ inline int chunks_per_row(int V, int dt)
     return (V + vec_elems(dt) - 1 + chunk_elems(dt) - 1) / chunk_elems(dt);
 }
 
+// Row statistics (sd_verify stage 1): a warp consumes "steps" of 32 lanes x kUnroll vectors,
+// kStatIters of them per CTA, so one CTA covers a segment of kWarps*kStatIters steps of a row.
+constexpr int kStatIters = 4;
+__host__ __device__ constexpr int stat_step_elems(int dt) { return 32 * kUnroll * vec_elems(dt); }
+__host__ __device__ constexpr int stat_segment_elems(int dt) { return kWarps * kStatIters * stat_step_elems(dt); }
+__host__ __device__ inline int stat_segments_per_row(int V, int dt)
+{
+    return (V + vec_elems(dt) - 1 + stat_segment_elems(dt) - 1) / stat_segment_elems(dt);
+}
+
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // ---------------------------------------------------------------- workspace layouts
@@ -59,12 +69,12 @@ struct SdWs {
     size_t seq_counters;     // int32 [B]      rows finished per sequence
     size_t counters_end;     // end of the zone cleared per call (includes the draw counters)
     size_t acc;              // uint8 [M]      0 reject, 1 accept, 2 invalid token
-    size_t part;             // float4 [M*C]   (max_p, sum_p, max_q, sum_q) per chunk
+    size_t part;             // float4 [M*S]   (max_p, sum_p, max_q, sum_q) per row segment
     size_t rowstats;         // float4 [M]     (max_p, ln Z_p, max_q, ln Z_q)
     DrawWs draw;             // correction draw, n = B
     size_t end;
 };
-__host__ __device__ inline SdWs sd_ws_layout(int B, int K, int C)
+__host__ __device__ inline SdWs sd_ws_layout(int B, int K, int S, int C)   // S stat segments, C draw chunks
 {
     const size_t M = (size_t)B * K;
     SdWs w;
@@ -74,7 +84,7 @@ __host__ __device__ inline SdWs sd_ws_layout(int B, int K, int C)
     w.counters_end = align_up(draw_counters + 4 * (size_t)B, 256);
     w.acc = w.counters_end;
     w.part = align_up(w.acc + M, 256);
-    w.rowstats = align_up(w.part + 16 * M * C, 256);
+    w.rowstats = align_up(w.part + 16 * M * S, 256);
     w.draw = draw_ws_layout(draw_counters, align_up(w.rowstats + 16 * M, 256), B, C);
     w.end = w.draw.end;
     return w;

@@ -144,16 +144,66 @@ __device__ __forceinline__ MS thread_ms(const uint4 (&raw)[kUnroll])
 }
 
 // ================================================================ sd_verify, stage 1
-// One CTA per (row, chunk): chunk statistics of the p row and the q row.  The CTA that
-// finishes a row last merges the chunks, runs the accept test for that position, and the
-// row that finishes a sequence last runs the first-rejection scan.
+// Lane-local online softmax statistics: folds kUnroll vectors into a running (max, sum of
+// exp(x - max)).  When the maximum grows the old sum is rescaled once per call.
+template <typename T>
+__device__ __forceinline__ void online_update(const uint4 (&raw)[kUnroll], float &m, float &s)
+{
+    constexpr int N = Vec<T>::N;
+    float g = Vec<T>::vmax(raw[0]);
+#pragma unroll
+    for (int j = 1; j < kUnroll; ++j) g = fmaxf(g, Vec<T>::vmax(raw[j]));
+    const float mn = fmaxf(m, g);
+    const float ref = (mn == neg_inf()) ? 0.f : mn;
+    const float off = -ref * kLog2e;
+    float acc[kUnroll];
+    acc[0] = s * ex2(fmaf(m, kLog2e, off));   // m = -inf: exp2(-inf) = 0
+#pragma unroll
+    for (int j = 1; j < kUnroll; ++j) acc[j] = 0.f;
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) {
+        float f[N];
+        Vec<T>::unpack(raw[j], f);
+#pragma unroll
+        for (int e = 0; e < N; ++e) acc[j] += ex2(fmaf(f[e], kLog2e, off));
+    }
+    m = mn;
+    s = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+}
+
+// The kUnroll vectors of one warp step: vector j of lane l starts at element
+// first + (j*32 + l)*N of the row (first may be negative or run past V at the row's ends).
+template <typename T>
+__device__ __forceinline__ void load_step(const T *__restrict__ row, int first, int V, int lane,
+                                          uint4 (&raw)[kUnroll])
+{
+    constexpr int N = Vec<T>::N;
+    constexpr int kStep = 32 * kUnroll * N;
+    if (first >= 0 && first + kStep <= V) {   // interior: aligned by construction
+        const uint4 *p = reinterpret_cast<const uint4 *>(row + first) + lane;
+#pragma unroll
+        for (int j = 0; j < kUnroll; ++j) raw[j] = ld_stream(p + j * 32);
+    } else {
+#pragma unroll
+        for (int j = 0; j < kUnroll; ++j) raw[j] = load_vec<T>(row, first + (j * 32 + lane) * N, V);
+    }
+}
+
+// One CTA per (row, segment): statistics of the p row and the q row over a segment of
+// kWarps*kStatIters warp steps (warp w takes steps w, w+8, ...; loads for a warp's next step
+// are issued before the current one is consumed).  The CTA that finishes a row last merges
+// the segments, runs the accept test for that position, and the row that finishes a
+// sequence last runs the first-rejection scan.
 template <typename T>
 __global__ void __launch_bounds__(kThreads) sd_row_stats_kernel(const SdParams prm)
 {
+    constexpr int N = Vec<T>::N;
+    constexpr int kStep = 32 * kUnroll * N;
+    constexpr int kSegment = kWarps * kStatIters * kStep;
     __shared__ float4 s_part[kWarps];
     __shared__ int s_last;
 
-    const int C = prm.chunks;
+    const int C = prm.chunks;            // segments per row
     const int64_t row = blockIdx.x / C;  // = b*K + k
     const int c = blockIdx.x % C;
     const int b = (int)(row / prm.K), k = (int)(row % prm.K);
@@ -161,16 +211,27 @@ __global__ void __launch_bounds__(kThreads) sd_row_stats_kernel(const SdParams p
 
     const T *prow = static_cast<const T *>(prm.p) + ((int64_t)b * prm.Kp + k) * prm.ldv;
     const T *qrow = static_cast<const T *>(prm.q) + row * prm.ldv;
-    const int pad_p = row_pad(prow), pad_q = row_pad(qrow);
+    // element index (may be negative) of this warp's first step in each row
+    const int first_p = c * kSegment + warp * kStep - row_pad(prow);
+    const int first_q = c * kSegment + warp * kStep - row_pad(qrow);
+    const int V = prm.V;
 
+    MS mp{neg_inf(), 0.f}, mq{neg_inf(), 0.f};
     uint4 rp[kUnroll], rq[kUnroll];
+    load_step<T>(prow, first_p, V, lane, rp);
+    load_step<T>(qrow, first_q, V, lane, rq);
 #pragma unroll
-    for (int j = 0; j < kUnroll; ++j) rp[j] = load_vec<T>(prow, vec_start<T>(c, j, tid, pad_p), prm.V);
-#pragma unroll
-    for (int j = 0; j < kUnroll; ++j) rq[j] = load_vec<T>(qrow, vec_start<T>(c, j, tid, pad_q), prm.V);
-
-    MS mp = warp_ms(thread_ms<T>(rp));
-    MS mq = warp_ms(thread_ms<T>(rq));
+    for (int it = 0; it < kStatIters; ++it) {
+        const int nxt = (it + 1) * kWarps * kStep;
+        const bool more = it + 1 < kStatIters && min(first_p, first_q) + nxt < V;   // warp-uniform
+        online_update<T>(rp, mp.m, mp.s);
+        if (more) load_step<T>(prow, first_p + nxt, V, lane, rp);
+        online_update<T>(rq, mq.m, mq.s);
+        if (more) load_step<T>(qrow, first_q + nxt, V, lane, rq);
+        if (!more) break;
+    }
+    mp = warp_ms(mp);
+    mq = warp_ms(mq);
     if (lane == 0) s_part[warp] = make_float4(mp.m, mp.s, mq.m, mq.s);
     __syncthreads();
     if (warp == 0) {
