@@ -194,8 +194,8 @@ int sd_verify_host(const void *p_logits, const void *q_logits, int64_t ldv, cons
  * until the process exits).  The call allocates and frees nothing.
  *
  * Limits: n <= SPR_STATIC_MAX_DRAWS and n * chunks <= SPR_STATIC_MAX_DRAW_CHUNKS, where
- * chunks = ceil((V + 7) / 8192) for bf16 and ceil((V + 3) / 4096) for f32 (16 for
- * V = 128256 bf16, so up to 1024 draws per call).  Larger requests return
+ * chunks = ceil((V + 7) / 32768) for bf16 and ceil((V + 3) / 16384) for f32 (4 for
+ * V = 128256 bf16; the draw count is then the binding limit: 1024 per call).  Larger requests return
  * SPR_ERR_WORKSPACE and launch nothing; split them or use replace_sample().
  *
  * First call on a device: looks up the device address of the array (the device must be

@@ -67,10 +67,10 @@ size_t spr_workspace_bytes(int op, int B, int K, int V, int d, int h, int dt)
         return verify_ws_bytes(B, K, h);
     case SPR_OP_REPLACE_SAMPLE:
         if (V <= 0) return 0;
-        return replace_ws_layout(B, chunks_per_row(V, dt)).end;
+        return replace_ws_layout(B, stat_segments_per_row(V, dt)).end;
     case SPR_OP_SD_VERIFY:
         if (K <= 0 || V <= 0 || (int64_t)B * K > 0x7fffffff) return 0;
-        return sd_ws_layout(B, K, stat_segments_per_row(V, dt), chunks_per_row(V, dt)).end;
+        return sd_ws_layout(B, K, stat_segments_per_row(V, dt)).end;
     default:
         return 0;
     }
@@ -151,7 +151,7 @@ int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, con
     if (!aligned(target_logits, elem_size(dt)) || !aligned(uniforms, 4) || !aligned(tokens, 4) ||
         (rows && !aligned(rows, 4)) || (first_reject && !aligned(first_reject, 4)))
         return SPR_ERR_INVALID_ARG;
-    const int C = chunks_per_row(V, dt);
+    const int C = stat_segments_per_row(V, dt);
     const DrawWs lay = replace_ws_layout(n, C);
     if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
     int rc = check_device();
@@ -200,8 +200,8 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
         (p_tok && !aligned(p_tok, 4)) || (q_tok && !aligned(q_tok, 4)) ||
         (residual_mass && !aligned(residual_mass, 4)))
         return SPR_ERR_INVALID_ARG;
-    const int C = chunks_per_row(V, dt), S = stat_segments_per_row(V, dt);
-    const SdWs lay = sd_ws_layout(B, K, S, C);
+    const int C = stat_segments_per_row(V, dt);
+    const SdWs lay = sd_ws_layout(B, K, C);
     if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
     int rc = check_device();
     if (rc != SPR_OK) return rc;
@@ -215,7 +215,7 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
     sp.V = V;
     sp.K = K;
     sp.Kp = Kp;
-    sp.chunks = S;
+    sp.chunks = C;
     sp.draft_tokens = draft_tokens;
     sp.uniforms = uniforms;
     sp.accepted_len = accepted_len;

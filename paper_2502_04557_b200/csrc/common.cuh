@@ -11,23 +11,18 @@ namespace spr {
 
 // ---------------------------------------------------------------- constants
 constexpr int kThreads = 256;           // CTA size of the vocabulary kernels
-constexpr int kUnroll = 4;              // 16-byte vectors per thread per chunk and row
+constexpr int kUnroll = 4;              // 16-byte vectors per lane per warp step
 constexpr int kWarps = kThreads / 32;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kHeaderBytes = 256;       // workspace header; word 0 is the sticky status
 
 __host__ __device__ constexpr int elem_size(int dt) { return dt == SPR_F32 ? 4 : 2; }
 __host__ __device__ constexpr int vec_elems(int dt) { return 16 / elem_size(dt); }
-// elements of one row that one CTA covers
-__host__ __device__ constexpr int chunk_elems(int dt) { return kThreads * kUnroll * vec_elems(dt); }
-// chunks per row; rows may start up to one vector minus one element past a 16-byte boundary
-__host__ __device__ inline int chunks_per_row(int V, int dt)
-{
-    return (V + vec_elems(dt) - 1 + chunk_elems(dt) - 1) / chunk_elems(dt);
-}
 
-// Row statistics (sd_verify stage 1): a warp consumes "steps" of 32 lanes x kUnroll vectors,
-// kStatIters of them per CTA, so one CTA covers a segment of kWarps*kStatIters steps of a row.
+// Vocabulary kernels: a warp consumes "steps" of 32 lanes x kUnroll vectors, kStatIters of
+// them per CTA, so one CTA covers a segment of kWarps*kStatIters = 32 steps of a row (32768
+// bf16 or 16384 fp32 elements).  Rows may start up to one vector minus one element past a
+// 16-byte boundary, hence the vec_elems - 1 below.
 constexpr int kStatIters = 4;
 __host__ __device__ constexpr int stat_step_elems(int dt) { return 32 * kUnroll * vec_elems(dt); }
 __host__ __device__ constexpr int stat_segment_elems(int dt) { return kWarps * kStatIters * stat_step_elems(dt); }
@@ -44,9 +39,9 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 // clears that zone on the stream before its first kernel, so a workspace may be shared by
 // calls of different ops and shapes.
 struct DrawWs {              // replace_sample, and the correction draw of sd_verify
-    size_t counters;         // int32 [n]      chunks finished per draw
-    size_t part_m;           // float [n*C]    chunk maximum (softmax draws)
-    size_t part_s;           // double [n*C]   chunk weight sum
+    size_t counters;         // int32 [n]      segments finished per draw
+    size_t part_m;           // float [n*C]    segment maximum (softmax draws)
+    size_t part_s;           // double [n*C]   segment weight sum
     size_t end;
 };
 __host__ __device__ inline DrawWs draw_ws_layout(size_t counters, size_t scratch, int n, int C)
@@ -65,7 +60,7 @@ __host__ __device__ inline DrawWs replace_ws_layout(int n, int C)
 }
 
 struct SdWs {
-    size_t row_counters;     // int32 [M]      chunks finished per row
+    size_t row_counters;     // int32 [M]      segments finished per row
     size_t seq_counters;     // int32 [B]      rows finished per sequence
     size_t counters_end;     // end of the zone cleared per call (includes the draw counters)
     size_t acc;              // uint8 [M]      0 reject, 1 accept, 2 invalid token
@@ -74,7 +69,7 @@ struct SdWs {
     DrawWs draw;             // correction draw, n = B
     size_t end;
 };
-__host__ __device__ inline SdWs sd_ws_layout(int B, int K, int S, int C)   // S stat segments, C draw chunks
+__host__ __device__ inline SdWs sd_ws_layout(int B, int K, int S)   // S segments per row
 {
     const size_t M = (size_t)B * K;
     SdWs w;
@@ -85,7 +80,7 @@ __host__ __device__ inline SdWs sd_ws_layout(int B, int K, int S, int C)   // S 
     w.acc = w.counters_end;
     w.part = align_up(w.acc + M, 256);
     w.rowstats = align_up(w.part + 16 * M * S, 256);
-    w.draw = draw_ws_layout(draw_counters, align_up(w.rowstats + 16 * M, 256), B, C);
+    w.draw = draw_ws_layout(draw_counters, align_up(w.rowstats + 16 * M, 256), B, S);
     w.end = w.draw.end;
     return w;
 }

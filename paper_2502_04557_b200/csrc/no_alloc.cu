@@ -62,8 +62,8 @@ extern "C" int replace_sample_static(const void *target_logits, int64_t ldv, int
         reinterpret_cast<uintptr_t>(tokens) % 4 || (rows && reinterpret_cast<uintptr_t>(rows) % 4) ||
         (first_reject && reinterpret_cast<uintptr_t>(first_reject) % 4))
         return SPR_ERR_INVALID_ARG;
-    const int C = chunks_per_row(V, dt);
-    // the built-in scratch has room for kMaxDraws tickets and kMaxDrawChunks chunk partials
+    const int C = stat_segments_per_row(V, dt);
+    // the built-in scratch has room for kMaxDraws tickets and kMaxDrawChunks segment partials
     if (n > kMaxDraws || (int64_t)n * C > kMaxDrawChunks) return SPR_ERR_WORKSPACE;
 
     int major = 0, dev = 0;

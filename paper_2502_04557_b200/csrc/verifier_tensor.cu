@@ -7,8 +7,8 @@
 //                              bias, ReLU and the W2 dot product in registers; A never
 //                              reaches HBM
 // One CTA computes a 128-token x BN-hidden-unit tile and writes one partial z per token.
-// The CTA that finishes last adds the partials in slice order, applies the sigmoid and the
-// threshold and runs the first-rejection scan (same tail as the SIMT kernel).
+// The CTA that completes a token tile adds its partials in slice order, applies the sigmoid
+// and the threshold and scans the sequences inside the tile (same tail as the SIMT kernel).
 //
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
 // warps 2..5 = epilogue (warp w reads TMEM lanes 32*(w%4) .. +31).
@@ -253,15 +253,27 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"((uint32_t)Cfg::kTmemCols)
                      : "memory");
     }
+    // Tickets: the CTA that completes a token tile (all slices written) turns its 128 partial
+    // sums into scores, accept bits and the scan of the sequences inside the tile; sequences
+    // cut by a tile boundary wait for the CTA that completes the last tile.
     if (tid == 0) {
         __threadfence();
-        const int total = (int)(gridDim.x * gridDim.y);
-        ctl->last = (atomicAdd(prm.counter, 1) == total - 1);
+        ctl->last = (atomicAdd(&prm.counter[1 + blockIdx.y], 1) == (int)gridDim.x - 1);
     }
     __syncthreads();
     if (!ctl->last) return;
     __threadfence();
-    finalise_scores(prm);
+    finalise_tile(prm, m0, min(m0 + kBM, M));
+    if (kBM % prm.K == 0) return;   // no sequence straddles a tile boundary
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        ctl->last = (atomicAdd(&prm.counter[0], 1) == (int)gridDim.y - 1);
+    }
+    __syncthreads();
+    if (!ctl->last) return;
+    __threadfence();
+    finalise_straddlers(prm, kBM);
 }
 
 // ---------------------------------------------------------------- host side

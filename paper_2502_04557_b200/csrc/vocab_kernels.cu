@@ -400,45 +400,115 @@ __device__ __forceinline__ void residual_weights(const uint4 &vp, const uint4 &v
         w[e] = fmaxf(0.f, ex2(fmaf(fp[e], kLog2e, -cp)) - ex2(fmaf(fq[e], kLog2e, -cq)));
 }
 
+static_assert(kWarps * kStatIters == 32, "a segment must hold exactly one warp's worth of steps");
+
 struct DrawSmem {
     float4 red[kWarps];
-    double scan[kWarps];
-    double base;
+    double step_sum[32];   // weight of each warp step of the rescanned segment
+    double base;           // weight before the crossing step
     double t_in;
     double total;
     float ref;
-    int chunk;
-    int first;
+    int segment;
+    int step;
     int lastpos;
     int token;
     int last;
 };
 
-// (chunk max, chunk sum) of softmax weights, or (0, chunk sum) of residual weights; the
-// result is valid in thread 0.
+__device__ __forceinline__ double warp_sum_f64(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+// inclusive prefix sum over the lanes of a warp, in lane order
+__device__ __forceinline__ double warp_scan_f64(double v, int lane)
+{
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += up;
+    }
+    return v;
+}
+
+// like load_step, for a row whose vectors need not be 16-byte aligned at `first`
 template <typename T>
-__device__ __forceinline__ MS block_chunk_stats(const Job<T> &job, int mode, int V, int c, DrawSmem &sm)
+__device__ __forceinline__ void load_step_any(const T *__restrict__ row, int first, int V, int lane,
+                                              uint4 (&raw)[kUnroll])
 {
     constexpr int N = Vec<T>::N;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int pad = row_pad(job.p_row);
-    uint4 rp[kUnroll];
+    if ((reinterpret_cast<uintptr_t>(row + first) & 15) == 0) {
+        load_step<T>(row, first, V, lane, raw);
+    } else {
 #pragma unroll
-    for (int j = 0; j < kUnroll; ++j) rp[j] = load_vec<T>(job.p_row, vec_start<T>(c, j, tid, pad), V);
-    MS v;
+        for (int j = 0; j < kUnroll; ++j) raw[j] = load_vec<T>(row, first + (j * 32 + lane) * N, V);
+    }
+}
+
+// lane-local sum of the residual weights of one warp step
+template <typename T>
+__device__ __forceinline__ float residual_step_sum(const uint4 (&rp)[kUnroll], const uint4 (&rq)[kUnroll],
+                                                   float cp, float cq)
+{
+    constexpr int N = Vec<T>::N;
+    float acc[kUnroll];
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) {
+        float w[N];
+        residual_weights<T>(rp[j], rq[j], cp, cq, w);
+        acc[j] = 0.f;
+#pragma unroll
+        for (int e = 0; e < N; ++e) acc[j] += w[e];
+    }
+    return (acc[0] + acc[1]) + (acc[2] + acc[3]);
+}
+
+// (segment max, segment sum) of softmax weights, or (0, segment sum) of residual weights over
+// segment c of the job's row(s); same step interleaving and prefetch as the row-statistics
+// kernel.  The result is valid in thread 0.
+template <typename T>
+__device__ __forceinline__ MS segment_stats(const Job<T> &job, int mode, int V, int c, DrawSmem &sm)
+{
+    constexpr int N = Vec<T>::N;
+    constexpr int kStep = 32 * kUnroll * N;
+    constexpr int kSegment = 32 * kStep;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int first = c * kSegment + warp * kStep - row_pad(job.p_row);
+    MS v{neg_inf(), 0.f};
+    uint4 rp[kUnroll];
+    load_step<T>(job.p_row, first, V, lane, rp);
     if (mode == MODE_SOFTMAX) {
-        v = warp_ms(thread_ms<T>(rp));
+#pragma unroll
+        for (int it = 0; it < kStatIters; ++it) {
+            const int nxt = (it + 1) * kWarps * kStep;
+            const bool more = it + 1 < kStatIters && first + nxt < V;
+            online_update<T>(rp, v.m, v.s);
+            if (!more) break;
+            load_step<T>(job.p_row, first + nxt, V, lane, rp);
+        }
+        v = warp_ms(v);
     } else {
         uint4 rq[kUnroll];
-#pragma unroll
-        for (int j = 0; j < kUnroll; ++j) rq[j] = load_vec<T>(job.q_row, vec_start<T>(c, j, tid, pad), V);
+        load_step_any<T>(job.q_row, first, V, lane, rq);
         float s = 0.f;
 #pragma unroll
-        for (int j = 0; j < kUnroll; ++j) {
-            float w[N];
-            residual_weights<T>(rp[j], rq[j], job.cp, job.cq, w);
+        for (int it = 0; it < kStatIters; ++it) {
+            const int nxt = (it + 1) * kWarps * kStep;
+            const bool more = it + 1 < kStatIters && first + nxt < V;
+            uint4 np[kUnroll], nq[kUnroll];
+            if (more) {
+                load_step<T>(job.p_row, first + nxt, V, lane, np);
+                load_step_any<T>(job.q_row, first + nxt, V, lane, nq);
+            }
+            s += residual_step_sum<T>(rp, rq, job.cp, job.cq);
+            if (!more) break;
 #pragma unroll
-            for (int e = 0; e < N; ++e) s += w[e];
+            for (int j = 0; j < kUnroll; ++j) {
+                rp[j] = np[j];
+                rq[j] = nq[j];
+            }
         }
         v.m = 0.f;
         v.s = warp_sum(s);
@@ -458,87 +528,129 @@ __device__ __forceinline__ MS block_chunk_stats(const Job<T> &job, int mode, int
     return v;
 }
 
-// Finds, inside chunk c, the first element whose running weight sum exceeds t_in (weights
-// taken relative to `ref` for softmax draws).  Falls back to the last positive-weight
-// element of the chunk when rounding leaves no crossing; -1 if the chunk has no weight.
+// weights of one vector of a step (softmax relative to `ref`, or residual)
 template <typename T>
-__device__ int block_locate(const Job<T> &job, int mode, int V, int c, double t_in, float ref,
-                            DrawSmem &sm)
+__device__ __forceinline__ void step_weights(const Job<T> &job, int mode, float off, const uint4 &vp,
+                                             const uint4 &vq, float (&w)[Vec<T>::N])
 {
     constexpr int N = Vec<T>::N;
+    if (mode == MODE_SOFTMAX) {
+        float f[N];
+        Vec<T>::unpack(vp, f);
+#pragma unroll
+        for (int e = 0; e < N; ++e) w[e] = ex2(fmaf(f[e], kLog2e, off));
+    } else {
+        residual_weights<T>(vp, vq, job.cp, job.cq, w);
+    }
+}
+
+// Finds, inside segment c, the first element whose running weight sum exceeds t_in (softmax
+// weights are taken relative to `ref`).  Three phases: per-step sums of the whole segment,
+// the step that holds the crossing (one warp scan), then the element inside that step (its
+// owner warp).  Falls back to the last positive-weight element of the segment when rounding
+// leaves no crossing; -1 if the segment has no weight.
+template <typename T>
+__device__ int segment_locate(const Job<T> &job, int mode, int V, int c, double t_in, float ref,
+                              DrawSmem &sm)
+{
+    constexpr int N = Vec<T>::N;
+    constexpr int kStep = 32 * kUnroll * N;
+    constexpr int kSegment = 32 * kStep;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int pad = row_pad(job.p_row);
+    const int first = c * kSegment + warp * kStep - row_pad(job.p_row);
     const float off = -ref * kLog2e;
     if (tid == 0) {
-        sm.first = INT_MAX;
         sm.lastpos = -1;
-        sm.base = 0.0;
         sm.token = -1;
+        sm.step = -1;
+        sm.base = 0.0;
     }
     __syncthreads();
-    for (int j = 0; j < kUnroll; ++j) {
-        const int i0 = vec_start<T>(c, j, tid, pad);
-        float w[N];
-        const uint4 vp = load_vec<T>(job.p_row, i0, V);
-        if (mode == MODE_SOFTMAX) {
-            float f[N];
-            Vec<T>::unpack(vp, f);
-#pragma unroll
-            for (int e = 0; e < N; ++e) w[e] = ex2(fmaf(f[e], kLog2e, off));
-        } else {
-            const uint4 vq = load_vec<T>(job.q_row, i0, V);
-            residual_weights<T>(vp, vq, job.cp, job.cq, w);
-        }
+    int lp = -1;
+    for (int it = 0; it < kStatIters; ++it) {
+        const int f0 = first + it * kWarps * kStep;
+        uint4 rp[kUnroll], rq[kUnroll] = {};
+        load_step<T>(job.p_row, f0, V, lane, rp);
+        if (mode == MODE_RESIDUAL) load_step_any<T>(job.q_row, f0, V, lane, rq);
         double ts = 0.0;
-        int lp = -1;
 #pragma unroll
-        for (int e = 0; e < N; ++e) {
-            ts += (double)w[e];
-            if (w[e] > 0.f) lp = i0 + e;
-        }
-        // inclusive scan of ts in thread order
-        double incl = ts;
+        for (int j = 0; j < kUnroll; ++j) {
+            float w[N];
+            step_weights<T>(job, mode, off, rp[j], rq[j], w);
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const double up = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += up;
-        }
-        if (lane == 31) sm.scan[warp] = incl;
-        __syncthreads();
-        double before = sm.base;
-        for (int ww = 0; ww < warp; ++ww) before += sm.scan[ww];
-        incl += before;
-        if (incl > t_in) atomicMin(&sm.first, tid);
-        if (lp >= 0) atomicMax(&sm.lastpos, lp);
-        __syncthreads();
-        if (sm.first != INT_MAX) {
-            if (tid == sm.first) {
-                double run = incl - ts;
-                int tok = -1;
-#pragma unroll
-                for (int e = 0; e < N; ++e) {
-                    run += (double)w[e];
-                    if (tok < 0 && run > t_in && w[e] > 0.f) tok = i0 + e;
-                }
-                sm.token = tok >= 0 ? tok : (lp >= 0 ? lp : sm.lastpos);
+            for (int e = 0; e < N; ++e) {
+                ts += (double)w[e];
+                if (w[e] > 0.f) lp = f0 + (j * 32 + lane) * N + e;
             }
-            __syncthreads();
-            return sm.token;
         }
-        if (tid == kThreads - 1) sm.base = incl;
-        __syncthreads();
+        ts = warp_sum_f64(ts);
+        if (lane == 0) sm.step_sum[it * kWarps + warp] = ts;
     }
-    return sm.lastpos;
+    lp = (int)__reduce_max_sync(0xffffffffu, lp);
+    if (lane == 0 && lp >= 0) atomicMax(&sm.lastpos, lp);
+    __syncthreads();
+    if (warp == 0) {
+        const double v = sm.step_sum[lane];
+        const double incl = warp_scan_f64(v, lane);
+        const unsigned cross = __ballot_sync(0xffffffffu, incl > t_in);
+        if (cross != 0u && lane == __ffs(cross) - 1) {
+            sm.step = lane;
+            sm.base = incl - v;
+        }
+    }
+    __syncthreads();
+    const int step = sm.step;
+    if (step < 0) return sm.lastpos;
+    if (warp == step % kWarps) {
+        const int f0 = first + (step / kWarps) * kWarps * kStep;
+        uint4 rp[kUnroll], rq[kUnroll] = {};
+        load_step<T>(job.p_row, f0, V, lane, rp);
+        if (mode == MODE_RESIDUAL) load_step_any<T>(job.q_row, f0, V, lane, rq);
+        double run = sm.base;
+        int tok = -1;
+#pragma unroll
+        for (int j = 0; j < kUnroll; ++j) {
+            float w[N];
+            step_weights<T>(job, mode, off, rp[j], rq[j], w);
+            double ts = 0.0;
+#pragma unroll
+            for (int e = 0; e < N; ++e) ts += (double)w[e];
+            const double incl = run + warp_scan_f64(ts, lane);
+            const unsigned cross = tok < 0 ? __ballot_sync(0xffffffffu, incl > t_in) : 0u;
+            if (tok < 0 && cross != 0u) {
+                const int owner = __ffs(cross) - 1;
+                int mine = -1;
+                if (lane == owner) {
+                    double r = incl - ts;
+                    int last_pos = -1;
+#pragma unroll
+                    for (int e = 0; e < N; ++e) {
+                        r += (double)w[e];
+                        if (w[e] > 0.f) last_pos = e;
+                        if (mine < 0 && r > t_in && w[e] > 0.f) mine = e;
+                    }
+                    if (mine < 0) mine = last_pos;   // rounding inside the vector
+                    if (mine >= 0) mine += f0 + (j * 32 + lane) * N;
+                }
+                tok = __shfl_sync(0xffffffffu, mine, owner);
+                if (tok < 0) tok = -2;   // crossing vector had no positive weight: use the fallback
+            }
+            run = __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (lane == 0) sm.token = tok >= 0 ? tok : sm.lastpos;
+    }
+    __syncthreads();
+    return sm.token;
 }
 
 template <typename T>
 __global__ void __launch_bounds__(kThreads) draw_kernel(const DrawParams prm)
 {
     __shared__ DrawSmem sm;
-    const int C = prm.chunks;
+    const int C = prm.chunks;   // segments per row
     const int i = blockIdx.x / C;
     const int c = blockIdx.x % C;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     Job<T> job = resolve_job<T>(prm, i);
     if (job.mode == MODE_NONE) {
@@ -552,7 +664,7 @@ __global__ void __launch_bounds__(kThreads) draw_kernel(const DrawParams prm)
     float *part_m = prm.part_m + (int64_t)i * C;
     double *part_s = prm.part_s + (int64_t)i * C;
 
-    const MS v = block_chunk_stats<T>(job, mode, prm.V, c, sm);
+    const MS v = segment_stats<T>(job, mode, prm.V, c, sm);
     if (tid == 0) {
         part_m[c] = v.m;
         part_s[c] = (double)v.s;
@@ -563,41 +675,57 @@ __global__ void __launch_bounds__(kThreads) draw_kernel(const DrawParams prm)
     if (!sm.last) return;
     __threadfence();
 
-    // ---- last CTA of this draw: total weight, crossing chunk, then the token inside it
+    // ---- last CTA of this draw: total weight and crossing segment (warp 0, segments in
+    //      order, 32 at a time), then the token inside that segment (whole CTA)
     for (int attempt = 0; attempt < 2; ++attempt) {
-        if (tid == 0) {
+        if (warp == 0) {
             float M = neg_inf();
-            for (int cc = 0; cc < C; ++cc) M = fmaxf(M, __ldcg(&part_m[cc]));
-            double total = 0.0;
-            for (int cc = 0; cc < C; ++cc) {
-                const double s = __ldcg(&part_s[cc]);
-                if (s > 0.0) total += s * exp((double)__ldcg(&part_m[cc]) - (double)M);
-            }
-            const double target = (double)job.u * total;
-            double prefix = 0.0, before = 0.0;
-            int chunk = -1, lastpos_chunk = -1;
-            for (int cc = 0; cc < C; ++cc) {
-                const double s = __ldcg(&part_s[cc]);
-                if (!(s > 0.0)) continue;
-                const double S = s * exp((double)__ldcg(&part_m[cc]) - (double)M);
-                if (S > 0.0) lastpos_chunk = cc;
-                if (prefix + S > target) {
-                    chunk = cc;
-                    before = prefix;
-                    break;
+            for (int cc = lane; cc < C; cc += 32) M = fmaxf(M, __ldcg(&part_m[cc]));
+            M = warp_max(M);
+            double carry = 0.0, before = 0.0;
+            int seg = -1, last_seg = -1;
+            for (int c0 = 0; c0 < C; c0 += 32) {      // pass 1: total
+                const int cc = c0 + lane;
+                double S = 0.0;
+                if (cc < C) {
+                    const double s = __ldcg(&part_s[cc]);
+                    if (s > 0.0) S = s * exp((double)__ldcg(&part_m[cc]) - (double)M);
                 }
-                prefix += S;
+                carry += __shfl_sync(0xffffffffu, warp_scan_f64(S, lane), 31);
             }
-            sm.total = total;
-            if (chunk >= 0) {
-                const float mc = __ldcg(&part_m[chunk]);
-                sm.chunk = chunk;
-                sm.ref = mc;
-                sm.t_in = (target - before) * exp((double)M - (double)mc);
-            } else {  // u*total not below total (rounding, or u >= 1): last positive weight
-                sm.chunk = lastpos_chunk;
-                sm.ref = lastpos_chunk >= 0 ? __ldcg(&part_m[lastpos_chunk]) : 0.f;
-                sm.t_in = __longlong_as_double(0x7ff0000000000000LL);
+            const double total = carry;
+            const double target = (double)job.u * total;
+            carry = 0.0;
+            for (int c0 = 0; c0 < C; c0 += 32) {      // pass 2: same sums, find the crossing
+                const int cc = c0 + lane;
+                double S = 0.0;
+                if (cc < C) {
+                    const double s = __ldcg(&part_s[cc]);
+                    if (s > 0.0) S = s * exp((double)__ldcg(&part_m[cc]) - (double)M);
+                }
+                const double incl = carry + warp_scan_f64(S, lane);
+                const unsigned pos = __ballot_sync(0xffffffffu, S > 0.0);
+                if (pos != 0u) last_seg = c0 + 31 - __clz(pos);
+                const unsigned cross = __ballot_sync(0xffffffffu, incl > target);
+                if (seg < 0 && cross != 0u) {
+                    const int owner = __ffs(cross) - 1;
+                    seg = c0 + owner;
+                    before = __shfl_sync(0xffffffffu, incl - S, owner);
+                }
+                carry = __shfl_sync(0xffffffffu, incl, 31);
+            }
+            if (lane == 0) {
+                sm.total = total;
+                if (seg >= 0) {
+                    const float mc = __ldcg(&part_m[seg]);
+                    sm.segment = seg;
+                    sm.ref = mc;
+                    sm.t_in = (target - before) * exp((double)M - (double)mc);
+                } else {  // u*total not below total (rounding, or u >= 1): last positive weight
+                    sm.segment = last_seg;
+                    sm.ref = last_seg >= 0 ? __ldcg(&part_m[last_seg]) : 0.f;
+                    sm.t_in = __longlong_as_double(0x7ff0000000000000LL);
+                }
             }
         }
         __syncthreads();
@@ -607,7 +735,7 @@ __global__ void __launch_bounds__(kThreads) draw_kernel(const DrawParams prm)
             // max(0, p - q) vanished: Eq. 1 is undefined, draw from p itself (one CTA, rare)
             mode = MODE_SOFTMAX;
             for (int cc = 0; cc < C; ++cc) {
-                const MS r = block_chunk_stats<T>(job, mode, prm.V, cc, sm);
+                const MS r = segment_stats<T>(job, mode, prm.V, cc, sm);
                 if (tid == 0) {
                     part_m[cc] = r.m;
                     part_s[cc] = (double)r.s;
@@ -620,15 +748,13 @@ __global__ void __launch_bounds__(kThreads) draw_kernel(const DrawParams prm)
         break;
     }
     int token = -1;
-    if (sm.chunk >= 0) {
-        const int chunk = sm.chunk;
+    if (sm.segment >= 0) {
+        const int seg = sm.segment;
         const double t_in = sm.t_in;
         const float ref = sm.ref;
-        token = block_locate<T>(job, mode, prm.V, chunk, t_in, ref, sm);
+        token = segment_locate<T>(job, mode, prm.V, seg, t_in, ref, sm);
     }
-    if (tid == 0) {
-        prm.tokens[i] = token;
-    }
+    if (tid == 0) prm.tokens[i] = token;
 }
 
 // ================================================================ host launchers

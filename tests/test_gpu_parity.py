@@ -424,7 +424,7 @@ def test_verifier_threshold_equality(spr):
 
 
 @pytest.mark.parametrize("B,K,d,h", [(4, 8, 64, 16), (40, 8, 256, 96), (130, 3, 136, 20), (32, 8, 768, 256),
-                                      (64, 1, 4096, 1024), (100, 16, 2048, 512)])
+                                      (64, 1, 4096, 1024), (100, 16, 2048, 512), (20, 33, 64, 16), (3, 200, 64, 16)])
 def test_verifier_tensor_core_path(spr, B, K, d, h):
     """tcgen05 kernel forced (PATH_TENSOR) on shapes with ragged M, h and d tails."""
     g = torch.Generator().manual_seed(B * 7 + K + d + h)
