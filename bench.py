@@ -36,7 +36,7 @@ NCU_TRAFFIC = {
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="llama3")
     ap.add_argument("--batch", type=int, default=None, help="sequences per GPU (default: the configuration's)")

@@ -497,18 +497,10 @@ __device__ __forceinline__ MS segment_stats(const Job<T> &job, int mode, int V, 
         for (int it = 0; it < kStatIters; ++it) {
             const int nxt = (it + 1) * kWarps * kStep;
             const bool more = it + 1 < kStatIters && first + nxt < V;
-            uint4 np[kUnroll], nq[kUnroll];
-            if (more) {
-                load_step<T>(job.p_row, first + nxt, V, lane, np);
-                load_step_any<T>(job.q_row, first + nxt, V, lane, nq);
-            }
             s += residual_step_sum<T>(rp, rq, job.cp, job.cq);
             if (!more) break;
-#pragma unroll
-            for (int j = 0; j < kUnroll; ++j) {
-                rp[j] = np[j];
-                rq[j] = nq[j];
-            }
+            load_step<T>(job.p_row, first + nxt, V, lane, rp);
+            load_step_any<T>(job.q_row, first + nxt, V, lane, rq);
         }
         v.m = 0.f;
         v.s = warp_sum(s);
@@ -644,7 +636,7 @@ __device__ int segment_locate(const Job<T> &job, int mode, int V, int c, double 
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kThreads) draw_kernel(const DrawParams prm)
+__global__ void __launch_bounds__(kThreads, 4) draw_kernel(const DrawParams prm)
 {
     __shared__ DrawSmem sm;
     const int C = prm.chunks;   // segments per row
