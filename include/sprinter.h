@@ -190,12 +190,12 @@ int sd_verify_host(const void *p_logits, const void *q_logits, int64_t ldv, cons
  * pool, a plugin whose host forbids cudaMalloc), or that runs where cudaMalloc would
  * stall everything (it synchronises the device).  They have nowhere to get a `ws` from.
  * Same operation, arguments and results as replace_sample(), but the scratch is a fixed
- * array inside the library image (about 200 KB on every GPU that loads the library, held
+ * array inside the library image (about 516 KB on every GPU that loads the library, held
  * until the process exits).  The call allocates and frees nothing.
  *
- * Limits: n <= SPR_STATIC_MAX_DRAWS and n * chunks <= SPR_STATIC_MAX_DRAW_CHUNKS, where
- * chunks = ceil((V + 7) / 32768) for bf16 and ceil((V + 3) / 16384) for f32 (4 for
- * V = 128256 bf16; the draw count is then the binding limit: 1024 per call).  Larger requests return
+ * Limits: n <= SPR_STATIC_MAX_DRAWS and n * steps <= SPR_STATIC_MAX_DRAW_STEPS, where
+ * steps = ceil((V + 7) / 1024) for bf16 and ceil((V + 3) / 512) for f32 (126 for
+ * V = 128256 bf16, so up to 520 draws per call; 1024 draws up to V = 65536 bf16).  Larger requests return
  * SPR_ERR_WORKSPACE and launch nothing; split them or use replace_sample().
  *
  * First call on a device: looks up the device address of the array (the device must be
@@ -208,7 +208,7 @@ int sd_verify_host(const void *p_logits, const void *q_logits, int64_t ldv, cons
  * back.
  */
 #define SPR_STATIC_MAX_DRAWS 1024
-#define SPR_STATIC_MAX_DRAW_CHUNKS 16384
+#define SPR_STATIC_MAX_DRAW_STEPS 65536
 int replace_sample_static(const void *target_logits, int64_t ldv, int V, int64_t R, const int32_t *rows,
                           const int32_t *first_reject, int K, int seq_stride, int n,
                           const float *uniforms, int dt, int32_t *tokens, void *cuda_stream);

@@ -351,7 +351,7 @@ def replace_sample_static(target_logits, V: int, uniforms, tokens, rows=None, fi
     """replace_sample on the library's built-in scratch: no workspace argument, and nothing is
     allocated here either - the caller passes the output tensor `tokens` (int32 [n]).  For
     code that must not allocate device memory around the call; limited to
-    n <= 1024 draws and n * chunks <= 16384 (see include/sprinter.h).  Calls that may overlap
+    n <= 1024 draws and n * steps <= 65536 (see include/sprinter.h).  Calls that may overlap
     on one GPU race on the shared scratch: keep them on one stream."""
     _dev(target_logits, name="target_logits")
     ldv = target_logits.shape[-1]

@@ -67,10 +67,10 @@ size_t spr_workspace_bytes(int op, int B, int K, int V, int d, int h, int dt)
         return verify_ws_bytes(B, K, h);
     case SPR_OP_REPLACE_SAMPLE:
         if (V <= 0) return 0;
-        return replace_ws_layout(B, stat_segments_per_row(V, dt)).end;
+        return replace_ws_layout(B, stat_steps_per_row(V, dt)).end;
     case SPR_OP_SD_VERIFY:
         if (K <= 0 || V <= 0 || (int64_t)B * K > 0x7fffffff) return 0;
-        return sd_ws_layout(B, K, stat_segments_per_row(V, dt)).end;
+        return sd_ws_layout(B, K, stat_segments_per_row(V, dt), stat_steps_per_row(V, dt)).end;
     default:
         return 0;
     }
@@ -151,8 +151,8 @@ int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, con
     if (!aligned(target_logits, elem_size(dt)) || !aligned(uniforms, 4) || !aligned(tokens, 4) ||
         (rows && !aligned(rows, 4)) || (first_reject && !aligned(first_reject, 4)))
         return SPR_ERR_INVALID_ARG;
-    const int C = stat_segments_per_row(V, dt);
-    const DrawWs lay = replace_ws_layout(n, C);
+    const int C = stat_segments_per_row(V, dt), T = stat_steps_per_row(V, dt);
+    const DrawWs lay = replace_ws_layout(n, T);
     if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
     int rc = check_device();
     if (rc != SPR_OK) return rc;
@@ -174,8 +174,8 @@ int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, con
     dp.tokens = tokens;
     dp.status = at<int>(ws, 0);
     dp.counters = at<int>(ws, lay.counters);
-    dp.part_m = at<float>(ws, lay.part_m);
-    dp.part_s = at<double>(ws, lay.part_s);
+    dp.steps = T;
+    dp.part = at<float2>(ws, lay.part);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaMemsetAsync(dp.counters, 0, sizeof(int) * (size_t)n, st);
     if (e == cudaSuccess) e = launch_draw(dp, n, dt, st);
@@ -200,8 +200,8 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
         (p_tok && !aligned(p_tok, 4)) || (q_tok && !aligned(q_tok, 4)) ||
         (residual_mass && !aligned(residual_mass, 4)))
         return SPR_ERR_INVALID_ARG;
-    const int C = stat_segments_per_row(V, dt);
-    const SdWs lay = sd_ws_layout(B, K, C);
+    const int C = stat_segments_per_row(V, dt), T = stat_steps_per_row(V, dt);
+    const SdWs lay = sd_ws_layout(B, K, C, T);
     if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
     int rc = check_device();
     if (rc != SPR_OK) return rc;
@@ -246,8 +246,8 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
     dp.residual_mass = residual_mass;
     dp.status = sp.status;
     dp.counters = at<int>(ws, lay.draw.counters);
-    dp.part_m = at<float>(ws, lay.draw.part_m);
-    dp.part_s = at<double>(ws, lay.draw.part_s);
+    dp.steps = T;
+    dp.part = at<float2>(ws, lay.draw.part);
 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaMemsetAsync(sp.row_counters, 0, lay.counters_end - lay.row_counters, st);

@@ -26,6 +26,10 @@ __host__ __device__ constexpr int vec_elems(int dt) { return 16 / elem_size(dt);
 constexpr int kStatIters = 4;
 __host__ __device__ constexpr int stat_step_elems(int dt) { return 32 * kUnroll * vec_elems(dt); }
 __host__ __device__ constexpr int stat_segment_elems(int dt) { return kWarps * kStatIters * stat_step_elems(dt); }
+__host__ __device__ inline int stat_steps_per_row(int V, int dt)
+{
+    return (V + vec_elems(dt) - 1 + stat_step_elems(dt) - 1) / stat_step_elems(dt);
+}
 __host__ __device__ inline int stat_segments_per_row(int V, int dt)
 {
     return (V + vec_elems(dt) - 1 + stat_segment_elems(dt) - 1) / stat_segment_elems(dt);
@@ -40,23 +44,21 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 // calls of different ops and shapes.
 struct DrawWs {              // replace_sample, and the correction draw of sd_verify
     size_t counters;         // int32 [n]      segments finished per draw
-    size_t part_m;           // float [n*C]    segment maximum (softmax draws)
-    size_t part_s;           // double [n*C]   segment weight sum
+    size_t part;             // float2 [n*T]   (max, weight) of every warp step
     size_t end;
 };
-__host__ __device__ inline DrawWs draw_ws_layout(size_t counters, size_t scratch, int n, int C)
+__host__ __device__ inline DrawWs draw_ws_layout(size_t counters, size_t scratch, int n, int T)
 {
     DrawWs w;
     w.counters = counters;
-    w.part_m = align_up(scratch, 256);
-    w.part_s = align_up(w.part_m + sizeof(float) * (size_t)n * C, 256);
-    w.end = align_up(w.part_s + sizeof(double) * (size_t)n * C, 256);
+    w.part = align_up(scratch, 256);
+    w.end = align_up(w.part + 8 * (size_t)n * T, 256);
     return w;
 }
 // replace_sample alone: counters [n] directly after the header
-__host__ __device__ inline DrawWs replace_ws_layout(int n, int C)
+__host__ __device__ inline DrawWs replace_ws_layout(int n, int T)
 {
-    return draw_ws_layout(kHeaderBytes, kHeaderBytes + align_up(sizeof(int32_t) * (size_t)n, 256), n, C);
+    return draw_ws_layout(kHeaderBytes, kHeaderBytes + align_up(sizeof(int32_t) * (size_t)n, 256), n, T);
 }
 
 struct SdWs {
@@ -69,7 +71,7 @@ struct SdWs {
     DrawWs draw;             // correction draw, n = B
     size_t end;
 };
-__host__ __device__ inline SdWs sd_ws_layout(int B, int K, int S)   // S segments per row
+__host__ __device__ inline SdWs sd_ws_layout(int B, int K, int S, int T)   // S segments, T steps per row
 {
     const size_t M = (size_t)B * K;
     SdWs w;
@@ -80,7 +82,7 @@ __host__ __device__ inline SdWs sd_ws_layout(int B, int K, int S)   // S segment
     w.acc = w.counters_end;
     w.part = align_up(w.acc + M, 256);
     w.rowstats = align_up(w.part + 16 * M * S, 256);
-    w.draw = draw_ws_layout(draw_counters, align_up(w.rowstats + 16 * M, 256), B, S);
+    w.draw = draw_ws_layout(draw_counters, align_up(w.rowstats + 16 * M, 256), B, T);
     w.end = w.draw.end;
     return w;
 }

@@ -33,7 +33,7 @@ struct DrawParams {
     const void *p;
     const void *q;
     int64_t ldv;
-    int V, chunks;
+    int V, chunks, steps;   // segments (CTAs) and warp steps per row
     // replace_sample
     int64_t R;
     const int32_t *rows;
@@ -49,8 +49,7 @@ struct DrawParams {
     // workspace
     int *status;
     int *counters;   // [n]
-    float *part_m;   // [n*chunks]
-    double *part_s;  // [n*chunks]
+    float2 *part;    // [n*steps] (max, weight) of every warp step
 };
 
 struct VerifyParams {

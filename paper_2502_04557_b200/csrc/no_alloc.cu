@@ -11,15 +11,13 @@ namespace {
 
 // Limits of the built-in scratch (see include/sprinter.h).
 constexpr int kMaxDraws = SPR_STATIC_MAX_DRAWS;
-constexpr int kMaxDrawChunks = SPR_STATIC_MAX_DRAW_CHUNKS;
+constexpr int kMaxDrawSteps = SPR_STATIC_MAX_DRAW_STEPS;
 constexpr size_t kOffCounters = kHeaderBytes;
-constexpr size_t kOffPartM = kOffCounters + sizeof(int32_t) * (size_t)kMaxDraws;
-constexpr size_t kOffPartS = kOffPartM + sizeof(float) * (size_t)kMaxDrawChunks;
-constexpr size_t kScratchBytes = kOffPartS + sizeof(double) * (size_t)kMaxDrawChunks;
-static_assert(kOffCounters % 256 == 0 && kOffPartM % 256 == 0 && kOffPartS % 256 == 0,
-              "scratch regions must stay 256-byte aligned");
+constexpr size_t kOffPart = kOffCounters + sizeof(int32_t) * (size_t)kMaxDraws;
+constexpr size_t kScratchBytes = kOffPart + sizeof(float2) * (size_t)kMaxDrawSteps;
+static_assert(kOffCounters % 256 == 0 && kOffPart % 256 == 0, "scratch regions must stay 256-byte aligned");
 
-// ~200 KB of device memory per GPU, held from library load until process exit.
+// ~516 KB of device memory per GPU, held from library load until process exit.
 static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
 
 // Device address of g_static_scratch per device ordinal.  In host code the array's name is
@@ -62,9 +60,9 @@ extern "C" int replace_sample_static(const void *target_logits, int64_t ldv, int
         reinterpret_cast<uintptr_t>(tokens) % 4 || (rows && reinterpret_cast<uintptr_t>(rows) % 4) ||
         (first_reject && reinterpret_cast<uintptr_t>(first_reject) % 4))
         return SPR_ERR_INVALID_ARG;
-    const int C = stat_segments_per_row(V, dt);
-    // the built-in scratch has room for kMaxDraws tickets and kMaxDrawChunks segment partials
-    if (n > kMaxDraws || (int64_t)n * C > kMaxDrawChunks) return SPR_ERR_WORKSPACE;
+    const int C = stat_segments_per_row(V, dt), T = stat_steps_per_row(V, dt);
+    // the built-in scratch has room for kMaxDraws tickets and kMaxDrawSteps step partials
+    if (n > kMaxDraws || (int64_t)n * T > kMaxDrawSteps) return SPR_ERR_WORKSPACE;
 
     int major = 0, dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -93,8 +91,8 @@ extern "C" int replace_sample_static(const void *target_logits, int64_t ldv, int
     dp.tokens = tokens;
     dp.status = reinterpret_cast<int *>(scratch);
     dp.counters = reinterpret_cast<int *>(scratch + kOffCounters);
-    dp.part_m = reinterpret_cast<float *>(scratch + kOffPartM);
-    dp.part_s = reinterpret_cast<double *>(scratch + kOffPartS);
+    dp.steps = T;
+    dp.part = reinterpret_cast<float2 *>(scratch + kOffPart);
 
     // The array keeps whatever the previous call left: the tickets must start at zero (the
     // partials are always written before they are read, and the status word is not reported).

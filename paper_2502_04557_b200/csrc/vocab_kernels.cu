@@ -400,28 +400,20 @@ __device__ __forceinline__ void residual_weights(const uint4 &vp, const uint4 &v
         w[e] = fmaxf(0.f, ex2(fmaf(fp[e], kLog2e, -cp)) - ex2(fmaf(fq[e], kLog2e, -cq)));
 }
 
-static_assert(kWarps * kStatIters == 32, "a segment must hold exactly one warp's worth of steps");
+constexpr int kCachedSteps = 512;   // step weights the last CTA of a draw keeps in shared memory
 
 struct DrawSmem {
-    float4 red[kWarps];
-    double step_sum[32];   // weight of each warp step of the rescanned segment
-    double base;           // weight before the crossing step
+    double weight[kCachedSteps];   // weight of each step, relative to the row maximum
+    double base;                   // weight before the crossing step
     double t_in;
     double total;
+    float row_max;
     float ref;
-    int segment;
     int step;
-    int lastpos;
     int token;
     int last;
 };
 
-__device__ __forceinline__ double warp_sum_f64(double v)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
 // inclusive prefix sum over the lanes of a warp, in lane order
 __device__ __forceinline__ double warp_scan_f64(double v, int lane)
 {
@@ -465,181 +457,126 @@ __device__ __forceinline__ float residual_step_sum(const uint4 (&rp)[kUnroll], c
     return (acc[0] + acc[1]) + (acc[2] + acc[3]);
 }
 
-// (segment max, segment sum) of softmax weights, or (0, segment sum) of residual weights over
-// segment c of the job's row(s); same step interleaving and prefetch as the row-statistics
-// kernel.  The result is valid in thread 0.
+// (max, sum of exp(x - max)) of one warp step of a softmax draw, in every lane
 template <typename T>
-__device__ __forceinline__ MS segment_stats(const Job<T> &job, int mode, int V, int c, DrawSmem &sm)
+__device__ __forceinline__ MS softmax_step(const uint4 (&raw)[kUnroll])
+{
+    const MS t = thread_ms<T>(raw);
+    MS r;
+    r.m = warp_max(t.m);
+    const float ref = (r.m == neg_inf()) ? 0.f : r.m;
+    r.s = warp_sum(t.s * ex2((t.m - ref) * kLog2e));
+    return r;
+}
+
+// Step partials (max, weight) of segment c of the job's row(s), written to part[step] for the
+// steps this CTA owns; same step interleaving and prefetch as the row-statistics kernel.
+// Residual draws store (0, sum of max(0, p - q)).
+template <typename T>
+__device__ __forceinline__ void segment_pass(const Job<T> &job, int mode, int V, int c, int steps,
+                                             float2 *__restrict__ part)
 {
     constexpr int N = Vec<T>::N;
     constexpr int kStep = 32 * kUnroll * N;
-    constexpr int kSegment = 32 * kStep;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int first = c * kSegment + warp * kStep - row_pad(job.p_row);
-    MS v{neg_inf(), 0.f};
-    uint4 rp[kUnroll];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int step0 = c * 32 + warp;                      // this warp's steps: step0 + it*kWarps
+    const int first = step0 * kStep - row_pad(job.p_row);
+    uint4 rp[kUnroll], rq[kUnroll];
+    if (step0 >= steps) return;
     load_step<T>(job.p_row, first, V, lane, rp);
-    if (mode == MODE_SOFTMAX) {
+    if (mode == MODE_RESIDUAL) load_step_any<T>(job.q_row, first, V, lane, rq);
 #pragma unroll
-        for (int it = 0; it < kStatIters; ++it) {
-            const int nxt = (it + 1) * kWarps * kStep;
-            const bool more = it + 1 < kStatIters && first + nxt < V;
-            online_update<T>(rp, v.m, v.s);
-            if (!more) break;
-            load_step<T>(job.p_row, first + nxt, V, lane, rp);
-        }
-        v = warp_ms(v);
-    } else {
-        uint4 rq[kUnroll];
-        load_step_any<T>(job.q_row, first, V, lane, rq);
-        float s = 0.f;
-#pragma unroll
-        for (int it = 0; it < kStatIters; ++it) {
-            const int nxt = (it + 1) * kWarps * kStep;
-            const bool more = it + 1 < kStatIters && first + nxt < V;
-            s += residual_step_sum<T>(rp, rq, job.cp, job.cq);
-            if (!more) break;
-            load_step<T>(job.p_row, first + nxt, V, lane, rp);
-            load_step_any<T>(job.q_row, first + nxt, V, lane, rq);
-        }
-        v.m = 0.f;
-        v.s = warp_sum(s);
-    }
-    __syncthreads();  // sm.red may still be read by the previous use
-    if (lane == 0) sm.red[warp] = make_float4(v.m, v.s, 0.f, 0.f);
-    __syncthreads();
-    if (warp == 0) {
-        const float4 r = lane < kWarps ? sm.red[lane] : make_float4(neg_inf(), 0.f, 0.f, 0.f);
+    for (int it = 0; it < kStatIters; ++it) {
+        const int step = step0 + it * kWarps;
+        const int nxt = (it + 1) * kWarps * kStep;
+        const bool more = it + 1 < kStatIters && step + kWarps < steps;
+        MS v;
         if (mode == MODE_SOFTMAX) {
-            v = warp_ms(MS{r.x, r.y});
+            uint4 cur[kUnroll];
+#pragma unroll
+            for (int j = 0; j < kUnroll; ++j) cur[j] = rp[j];
+            if (more) load_step<T>(job.p_row, first + nxt, V, lane, rp);   // in flight during the math
+            v = softmax_step<T>(cur);
         } else {
             v.m = 0.f;
-            v.s = warp_sum(lane < kWarps ? r.y : 0.f);
+            v.s = warp_sum(residual_step_sum<T>(rp, rq, job.cp, job.cq));
+            if (more) {
+                load_step<T>(job.p_row, first + nxt, V, lane, rp);
+                load_step_any<T>(job.q_row, first + nxt, V, lane, rq);
+            }
         }
+        if (lane == 0) part[step] = make_float2(v.m, v.s);
+        if (!more) break;
     }
-    return v;
+    __threadfence();
 }
 
-// weights of one vector of a step (softmax relative to `ref`, or residual)
+// Inside step `step` of the row, the first element whose running weight exceeds t_in (softmax
+// weights relative to `ref`); the last positive-weight element of the step if rounding
+// leaves no crossing, -1 if the step has no weight.  One warp; result in every lane.
 template <typename T>
-__device__ __forceinline__ void step_weights(const Job<T> &job, int mode, float off, const uint4 &vp,
-                                             const uint4 &vq, float (&w)[Vec<T>::N])
-{
-    constexpr int N = Vec<T>::N;
-    if (mode == MODE_SOFTMAX) {
-        float f[N];
-        Vec<T>::unpack(vp, f);
-#pragma unroll
-        for (int e = 0; e < N; ++e) w[e] = ex2(fmaf(f[e], kLog2e, off));
-    } else {
-        residual_weights<T>(vp, vq, job.cp, job.cq, w);
-    }
-}
-
-// Finds, inside segment c, the first element whose running weight sum exceeds t_in (softmax
-// weights are taken relative to `ref`).  Three phases: per-step sums of the whole segment,
-// the step that holds the crossing (one warp scan), then the element inside that step (its
-// owner warp).  Falls back to the last positive-weight element of the segment when rounding
-// leaves no crossing; -1 if the segment has no weight.
-template <typename T>
-__device__ int segment_locate(const Job<T> &job, int mode, int V, int c, double t_in, float ref,
-                              DrawSmem &sm)
+__device__ int step_locate(const Job<T> &job, int mode, int V, int step, double t_in, float ref)
 {
     constexpr int N = Vec<T>::N;
     constexpr int kStep = 32 * kUnroll * N;
-    constexpr int kSegment = 32 * kStep;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int first = c * kSegment + warp * kStep - row_pad(job.p_row);
+    const int lane = threadIdx.x & 31;
+    const int f0 = step * kStep - row_pad(job.p_row);
     const float off = -ref * kLog2e;
-    if (tid == 0) {
-        sm.lastpos = -1;
-        sm.token = -1;
-        sm.step = -1;
-        sm.base = 0.0;
-    }
-    __syncthreads();
-    int lp = -1;
-    for (int it = 0; it < kStatIters; ++it) {
-        const int f0 = first + it * kWarps * kStep;
-        uint4 rp[kUnroll], rq[kUnroll] = {};
-        load_step<T>(job.p_row, f0, V, lane, rp);
-        if (mode == MODE_RESIDUAL) load_step_any<T>(job.q_row, f0, V, lane, rq);
+    uint4 rp[kUnroll], rq[kUnroll] = {};
+    load_step<T>(job.p_row, f0, V, lane, rp);
+    if (mode == MODE_RESIDUAL) load_step_any<T>(job.q_row, f0, V, lane, rq);
+    double run = 0.0;
+    int tok = -1, lastpos = -1;
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) {
+        float w[N];
+        if (mode == MODE_SOFTMAX) {
+            float f[N];
+            Vec<T>::unpack(rp[j], f);
+#pragma unroll
+            for (int e = 0; e < N; ++e) w[e] = ex2(fmaf(f[e], kLog2e, off));
+        } else {
+            residual_weights<T>(rp[j], rq[j], job.cp, job.cq, w);
+        }
+        const int e0 = f0 + (j * 32 + lane) * N;
         double ts = 0.0;
 #pragma unroll
-        for (int j = 0; j < kUnroll; ++j) {
-            float w[N];
-            step_weights<T>(job, mode, off, rp[j], rq[j], w);
-#pragma unroll
-            for (int e = 0; e < N; ++e) {
-                ts += (double)w[e];
-                if (w[e] > 0.f) lp = f0 + (j * 32 + lane) * N + e;
-            }
+        for (int e = 0; e < N; ++e) {
+            ts += (double)w[e];
+            if (w[e] > 0.f) lastpos = e0 + e;
         }
-        ts = warp_sum_f64(ts);
-        if (lane == 0) sm.step_sum[it * kWarps + warp] = ts;
-    }
-    lp = (int)__reduce_max_sync(0xffffffffu, lp);
-    if (lane == 0 && lp >= 0) atomicMax(&sm.lastpos, lp);
-    __syncthreads();
-    if (warp == 0) {
-        const double v = sm.step_sum[lane];
-        const double incl = warp_scan_f64(v, lane);
+        const double incl = run + warp_scan_f64(ts, lane);
         const unsigned cross = __ballot_sync(0xffffffffu, incl > t_in);
-        if (cross != 0u && lane == __ffs(cross) - 1) {
-            sm.step = lane;
-            sm.base = incl - v;
-        }
-    }
-    __syncthreads();
-    const int step = sm.step;
-    if (step < 0) return sm.lastpos;
-    if (warp == step % kWarps) {
-        const int f0 = first + (step / kWarps) * kWarps * kStep;
-        uint4 rp[kUnroll], rq[kUnroll] = {};
-        load_step<T>(job.p_row, f0, V, lane, rp);
-        if (mode == MODE_RESIDUAL) load_step_any<T>(job.q_row, f0, V, lane, rq);
-        double run = sm.base;
-        int tok = -1;
+        if (tok < 0 && cross != 0u) {
+            const int owner = __ffs(cross) - 1;
+            int mine = -1;
+            if (lane == owner) {
+                double r = incl - ts;
+                int last_e = -1;
 #pragma unroll
-        for (int j = 0; j < kUnroll; ++j) {
-            float w[N];
-            step_weights<T>(job, mode, off, rp[j], rq[j], w);
-            double ts = 0.0;
-#pragma unroll
-            for (int e = 0; e < N; ++e) ts += (double)w[e];
-            const double incl = run + warp_scan_f64(ts, lane);
-            const unsigned cross = tok < 0 ? __ballot_sync(0xffffffffu, incl > t_in) : 0u;
-            if (tok < 0 && cross != 0u) {
-                const int owner = __ffs(cross) - 1;
-                int mine = -1;
-                if (lane == owner) {
-                    double r = incl - ts;
-                    int last_pos = -1;
-#pragma unroll
-                    for (int e = 0; e < N; ++e) {
-                        r += (double)w[e];
-                        if (w[e] > 0.f) last_pos = e;
-                        if (mine < 0 && r > t_in && w[e] > 0.f) mine = e;
-                    }
-                    if (mine < 0) mine = last_pos;   // rounding inside the vector
-                    if (mine >= 0) mine += f0 + (j * 32 + lane) * N;
+                for (int e = 0; e < N; ++e) {
+                    r += (double)w[e];
+                    if (w[e] > 0.f) last_e = e;
+                    if (mine < 0 && r > t_in && w[e] > 0.f) mine = e;
                 }
-                tok = __shfl_sync(0xffffffffu, mine, owner);
-                if (tok < 0) tok = -2;   // crossing vector had no positive weight: use the fallback
+                if (mine < 0) mine = last_e;       // rounding inside the vector
+                if (mine >= 0) mine += e0;
             }
-            run = __shfl_sync(0xffffffffu, incl, 31);
+            tok = __shfl_sync(0xffffffffu, mine, owner);
+            if (tok < 0) tok = -2;                 // no weight in the crossing vector: fall back
         }
-        if (lane == 0) sm.token = tok >= 0 ? tok : sm.lastpos;
+        run = __shfl_sync(0xffffffffu, incl, 31);
     }
-    __syncthreads();
-    return sm.token;
+    lastpos = (int)__reduce_max_sync(0xffffffffu, lastpos);
+    return tok >= 0 ? tok : lastpos;
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kThreads, 4) draw_kernel(const DrawParams prm)
+__global__ void __launch_bounds__(kThreads, 3) draw_kernel(const DrawParams prm)
 {
     __shared__ DrawSmem sm;
-    const int C = prm.chunks;   // segments per row
+    const int C = prm.chunks;   // segments (CTAs) per row
+    const int steps = prm.steps;
     const int i = blockIdx.x / C;
     const int c = blockIdx.x % C;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -653,13 +590,11 @@ __global__ void __launch_bounds__(kThreads, 4) draw_kernel(const DrawParams prm)
         return;
     }
     int mode = job.mode;
-    float *part_m = prm.part_m + (int64_t)i * C;
-    double *part_s = prm.part_s + (int64_t)i * C;
+    float2 *part = prm.part + (int64_t)i * steps;
 
-    const MS v = segment_stats<T>(job, mode, prm.V, c, sm);
+    segment_pass<T>(job, mode, prm.V, c, steps, part);
+    __syncthreads();
     if (tid == 0) {
-        part_m[c] = v.m;
-        part_s[c] = (double)v.s;
         __threadfence();
         sm.last = (atomicAdd(&prm.counters[i], 1) == C - 1);
     }
@@ -667,55 +602,63 @@ __global__ void __launch_bounds__(kThreads, 4) draw_kernel(const DrawParams prm)
     if (!sm.last) return;
     __threadfence();
 
-    // ---- last CTA of this draw: total weight and crossing segment (warp 0, segments in
-    //      order, 32 at a time), then the token inside that segment (whole CTA)
+    // ---- last CTA of this draw: warp 0 adds the step weights in step order, finds the step
+    //      where the running sum crosses u * total, and then the token inside that step
     for (int attempt = 0; attempt < 2; ++attempt) {
         if (warp == 0) {
             float M = neg_inf();
-            for (int cc = lane; cc < C; cc += 32) M = fmaxf(M, __ldcg(&part_m[cc]));
+            for (int t = lane; t < steps; t += 32) M = fmaxf(M, __ldcg(&part[t]).x);
             M = warp_max(M);
-            double carry = 0.0, before = 0.0;
-            int seg = -1, last_seg = -1;
-            for (int c0 = 0; c0 < C; c0 += 32) {      // pass 1: total
-                const int cc = c0 + lane;
+            double carry = 0.0;
+            for (int t0 = 0; t0 < steps; t0 += 32) {      // pass 1: weights and their total
+                const int t = t0 + lane;
                 double S = 0.0;
-                if (cc < C) {
-                    const double s = __ldcg(&part_s[cc]);
-                    if (s > 0.0) S = s * exp((double)__ldcg(&part_m[cc]) - (double)M);
+                if (t < steps) {
+                    const float2 ms = __ldcg(&part[t]);
+                    if (ms.y > 0.f) S = (double)ms.y * exp((double)ms.x - (double)M);
+                    if (t < kCachedSteps) sm.weight[t] = S;
                 }
                 carry += __shfl_sync(0xffffffffu, warp_scan_f64(S, lane), 31);
             }
             const double total = carry;
             const double target = (double)job.u * total;
+            __syncwarp();
             carry = 0.0;
-            for (int c0 = 0; c0 < C; c0 += 32) {      // pass 2: same sums, find the crossing
-                const int cc = c0 + lane;
+            double before = 0.0;
+            int hit = -1, last_pos = -1;
+            for (int t0 = 0; t0 < steps && hit < 0; t0 += 32) {   // pass 2: the crossing step
+                const int t = t0 + lane;
                 double S = 0.0;
-                if (cc < C) {
-                    const double s = __ldcg(&part_s[cc]);
-                    if (s > 0.0) S = s * exp((double)__ldcg(&part_m[cc]) - (double)M);
+                if (t < steps) {
+                    if (t < kCachedSteps) {
+                        S = sm.weight[t];
+                    } else {
+                        const float2 ms = __ldcg(&part[t]);
+                        if (ms.y > 0.f) S = (double)ms.y * exp((double)ms.x - (double)M);
+                    }
                 }
                 const double incl = carry + warp_scan_f64(S, lane);
                 const unsigned pos = __ballot_sync(0xffffffffu, S > 0.0);
-                if (pos != 0u) last_seg = c0 + 31 - __clz(pos);
+                if (pos != 0u) last_pos = t0 + 31 - __clz(pos);
                 const unsigned cross = __ballot_sync(0xffffffffu, incl > target);
-                if (seg < 0 && cross != 0u) {
+                if (cross != 0u) {
                     const int owner = __ffs(cross) - 1;
-                    seg = c0 + owner;
+                    hit = t0 + owner;
                     before = __shfl_sync(0xffffffffu, incl - S, owner);
                 }
                 carry = __shfl_sync(0xffffffffu, incl, 31);
             }
             if (lane == 0) {
                 sm.total = total;
-                if (seg >= 0) {
-                    const float mc = __ldcg(&part_m[seg]);
-                    sm.segment = seg;
+                sm.row_max = M;
+                if (hit >= 0) {
+                    const float mc = __ldcg(&part[hit]).x;
+                    sm.step = hit;
                     sm.ref = mc;
                     sm.t_in = (target - before) * exp((double)M - (double)mc);
                 } else {  // u*total not below total (rounding, or u >= 1): last positive weight
-                    sm.segment = last_seg;
-                    sm.ref = last_seg >= 0 ? __ldcg(&part_m[last_seg]) : 0.f;
+                    sm.step = last_pos;
+                    sm.ref = last_pos >= 0 ? __ldcg(&part[last_pos]).x : 0.f;
                     sm.t_in = __longlong_as_double(0x7ff0000000000000LL);
                 }
             }
@@ -726,27 +669,16 @@ __global__ void __launch_bounds__(kThreads, 4) draw_kernel(const DrawParams prm)
         if (mode == MODE_RESIDUAL && !(sm.total > 0.0)) {
             // max(0, p - q) vanished: Eq. 1 is undefined, draw from p itself (one CTA, rare)
             mode = MODE_SOFTMAX;
-            for (int cc = 0; cc < C; ++cc) {
-                const MS r = segment_stats<T>(job, mode, prm.V, cc, sm);
-                if (tid == 0) {
-                    part_m[cc] = r.m;
-                    part_s[cc] = (double)r.s;
-                }
-            }
-            __threadfence();
+            for (int cc = 0; cc < C; ++cc) segment_pass<T>(job, mode, prm.V, cc, steps, part);
             __syncthreads();
             continue;
         }
         break;
     }
+    if (warp != 0) return;
     int token = -1;
-    if (sm.segment >= 0) {
-        const int seg = sm.segment;
-        const double t_in = sm.t_in;
-        const float ref = sm.ref;
-        token = segment_locate<T>(job, mode, prm.V, seg, t_in, ref, sm);
-    }
-    if (tid == 0) prm.tokens[i] = token;
+    if (sm.step >= 0) token = step_locate<T>(job, mode, prm.V, sm.step, sm.t_in, sm.ref);
+    if (lane == 0) prm.tokens[i] = token;
 }
 
 // ================================================================ host launchers

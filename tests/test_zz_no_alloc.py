@@ -67,11 +67,11 @@ def test_static_scratch_rejects_oversized_requests():
     tok = torch.zeros(1025, dtype=torch.int32, device="cuda")
     rows = torch.zeros(1025, dtype=torch.int32, device="cuda")
     assert _call_static(L, tl, 64, u, tok, rows=rows) == 3          # SPR_ERR_WORKSPACE
-    # fewer draws, but too many segment partials: n * ceil(V / 16384) = 1000 * 19 > 16384
-    V = 300000
+    # fewer draws, but too many step partials: n * ceil(V / 512) = 600 * 254 > 65536
+    V = 130000
     big = torch.zeros((1, V), device="cuda")
-    u = torch.zeros(1000, device="cuda")
-    tok = torch.zeros(1000, dtype=torch.int32, device="cuda")
-    rows = torch.zeros(1000, dtype=torch.int32, device="cuda")
+    u = torch.zeros(600, device="cuda")
+    tok = torch.zeros(600, dtype=torch.int32, device="cuda")
+    rows = torch.zeros(600, dtype=torch.int32, device="cuda")
     assert _call_static(L, big, V, u, tok, rows=rows) == 3
     assert "workspace" in L.spr_status_string(3).decode()
