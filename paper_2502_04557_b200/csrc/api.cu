@@ -251,7 +251,8 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaMemsetAsync(sp.row_counters, 0, lay.counters_end - lay.row_counters, st);
-    if (e == cudaSuccess) e = launch_sd_verify(sp, dp, B, K, dt, st);
+    if (e == cudaSuccess) e = launch_sd_row_stats(sp, B, K, dt, st);
+    if (e == cudaSuccess) e = launch_draw(dp, B, dt, st);
     return e == cudaSuccess ? SPR_OK : cuda_fail(e);
 }
 

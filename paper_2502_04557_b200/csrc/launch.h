@@ -69,8 +69,7 @@ struct VerifyParams {
     int slices;
 };
 
-cudaError_t launch_sd_verify(const SdParams &sp, const DrawParams &dp, int B, int K, int dt,
-                             cudaStream_t st);
+cudaError_t launch_sd_row_stats(const SdParams &sp, int B, int K, int dt, cudaStream_t st);
 int report_cuda_error(cudaError_t e);  // records the text, returns SPR_ERR_CUDA
 void set_stage_events(cudaEvent_t before, cudaEvent_t after);
 cudaError_t launch_draw(const DrawParams &dp, int n, int dt, cudaStream_t st);

@@ -1,0 +1,174 @@
+// sd_verify, stage 1: softmax statistics of every (p, q) row pair, the min(1, p/q) accept test
+// and the first-rejection scan.  Streams each logits row from HBM exactly once in 16-byte
+// vectors; per-segment partial results go to the last CTA that finishes a row ("last block
+// done" tickets: nothing ever waits on another CTA).
+#include "vocab_common.cuh"
+
+namespace spr {
+
+// One CTA per (row, segment): statistics of the p row and the q row over a segment of
+// kWarps*kStatIters warp steps (warp w takes steps w, w+8, ...; loads for a warp's next step
+// are issued before the current one is consumed).  The CTA that finishes a row last merges
+// the segments, runs the accept test for that position, and the row that finishes a
+// sequence last runs the first-rejection scan.
+template <typename T>
+__global__ void __launch_bounds__(kThreads) sd_row_stats_kernel(const SdParams prm)
+{
+    constexpr int N = Vec<T>::N;
+    constexpr int kStep = 32 * kUnroll * N;
+    constexpr int kSegment = kWarps * kStatIters * kStep;
+    __shared__ float4 s_part[kWarps];
+    __shared__ int s_last;
+
+    const int C = prm.chunks;            // segments per row
+    const int64_t row = blockIdx.x / C;  // = b*K + k
+    const int c = blockIdx.x % C;
+    const int b = (int)(row / prm.K), k = (int)(row % prm.K);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    const T *prow = static_cast<const T *>(prm.p) + ((int64_t)b * prm.Kp + k) * prm.ldv;
+    const T *qrow = static_cast<const T *>(prm.q) + row * prm.ldv;
+    // element index (may be negative) of this warp's first step in each row
+    const int first_p = c * kSegment + warp * kStep - row_pad(prow);
+    const int first_q = c * kSegment + warp * kStep - row_pad(qrow);
+    const int V = prm.V;
+
+    MS mp{neg_inf(), 0.f}, mq{neg_inf(), 0.f};
+    uint4 rp[kUnroll], rq[kUnroll];
+    load_step<T>(prow, first_p, V, lane, rp);
+    load_step<T>(qrow, first_q, V, lane, rq);
+#pragma unroll
+    for (int it = 0; it < kStatIters; ++it) {
+        const int nxt = (it + 1) * kWarps * kStep;
+        const bool more = it + 1 < kStatIters && min(first_p, first_q) + nxt < V;   // warp-uniform
+        online_update<T>(rp, mp.m, mp.s);
+        if (more) load_step<T>(prow, first_p + nxt, V, lane, rp);
+        online_update<T>(rq, mq.m, mq.s);
+        if (more) load_step<T>(qrow, first_q + nxt, V, lane, rq);
+        if (!more) break;
+    }
+    mp = warp_ms(mp);
+    mq = warp_ms(mq);
+    if (lane == 0) s_part[warp] = make_float4(mp.m, mp.s, mq.m, mq.s);
+    __syncthreads();
+    if (warp == 0) {
+        float4 v = lane < kWarps ? s_part[lane] : make_float4(neg_inf(), 0.f, neg_inf(), 0.f);
+        mp = warp_ms(MS{v.x, v.y});
+        mq = warp_ms(MS{v.z, v.w});
+        if (lane == 0) {
+            prm.part[row * C + c] = make_float4(mp.m, mp.s, mq.m, mq.s);
+            __threadfence();
+            const int ticket = atomicAdd(&prm.row_counters[row], 1);
+            s_last = (ticket == C - 1);
+        }
+    }
+    __syncthreads();
+    if (!s_last || warp != 0) return;
+
+    // ---- this CTA saw the last chunk of the row: merge chunks in chunk order (warp 0)
+    __threadfence();
+    float m_p = neg_inf(), m_q = neg_inf();
+    for (int cc = lane; cc < C; cc += 32) {
+        const float4 v = __ldcg(&prm.part[row * C + cc]);
+        m_p = fmaxf(m_p, v.x);
+        m_q = fmaxf(m_q, v.z);
+    }
+    m_p = warp_max(m_p);
+    m_q = warp_max(m_q);
+    double z_p = 0.0, z_q = 0.0;
+    for (int c0 = 0; c0 < C; c0 += 32) {  // fixed order: chunk groups ascending, butterfly inside
+        const int cc = c0 + lane;
+        double a = 0.0, bq = 0.0;
+        if (cc < C) {
+            const float4 v = __ldcg(&prm.part[row * C + cc]);
+            a = v.y > 0.f ? (double)v.y * exp((double)v.x - (double)m_p) : 0.0;
+            bq = v.w > 0.f ? (double)v.w * exp((double)v.z - (double)m_q) : 0.0;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            a += __shfl_xor_sync(0xffffffffu, a, o);
+            bq += __shfl_xor_sync(0xffffffffu, bq, o);
+        }
+        z_p += a;
+        z_q += bq;
+    }
+    int last_row = 0;
+    if (lane == 0) {
+        const double lnz_p = log(z_p), lnz_q = log(z_q);
+        const int x = prm.draft_tokens[row];
+        unsigned char acc;
+        float P = -1.f, Q = -1.f;
+        if (x < 0 || x >= prm.V) {
+            raise_status(prm.status, SPR_ERR_BAD_TOKEN);
+            acc = 2;
+        } else {
+            float lpx, lqx;
+            if (sizeof(T) == 4) {
+                lpx = reinterpret_cast<const float *>(prow)[x];
+                lqx = reinterpret_cast<const float *>(qrow)[x];
+            } else {
+                lpx = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(prow)[x]);
+                lqx = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(qrow)[x]);
+            }
+            const double logP = (double)lpx - (double)m_p - lnz_p;
+            const double logQ = (double)lqx - (double)m_q - lnz_q;
+            const double ratio = exp(logP - logQ);
+            const double u = (double)prm.uniforms[(int64_t)b * (prm.K + 1) + k];
+            acc = (u <= fmin(1.0, ratio)) ? 1 : 0;
+            P = (float)exp(logP);
+            Q = (float)exp(logQ);
+        }
+        prm.acc[row] = acc;
+        if (prm.accept) prm.accept[row] = acc == 1 ? 1 : 0;
+        if (prm.p_tok) prm.p_tok[row] = P;
+        if (prm.q_tok) prm.q_tok[row] = Q;
+        prm.rowstats[row] = make_float4(m_p, (float)lnz_p, m_q, (float)lnz_q);
+        __threadfence();
+        last_row = (atomicAdd(&prm.seq_counters[b], 1) == prm.K - 1);
+    }
+    last_row = __shfl_sync(0xffffffffu, last_row, 0);
+    if (!last_row) return;
+
+    // ---- last row of the sequence: first rejection = lowest set bit of the reject ballot
+    __threadfence();
+    int first = prm.K;
+    bool bad = false;
+    for (int k0 = 0; k0 < prm.K; k0 += 32) {
+        const int kk = k0 + lane;
+        const unsigned v = kk < prm.K ? (unsigned)__ldcg(&prm.acc[(int64_t)b * prm.K + kk]) : 1u;
+        const unsigned rej = __ballot_sync(0xffffffffu, v != 1u);
+        bad |= __ballot_sync(0xffffffffu, v == 2u) != 0u;
+        if (rej != 0u && first == prm.K) first = k0 + __ffs(rej) - 1;
+    }
+    if (lane == 0) {
+        prm.accepted_len[b] = bad ? -1 : first;
+        if (bad && prm.accept)
+            for (int kk = 0; kk < prm.K; ++kk) prm.accept[(int64_t)b * prm.K + kk] = 0;
+    }
+}
+
+// Optional CUDA events recorded right before and after the row-statistics kernel (the
+// launch that moves almost all the bytes), so a caller can time it inside a longer step.
+static thread_local cudaEvent_t g_stage_before = nullptr, g_stage_after = nullptr;
+void set_stage_events(cudaEvent_t before, cudaEvent_t after)
+{
+    g_stage_before = before;
+    g_stage_after = after;
+}
+
+cudaError_t launch_sd_row_stats(const SdParams &sp, int B, int K, int dt, cudaStream_t st)
+{
+    const int64_t grid = (int64_t)B * K * sp.chunks;
+    if (grid > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    if (grid == 0) return cudaSuccess;
+    if (g_stage_before) cudaEventRecord(g_stage_before, st);
+    if (dt == SPR_F32)
+        sd_row_stats_kernel<float><<<(unsigned)grid, kThreads, 0, st>>>(sp);
+    else
+        sd_row_stats_kernel<__nv_bfloat16><<<(unsigned)grid, kThreads, 0, st>>>(sp);
+    const cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess && g_stage_after) cudaEventRecord(g_stage_after, st);
+    return e;
+}
+
+}  // namespace spr
