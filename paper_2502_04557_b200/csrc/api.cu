@@ -39,6 +39,9 @@ int check_device()
     return major == 10 ? SPR_OK : SPR_ERR_UNSUPPORTED;
 }
 
+// AUTO hands batches of at least this many tokens to the tensor-core verifier
+constexpr int kTensorMinTokens = 32;
+
 bool dtype_ok(int dt) { return dt == SPR_F32 || dt == SPR_BF16; }
 bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
@@ -129,7 +132,8 @@ int sprinter_verify(const void *hidden, const void *W1, const float *b1, const v
     if (ce != cudaSuccess) return cuda_fail(ce);
 
     if (path != SPR_VERIFIER_SIMT) {
-        const int tensor_rc = launch_verifier_tensor(vp, dt, st);  // < 0: shape not taken
+        const int min_tokens = path == SPR_VERIFIER_TENSOR ? 1 : kTensorMinTokens;
+        const int tensor_rc = launch_verifier_tensor(vp, dt, min_tokens, st);  // < 0: shape not taken
         if (tensor_rc == 0) return SPR_OK;
         if (tensor_rc > 0) return cuda_fail((cudaError_t)tensor_rc);
         if (path == SPR_VERIFIER_TENSOR) return SPR_ERR_UNSUPPORTED;

@@ -80,7 +80,8 @@ cudaError_t launch_verifier_simt(const VerifyParams &vp, int dt, cudaStream_t st
 
 // Tensor-core (tcgen05) verifier for bf16 MLPs.  Returns 0 when launched, a negative
 // value when it does not take this shape or dtype (nothing launched), or a positive
-// cudaError_t.  It sets the slice count itself.
-int launch_verifier_tensor(const VerifyParams &vp, int dt, cudaStream_t st);
+// cudaError_t.  It sets the slice count itself.  Batches of fewer than min_tokens tokens
+// are left to the SIMT kernel.
+int launch_verifier_tensor(const VerifyParams &vp, int dt, int min_tokens, cudaStream_t st);
 
 }  // namespace spr

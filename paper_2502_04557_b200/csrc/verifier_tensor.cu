@@ -16,6 +16,7 @@
 // SPR_ERR_TIMEOUT in the status word, all roles leave their loops, TMEM is released and
 // the CTA exits.
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 #include "launch.h"
@@ -29,6 +30,7 @@ constexpr int kBM = 128;        // tokens per tile (UMMA M)
 constexpr int kBK = 64;         // bf16 elements per k-block: one 128-byte swizzle row
 constexpr int kUmmaK = 16;      // K of one tcgen05.mma for 16-bit operands
 constexpr int kTcThreads = 192;
+constexpr int kMaxChains = 4;    // independent accumulators the k-blocks are dealt to
 constexpr uint32_t kSpinLimit = 1u << 24;   // polls of mbarrier.try_wait before giving up
 
 template <int BN>
@@ -37,7 +39,8 @@ struct TileCfg {
     static constexpr int kBytesA = kBM * kBK * 2;
     static constexpr int kBytesB = BN * kBK * 2;
     static constexpr int kStageBytes = kBytesA + kBytesB;
-    static constexpr int kTmemCols = BN < 32 ? 32 : BN;
+    // kMaxChains accumulators of BN columns each (see the MMA issuer)
+    static constexpr int kTmemCols = BN * kMaxChains < 32 ? 32 : BN * kMaxChains;
     // stages, slack to align them to 1024 bytes, control block
     static constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 + 3072;
 };
@@ -148,7 +151,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
 template <int BN>
 __global__ void __launch_bounds__(kTcThreads, 1)
 verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w,
-                        const VerifyParams prm)
+                        const VerifyParams prm, const int chains)
 {
     using Cfg = TileCfg<BN>;
     extern __shared__ unsigned char smem_raw[];
@@ -220,7 +223,10 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
                 for (int k = 0; k < kBK / kUmmaK; ++k) {
                     // next 16 elements along K: 32 bytes further inside the swizzle row
                     const uint64_t adv = (uint64_t)((k * kUmmaK * 2) >> 4);
-                    umma_bf16(tmem_acc, da + adv, db + adv, idesc, (kb | k) != 0 ? 1u : 0u);
+                    // k-block kb accumulates into chain kb % chains: consecutive MMAs do not
+                    // depend on each other, the chains are added up in the epilogue
+                    umma_bf16(tmem_acc + (uint32_t)((kb % chains) * BN), da + adv, db + adv, idesc,
+                              (kb >= chains || k != 0) ? 1u : 0u);
                 }
                 umma_commit(&ctl->empty[s]);       // stage is free once these MMAs have read it
             }
@@ -238,6 +244,12 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
             for (int c0 = 0; c0 < BN; c0 += 16) {
                 float v[16];
                 tmem_ld16(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
+                for (int c = 1; c < min(chains, num_kb); ++c) {
+                    float w[16];
+                    tmem_ld16(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * BN + c0), w);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] += w[j];
+                }
 #pragma unroll
                 for (int j = 0; j < 16; ++j) z = fmaf(ctl->w2[c0 + j], fmaxf(v[j] + ctl->b1[c0 + j], 0.f), z);
             }
@@ -327,16 +339,21 @@ int launch_bn(const CUtensorMap &mh, const CUtensorMap &mw, VerifyParams vp, int
     }
     vp.slices = (vp.h + BN - 1) / BN;
     dim3 grid((unsigned)vp.slices, (unsigned)tiles_m);
-    verifier_tcgen05_kernel<BN><<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(mh, mw, vp);
+    int chains = kMaxChains;
+    if (const char *env = getenv("SPR_VERIFIER_CHAINS")) {   // tuning aid
+        const int v = atoi(env);
+        if (v == 1 || v == 2 || v == 4) chains = v;
+    }
+    verifier_tcgen05_kernel<BN><<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(mh, mw, vp, chains);
     return (int)cudaGetLastError();
 }
 
 }  // namespace
 
-int launch_verifier_tensor(const VerifyParams &vp, int dt, cudaStream_t st)
+int launch_verifier_tensor(const VerifyParams &vp, int dt, int min_tokens, cudaStream_t st)
 {
     const int64_t M = (int64_t)vp.B * vp.K;
-    if (dt != SPR_BF16 || vp.h <= 0 || vp.d % 8 != 0 || M < 32) return -1;
+    if (dt != SPR_BF16 || vp.h <= 0 || vp.d % 8 != 0 || M < min_tokens) return -1;
     if ((reinterpret_cast<uintptr_t>(vp.hidden) & 15) || (reinterpret_cast<uintptr_t>(vp.W1) & 15)) return -1;
     const int tiles_m = (int)((M + kBM - 1) / kBM);
     if (tiles_m > 65535) return -1;
@@ -347,6 +364,11 @@ int launch_verifier_tensor(const VerifyParams &vp, int dt, cudaStream_t st)
             bn = cand;
             break;
         }
+    }
+    // tuning aid: SPR_VERIFIER_BN=16|32|64|128 overrides the slice width
+    if (const char *env = getenv("SPR_VERIFIER_BN")) {
+        const int v = atoi(env);
+        if (v == 16 || v == 32 || v == 64 || v == 128) bn = v;
     }
     CUtensorMap mh, mw;
     if (!make_map(&mh, vp.hidden, (int)M, vp.d, kBM)) return -1;
