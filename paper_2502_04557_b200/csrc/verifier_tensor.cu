@@ -27,18 +27,24 @@ namespace spr {
 namespace {
 
 constexpr int kBM = 128;        // tokens per tile (UMMA M)
-constexpr int kBK = 64;         // bf16 elements per k-block: one 128-byte swizzle row
+constexpr int kAtomK = 64;      // bf16 elements of one 128-byte swizzle row (one TMA box)
+constexpr int kAtoms = 2;       // swizzle atoms per pipeline stage
+constexpr int kBK = kAtomK * kAtoms;   // bf16 elements per k-block (pipeline stage)
 constexpr int kUmmaK = 16;      // K of one tcgen05.mma for 16-bit operands
 constexpr int kTcThreads = 192;
+constexpr int kMaxStages = 12;
 constexpr int kMaxChains = 4;    // independent accumulators the k-blocks are dealt to
 constexpr uint32_t kSpinLimit = 1u << 24;   // polls of mbarrier.try_wait before giving up
 
 template <int BN>
 struct TileCfg {
-    static constexpr int kStages = BN >= 128 ? 5 : 6;
     static constexpr int kBytesA = kBM * kBK * 2;
     static constexpr int kBytesB = BN * kBK * 2;
     static constexpr int kStageBytes = kBytesA + kBytesB;
+    // The k-loop is bound by the time a stage takes to come round again (MMA done -> commit ->
+    // producer -> TMA -> full, about 2 us), so throughput is stages / that time: use all the
+    // shared memory there is (one CTA per SM either way).
+    static constexpr int kStages = (220 * 1024) / kStageBytes < kMaxStages ? (220 * 1024) / kStageBytes : kMaxStages;
     // kMaxChains accumulators of BN columns each (see the MMA issuer)
     static constexpr int kTmemCols = BN * kMaxChains < 32 ? 32 : BN * kMaxChains;
     // stages, slack to align them to 1024 bytes, control block
@@ -46,8 +52,8 @@ struct TileCfg {
 };
 
 struct Control {                 // lives behind the stages in dynamic shared memory
-    uint64_t full[8];
-    uint64_t empty[8];
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
     uint64_t tmem_full;
     uint32_t tmem_base;
     int abort;
@@ -201,8 +207,11 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
                 unsigned char *a_dst = stages + (size_t)s * Cfg::kStageBytes;
                 unsigned char *b_dst = a_dst + Cfg::kBytesA;
                 mbar_expect_tx(&ctl->full[s], (uint32_t)Cfg::kStageBytes);
-                tma_load_2d(a_dst, &map_h, kb * kBK, m0, &ctl->full[s]);
-                tma_load_2d(b_dst, &map_w, kb * kBK, n0, &ctl->full[s]);
+#pragma unroll
+                for (int a = 0; a < kAtoms; ++a) {   // one box per 64-wide swizzle atom
+                    tma_load_2d(a_dst + a * (Cfg::kBytesA / kAtoms), &map_h, kb * kBK + a * kAtomK, m0, &ctl->full[s]);
+                    tma_load_2d(b_dst + a * (Cfg::kBytesB / kAtoms), &map_w, kb * kBK + a * kAtomK, n0, &ctl->full[s]);
+                }
             }
         }
     } else if (warp == 1) {
@@ -218,15 +227,19 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t a_addr = smem_u32(stages + (size_t)s * Cfg::kStageBytes);
                 const uint32_t b_addr = a_addr + Cfg::kBytesA;
-                const uint64_t da = umma_smem_desc(a_addr), db = umma_smem_desc(b_addr);
 #pragma unroll
-                for (int k = 0; k < kBK / kUmmaK; ++k) {
-                    // next 16 elements along K: 32 bytes further inside the swizzle row
-                    const uint64_t adv = (uint64_t)((k * kUmmaK * 2) >> 4);
-                    // k-block kb accumulates into chain kb % chains: consecutive MMAs do not
-                    // depend on each other, the chains are added up in the epilogue
-                    umma_bf16(tmem_acc + (uint32_t)((kb % chains) * BN), da + adv, db + adv, idesc,
-                              (kb >= chains || k != 0) ? 1u : 0u);
+                for (int a = 0; a < kAtoms; ++a) {
+                    const uint64_t da = umma_smem_desc(a_addr + a * (Cfg::kBytesA / kAtoms));
+                    const uint64_t db = umma_smem_desc(b_addr + a * (Cfg::kBytesB / kAtoms));
+#pragma unroll
+                    for (int k = 0; k < kAtomK / kUmmaK; ++k) {
+                        // next 16 elements along K: 32 bytes further inside the swizzle row.
+                        // k-block kb accumulates into chain kb % chains: consecutive k-blocks do
+                        // not depend on each other, the chains are added up in the epilogue
+                        const uint64_t adv = (uint64_t)((k * kUmmaK * 2) >> 4);
+                        umma_bf16(tmem_acc + (uint32_t)((kb % chains) * BN), da + adv, db + adv, idesc,
+                                  (kb >= chains || (a | k) != 0) ? 1u : 0u);
+                    }
                 }
                 umma_commit(&ctl->empty[s]);       // stage is free once these MMAs have read it
             }
@@ -317,7 +330,7 @@ bool make_map(CUtensorMap *map, const void *base, int rows, int cols, int box_ro
     if (!fn) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
+    const cuuint32_t box[2] = {(cuuint32_t)kAtomK, (cuuint32_t)box_rows};
     const cuuint32_t elem[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, elem,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
