@@ -40,7 +40,7 @@ int check_device()
 }
 
 // AUTO hands batches of at least this many tokens to the tensor-core verifier
-constexpr int kTensorMinTokens = 32;
+constexpr int kTensorMinTokens = 4;
 
 bool dtype_ok(int dt) { return dt == SPR_F32 || dt == SPR_BF16; }
 bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
@@ -54,7 +54,7 @@ T *at(void *ws, size_t off)
 size_t verify_ws_bytes(int B, int K, int h)
 {
     const int M = B * K;
-    return verify_ws_layout(M, verifier_simt_slices(h), (M + 127) / 128).end;
+    return verify_ws_layout(M, verifier_simt_slices(h), (M + 63) / 64).end;
 }
 
 }  // namespace
@@ -125,7 +125,7 @@ int sprinter_verify(const void *hidden, const void *W1, const float *b1, const v
     vp.accept = accept;
     vp.first_reject = first_reject;
     vp.status = at<int>(ws, 0);
-    const VerifyWs lay = verify_ws_layout(M, verifier_simt_slices(h), (M + 127) / 128);
+    const VerifyWs lay = verify_ws_layout(M, verifier_simt_slices(h), (M + 63) / 64);
     vp.counter = at<int>(ws, lay.counter);
     vp.part_z = at<float>(ws, lay.part_z);
     cudaError_t ce = cudaMemsetAsync(vp.counter, 0, lay.counters_end - lay.counter, st);

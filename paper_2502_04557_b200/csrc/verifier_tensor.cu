@@ -6,7 +6,8 @@
 //                              lane), reads its accumulator row with tcgen05.ld and folds
 //                              bias, ReLU and the W2 dot product in registers; A never
 //                              reaches HBM
-// One CTA computes a 128-token x BN-hidden-unit tile and writes one partial z per token.
+// One CTA computes a BM-token x BN-hidden-unit tile (BM, BN in {64, 128}) and writes one
+// partial z per token.
 // The CTA that completes a token tile adds its partials in slice order, applies the sigmoid
 // and the threshold and scans the sequences inside the tile (same tail as the SIMT kernel).
 //
@@ -26,27 +27,24 @@ namespace spr {
 
 namespace {
 
-constexpr int kBM = 128;        // tokens per tile (UMMA M)
 constexpr int kAtomK = 64;      // bf16 elements of one 128-byte swizzle row (one TMA box)
 constexpr int kAtoms = 2;       // swizzle atoms per pipeline stage
 constexpr int kBK = kAtomK * kAtoms;   // bf16 elements per k-block (pipeline stage)
 constexpr int kUmmaK = 16;      // K of one tcgen05.mma for 16-bit operands
 constexpr int kTcThreads = 192;
 constexpr int kMaxStages = 12;
-constexpr int kMaxChains = 4;    // independent accumulators the k-blocks are dealt to
 constexpr uint32_t kSpinLimit = 1u << 24;   // polls of mbarrier.try_wait before giving up
 
-template <int BN>
+template <int BM, int BN>
 struct TileCfg {
-    static constexpr int kBytesA = kBM * kBK * 2;
+    static constexpr int kBytesA = BM * kBK * 2;
     static constexpr int kBytesB = BN * kBK * 2;
     static constexpr int kStageBytes = kBytesA + kBytesB;
     // The k-loop is bound by the time a stage takes to come round again (MMA done -> commit ->
     // producer -> TMA -> full, about 2 us), so throughput is stages / that time: use all the
     // shared memory there is (one CTA per SM either way).
     static constexpr int kStages = (220 * 1024) / kStageBytes < kMaxStages ? (220 * 1024) / kStageBytes : kMaxStages;
-    // kMaxChains accumulators of BN columns each (see the MMA issuer)
-    static constexpr int kTmemCols = BN * kMaxChains < 32 ? 32 : BN * kMaxChains;
+    static constexpr int kTmemCols = BN < 32 ? 32 : BN;
     // stages, slack to align them to 1024 bytes, control block
     static constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 + 3072;
 };
@@ -58,8 +56,8 @@ struct Control {                 // lives behind the stages in dynamic shared me
     uint32_t tmem_base;
     int abort;
     int last;
-    float b1[256];
-    float w2[256];
+    float b1[128];
+    float w2[128];
 };
 static_assert(sizeof(Control) <= 3072, "control block must fit its reservation");
 
@@ -120,11 +118,11 @@ __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr)
     return d;
 }
 
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = BN.
-template <int BN>
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = BM, N = BN.
+template <int BM, int BN>
 __device__ __forceinline__ constexpr uint32_t umma_instr_desc()
 {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 }
 
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc)
@@ -154,12 +152,12 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-template <int BN>
+template <int BM, int BN>
 __global__ void __launch_bounds__(kTcThreads, 1)
 verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w,
-                        const VerifyParams prm, const int chains)
+                        const VerifyParams prm)
 {
-    using Cfg = TileCfg<BN>;
+    using Cfg = TileCfg<BM, BN>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *stages = reinterpret_cast<unsigned char *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -168,7 +166,7 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int M = prm.B * prm.K;
     const int n0 = blockIdx.x * BN;      // first hidden unit of this slice
-    const int m0 = blockIdx.y * kBM;     // first token of this tile
+    const int m0 = blockIdx.y * BM;      // first token of this tile
     const int num_kb = (prm.d + kBK - 1) / kBK;
 
     if (tid == 0) {
@@ -217,7 +215,7 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
     } else if (warp == 1) {
         // ---------------- MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_instr_desc<BN>();
+            constexpr uint32_t idesc = umma_instr_desc<BM, BN>();
             bool ok = true;
             for (int kb = 0; kb < num_kb && ok; ++kb) {
                 const int s = kb % Cfg::kStages;
@@ -233,12 +231,9 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
                     const uint64_t db = umma_smem_desc(b_addr + a * (Cfg::kBytesB / kAtoms));
 #pragma unroll
                     for (int k = 0; k < kAtomK / kUmmaK; ++k) {
-                        // next 16 elements along K: 32 bytes further inside the swizzle row.
-                        // k-block kb accumulates into chain kb % chains: consecutive k-blocks do
-                        // not depend on each other, the chains are added up in the epilogue
+                        // next 16 elements along K: 32 bytes further inside the swizzle row
                         const uint64_t adv = (uint64_t)((k * kUmmaK * 2) >> 4);
-                        umma_bf16(tmem_acc + (uint32_t)((kb % chains) * BN), da + adv, db + adv, idesc,
-                                  (kb >= chains || (a | k) != 0) ? 1u : 0u);
+                        umma_bf16(tmem_acc, da + adv, db + adv, idesc, (kb | a | k) != 0 ? 1u : 0u);
                     }
                 }
                 umma_commit(&ctl->empty[s]);       // stage is free once these MMAs have read it
@@ -247,8 +242,11 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
         }
     } else {
         // ---------------- epilogue: thread = token, TMEM lane = 32*(warp%4) + lane
+        // BM = 128: accumulator row r lives in TMEM lane r.  BM = 64: the 64 rows use lanes
+        // 0-15 of each 32-lane quarter (row r in lane 32*(r/16) + r%16).
         const int quarter = warp & 3;
-        const int row = m0 + quarter * 32 + lane;
+        const bool has_row = BM == 128 || lane < 16;
+        const int row = m0 + (BM == 128 ? quarter * 32 + lane : quarter * 16 + lane);
         const bool ok = __all_sync(0xffffffffu, mbar_wait(&ctl->tmem_full, 0, ctl, prm.status));
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (ok) {
@@ -257,16 +255,10 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
             for (int c0 = 0; c0 < BN; c0 += 16) {
                 float v[16];
                 tmem_ld16(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
-                for (int c = 1; c < min(chains, num_kb); ++c) {
-                    float w[16];
-                    tmem_ld16(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * BN + c0), w);
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] += w[j];
-                }
 #pragma unroll
                 for (int j = 0; j < 16; ++j) z = fmaf(ctl->w2[c0 + j], fmaxf(v[j] + ctl->b1[c0 + j], 0.f), z);
             }
-            if (row < M) prm.part_z[(int64_t)blockIdx.x * M + row] = z;
+            if (has_row && row < M) prm.part_z[(int64_t)blockIdx.x * M + row] = z;
         }
     }
 
@@ -288,8 +280,8 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
     __syncthreads();
     if (!ctl->last) return;
     __threadfence();
-    finalise_tile(prm, m0, min(m0 + kBM, M));
-    if (kBM % prm.K == 0) return;   // no sequence straddles a tile boundary
+    finalise_tile(prm, m0, min(m0 + BM, M));
+    if (BM % prm.K == 0) return;   // no sequence straddles a tile boundary
     __syncthreads();
     if (tid == 0) {
         __threadfence();
@@ -298,7 +290,7 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
     __syncthreads();
     if (!ctl->last) return;
     __threadfence();
-    finalise_straddlers(prm, kBM);
+    finalise_straddlers(prm, BM);
 }
 
 // ---------------------------------------------------------------- host side
@@ -337,27 +329,22 @@ bool make_map(CUtensorMap *map, const void *base, int rows, int cols, int box_ro
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN>
-int launch_bn(const CUtensorMap &mh, const CUtensorMap &mw, VerifyParams vp, int tiles_m, cudaStream_t st)
+template <int BM, int BN>
+int launch_tile(const CUtensorMap &mh, const CUtensorMap &mw, VerifyParams vp, int tiles_m, cudaStream_t st)
 {
-    using Cfg = TileCfg<BN>;
+    using Cfg = TileCfg<BM, BN>;
     static bool attr_set[64];
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(verifier_tcgen05_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(verifier_tcgen05_kernel<BM, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)Cfg::kSmemBytes);
         if (e != cudaSuccess) return (int)e;
         attr_set[dev] = true;
     }
     vp.slices = (vp.h + BN - 1) / BN;
     dim3 grid((unsigned)vp.slices, (unsigned)tiles_m);
-    int chains = kMaxChains;
-    if (const char *env = getenv("SPR_VERIFIER_CHAINS")) {   // tuning aid
-        const int v = atoi(env);
-        if (v == 1 || v == 2 || v == 4) chains = v;
-    }
-    verifier_tcgen05_kernel<BN><<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(mh, mw, vp, chains);
+    verifier_tcgen05_kernel<BM, BN><<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(mh, mw, vp);
     return (int)cudaGetLastError();
 }
 
@@ -368,30 +355,44 @@ int launch_verifier_tensor(const VerifyParams &vp, int dt, int min_tokens, cudaS
     const int64_t M = (int64_t)vp.B * vp.K;
     if (dt != SPR_BF16 || vp.h <= 0 || vp.d % 8 != 0 || M < min_tokens) return -1;
     if ((reinterpret_cast<uintptr_t>(vp.hidden) & 15) || (reinterpret_cast<uintptr_t>(vp.W1) & 15)) return -1;
-    const int tiles_m = (int)((M + kBM - 1) / kBM);
-    if (tiles_m > 65535) return -1;
-    // widest slice that still gives the GPU enough CTAs
-    int bn = 16;
-    for (int cand : {128, 64, 32}) {
-        if ((int64_t)tiles_m * ((vp.h + cand - 1) / cand) >= 96) {
-            bn = cand;
+    // Measured on B200: a CTA's k-loop costs about the same per tcgen05.mma (140-250 cycles)
+    // whatever the tile shape up to 128 x 128, so time is set by the d/16 instructions each CTA
+    // issues in a row and by how many CTAs run at once.  Take the largest of the four tile
+    // shapes that still gives the GPU about a wave of CTAs; 64 x 64 if none does, 128 x 128
+    // once even that exceeds a wave.
+    auto ctas = [&](int m, int n) { return ((M + m - 1) / m) * (int64_t)((vp.h + n - 1) / n); };
+    static const int kShapes[4][2] = {{128, 128}, {64, 128}, {128, 64}, {64, 64}};
+    int bm = 64, bn = 64;
+    for (const auto &sh : kShapes) {
+        if (ctas(sh[0], sh[1]) >= 96) {
+            bm = sh[0];
+            bn = sh[1];
             break;
         }
     }
-    // tuning aid: SPR_VERIFIER_BN=16|32|64|128 overrides the slice width
+    // tuning aids: SPR_VERIFIER_BM=64|128, SPR_VERIFIER_BN=64|128
+    if (const char *env = getenv("SPR_VERIFIER_BM")) {
+        const int v = atoi(env);
+        if (v == 64 || v == 128) bm = v;
+    }
     if (const char *env = getenv("SPR_VERIFIER_BN")) {
         const int v = atoi(env);
-        if (v == 16 || v == 32 || v == 64 || v == 128) bn = v;
+        if (v == 64 || v == 128) bn = v;
     }
+    const int64_t tiles64 = (M + bm - 1) / bm;
+    if (tiles64 > 65535) return -1;
+    const int tiles_m = (int)tiles64;
     CUtensorMap mh, mw;
-    if (!make_map(&mh, vp.hidden, (int)M, vp.d, kBM)) return -1;
+    if (!make_map(&mh, vp.hidden, (int)M, vp.d, bm)) return -1;
     if (!make_map(&mw, vp.W1, vp.h, vp.d, bn)) return -1;
-    switch (bn) {
-    case 128: return launch_bn<128>(mh, mw, vp, tiles_m, st);
-    case 64: return launch_bn<64>(mh, mw, vp, tiles_m, st);
-    case 32: return launch_bn<32>(mh, mw, vp, tiles_m, st);
-    default: return launch_bn<16>(mh, mw, vp, tiles_m, st);
-    }
+#define SPR_TILE(BM_, BN_) \
+    if (bm == BM_ && bn == BN_) return launch_tile<BM_, BN_>(mh, mw, vp, tiles_m, st)
+    SPR_TILE(64, 64);
+    SPR_TILE(64, 128);
+    SPR_TILE(128, 64);
+    SPR_TILE(128, 128);
+#undef SPR_TILE
+    return -1;
 }
 
 }  // namespace spr
