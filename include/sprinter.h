@@ -56,7 +56,12 @@ typedef enum {
 
 typedef enum { SPR_F32 = 0, SPR_BF16 = 1 } spr_dtype;
 
-typedef enum { SPR_OP_SPRINTER_VERIFY = 0, SPR_OP_REPLACE_SAMPLE = 1, SPR_OP_SD_VERIFY = 2 } spr_op;
+typedef enum {
+    SPR_OP_SPRINTER_VERIFY = 0,
+    SPR_OP_REPLACE_SAMPLE = 1,
+    SPR_OP_SD_VERIFY = 2,
+    SPR_OP_SPRINTER_STEP = 3
+} spr_op;
 
 /* Which verifier kernel sprinter_verify() uses.  AUTO picks the tensor-core
  * kernel for bf16 MLPs whose shapes it supports and the SIMT kernel otherwise. */
@@ -64,8 +69,9 @@ typedef enum { SPR_VERIFIER_AUTO = 0, SPR_VERIFIER_SIMT = 1, SPR_VERIFIER_TENSOR
 
 /* Bytes of device scratch one call of `op` needs.  For SPR_OP_REPLACE_SAMPLE,
  * B is the number of draws n and K, d, h are ignored; for SPR_OP_SD_VERIFY d
- * and h are ignored; for SPR_OP_SPRINTER_VERIFY V is ignored.  Returns 0 for
- * invalid arguments.  A workspace sized for the largest op serves all three. */
+ * and h are ignored; for SPR_OP_SPRINTER_VERIFY V is ignored; SPR_OP_SPRINTER_STEP
+ * uses all of them.  Returns 0 for invalid arguments.  A workspace sized for the
+ * largest op serves all of them. */
 size_t spr_workspace_bytes(int op, int B, int K, int V, int d, int h, int dt);
 
 /* Clears a freshly allocated workspace (enqueues a memset on the stream). */
@@ -119,6 +125,27 @@ int sprinter_verify(const void *hidden, const void *W1, const float *b1, const v
 int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, const int32_t *rows,
                    const int32_t *first_reject, int K, int seq_stride, int n, const float *uniforms,
                    int dt, int32_t *tokens, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * sprinter_step - one SPRINTER verification-and-replacement step in a single call.
+ *
+ * Defined by: Algorithm 2 as a whole: the verifier loop over the K draft positions
+ * (sprinter_verify) followed by the single target call for the position where the
+ * verifier stopped (replace_sample on row b*seq_stride + first_reject[b], skipped
+ * when every token passed).  Same arguments, results and error behaviour as those
+ * two calls made one after the other with first_reject passed along; here the
+ * replacement kernel is launched programmatically behind the verifier kernel, so
+ * its launch latency hides in the verifier's tail, and one clear serves both.
+ *
+ * target_logits [B, seq_stride, ldv] dt with seq_stride >= K rows per sequence (K, or
+ * K+1 when a bonus row is kept); uniforms [B] f32; tokens [B] int32 (-1 where nothing
+ * was rejected).  Workspace: spr_workspace_bytes(SPR_OP_SPRINTER_STEP, ...).
+ */
+int sprinter_step(const void *hidden, const void *W1, const float *b1, const void *W2, const float *b2,
+                  float threshold, int B, int K, int d, int h, const void *target_logits, int64_t ldv,
+                  int V, int seq_stride, const float *uniforms, int dt, int path, float *scores,
+                  uint8_t *accept, int32_t *first_reject, int32_t *tokens, void *ws, size_t ws_bytes,
+                  void *cuda_stream);
 
 /*
  * sd_verify - exact verification of standard speculative decoding.

@@ -15,14 +15,14 @@ import torch
 from . import build as _build
 
 F32, BF16 = 0, 1
-OP_SPRINTER_VERIFY, OP_REPLACE_SAMPLE, OP_SD_VERIFY = 0, 1, 2
+OP_SPRINTER_VERIFY, OP_REPLACE_SAMPLE, OP_SD_VERIFY, OP_SPRINTER_STEP = 0, 1, 2, 3
 PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
 
 EXPORTS = [
     "spr_workspace_bytes", "spr_workspace_init", "sprinter_verify", "replace_sample", "sd_verify",
     "spr_device_status", "spr_status_string", "spr_last_cuda_error", "spr_version",
     "spr_host_arena_bytes", "sprinter_verify_host", "replace_sample_host", "sd_verify_host",
-    "spr_set_stage_events", "replace_sample_static",
+    "spr_set_stage_events", "replace_sample_static", "sprinter_step",
 ]
 
 
@@ -60,6 +60,9 @@ def lib():
         L.sprinter_verify.restype = i32
         L.sprinter_verify.argtypes = [vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32,
                                       vp, vp, vp, vp, sz, vp]
+        L.sprinter_step.restype = i32
+        L.sprinter_step.argtypes = [vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, vp, i64, i32, i32, vp,
+                                    i32, i32, vp, vp, vp, vp, vp, sz, vp]
         L.replace_sample.restype = i32
         L.replace_sample.argtypes = [vp, i64, i32, i64, vp, vp, i32, i32, i32, vp, i32, vp, vp, sz, vp]
         L.sd_verify.restype = i32
@@ -148,7 +151,8 @@ class Workspace:
     def for_problem(cls, B: int, K: int, V: int, d: int, h: int, dt: int, device="cuda"):
         n = max(workspace_bytes(OP_SPRINTER_VERIFY, B, K, V, d, h, dt),
                 workspace_bytes(OP_REPLACE_SAMPLE, B, K, V, d, h, dt),
-                workspace_bytes(OP_SD_VERIFY, B, K, V, d, h, dt))
+                workspace_bytes(OP_SD_VERIFY, B, K, V, d, h, dt),
+                workspace_bytes(OP_SPRINTER_STEP, B, K, V, d, h, dt))
         return cls(n, device)
 
 
@@ -183,6 +187,46 @@ def sprinter_verify(hidden, W1, b1, W2, b2, threshold: float, ws: Workspace, pat
                                _ptr(ws.buf), ws.nbytes, _stream())
     _check("sprinter_verify", rc)
     return scores, accept, first_reject
+
+
+def sprinter_step(hidden, W1, b1, W2, b2, threshold: float, target_logits, V: int, uniforms,
+                  ws: Workspace, path: int = PATH_AUTO, want_scores: bool = True, out=None):
+    """sprinter_verify followed by the gated replace_sample, as one library call.
+
+    target_logits [B, seq_stride, ldv]; uniforms f32 [B].
+    Returns (scores or None, accept u8 [B,K], first_reject i32 [B], tokens i32 [B])."""
+    _dev(hidden, name="hidden")
+    B, K, d = hidden.shape
+    dt = _dt(hidden)
+    _dev(W1, hidden.dtype, "W1")
+    h = 0 if W1.dim() == 1 else W1.shape[0]
+    _dev(b2, torch.float32, "b2")
+    if h:
+        _dev(b1, torch.float32, "b1")
+        _dev(W2, hidden.dtype, "W2")
+    else:
+        b1 = W2 = None
+    _dev(target_logits, hidden.dtype, "target_logits")
+    if target_logits.dim() != 3 or target_logits.shape[0] != B:
+        raise ValueError("target_logits must be [B, seq_stride, ldv]")
+    seq_stride, ldv = target_logits.shape[1], target_logits.shape[2]
+    _dev(uniforms, torch.float32, "uniforms")
+    if uniforms.numel() != B:
+        raise ValueError("uniforms must have one entry per sequence")
+    if out is None:
+        dev = hidden.device
+        scores = torch.empty((B, K), dtype=torch.float32, device=dev) if want_scores else None
+        accept = torch.empty((B, K), dtype=torch.uint8, device=dev)
+        first_reject = torch.empty((B,), dtype=torch.int32, device=dev)
+        tokens = torch.empty((B,), dtype=torch.int32, device=dev)
+    else:
+        scores, accept, first_reject, tokens = out
+    rc = lib().sprinter_step(_ptr(hidden), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), float(threshold),
+                             B, K, d, h, _ptr(target_logits), ldv, V, seq_stride, _ptr(uniforms), dt, path,
+                             _ptr(scores), _ptr(accept), _ptr(first_reject), _ptr(tokens),
+                             _ptr(ws.buf), ws.nbytes, _stream())
+    _check("sprinter_step", rc)
+    return scores, accept, first_reject, tokens
 
 
 def replace_sample(target_logits, V: int, uniforms, ws: Workspace, rows=None, first_reject=None,

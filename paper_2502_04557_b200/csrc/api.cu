@@ -51,6 +51,21 @@ T *at(void *ws, size_t off)
     return reinterpret_cast<T *>(static_cast<char *>(ws) + off);
 }
 
+// tensor-core kernel where it applies (or is forced), SIMT kernel otherwise
+int launch_verifier(VerifyParams &vp, int dt, int path, cudaStream_t st)
+{
+    if (path != SPR_VERIFIER_SIMT) {
+        const int min_tokens = path == SPR_VERIFIER_TENSOR ? 1 : kTensorMinTokens;
+        const int tensor_rc = launch_verifier_tensor(vp, dt, min_tokens, st);  // < 0: shape not taken
+        if (tensor_rc == 0) return SPR_OK;
+        if (tensor_rc > 0) return cuda_fail((cudaError_t)tensor_rc);
+        if (path == SPR_VERIFIER_TENSOR) return SPR_ERR_UNSUPPORTED;
+    }
+    vp.slices = verifier_simt_slices(vp.h);
+    cudaError_t e = launch_verifier_simt(vp, dt, st);
+    return e == cudaSuccess ? SPR_OK : cuda_fail(e);
+}
+
 size_t verify_ws_bytes(int B, int K, int h)
 {
     const int M = B * K;
@@ -71,6 +86,9 @@ size_t spr_workspace_bytes(int op, int B, int K, int V, int d, int h, int dt)
     case SPR_OP_REPLACE_SAMPLE:
         if (V <= 0) return 0;
         return replace_ws_layout(B, stat_steps_per_row(V, dt)).end;
+    case SPR_OP_SPRINTER_STEP:
+        if (K <= 0 || d <= 0 || h < 0 || V <= 0 || (int64_t)B * K > 0x7fffffff) return 0;
+        return step_ws_layout(B, K, verifier_simt_slices(h), (B * K + 63) / 64, stat_steps_per_row(V, dt)).end;
     case SPR_OP_SD_VERIFY:
         if (K <= 0 || V <= 0 || (int64_t)B * K > 0x7fffffff) return 0;
         return sd_ws_layout(B, K, stat_segments_per_row(V, dt), stat_steps_per_row(V, dt)).end;
@@ -131,16 +149,7 @@ int sprinter_verify(const void *hidden, const void *W1, const float *b1, const v
     cudaError_t ce = cudaMemsetAsync(vp.counter, 0, lay.counters_end - lay.counter, st);
     if (ce != cudaSuccess) return cuda_fail(ce);
 
-    if (path != SPR_VERIFIER_SIMT) {
-        const int min_tokens = path == SPR_VERIFIER_TENSOR ? 1 : kTensorMinTokens;
-        const int tensor_rc = launch_verifier_tensor(vp, dt, min_tokens, st);  // < 0: shape not taken
-        if (tensor_rc == 0) return SPR_OK;
-        if (tensor_rc > 0) return cuda_fail((cudaError_t)tensor_rc);
-        if (path == SPR_VERIFIER_TENSOR) return SPR_ERR_UNSUPPORTED;
-    }
-    vp.slices = verifier_simt_slices(h);
-    cudaError_t e = launch_verifier_simt(vp, dt, st);
-    return e == cudaSuccess ? SPR_OK : cuda_fail(e);
+    return launch_verifier(vp, dt, path, st);
 }
 
 int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, const int32_t *rows,
@@ -183,6 +192,81 @@ int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, con
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaMemsetAsync(dp.counters, 0, sizeof(int) * (size_t)n, st);
     if (e == cudaSuccess) e = launch_draw(dp, n, dt, st);
+    return e == cudaSuccess ? SPR_OK : cuda_fail(e);
+}
+
+int sprinter_step(const void *hidden, const void *W1, const float *b1, const void *W2, const float *b2,
+                  float threshold, int B, int K, int d, int h, const void *target_logits, int64_t ldv,
+                  int V, int seq_stride, const float *uniforms, int dt, int path, float *scores,
+                  uint8_t *accept, int32_t *first_reject, int32_t *tokens, void *ws, size_t ws_bytes,
+                  void *cuda_stream)
+{
+    if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
+    if (path != SPR_VERIFIER_AUTO && path != SPR_VERIFIER_SIMT && path != SPR_VERIFIER_TENSOR)
+        return SPR_ERR_UNSUPPORTED;
+    if (B < 0 || K <= 0 || d <= 0 || h < 0 || V <= 0 || ldv < V || seq_stride < K ||
+        (int64_t)B * K > 0x7fffffff)
+        return SPR_ERR_INVALID_ARG;
+    if (B == 0) return SPR_OK;
+    if (!hidden || !W1 || !b2 || !accept || !first_reject || !target_logits || !uniforms || !tokens)
+        return SPR_ERR_INVALID_ARG;
+    if (h > 0 && (!b1 || !W2)) return SPR_ERR_INVALID_ARG;
+    const size_t es = elem_size(dt);
+    if (!aligned(hidden, es) || !aligned(W1, es) || (W2 && !aligned(W2, es)) || !aligned(b2, 4) ||
+        (b1 && !aligned(b1, 4)) || (scores && !aligned(scores, 4)) || !aligned(first_reject, 4) ||
+        !aligned(target_logits, es) || !aligned(uniforms, 4) || !aligned(tokens, 4))
+        return SPR_ERR_INVALID_ARG;
+    const int M = B * K;
+    const int C = stat_segments_per_row(V, dt), T = stat_steps_per_row(V, dt);
+    const StepWs lay = step_ws_layout(B, K, verifier_simt_slices(h), (M + 63) / 64, T);
+    if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
+    int rc = check_device();
+    if (rc != SPR_OK) return rc;
+
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    VerifyParams vp;
+    memset(&vp, 0, sizeof vp);
+    vp.hidden = hidden;
+    vp.W1 = W1;
+    vp.b1 = b1;
+    vp.W2 = W2;
+    vp.b2 = b2;
+    vp.threshold = threshold;
+    vp.B = B;
+    vp.K = K;
+    vp.d = d;
+    vp.h = h;
+    vp.scores = scores;
+    vp.accept = accept;
+    vp.first_reject = first_reject;
+    vp.status = at<int>(ws, 0);
+    vp.counter = at<int>(ws, lay.verify_counter);
+    vp.part_z = at<float>(ws, lay.part_z);
+
+    DrawParams dp;
+    memset(&dp, 0, sizeof dp);
+    dp.kind = DRAW_REPLACE;
+    dp.p = target_logits;
+    dp.ldv = ldv;
+    dp.V = V;
+    dp.chunks = C;
+    dp.steps = T;
+    dp.R = (int64_t)B * seq_stride;
+    dp.gate = first_reject;
+    dp.seq_stride = seq_stride;
+    dp.K = K;
+    dp.uniforms = uniforms;
+    dp.tokens = tokens;
+    dp.status = vp.status;
+    dp.counters = at<int>(ws, lay.draw.counters);
+    dp.part = at<float2>(ws, lay.draw.part);
+
+    // one clear for both kernels' tickets, then the draw is launched behind the verifier
+    cudaError_t e = cudaMemsetAsync(vp.counter, 0, lay.counters_end - lay.verify_counter, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    rc = launch_verifier(vp, dt, path, st);
+    if (rc != SPR_OK) return rc;
+    e = launch_draw(dp, B, dt, st, /*after_kernel=*/true);
     return e == cudaSuccess ? SPR_OK : cuda_fail(e);
 }
 
@@ -256,7 +340,7 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaMemsetAsync(sp.row_counters, 0, lay.counters_end - lay.row_counters, st);
     if (e == cudaSuccess) e = launch_sd_row_stats(sp, B, K, dt, st);
-    if (e == cudaSuccess) e = launch_draw(dp, B, dt, st);
+    if (e == cudaSuccess) e = launch_draw(dp, B, dt, st, /*after_kernel=*/true);
     return e == cudaSuccess ? SPR_OK : cuda_fail(e);
 }
 

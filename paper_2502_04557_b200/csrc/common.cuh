@@ -103,8 +103,37 @@ __host__ __device__ inline VerifyWs verify_ws_layout(int M, int slices, int tile
     return w;
 }
 
+struct StepWs {              // sprinter_step: verifier and replacement draw in one call
+    size_t verify_counter;   // int32 [1 + row tiles]
+    size_t draw_counters;    // int32 [B]
+    size_t counters_end;
+    size_t part_z;           // float [slices * M]
+    DrawWs draw;
+    size_t end;
+};
+__host__ __device__ inline StepWs step_ws_layout(int B, int K, int slices, int tiles, int T)
+{
+    const size_t M = (size_t)B * K;
+    StepWs w;
+    w.verify_counter = kHeaderBytes;
+    w.draw_counters = w.verify_counter + 4 * (size_t)(1 + tiles);
+    w.counters_end = align_up(w.draw_counters + 4 * (size_t)B, 256);
+    w.part_z = w.counters_end;
+    w.draw = draw_ws_layout(w.draw_counters, align_up(w.part_z + 4 * (size_t)slices * M, 256), B, T);
+    w.end = w.draw.end;
+    return w;
+}
+
 // ---------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
+
+// Programmatic dependent launch: a kernel launched with the programmatic-serialisation
+// attribute may start while the kernel before it in the stream is still running; it must
+// call pdl_wait() before touching anything that kernel writes.  pdl_trigger() in the earlier
+// kernel allows the next one to be scheduled as soon as every CTA has got this far.  Both are
+// no-ops for ordinary launches.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
 

@@ -257,6 +257,7 @@ __global__ void __launch_bounds__(kThreads, 3) draw_kernel(const DrawParams prm)
     const int c = blockIdx.x % C;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
+    pdl_wait();   // the kernel before this one may still be writing first_reject / accepted_len
     Job<T> job = resolve_job<T>(prm, i);
     if (job.mode == MODE_NONE) {
         if (c == 0 && tid == 0) {
@@ -357,16 +358,24 @@ __global__ void __launch_bounds__(kThreads, 3) draw_kernel(const DrawParams prm)
     if (lane == 0) prm.tokens[i] = token;
 }
 
-cudaError_t launch_draw(const DrawParams &dp, int n, int dt, cudaStream_t st)
+cudaError_t launch_draw(const DrawParams &dp, int n, int dt, cudaStream_t st, bool after_kernel)
 {
     const int64_t grid = (int64_t)n * dp.chunks;
     if (grid > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     if (grid == 0) return cudaSuccess;
-    if (dt == SPR_F32)
-        draw_kernel<float><<<(unsigned)grid, kThreads, 0, st>>>(dp);
-    else
-        draw_kernel<__nv_bfloat16><<<(unsigned)grid, kThreads, 0, st>>>(dp);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    if (after_kernel) {   // overlap this launch with the tail of the kernel that feeds it
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    return dt == SPR_F32 ? cudaLaunchKernelEx(&cfg, draw_kernel<float>, dp)
+                         : cudaLaunchKernelEx(&cfg, draw_kernel<__nv_bfloat16>, dp);
 }
 
 }  // namespace spr

@@ -72,7 +72,9 @@ struct VerifyParams {
 cudaError_t launch_sd_row_stats(const SdParams &sp, int B, int K, int dt, cudaStream_t st);
 int report_cuda_error(cudaError_t e);  // records the text, returns SPR_ERR_CUDA
 void set_stage_events(cudaEvent_t before, cudaEvent_t after);
-cudaError_t launch_draw(const DrawParams &dp, int n, int dt, cudaStream_t st);
+// after_kernel: the launch directly follows, in the same stream, the kernel whose output
+// selects the rows (programmatic dependent launch)
+cudaError_t launch_draw(const DrawParams &dp, int n, int dt, cudaStream_t st, bool after_kernel = false);
 
 // SIMT verifier: any dtype and shape.  `slices` must equal verifier_simt_slices(h).
 int verifier_simt_slices(int h);

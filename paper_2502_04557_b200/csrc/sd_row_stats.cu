@@ -20,6 +20,7 @@ __global__ void __launch_bounds__(kThreads) sd_row_stats_kernel(const SdParams p
     __shared__ float4 s_part[kWarps];
     __shared__ int s_last;
 
+    pdl_trigger();                       // the correction draw may be scheduled behind this grid
     const int C = prm.chunks;            // segments per row
     const int64_t row = blockIdx.x / C;  // = b*K + k
     const int c = blockIdx.x % C;

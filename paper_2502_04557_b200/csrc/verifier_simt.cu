@@ -78,6 +78,7 @@ __global__ void __launch_bounds__(kThreads) verifier_simt_kernel(const VerifyPar
 {
     __shared__ float s_z[kWarps][kTokTile];
     __shared__ int s_last;
+    pdl_trigger();   // a replacement draw launched behind this grid may be scheduled now
     const int M = prm.B * prm.K;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const T *hid = static_cast<const T *>(prm.hidden);

@@ -163,6 +163,7 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     Control *ctl = reinterpret_cast<Control *>(stages + (size_t)Cfg::kStages * Cfg::kStageBytes);
 
+    pdl_trigger();   // a replacement draw launched behind this grid may be scheduled now
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int M = prm.B * prm.K;
     const int n0 = blockIdx.x * BN;      // first hidden unit of this slice

@@ -464,3 +464,32 @@ def test_verifier_tensor_path_refuses_unsupported_shapes(spr):
         spr.sprinter_verify(H, z(8, 64).cuda(), z(8).cuda(), z(8).cuda(), z(1).cuda(), 0.5, ws,
                             path=spr.PATH_TENSOR)
     assert e.value.status == 2
+
+
+@pytest.mark.parametrize("name,kw", [("tiny", {}), ("gpt2", {"B": 6}), ("gpt2", {"B": 5, "ldv": 50264, "bonus_row": False}),
+                                     ("sequential", {"B": 16, "bonus_row": False}), ("llama2", {"B": 40})],
+                         ids=["tiny", "gpt2", "gpt2-padded", "sequential16", "llama2"])
+def test_sprinter_step_fused_call(spr, name, kw):
+    """sprinter_step = sprinter_verify + gated replace_sample in one call: same bits as the two
+    calls made separately, and as the oracle."""
+    wl_cpu = spr.workloads.make(name, "cpu", **kw)
+    enforce_margins(wl_cpu)
+    wl = to_device(wl_cpu)
+    cfg = wl.cfg
+    dtc = spr.binding._dt(wl.hidden)
+    ws = spr.Workspace.for_problem(wl.B, wl.K, wl.V, cfg.d, cfg.h, dtc)
+    scores, accept, fr, tokens = spr.sprinter_step(wl.hidden, wl.W1, wl.b1, wl.W2, wl.b2, 0.5, wl.p_logits,
+                                                   wl.V, wl.u_replace, ws)
+    assert ws.device_status() == 0
+    s2, a2, fr2 = spr.sprinter_verify(wl.hidden, wl.W1, wl.b1, wl.W2, wl.b2, 0.5, ws)
+    t2 = spr.replace_sample(wl.p_logits, wl.V, wl.u_replace, ws, first_reject=fr2, K=wl.K, seq_stride=wl.Kp)
+    assert torch.equal(scores, s2) and torch.equal(accept, a2) and torch.equal(fr, fr2) and torch.equal(tokens, t2)
+    s_ref, a_ref, fr_ref = oracle_verify(wl_cpu, 0.5)
+    P = to_np(wl_cpu.p_logits).reshape(wl.B * wl.Kp, wl.ldv)
+    t_ref = oracle.replace_sample(P, wl.V, to_np(wl_cpu.u_replace), first_reject=fr_ref, K=wl.K, seq_stride=wl.Kp)
+    eq(accept, a_ref, "accept")
+    eq(fr, fr_ref, "first_reject")
+    eq(tokens, t_ref, "tokens")
+    # a second fused call on the same workspace gives the same bits
+    again = spr.sprinter_step(wl.hidden, wl.W1, wl.b1, wl.W2, wl.b2, 0.5, wl.p_logits, wl.V, wl.u_replace, ws)
+    assert torch.equal(again[3], tokens) and torch.equal(again[2], fr)
