@@ -2,8 +2,9 @@
 """Throughput of the verification-and-replacement hot path on synthetic inputs.
 
 One step = one pass of the whole path over one batch: sprinter_verify (verifier scores,
-threshold, first-rejection scan) -> replace_sample gated by first_reject (replacement tokens)
--> sd_verify (exact speculative-decoding verification of the same draft tokens).  The
+threshold, first-rejection scan) -> replace_sample gated by first_reject (replacement tokens),
+issued as the fused sprinter_step call, and sd_verify (exact speculative-decoding verification
+of the same draft tokens) on a second stream.  The
 metric is draft tokens taken through that step per second, summed over all GPUs (each rank
 verifies its own batch: weak scaling, no data-path collective).
 
@@ -234,10 +235,9 @@ def main():
     def step():
         with torch.cuda.stream(st_sd):
             spr.sd_verify(wl.p_logits, wl.q_logits, V, wl.draft_tokens, wl.uniforms, ws_sd, out=sd_out)
-        with torch.cuda.stream(st_spr):
-            _, _, fr = spr.sprinter_verify(wl.hidden, wl.W1, wl.b1, wl.W2, wl.b2, tau, ws, out=ver_out)
-            spr.replace_sample(wl.p_logits, V, wl.u_replace, ws, first_reject=fr, K=K, seq_stride=wl.Kp,
-                               out=tok_out)
+        with torch.cuda.stream(st_spr):   # sprinter_verify + gated replace_sample as one call
+            spr.sprinter_step(wl.hidden, wl.W1, wl.b1, wl.W2, wl.b2, tau, wl.p_logits, V, wl.u_replace, ws,
+                              out=(ver_out[0], ver_out[1], ver_out[2], tok_out))
 
     def fork():
         st_spr.wait_stream(torch.cuda.current_stream())
@@ -365,7 +365,7 @@ def main():
             "steps": nsteps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16"
             if cfg.dtype == torch.bfloat16 else "f32", "data": "synthetic",
-            "config": {"workload": workload_label(wl), "step": "sd_verify (stream 1) || sprinter_verify + gated replace_sample (stream 2)",
+            "config": {"workload": workload_label(wl), "step": "sd_verify (stream 1) || sprinter_step = sprinter_verify + gated replace_sample (stream 2)",
                        "l2": f"inputs per step ({(alg_bytes + wl.p_logits[:, K:].numel() * es) / 1e9:.2f} GB of logits) "
                              "exceed the 126 MB L2; no flush needed",
                        "threshold": tau, "mean_sd_accepted_len": acc_len, "mean_first_reject": fr_mean},
