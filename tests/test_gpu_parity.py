@@ -175,6 +175,23 @@ def test_llama3_full_size_sampled(spr):
     t = tokens.cpu().numpy()
     frn = fr.cpu().numpy()
     assert ((t >= 0) == (frn < wl.K)).all() and (t < wl.V).all()
+    # the launch configuration the benchmark times: sd_verify on one stream, the fused
+    # sprinter_step on another, separate workspaces; must give the same bits
+    cfg = wl.cfg
+    ws1 = spr.Workspace.for_problem(wl.B, wl.K, wl.V, cfg.d, cfg.h, spr.BF16)
+    ws2 = spr.Workspace.for_problem(wl.B, wl.K, wl.V, cfg.d, cfg.h, spr.BF16)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for _ in range(2):
+        with torch.cuda.stream(s1):
+            out2 = spr.sd_verify(wl.p_logits, wl.q_logits, wl.V, wl.draft_tokens, wl.uniforms, ws1)
+        with torch.cuda.stream(s2):
+            _, acc2, fr2, tok2 = spr.sprinter_step(wl.hidden, wl.W1, wl.b1, wl.W2, wl.b2, 0.5, wl.p_logits,
+                                                   wl.V, wl.u_replace, ws2)
+    torch.cuda.synchronize()
+    for k in out:
+        assert torch.equal(out[k], out2[k]), k
+    assert torch.equal(fr, fr2) and torch.equal(tokens, tok2)
 
 
 def test_sequential_1024_sampled(spr):
