@@ -66,6 +66,10 @@ def lib():
         L.oracle_softmax_draw_margin.argtypes = [vp, i32, i32, f64, vp]
         L.oracle_residual_draw_margin.restype = f64
         L.oracle_residual_draw_margin.argtypes = [vp, vp, i32, i32, f64, vp]
+        L.oracle_philox4x32_10.restype = None
+        L.oracle_philox4x32_10.argtypes = [vp, vp, vp]
+        L.oracle_simulate_runs.restype = i32
+        L.oracle_simulate_runs.argtypes = [C.c_uint64, i64, i64, i32, f32, f32, i32, vp, vp]
         _lib = L
     return _lib
 
@@ -219,3 +223,24 @@ def residual_draw_margin(p_row, q_row, u: float):
     m = lib().oracle_residual_draw_margin(_p(p_row), _p(q_row), _dt(p_row), p_row.shape[0],
                                           float(u), C.byref(t))
     return float(m), int(t.value)
+
+
+def philox4x32_10(counter, key) -> np.ndarray:
+    c = _c(counter, np.uint32)
+    k = _c(key, np.uint32)
+    assert c.shape == (4,) and k.shape == (2,)
+    out = np.empty(4, np.uint32)
+    lib().oracle_philox4x32_10(_p(c), _p(k), _p(out))
+    return out
+
+
+def simulate_runs(seed: int, runs: int, r: int, eta_tp: float, eta_fp: float, max_tokens: int,
+                  first_run: int = 0):
+    """Returns (n_accepted int32 [runs], histogram uint64 [max_tokens + 1])."""
+    n = np.empty((runs,), np.int32)
+    hist = np.empty((max_tokens + 1,), np.uint64)
+    rc = lib().oracle_simulate_runs(int(seed), int(first_run), int(runs), int(r), float(eta_tp),
+                                    float(eta_fp), int(max_tokens), _p(n), _p(hist))
+    if rc != OK:
+        raise ValueError(f"oracle_simulate_runs: error {rc}")
+    return n, hist

@@ -19,6 +19,9 @@
  *   oracle_sd_verify        - accept with probability min(1, p(x)/q(x)), else
  *                             resample from norm(max(0, p - q)) (Section 2 and
  *                             Eq. 1; Algorithm 2, branch c > n).
+ *   oracle_simulate_runs    - the number of tokens an i.i.d. verifier accepts in a
+ *                             row (the scenario of Theorems 2 and 3), one
+ *                             Philox4x32-10 stream per run.
  *
  * Readings of points the paper leaves open (all restated in the design notes):
  *   - a token is accepted by the verifier iff score >= tau (Algorithm 2; the
@@ -392,4 +395,72 @@ double oracle_residual_draw_margin(const void *p_row, const void *q_row, int dt,
         m = oracle_softmax_draw_margin(p_row, dt, V, u, t_out);
     free(w);
     return m;
+}
+
+/* ---- decode-loop statistics with an i.i.d. verifier (Section 3.1, Theorems 2 and 3) ----
+ *
+ * Scenario of Fig. "token generation": the draft produces r acceptable tokens followed by
+ * unacceptable ones; the verifier accepts an acceptable token with probability eta_TP and an
+ * unacceptable one with probability eta_FP, independently; N = number of consecutive tokens
+ * it accepts before its first rejection.  Run i draws its uniforms from the counter-based
+ * generator Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as
+ * 1, 2, 3", SC'11): block j of run i is Philox(counter = {lo(i), hi(i), j, 0},
+ * key = {lo(seed), hi(seed)}), token k uses word k % 4 of block k / 4, and
+ * u = (word >> 8) * 2^-24.  Token k (0-based) is accepted iff u < (k < r ? eta_TP : eta_FP).
+ * N is capped at max_tokens.
+ */
+void oracle_philox4x32_10(const uint32_t ctr_in[4], const uint32_t key_in[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr_in[0], c1 = ctr_in[1], c2 = ctr_in[2], c3 = ctr_in[3];
+    uint32_t k0 = key_in[0], k1 = key_in[1];
+    for (int round = 0; round < 10; ++round) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        const uint32_t n1 = (uint32_t)p1;
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        const uint32_t n3 = (uint32_t)p0;
+        c0 = n0;
+        c1 = n1;
+        c2 = n2;
+        c3 = n3;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0;
+    out[1] = c1;
+    out[2] = c2;
+    out[3] = c3;
+}
+
+int oracle_simulate_runs(uint64_t seed, int64_t first_run, int64_t runs, int r, float eta_tp,
+                         float eta_fp, int max_tokens, int32_t *n_accepted, uint64_t *histogram)
+{
+    if (runs < 0 || r < 0 || max_tokens < 0 || (!n_accepted && !histogram))
+        return ORC_ERR_ARG;
+    if (histogram)
+        for (int i = 0; i <= max_tokens; ++i)
+            histogram[i] = 0;
+    const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    for (int64_t j = 0; j < runs; ++j) {
+        const uint64_t run = (uint64_t)(first_run + j);
+        int n = 0;
+        uint32_t w[4] = {0, 0, 0, 0};
+        while (n < max_tokens) {
+            if (n % 4 == 0) {
+                const uint32_t ctr[4] = {(uint32_t)run, (uint32_t)(run >> 32), (uint32_t)(n / 4), 0u};
+                oracle_philox4x32_10(ctr, key, w);
+            }
+            const float u = (float)(w[n % 4] >> 8) * 5.9604644775390625e-8f; /* 2^-24 */
+            const float eta = n < r ? eta_tp : eta_fp;
+            if (!(u < eta))
+                break;
+            ++n;
+        }
+        if (n_accepted)
+            n_accepted[j] = n;
+        if (histogram)
+            histogram[n] += 1;
+    }
+    return ORC_OK;
 }
