@@ -180,6 +180,26 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
               float *residual_mass, void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * sprinter_simulate - run lengths of an i.i.d. verifier (Monte-Carlo of Theorems 2 and 3).
+ *
+ * Defined by: Section 3.1(b), the scenario of Theorem 2: the draft produces r acceptable
+ * tokens followed by unacceptable ones; the verifier accepts an acceptable token with
+ * probability eta_tp and an unacceptable one with probability eta_fp, independently;
+ * N = number of consecutive tokens accepted before the first rejection (capped at
+ * max_tokens).  Theorem 2 gives the law and mean of N, Theorem 3 the stopping time
+ * t_d (N + 1).
+ *
+ * Run i (i = first_run .. first_run + runs - 1) owns one Philox4x32-10 stream: block j
+ * = Philox(counter {lo(i), hi(i), j, 0}, key {lo(seed), hi(seed)}); token k uses word
+ * k % 4 of block k / 4 with u = (word >> 8) * 2^-24 and is accepted iff
+ * u < (k < r ? eta_tp : eta_fp).  Results therefore do not depend on the launch shape.
+ * n_accepted [runs] int32 (device, optional), histogram [max_tokens + 1] uint64 (device,
+ * optional, overwritten): at least one must be given.  No workspace.
+ */
+int sprinter_simulate(uint64_t seed, int64_t first_run, int64_t runs, int r, float eta_tp, float eta_fp,
+                      int max_tokens, int32_t *n_accepted, uint64_t *histogram, void *cuda_stream);
+
+/*
  * Host-buffer variants.  Same operations and arguments as the calls above, but every
  * tensor pointer is a HOST pointer (pinned memory makes the copies asynchronous and
  * fast).  Each call copies its inputs into `arena` - caller-owned device memory of at

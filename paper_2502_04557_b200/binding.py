@@ -22,7 +22,7 @@ EXPORTS = [
     "spr_workspace_bytes", "spr_workspace_init", "sprinter_verify", "replace_sample", "sd_verify",
     "spr_device_status", "spr_status_string", "spr_last_cuda_error", "spr_version",
     "spr_host_arena_bytes", "sprinter_verify_host", "replace_sample_host", "sd_verify_host",
-    "spr_set_stage_events", "replace_sample_static", "sprinter_step",
+    "spr_set_stage_events", "replace_sample_static", "sprinter_step", "sprinter_simulate",
 ]
 
 
@@ -63,6 +63,8 @@ def lib():
         L.sprinter_step.restype = i32
         L.sprinter_step.argtypes = [vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, vp, i64, i32, i32, vp,
                                     i32, i32, vp, vp, vp, vp, vp, sz, vp]
+        L.sprinter_simulate.restype = i32
+        L.sprinter_simulate.argtypes = [C.c_uint64, i64, i64, i32, f32, f32, i32, vp, vp, vp]
         L.replace_sample.restype = i32
         L.replace_sample.argtypes = [vp, i64, i32, i64, vp, vp, i32, i32, i32, vp, i32, vp, vp, sz, vp]
         L.sd_verify.restype = i32
@@ -410,3 +412,16 @@ def replace_sample_static(target_logits, V: int, uniforms, tokens, rows=None, fi
                                      _stream())
     _check("replace_sample_static", rc)
     return tokens
+
+
+def sprinter_simulate(seed: int, runs: int, r: int, eta_tp: float, eta_fp: float, max_tokens: int,
+                      first_run: int = 0, want_runs: bool = True, device="cuda"):
+    """Run lengths of an i.i.d. verifier (Theorems 2 and 3).
+
+    Returns (n_accepted int32 [runs] or None, histogram int64 [max_tokens + 1])."""
+    n = torch.empty((runs,), dtype=torch.int32, device=device) if want_runs else None
+    hist = torch.empty((max_tokens + 1,), dtype=torch.int64, device=device)
+    rc = lib().sprinter_simulate(int(seed), int(first_run), int(runs), int(r), float(eta_tp), float(eta_fp),
+                                 int(max_tokens), _ptr(n), _ptr(hist), _stream())
+    _check("sprinter_simulate", rc)
+    return n, hist

@@ -344,6 +344,35 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
     return e == cudaSuccess ? SPR_OK : cuda_fail(e);
 }
 
+int sprinter_simulate(uint64_t seed, int64_t first_run, int64_t runs, int r, float eta_tp, float eta_fp,
+                      int max_tokens, int32_t *n_accepted, uint64_t *histogram, void *cuda_stream)
+{
+    if (runs < 0 || first_run < 0 || r < 0 || max_tokens < 0 || (!n_accepted && !histogram))
+        return SPR_ERR_INVALID_ARG;
+    if (!(eta_tp >= 0.f && eta_tp <= 1.f) || !(eta_fp >= 0.f && eta_fp <= 1.f)) return SPR_ERR_INVALID_ARG;
+    if ((n_accepted && !aligned(n_accepted, 4)) || (histogram && !aligned(histogram, 8)))
+        return SPR_ERR_INVALID_ARG;
+    int rc = check_device();
+    if (rc != SPR_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (histogram) {
+        cudaError_t e = cudaMemsetAsync(histogram, 0, sizeof(uint64_t) * ((size_t)max_tokens + 1), st);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    SimParams sp;
+    sp.seed = seed;
+    sp.first_run = first_run;
+    sp.runs = runs;
+    sp.r = r;
+    sp.max_tokens = max_tokens;
+    sp.eta_tp = eta_tp;
+    sp.eta_fp = eta_fp;
+    sp.n_accepted = n_accepted;
+    sp.histogram = reinterpret_cast<unsigned long long *>(histogram);
+    cudaError_t e = launch_simulate(sp, st);
+    return e == cudaSuccess ? SPR_OK : cuda_fail(e);
+}
+
 int spr_device_status(void *ws, void *cuda_stream)
 {
     if (!ws) return SPR_ERR_WORKSPACE;

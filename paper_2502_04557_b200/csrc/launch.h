@@ -69,6 +69,16 @@ struct VerifyParams {
     int slices;
 };
 
+struct SimParams {
+    uint64_t seed;
+    int64_t first_run, runs;
+    int r, max_tokens;
+    float eta_tp, eta_fp;
+    int32_t *n_accepted;              // [runs] or null
+    unsigned long long *histogram;    // [max_tokens + 1] or null
+};
+cudaError_t launch_simulate(const SimParams &sp, cudaStream_t st);
+
 cudaError_t launch_sd_row_stats(const SdParams &sp, int B, int K, int dt, cudaStream_t st);
 int report_cuda_error(cudaError_t e);  // records the text, returns SPR_ERR_CUDA
 void set_stage_events(cudaEvent_t before, cudaEvent_t after);
