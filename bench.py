@@ -56,6 +56,8 @@ def parse_args():
     ap.add_argument("--threshold", type=float, default=0.5)
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--simulator-runs", type=int, default=0,
+                    help="also time sprinter_simulate on this many runs (r=5, eta_TP=0.9, eta_FP=0.5)")
     return ap.parse_args()
 
 
@@ -356,6 +358,27 @@ def main():
                         "sample": f"first {sample} of {B} sequences ({sample * K} draft tokens), one pass, "
                                   f"{dt:.1f} s"}
 
+    simulator = None
+    if args.simulator_runs > 0:
+        runs = args.simulator_runs
+        for _ in range(3):
+            spr.sprinter_simulate(1, runs, 5, 0.9, 0.5, 255, want_runs=False, device=dev)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(10):
+            _, hist = spr.sprinter_simulate(1, runs, 5, 0.9, 0.5, 255, want_runs=False, device=dev)
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / 10
+        tokens = float((hist * torch.arange(256, device=dev)).sum() + runs)   # uniforms consumed
+        # every 4 uniforms cost one Philox block: 10 rounds x (2 mul.hi + 2 mul.lo + 4 xor + 2 add)
+        blocks = float(((hist * ((torch.arange(256, device=dev) + 4) // 4)).sum()))
+        int_ops = blocks * 100.0
+        alu_peak = 148 * 128 * 1.965e9      # 32-bit ALU lane-operations per second, all SMs
+        simulator = {"runs": runs, "ms": ms, "runs_per_s": runs / (ms * 1e-3), "uniforms_per_s": tokens / (ms * 1e-3),
+                     "roofline": {"bound": "alu", "achieved": int_ops / (ms * 1e-3) / 1e12, "peak": alu_peak / 1e12,
+                                  "unit": "Tlane-op/s", "frac": int_ops / (ms * 1e-3) / alu_peak}}
+
     if rank == 0:
         sampler.stop()
         acc_len = sd_out["accepted_len"].float().mean().item()
@@ -375,6 +398,7 @@ def main():
                          "traffic": traffic, "algorithmic_bytes_per_launch": alg_bytes,
                          "avg_launch_ms": stats_ms},
             "cpu_baseline": cpu_baseline,
+            **({"simulator": simulator} if simulator else {}),
         }))
     if world > 1:
         dist.destroy_process_group()
