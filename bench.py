@@ -30,10 +30,10 @@ if ROOT not in sys.path:
 # capture summarised under profiles/; reported only while the kernel source is unchanged.
 NCU_TRAFFIC = {
     "sources": ("sd_row_stats.cu", "vocab_common.cuh", "common.cuh"),
-    "sha256": "468c5a905fd148ba26ac74403665cbc469b6c6fe8065a64a6f1b78d88bf6539b",
-    # (262,771,968 read + 3,382,016 written) / 512 tokens in the B = 32 capture; traffic grows
+    "sha256": "7a0264a12ad9f730d10325ef514e4549e5abd5e8f0722d8a22f1cce9de696c17",
+    # (262,795,520 read + 3,676,160 written) / 512 tokens in the B = 32 capture; traffic grows
     # in proportion to the tokens, so a full launch is this times B*K
-    "bytes_per_unit": 519832,   # DRAM bytes per verified token at V = 128256, bf16
+    "bytes_per_unit": 520452,   # DRAM bytes per verified token at V = 128256, bf16
 }
 
 
