@@ -29,7 +29,7 @@
  *     first such code, and spr_device_status() returns and clears it.
  *   - Outputs are fully overwritten and are bit-identical from run to run for
  *     identical inputs (fixed reduction orders, no floating-point atomics).
- *   - Logits must be finite or -inf; uniforms must lie in [0,1).
+ *   - Logits must be finite or -inf; uniforms must lie in [0,1); V <= 2^30.
  *   - The library runs only on compute capability 10.x devices; there is no
  *     CPU or other fallback (SPR_ERR_UNSUPPORTED).
  */

@@ -42,6 +42,9 @@ int check_device()
 // AUTO hands batches of at least this many tokens to the tensor-core verifier
 constexpr int kTensorMinTokens = 4;
 
+// row indices are 32-bit inside the kernels; leave room for the padding of the last step
+constexpr int kMaxVocab = 1 << 30;
+
 bool dtype_ok(int dt) { return dt == SPR_F32 || dt == SPR_BF16; }
 bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
@@ -157,7 +160,7 @@ int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, con
                    int dt, int32_t *tokens, void *ws, size_t ws_bytes, void *cuda_stream)
 {
     if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
-    if (V <= 0 || ldv < V || R < 0 || n < 0 || seq_stride < 0) return SPR_ERR_INVALID_ARG;
+    if (V <= 0 || V > kMaxVocab || ldv < V || R < 0 || n < 0 || seq_stride < 0) return SPR_ERR_INVALID_ARG;
     if (n == 0) return SPR_OK;  // no draws: pointers may be null
     if (!target_logits || !uniforms || !tokens || R == 0) return SPR_ERR_INVALID_ARG;
     if (first_reject && K <= 0) return SPR_ERR_INVALID_ARG;
@@ -204,7 +207,7 @@ int sprinter_step(const void *hidden, const void *W1, const float *b1, const voi
     if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
     if (path != SPR_VERIFIER_AUTO && path != SPR_VERIFIER_SIMT && path != SPR_VERIFIER_TENSOR)
         return SPR_ERR_UNSUPPORTED;
-    if (B < 0 || K <= 0 || d <= 0 || h < 0 || V <= 0 || ldv < V || seq_stride < K ||
+    if (B < 0 || K <= 0 || d <= 0 || h < 0 || V <= 0 || V > kMaxVocab || ldv < V || seq_stride < K ||
         (int64_t)B * K > 0x7fffffff)
         return SPR_ERR_INVALID_ARG;
     if (B == 0) return SPR_OK;
@@ -276,7 +279,7 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
               float *residual_mass, void *ws, size_t ws_bytes, void *cuda_stream)
 {
     if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
-    if (B < 0 || K <= 0 || V <= 0 || ldv < V || (Kp != K && Kp != K + 1) ||
+    if (B < 0 || K <= 0 || V <= 0 || V > kMaxVocab || ldv < V || (Kp != K && Kp != K + 1) ||
         (int64_t)B * K > 0x7fffffff)
         return SPR_ERR_INVALID_ARG;
     if (B == 0) return SPR_OK;  // empty batch: pointers may be null

@@ -510,3 +510,37 @@ def test_sprinter_step_fused_call(spr, name, kw):
     # a second fused call on the same workspace gives the same bits
     again = spr.sprinter_step(wl.hidden, wl.W1, wl.b1, wl.W2, wl.b2, 0.5, wl.p_logits, wl.V, wl.u_replace, ws)
     assert torch.equal(again[3], tokens) and torch.equal(again[2], fr)
+
+
+@pytest.mark.parametrize("dtype,V", [(torch.bfloat16, 600_011), (torch.float32, 300_007)], ids=["bf16", "f32"])
+def test_very_large_vocabulary(spr, dtype, V):
+    """More warp steps per row (586) than the last CTA of a draw caches in shared memory (512)."""
+    B, K = 3, 2
+    p, q, x, u = _rand_problem(B, K, V, dtype, seed=V, Kp=K + 1, scale=3.0)
+    # put most of the mass of one row near the end of the vocabulary so draws land in late steps
+    p[0, 0, V - 5000:] += 6.0
+    ref = _clear_sd(p, q, V, x, u)
+    ws = spr.Workspace(max(spr.workspace_bytes(2, B, K, V, 1, 0, spr.binding._dt(p)),
+                           spr.workspace_bytes(1, B * (K + 1), 1, V, 1, 0, spr.binding._dt(p))))
+    out = spr.sd_verify(p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), ws)
+    assert ws.device_status() == 0
+    eq(out["accept"], ref["accept"], "accept")
+    eq(out["accepted_len"], ref["accepted_len"], "accepted_len")
+    eq(out["correction_token"], ref["correction_token"], "correction_token")
+    assert_close_rel(out["p_tok"], ref["p_tok"], RTOL[dtype], "p_tok")
+    # plain draws from every target row, uniforms spread over [0, 1)
+    rows = p.reshape(B * (K + 1), V)
+    g = torch.Generator().manual_seed(1)
+    uu = torch.rand(B * (K + 1), generator=g)
+    uu[0] = 0.97
+    R = to_np(rows)
+    for i in range(len(uu)):
+        for _ in range(50):
+            m, _t = oracle.softmax_draw_margin(R[i, :V], float(uu[i]))
+            if m >= 1e-6:
+                break
+            uu[i] = torch.rand((), generator=g)
+    got = spr.replace_sample(rows.cuda(), V, uu.cuda(), ws)
+    want = oracle.replace_sample(R, V, uu.numpy())
+    eq(got, want, "tokens")
+    assert want[0] >= V - 5000
