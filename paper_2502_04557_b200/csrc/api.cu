@@ -167,7 +167,9 @@ int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, con
     if (!aligned(target_logits, elem_size(dt)) || !aligned(uniforms, 4) || !aligned(tokens, 4) ||
         (rows && !aligned(rows, 4)) || (first_reject && !aligned(first_reject, 4)))
         return SPR_ERR_INVALID_ARG;
-    const int C = stat_segments_per_row(V, dt), T = stat_steps_per_row(V, dt);
+    const int T = stat_steps_per_row(V, dt);
+    int C, iters;
+    draw_geometry(n, T, &C, &iters);
     const DrawWs lay = replace_ws_layout(n, T);
     if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
     int rc = check_device();
@@ -181,6 +183,7 @@ int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, con
     dp.ldv = ldv;
     dp.V = V;
     dp.chunks = C;
+    dp.iters = iters;
     dp.R = R;
     dp.rows = rows;
     dp.gate = first_reject;
@@ -220,7 +223,9 @@ int sprinter_step(const void *hidden, const void *W1, const float *b1, const voi
         !aligned(target_logits, es) || !aligned(uniforms, 4) || !aligned(tokens, 4))
         return SPR_ERR_INVALID_ARG;
     const int M = B * K;
-    const int C = stat_segments_per_row(V, dt), T = stat_steps_per_row(V, dt);
+    const int T = stat_steps_per_row(V, dt);
+    int C, iters;
+    draw_geometry(B, T, &C, &iters);
     const StepWs lay = step_ws_layout(B, K, verifier_simt_slices(h), (M + 63) / 64, T);
     if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
     int rc = check_device();
@@ -253,6 +258,7 @@ int sprinter_step(const void *hidden, const void *W1, const float *b1, const voi
     dp.ldv = ldv;
     dp.V = V;
     dp.chunks = C;
+    dp.iters = iters;
     dp.steps = T;
     dp.R = (int64_t)B * seq_stride;
     dp.gate = first_reject;
@@ -327,7 +333,7 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
     dp.q = q_logits;
     dp.ldv = ldv;
     dp.V = V;
-    dp.chunks = C;
+    draw_geometry(B, T, &dp.chunks, &dp.iters);
     dp.K = K;
     dp.Kp = Kp;
     dp.accepted_len = accepted_len;

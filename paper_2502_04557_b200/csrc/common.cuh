@@ -35,6 +35,16 @@ __host__ __device__ inline int stat_segments_per_row(int V, int dt)
     return (V + vec_elems(dt) - 1 + stat_segment_elems(dt) - 1) / stat_segment_elems(dt);
 }
 
+// Draw kernels: with few draws a row is spread over more CTAs (fewer steps per warp), which
+// shortens the chain of dependent loads each CTA goes through.
+inline void draw_geometry(int n, int steps, int *segments, int *iters)
+{
+    int it = kStatIters;
+    while (it > 1 && (int64_t)n * ((steps + kWarps * it - 1) / (kWarps * it)) < 148) it /= 2;
+    *iters = it;
+    *segments = (steps + kWarps * it - 1) / (kWarps * it);
+}
+
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // ---------------------------------------------------------------- workspace layouts

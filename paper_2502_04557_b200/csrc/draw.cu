@@ -146,16 +146,17 @@ __device__ __forceinline__ MS softmax_step(const uint4 (&raw)[kUnroll])
 }
 
 // Step partials (max, weight) of segment c of the job's row(s), written to part[step] for the
-// steps this CTA owns; same step interleaving and prefetch as the row-statistics kernel.
+// steps this CTA owns (iters per warp; fewer when there are few draws, so that more CTAs
+// share a row); same step interleaving and prefetch as the row-statistics kernel.
 // Residual draws store (0, sum of max(0, p - q)).
 template <typename T>
-__device__ __forceinline__ void segment_pass(const Job<T> &job, int mode, int V, int c, int steps,
+__device__ __forceinline__ void segment_pass(const Job<T> &job, int mode, int V, int c, int steps, int iters,
                                              float2 *__restrict__ part)
 {
     constexpr int N = Vec<T>::N;
     constexpr int kStep = 32 * kUnroll * N;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int step0 = c * 32 + warp;                      // this warp's steps: step0 + it*kWarps
+    const int step0 = c * kWarps * iters + warp;          // this warp's steps: step0 + it*kWarps
     const int first = step0 * kStep - row_pad(job.p_row);
     uint4 rp[kUnroll], rq[kUnroll];
     if (step0 >= steps) return;
@@ -165,7 +166,7 @@ __device__ __forceinline__ void segment_pass(const Job<T> &job, int mode, int V,
     for (int it = 0; it < kStatIters; ++it) {
         const int step = step0 + it * kWarps;
         const int nxt = (it + 1) * kWarps * kStep;
-        const bool more = it + 1 < kStatIters && step + kWarps < steps;
+        const bool more = it + 1 < iters && step + kWarps < steps;
         MS v;
         if (mode == MODE_SOFTMAX) {
             uint4 cur[kUnroll];
@@ -251,7 +252,7 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads, 3) draw_kernel(const DrawParams prm)
 {
     __shared__ DrawSmem sm;
-    const int C = prm.chunks;   // segments (CTAs) per row
+    const int C = prm.chunks;   // segments (CTAs) per row, of kWarps * prm.iters steps each
     const int steps = prm.steps;
     const int i = blockIdx.x / C;
     const int c = blockIdx.x % C;
@@ -269,7 +270,7 @@ __global__ void __launch_bounds__(kThreads, 3) draw_kernel(const DrawParams prm)
     int mode = job.mode;
     float2 *part = prm.part + (int64_t)i * steps;
 
-    segment_pass<T>(job, mode, prm.V, c, steps, part);
+    segment_pass<T>(job, mode, prm.V, c, steps, prm.iters, part);
     __syncthreads();
     if (tid == 0) {
         __threadfence();
@@ -346,7 +347,7 @@ __global__ void __launch_bounds__(kThreads, 3) draw_kernel(const DrawParams prm)
         if (mode == MODE_RESIDUAL && !(sm.total > 0.0)) {
             // max(0, p - q) vanished: Eq. 1 is undefined, draw from p itself (one CTA, rare)
             mode = MODE_SOFTMAX;
-            for (int cc = 0; cc < C; ++cc) segment_pass<T>(job, mode, prm.V, cc, steps, part);
+            for (int cc = 0; cc < C; ++cc) segment_pass<T>(job, mode, prm.V, cc, steps, prm.iters, part);
             __syncthreads();
             continue;
         }

@@ -34,6 +34,7 @@ struct DrawParams {
     const void *q;
     int64_t ldv;
     int V, chunks, steps;   // segments (CTAs) and warp steps per row
+    int iters;              // warp steps each warp of a CTA takes (1, 2 or 4)
     // replace_sample
     int64_t R;
     const int32_t *rows;

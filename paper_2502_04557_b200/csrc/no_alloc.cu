@@ -60,7 +60,9 @@ extern "C" int replace_sample_static(const void *target_logits, int64_t ldv, int
         reinterpret_cast<uintptr_t>(tokens) % 4 || (rows && reinterpret_cast<uintptr_t>(rows) % 4) ||
         (first_reject && reinterpret_cast<uintptr_t>(first_reject) % 4))
         return SPR_ERR_INVALID_ARG;
-    const int C = stat_segments_per_row(V, dt), T = stat_steps_per_row(V, dt);
+    const int T = stat_steps_per_row(V, dt);
+    int C, iters;
+    draw_geometry(n, T, &C, &iters);
     // the built-in scratch has room for kMaxDraws tickets and kMaxDrawSteps step partials
     if (n > kMaxDraws || (int64_t)n * T > kMaxDrawSteps) return SPR_ERR_WORKSPACE;
 
@@ -82,6 +84,7 @@ extern "C" int replace_sample_static(const void *target_logits, int64_t ldv, int
     dp.ldv = ldv;
     dp.V = V;
     dp.chunks = C;
+    dp.iters = iters;
     dp.R = R;
     dp.rows = rows;
     dp.gate = first_reject;
