@@ -94,7 +94,7 @@ size_t spr_workspace_bytes(int op, int B, int K, int V, int d, int h, int dt)
         return step_ws_layout(B, K, verifier_simt_slices(h), (B * K + 63) / 64, stat_steps_per_row(V, dt)).end;
     case SPR_OP_SD_VERIFY:
         if (K <= 0 || V <= 0 || (int64_t)B * K > 0x7fffffff) return 0;
-        return sd_ws_layout(B, K, stat_segments_per_row(V, dt), stat_steps_per_row(V, dt)).end;
+        return sd_ws_layout(B, K, stat_max_segments_per_row(V, dt), stat_steps_per_row(V, dt)).end;
     default:
         return 0;
     }
@@ -297,8 +297,10 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
         (p_tok && !aligned(p_tok, 4)) || (q_tok && !aligned(q_tok, 4)) ||
         (residual_mass && !aligned(residual_mass, 4)))
         return SPR_ERR_INVALID_ARG;
-    const int C = stat_segments_per_row(V, dt), T = stat_steps_per_row(V, dt);
-    const SdWs lay = sd_ws_layout(B, K, C, T);
+    const int T = stat_steps_per_row(V, dt);
+    int C, stat_iters;
+    draw_geometry(B * K, T, &C, &stat_iters);   // same rule for the row-statistics pass, over B*K rows
+    const SdWs lay = sd_ws_layout(B, K, stat_max_segments_per_row(V, dt), T);
     if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
     int rc = check_device();
     if (rc != SPR_OK) return rc;
@@ -313,6 +315,7 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
     sp.K = K;
     sp.Kp = Kp;
     sp.chunks = C;
+    sp.iters = stat_iters;
     sp.draft_tokens = draft_tokens;
     sp.uniforms = uniforms;
     sp.accepted_len = accepted_len;

@@ -30,12 +30,17 @@ __host__ __device__ inline int stat_steps_per_row(int V, int dt)
 {
     return (V + vec_elems(dt) - 1 + stat_step_elems(dt) - 1) / stat_step_elems(dt);
 }
+// most segments a row can be cut into (one step per warp)
+__host__ __device__ inline int stat_max_segments_per_row(int V, int dt)
+{
+    return (stat_steps_per_row(V, dt) + kWarps - 1) / kWarps;
+}
 __host__ __device__ inline int stat_segments_per_row(int V, int dt)
 {
     return (V + vec_elems(dt) - 1 + stat_segment_elems(dt) - 1) / stat_segment_elems(dt);
 }
 
-// Draw kernels: with few draws a row is spread over more CTAs (fewer steps per warp), which
+// With few rows to read, a row is spread over more CTAs (fewer steps per warp), which
 // shortens the chain of dependent loads each CTA goes through.
 inline void draw_geometry(int n, int steps, int *segments, int *iters)
 {

@@ -10,7 +10,8 @@ struct SdParams {
     const void *p;  // [B,Kp,ldv]
     const void *q;  // [B,K,ldv]
     int64_t ldv;
-    int V, K, Kp, chunks;
+    int V, K, Kp, chunks;   // chunks = segments (CTAs) per row
+    int iters;              // warp steps each warp of a CTA takes (1, 2 or 4)
     const int32_t *draft_tokens;  // [B,K]
     const float *uniforms;        // [B,K+1]
     // outputs

@@ -11,12 +11,12 @@ namespace spr {
 // are issued before the current one is consumed).  The CTA that finishes a row last merges
 // the segments, runs the accept test for that position, and the row that finishes a
 // sequence last runs the first-rejection scan.
-template <typename T>
+template <typename T, int ITERS>
 __global__ void __launch_bounds__(kThreads) sd_row_stats_kernel(const SdParams prm)
 {
     constexpr int N = Vec<T>::N;
     constexpr int kStep = 32 * kUnroll * N;
-    constexpr int kSegment = kWarps * kStatIters * kStep;
+    constexpr int kSegment = kWarps * ITERS * kStep;      // ITERS steps per warp: 4, fewer for small batches
     __shared__ float4 s_part[kWarps];
     __shared__ int s_last;
 
@@ -39,9 +39,9 @@ __global__ void __launch_bounds__(kThreads) sd_row_stats_kernel(const SdParams p
     load_step<T>(prow, first_p, V, lane, rp);
     load_step<T>(qrow, first_q, V, lane, rq);
 #pragma unroll
-    for (int it = 0; it < kStatIters; ++it) {
+    for (int it = 0; it < ITERS; ++it) {
         const int nxt = (it + 1) * kWarps * kStep;
-        const bool more = it + 1 < kStatIters && min(first_p, first_q) + nxt < V;   // warp-uniform
+        const bool more = it + 1 < ITERS && min(first_p, first_q) + nxt < V;   // warp-uniform
         online_update<T>(rp, mp.m, mp.s);
         if (more) load_step<T>(prow, first_p + nxt, V, lane, rp);
         online_update<T>(rq, mq.m, mq.s);
@@ -163,10 +163,17 @@ cudaError_t launch_sd_row_stats(const SdParams &sp, int B, int K, int dt, cudaSt
     if (grid > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     if (grid == 0) return cudaSuccess;
     if (g_stage_before) cudaEventRecord(g_stage_before, st);
-    if (dt == SPR_F32)
-        sd_row_stats_kernel<float><<<(unsigned)grid, kThreads, 0, st>>>(sp);
-    else
-        sd_row_stats_kernel<__nv_bfloat16><<<(unsigned)grid, kThreads, 0, st>>>(sp);
+#define SPR_STATS(T_, I_) sd_row_stats_kernel<T_, I_><<<(unsigned)grid, kThreads, 0, st>>>(sp)
+    if (dt == SPR_F32) {
+        if (sp.iters == 4) SPR_STATS(float, 4);
+        else if (sp.iters == 2) SPR_STATS(float, 2);
+        else SPR_STATS(float, 1);
+    } else {
+        if (sp.iters == 4) SPR_STATS(__nv_bfloat16, 4);
+        else if (sp.iters == 2) SPR_STATS(__nv_bfloat16, 2);
+        else SPR_STATS(__nv_bfloat16, 1);
+    }
+#undef SPR_STATS
     const cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess && g_stage_after) cudaEventRecord(g_stage_after, st);
     return e;
