@@ -12,7 +12,7 @@ namespace spr {
 // the segments, runs the accept test for that position, and the row that finishes a
 // sequence last runs the first-rejection scan.
 template <typename T, int ITERS>
-__global__ void __launch_bounds__(kThreads) sd_row_stats_kernel(const SdParams prm)
+__global__ void __launch_bounds__(kThreads, 4) sd_row_stats_kernel(const SdParams prm)
 {
     constexpr int N = Vec<T>::N;
     constexpr int kStep = 32 * kUnroll * N;

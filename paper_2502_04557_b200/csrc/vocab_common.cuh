@@ -133,6 +133,32 @@ __device__ __forceinline__ MS thread_ms(const uint4 (&raw)[kUnroll])
     return r;
 }
 
+// Two fp32 lanes per instruction (sm_100 packed fp32): halves the issue slots of the multiply-
+// add and of the accumulation, which matter here because the exp pipe and the issue rate are
+// the co-limiters of the streaming kernels.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
 // Lane-local online softmax statistics: folds kUnroll vectors into a running (max, sum of
 // exp(x - max)).  When the maximum grows the old sum is rescaled once per call.
 template <typename T>
@@ -145,19 +171,27 @@ __device__ __forceinline__ void online_update(const uint4 (&raw)[kUnroll], float
     const float mn = fmaxf(m, g);
     const float ref = (mn == neg_inf()) ? 0.f : mn;
     const float off = -ref * kLog2e;
-    float acc[kUnroll];
-    acc[0] = s * ex2(fmaf(m, kLog2e, off));   // m = -inf: exp2(-inf) = 0
+    const uint64_t scale2 = pack2(kLog2e, kLog2e), off2 = pack2(off, off);
+    uint64_t acc[kUnroll];
+    acc[0] = pack2(s * ex2(fmaf(m, kLog2e, off)), 0.f);   // m = -inf: exp2(-inf) = 0
 #pragma unroll
-    for (int j = 1; j < kUnroll; ++j) acc[j] = 0.f;
+    for (int j = 1; j < kUnroll; ++j) acc[j] = pack2(0.f, 0.f);
 #pragma unroll
     for (int j = 0; j < kUnroll; ++j) {
         float f[N];
         Vec<T>::unpack(raw[j], f);
 #pragma unroll
-        for (int e = 0; e < N; ++e) acc[j] += ex2(fmaf(f[e], kLog2e, off));
+        for (int e = 0; e < N; e += 2) {
+            float t0, t1;
+            unpack2(fma2(pack2(f[e], f[e + 1]), scale2, off2), t0, t1);
+            acc[j] = add2(acc[j], pack2(ex2(t0), ex2(t1)));
+        }
     }
     m = mn;
-    s = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+    float a0, a1, b0, b1;
+    unpack2(add2(acc[0], acc[1]), a0, a1);
+    unpack2(add2(acc[2], acc[3]), b0, b1);
+    s = (a0 + a1) + (b0 + b1);
 }
 
 // The kUnroll vectors of one warp step: vector j of lane l starts at element
