@@ -69,6 +69,91 @@ int launch_verifier(VerifyParams &vp, int dt, int path, cudaStream_t st)
     return e == cudaSuccess ? SPR_OK : cuda_fail(e);
 }
 
+VerifyParams verify_params(const void *hidden, const void *W1, const float *b1, const void *W2, const float *b2,
+                           float threshold, int B, int K, int d, int h, float *scores, uint8_t *accept,
+                           int32_t *first_reject)
+{
+    VerifyParams vp;
+    memset(&vp, 0, sizeof vp);
+    vp.hidden = hidden;
+    vp.W1 = W1;
+    vp.b1 = b1;
+    vp.W2 = W2;
+    vp.b2 = b2;
+    vp.threshold = threshold;
+    vp.B = B;
+    vp.K = K;
+    vp.d = d;
+    vp.h = h;
+    vp.scores = scores;
+    vp.accept = accept;
+    vp.first_reject = first_reject;
+    return vp;
+}
+
+// sizes first (an empty batch may come with null pointers), then pointers and alignment
+int check_verify_args(const VerifyParams &vp, int dt, int path)
+{
+    if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
+    if (path != SPR_VERIFIER_AUTO && path != SPR_VERIFIER_SIMT && path != SPR_VERIFIER_TENSOR)
+        return SPR_ERR_UNSUPPORTED;
+    if (vp.B < 0 || vp.K <= 0 || vp.d <= 0 || vp.h < 0 || (int64_t)vp.B * vp.K > 0x7fffffff)
+        return SPR_ERR_INVALID_ARG;
+    if (vp.B == 0) return SPR_OK;
+    if (!vp.hidden || !vp.W1 || !vp.b2 || !vp.accept || !vp.first_reject) return SPR_ERR_INVALID_ARG;
+    if (vp.h > 0 && (!vp.b1 || !vp.W2)) return SPR_ERR_INVALID_ARG;
+    const size_t es = elem_size(dt);
+    if (!aligned(vp.hidden, es) || !aligned(vp.W1, es) || (vp.W2 && !aligned(vp.W2, es)) || !aligned(vp.b2, 4) ||
+        (vp.b1 && !aligned(vp.b1, 4)) || (vp.scores && !aligned(vp.scores, 4)) || !aligned(vp.first_reject, 4))
+        return SPR_ERR_INVALID_ARG;
+    return SPR_OK;
+}
+
+int check_replace_args(const DrawParams &dp, int n, int dt)
+{
+    if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
+    if (dp.V <= 0 || dp.V > kMaxVocab || dp.ldv < dp.V || dp.R < 0 || n < 0 || dp.seq_stride < 0)
+        return SPR_ERR_INVALID_ARG;
+    if (n == 0) return SPR_OK;
+    if (!dp.p || !dp.uniforms || !dp.tokens || dp.R == 0) return SPR_ERR_INVALID_ARG;
+    if (dp.gate && dp.K <= 0) return SPR_ERR_INVALID_ARG;
+    if (!aligned(dp.p, elem_size(dt)) || !aligned(dp.uniforms, 4) || !aligned(dp.tokens, 4) ||
+        (dp.rows && !aligned(dp.rows, 4)) || (dp.gate && !aligned(dp.gate, 4)))
+        return SPR_ERR_INVALID_ARG;
+    return SPR_OK;
+}
+
+}  // namespace
+
+namespace spr {
+// everything of a replacement draw except the scratch pointers
+DrawParams replace_params(const void *target_logits, int64_t ldv, int V, int64_t R, const int32_t *rows,
+                          const int32_t *first_reject, int K, int seq_stride, int n, const float *uniforms,
+                          int dt, int32_t *tokens)
+{
+    DrawParams dp;
+    memset(&dp, 0, sizeof dp);
+    dp.kind = DRAW_REPLACE;
+    dp.p = target_logits;
+    dp.ldv = ldv;
+    dp.V = V;
+    dp.R = R;
+    dp.rows = rows;
+    dp.gate = first_reject;
+    dp.seq_stride = seq_stride;
+    dp.K = K;
+    dp.uniforms = uniforms;
+    dp.tokens = tokens;
+    if (V > 0 && n >= 0 && dtype_ok(dt)) {
+        dp.steps = stat_steps_per_row(V, dt);
+        draw_geometry(n, dp.steps, &dp.chunks, &dp.iters);
+    }
+    return dp;
+}
+}  // namespace spr
+
+namespace {
+
 size_t verify_ws_bytes(int B, int K, int h)
 {
     const int M = B * K;
@@ -112,46 +197,19 @@ int sprinter_verify(const void *hidden, const void *W1, const float *b1, const v
                     float *scores, uint8_t *accept, int32_t *first_reject, void *ws, size_t ws_bytes,
                     void *cuda_stream)
 {
-    if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
-    if (path != SPR_VERIFIER_AUTO && path != SPR_VERIFIER_SIMT && path != SPR_VERIFIER_TENSOR)
-        return SPR_ERR_UNSUPPORTED;
-    if (B < 0 || K <= 0 || d <= 0 || h < 0 || (int64_t)B * K > 0x7fffffff) return SPR_ERR_INVALID_ARG;
-    if (B == 0) return SPR_OK;  // empty batch: nothing to read or write, pointers may be null
-    if (!hidden || !W1 || !b2 || !accept || !first_reject) return SPR_ERR_INVALID_ARG;
-    if (h > 0 && (!b1 || !W2)) return SPR_ERR_INVALID_ARG;
-    const size_t es = elem_size(dt);
-    if (!aligned(hidden, es) || !aligned(W1, es) || (W2 && !aligned(W2, es)) || !aligned(b2, 4) ||
-        (b1 && !aligned(b1, 4)) || (scores && !aligned(scores, 4)) || !aligned(first_reject, 4))
-        return SPR_ERR_INVALID_ARG;
-    if (!ws || !aligned(ws, 256) || ws_bytes < verify_ws_bytes(B, K, h)) return SPR_ERR_WORKSPACE;
-    int rc = check_device();
-    if (rc != SPR_OK) return rc;
-    if (B == 0) return SPR_OK;
+    VerifyParams vp = verify_params(hidden, W1, b1, W2, b2, threshold, B, K, d, h, scores, accept, first_reject);
+    int rc = check_verify_args(vp, dt, path);
+    if (rc != SPR_OK || B == 0) return rc;  // empty batch: nothing to read or write
+    const VerifyWs lay = verify_ws_layout(B * K, verifier_simt_slices(h), (B * K + 63) / 64);
+    if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
+    if ((rc = check_device()) != SPR_OK) return rc;
 
-    const int M = B * K;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    VerifyParams vp;
-    memset(&vp, 0, sizeof vp);
-    vp.hidden = hidden;
-    vp.W1 = W1;
-    vp.b1 = b1;
-    vp.W2 = W2;
-    vp.b2 = b2;
-    vp.threshold = threshold;
-    vp.B = B;
-    vp.K = K;
-    vp.d = d;
-    vp.h = h;
-    vp.scores = scores;
-    vp.accept = accept;
-    vp.first_reject = first_reject;
     vp.status = at<int>(ws, 0);
-    const VerifyWs lay = verify_ws_layout(M, verifier_simt_slices(h), (M + 63) / 64);
     vp.counter = at<int>(ws, lay.counter);
     vp.part_z = at<float>(ws, lay.part_z);
-    cudaError_t ce = cudaMemsetAsync(vp.counter, 0, lay.counters_end - lay.counter, st);
-    if (ce != cudaSuccess) return cuda_fail(ce);
-
+    cudaError_t e = cudaMemsetAsync(vp.counter, 0, lay.counters_end - lay.counter, st);
+    if (e != cudaSuccess) return cuda_fail(e);
     return launch_verifier(vp, dt, path, st);
 }
 
@@ -159,43 +217,18 @@ int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, con
                    const int32_t *first_reject, int K, int seq_stride, int n, const float *uniforms,
                    int dt, int32_t *tokens, void *ws, size_t ws_bytes, void *cuda_stream)
 {
-    if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
-    if (V <= 0 || V > kMaxVocab || ldv < V || R < 0 || n < 0 || seq_stride < 0) return SPR_ERR_INVALID_ARG;
-    if (n == 0) return SPR_OK;  // no draws: pointers may be null
-    if (!target_logits || !uniforms || !tokens || R == 0) return SPR_ERR_INVALID_ARG;
-    if (first_reject && K <= 0) return SPR_ERR_INVALID_ARG;
-    if (!aligned(target_logits, elem_size(dt)) || !aligned(uniforms, 4) || !aligned(tokens, 4) ||
-        (rows && !aligned(rows, 4)) || (first_reject && !aligned(first_reject, 4)))
-        return SPR_ERR_INVALID_ARG;
-    const int T = stat_steps_per_row(V, dt);
-    int C, iters;
-    draw_geometry(n, T, &C, &iters);
-    const DrawWs lay = replace_ws_layout(n, T);
+    DrawParams dp = replace_params(target_logits, ldv, V, R, rows, first_reject, K, seq_stride, n, uniforms, dt,
+                                   tokens);
+    int rc = check_replace_args(dp, n, dt);
+    if (rc != SPR_OK || n == 0) return rc;  // no draws: pointers may be null
+    const DrawWs lay = replace_ws_layout(n, dp.steps);
     if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
-    int rc = check_device();
-    if (rc != SPR_OK) return rc;
-    if (n == 0) return SPR_OK;
+    if ((rc = check_device()) != SPR_OK) return rc;
 
-    DrawParams dp;
-    memset(&dp, 0, sizeof dp);
-    dp.kind = DRAW_REPLACE;
-    dp.p = target_logits;
-    dp.ldv = ldv;
-    dp.V = V;
-    dp.chunks = C;
-    dp.iters = iters;
-    dp.R = R;
-    dp.rows = rows;
-    dp.gate = first_reject;
-    dp.seq_stride = seq_stride;
-    dp.K = K;
-    dp.uniforms = uniforms;
-    dp.tokens = tokens;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     dp.status = at<int>(ws, 0);
     dp.counters = at<int>(ws, lay.counters);
-    dp.steps = T;
     dp.part = at<float2>(ws, lay.part);
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaMemsetAsync(dp.counters, 0, sizeof(int) * (size_t)n, st);
     if (e == cudaSuccess) e = launch_draw(dp, n, dt, st);
     return e == cudaSuccess ? SPR_OK : cuda_fail(e);
@@ -207,74 +240,28 @@ int sprinter_step(const void *hidden, const void *W1, const float *b1, const voi
                   uint8_t *accept, int32_t *first_reject, int32_t *tokens, void *ws, size_t ws_bytes,
                   void *cuda_stream)
 {
-    if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
-    if (path != SPR_VERIFIER_AUTO && path != SPR_VERIFIER_SIMT && path != SPR_VERIFIER_TENSOR)
-        return SPR_ERR_UNSUPPORTED;
-    if (B < 0 || K <= 0 || d <= 0 || h < 0 || V <= 0 || V > kMaxVocab || ldv < V || seq_stride < K ||
-        (int64_t)B * K > 0x7fffffff)
-        return SPR_ERR_INVALID_ARG;
-    if (B == 0) return SPR_OK;
-    if (!hidden || !W1 || !b2 || !accept || !first_reject || !target_logits || !uniforms || !tokens)
-        return SPR_ERR_INVALID_ARG;
-    if (h > 0 && (!b1 || !W2)) return SPR_ERR_INVALID_ARG;
-    const size_t es = elem_size(dt);
-    if (!aligned(hidden, es) || !aligned(W1, es) || (W2 && !aligned(W2, es)) || !aligned(b2, 4) ||
-        (b1 && !aligned(b1, 4)) || (scores && !aligned(scores, 4)) || !aligned(first_reject, 4) ||
-        !aligned(target_logits, es) || !aligned(uniforms, 4) || !aligned(tokens, 4))
-        return SPR_ERR_INVALID_ARG;
-    const int M = B * K;
-    const int T = stat_steps_per_row(V, dt);
-    int C, iters;
-    draw_geometry(B, T, &C, &iters);
-    const StepWs lay = step_ws_layout(B, K, verifier_simt_slices(h), (M + 63) / 64, T);
-    if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
-    int rc = check_device();
+    VerifyParams vp = verify_params(hidden, W1, b1, W2, b2, threshold, B, K, d, h, scores, accept, first_reject);
+    int rc = check_verify_args(vp, dt, path);
     if (rc != SPR_OK) return rc;
+    if (seq_stride < K) return SPR_ERR_INVALID_ARG;
+    DrawParams dp = replace_params(target_logits, ldv, V, (int64_t)B * seq_stride, nullptr, first_reject, K,
+                                   seq_stride, B, uniforms, dt, tokens);
+    rc = check_replace_args(dp, B, dt);
+    if (rc != SPR_OK || B == 0) return rc;
+    const StepWs lay = step_ws_layout(B, K, verifier_simt_slices(h), (B * K + 63) / 64, dp.steps);
+    if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
+    if ((rc = check_device()) != SPR_OK) return rc;
 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    VerifyParams vp;
-    memset(&vp, 0, sizeof vp);
-    vp.hidden = hidden;
-    vp.W1 = W1;
-    vp.b1 = b1;
-    vp.W2 = W2;
-    vp.b2 = b2;
-    vp.threshold = threshold;
-    vp.B = B;
-    vp.K = K;
-    vp.d = d;
-    vp.h = h;
-    vp.scores = scores;
-    vp.accept = accept;
-    vp.first_reject = first_reject;
-    vp.status = at<int>(ws, 0);
+    vp.status = dp.status = at<int>(ws, 0);
     vp.counter = at<int>(ws, lay.verify_counter);
     vp.part_z = at<float>(ws, lay.part_z);
-
-    DrawParams dp;
-    memset(&dp, 0, sizeof dp);
-    dp.kind = DRAW_REPLACE;
-    dp.p = target_logits;
-    dp.ldv = ldv;
-    dp.V = V;
-    dp.chunks = C;
-    dp.iters = iters;
-    dp.steps = T;
-    dp.R = (int64_t)B * seq_stride;
-    dp.gate = first_reject;
-    dp.seq_stride = seq_stride;
-    dp.K = K;
-    dp.uniforms = uniforms;
-    dp.tokens = tokens;
-    dp.status = vp.status;
     dp.counters = at<int>(ws, lay.draw.counters);
     dp.part = at<float2>(ws, lay.draw.part);
-
     // one clear for both kernels' tickets, then the draw is launched behind the verifier
     cudaError_t e = cudaMemsetAsync(vp.counter, 0, lay.counters_end - lay.verify_counter, st);
     if (e != cudaSuccess) return cuda_fail(e);
-    rc = launch_verifier(vp, dt, path, st);
-    if (rc != SPR_OK) return rc;
+    if ((rc = launch_verifier(vp, dt, path, st)) != SPR_OK) return rc;
     e = launch_draw(dp, B, dt, st, /*after_kernel=*/true);
     return e == cudaSuccess ? SPR_OK : cuda_fail(e);
 }

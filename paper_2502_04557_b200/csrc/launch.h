@@ -84,6 +84,10 @@ cudaError_t launch_simulate(const SimParams &sp, cudaStream_t st);
 cudaError_t launch_sd_row_stats(const SdParams &sp, int B, int K, int dt, cudaStream_t st);
 int report_cuda_error(cudaError_t e);  // records the text, returns SPR_ERR_CUDA
 void set_stage_events(cudaEvent_t before, cudaEvent_t after);
+// everything of a replacement draw except the scratch pointers (status, counters, part)
+DrawParams replace_params(const void *target_logits, int64_t ldv, int V, int64_t R, const int32_t *rows,
+                          const int32_t *first_reject, int K, int seq_stride, int n, const float *uniforms,
+                          int dt, int32_t *tokens);
 // after_kernel: the launch directly follows, in the same stream, the kernel whose output
 // selects the rows (programmatic dependent launch)
 cudaError_t launch_draw(const DrawParams &dp, int n, int dt, cudaStream_t st, bool after_kernel = false);

@@ -60,11 +60,10 @@ extern "C" int replace_sample_static(const void *target_logits, int64_t ldv, int
         reinterpret_cast<uintptr_t>(tokens) % 4 || (rows && reinterpret_cast<uintptr_t>(rows) % 4) ||
         (first_reject && reinterpret_cast<uintptr_t>(first_reject) % 4))
         return SPR_ERR_INVALID_ARG;
-    const int T = stat_steps_per_row(V, dt);
-    int C, iters;
-    draw_geometry(n, T, &C, &iters);
+    DrawParams dp = replace_params(target_logits, ldv, V, R, rows, first_reject, K, seq_stride, n, uniforms, dt,
+                                   tokens);
     // the built-in scratch has room for kMaxDraws tickets and kMaxDrawSteps step partials
-    if (n > kMaxDraws || (int64_t)n * T > kMaxDrawSteps) return SPR_ERR_WORKSPACE;
+    if (n > kMaxDraws || (int64_t)n * dp.steps > kMaxDrawSteps) return SPR_ERR_WORKSPACE;
 
     int major = 0, dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -76,25 +75,8 @@ extern "C" int replace_sample_static(const void *target_logits, int64_t ldv, int
     int rc = scratch_for_current_device(&base);
     if (rc != SPR_OK) return rc;
     char *scratch = static_cast<char *>(base);
-
-    DrawParams dp;
-    memset(&dp, 0, sizeof dp);
-    dp.kind = DRAW_REPLACE;
-    dp.p = target_logits;
-    dp.ldv = ldv;
-    dp.V = V;
-    dp.chunks = C;
-    dp.iters = iters;
-    dp.R = R;
-    dp.rows = rows;
-    dp.gate = first_reject;
-    dp.seq_stride = seq_stride;
-    dp.K = K;
-    dp.uniforms = uniforms;
-    dp.tokens = tokens;
     dp.status = reinterpret_cast<int *>(scratch);
     dp.counters = reinterpret_cast<int *>(scratch + kOffCounters);
-    dp.steps = T;
     dp.part = reinterpret_cast<float2 *>(scratch + kOffPart);
 
     // The array keeps whatever the previous call left: the tickets must start at zero (the
