@@ -544,3 +544,33 @@ def test_very_large_vocabulary(spr, dtype, V):
     want = oracle.replace_sample(R, V, uu.numpy())
     eq(got, want, "tokens")
     assert want[0] >= V - 5000
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_sd_rows_with_huge_dynamic_range(spr, dtype):
+    """Logits that jump by far more than exp() can hold in fp32 between the start and the rest
+    of a row (and rows that start with -inf): the row statistics must stay exact."""
+    B, K, V = 4, 2, 70_001
+    p, q, x, u = _rand_problem(B, K, V, dtype, seed=77, Kp=K, scale=2.0)
+    p[0, 0, :40_000] -= 150.0            # everything the first steps see is e^-150 below the rest
+    q[0, 1, :20_000] = float("-inf")     # a masked prefix
+    p[1, 0, 5_000:] += 120.0
+    q[2, 1, 60_000:] += 200.0
+    p[3, 1, :] -= 300.0                  # a uniformly tiny row
+    x[0, 0] = 50_000
+    x[0, 1] = 30_000
+    x[2, 1] = 65_000
+    ref = _clear_sd(p, q, V, x, u)
+    ws = spr.Workspace(spr.workspace_bytes(2, B, K, V, 1, 0, spr.binding._dt(p)))
+    out = spr.sd_verify(p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), ws)
+    assert ws.device_status() == 0
+    eq(out["accept"], ref["accept"], "accept")
+    eq(out["accepted_len"], ref["accepted_len"], "accepted_len")
+    eq(out["correction_token"], ref["correction_token"], "correction_token")
+    ok = ref["p_tok"] > 1e-30
+    got_p = out["p_tok"].cpu().double().numpy()
+    assert np.all(np.abs(got_p[ok] - ref["p_tok"][ok]) <= RTOL[dtype] * ref["p_tok"][ok])
+    ok = ref["q_tok"] > 1e-30
+    got_q = out["q_tok"].cpu().double().numpy()
+    assert np.all(np.abs(got_q[ok] - ref["q_tok"][ok]) <= RTOL[dtype] * ref["q_tok"][ok])
+    assert_close_rel(out["residual_mass"], ref["residual_mass"], RTOL[dtype], "residual_mass")
