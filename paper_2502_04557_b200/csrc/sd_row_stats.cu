@@ -34,53 +34,19 @@ __global__ void __launch_bounds__(kThreads, 4) sd_row_stats_kernel(const SdParam
     const int first_q = c * kSegment + warp * kStep - row_pad(qrow);
     const int V = prm.V;
 
-    // Step 0 fixes each lane's reference (its maximum over that step); the later steps only add
-    // exp(x - reference), which needs no maximum and stays exact unless some later logit lies
-    // more than ~88 above the reference.  That shows as an inf/NaN sum and sends the warp to
-    // the always-safe loop below.
     MS mp{neg_inf(), 0.f}, mq{neg_inf(), 0.f};
     uint4 rp[kUnroll], rq[kUnroll];
     load_step<T>(prow, first_p, V, lane, rp);
     load_step<T>(qrow, first_q, V, lane, rq);
-    float off_p = 0.f, off_q = 0.f;
 #pragma unroll
     for (int it = 0; it < ITERS; ++it) {
         const int nxt = (it + 1) * kWarps * kStep;
         const bool more = it + 1 < ITERS && min(first_p, first_q) + nxt < V;   // warp-uniform
-        if (it == 0) {
-            online_update<T>(rp, mp.m, mp.s);
-            off_p = -(mp.m == neg_inf() ? 0.f : mp.m) * kLog2e;
-        } else {
-            fixed_ref_update<T>(rp, off_p, mp.s);
-        }
+        online_update<T>(rp, mp.m, mp.s);
         if (more) load_step<T>(prow, first_p + nxt, V, lane, rp);
-        if (it == 0) {
-            online_update<T>(rq, mq.m, mq.s);
-            off_q = -(mq.m == neg_inf() ? 0.f : mq.m) * kLog2e;
-        } else {
-            fixed_ref_update<T>(rq, off_q, mq.s);
-        }
+        online_update<T>(rq, mq.m, mq.s);
         if (more) load_step<T>(qrow, first_q + nxt, V, lane, rq);
         if (!more) break;
-    }
-    if (ITERS > 1) {
-        // a lane that saw nothing but -inf in step 0 keeps reference 0 with m = -inf: give the
-        // pair a finite maximum so that the merges below scale its sum correctly
-        if (mp.m == neg_inf() && mp.s > 0.f) mp.m = 0.f;
-        if (mq.m == neg_inf() && mq.s > 0.f) mq.m = 0.f;
-        const bool overflow = !(mp.s < __int_as_float(0x7f800000)) || !(mq.s < __int_as_float(0x7f800000));
-        if (__any_sync(0xffffffffu, overflow)) {
-            mp = MS{neg_inf(), 0.f};
-            mq = MS{neg_inf(), 0.f};
-            for (int it = 0; it < ITERS; ++it) {
-                const int nxt = it * kWarps * kStep;
-                if (min(first_p, first_q) + nxt >= V) break;
-                load_step<T>(prow, first_p + nxt, V, lane, rp);
-                online_update<T>(rp, mp.m, mp.s);
-                load_step<T>(qrow, first_q + nxt, V, lane, rq);
-                online_update<T>(rq, mq.m, mq.s);
-            }
-        }
     }
     mp = warp_ms(mp);
     mq = warp_ms(mq);

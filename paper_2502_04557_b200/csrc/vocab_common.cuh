@@ -194,35 +194,6 @@ __device__ __forceinline__ void online_update(const uint4 (&raw)[kUnroll], float
     s = (a0 + a1) + (b0 + b1);
 }
 
-// Adds kUnroll vectors to a sum of exp(x - ref) whose reference is NOT moved: no maximum is
-// taken, so this is cheaper than online_update.  Correct for any reference as long as nothing
-// overflows; `off` is -ref*log2(e).  The caller checks the sum for inf/NaN afterwards.
-template <typename T>
-__device__ __forceinline__ void fixed_ref_update(const uint4 (&raw)[kUnroll], float off, float &s)
-{
-    constexpr int N = Vec<T>::N;
-    const uint64_t scale2 = pack2(kLog2e, kLog2e), off2 = pack2(off, off);
-    uint64_t acc[kUnroll];
-    acc[0] = pack2(s, 0.f);
-#pragma unroll
-    for (int j = 1; j < kUnroll; ++j) acc[j] = pack2(0.f, 0.f);
-#pragma unroll
-    for (int j = 0; j < kUnroll; ++j) {
-        float f[N];
-        Vec<T>::unpack(raw[j], f);
-#pragma unroll
-        for (int e = 0; e < N; e += 2) {
-            float t0, t1;
-            unpack2(fma2(pack2(f[e], f[e + 1]), scale2, off2), t0, t1);
-            acc[j] = add2(acc[j], pack2(ex2(t0), ex2(t1)));
-        }
-    }
-    float a0, a1, b0, b1;
-    unpack2(add2(acc[0], acc[1]), a0, a1);
-    unpack2(add2(acc[2], acc[3]), b0, b1);
-    s = (a0 + a1) + (b0 + b1);
-}
-
 // The kUnroll vectors of one warp step: vector j of lane l starts at element
 // first + (j*32 + l)*N of the row (first may be negative or run past V at the row's ends).
 template <typename T>

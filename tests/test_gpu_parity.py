@@ -573,4 +573,5 @@ def test_sd_rows_with_huge_dynamic_range(spr, dtype):
     ok = ref["q_tok"] > 1e-30
     got_q = out["q_tok"].cpu().double().numpy()
     assert np.all(np.abs(got_q[ok] - ref["q_tok"][ok]) <= RTOL[dtype] * ref["q_tok"][ok])
-    assert_close_rel(out["residual_mass"], ref["residual_mass"], RTOL[dtype], "residual_mass")
+    # logits of magnitude ~300 carry an absolute fp32 rounding error of ~2e-5 into the exponent
+    assert_close_rel(out["residual_mass"], ref["residual_mass"], max(RTOL[dtype], 1e-4), "residual_mass")
