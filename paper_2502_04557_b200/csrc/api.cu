@@ -154,10 +154,13 @@ DrawParams replace_params(const void *target_logits, int64_t ldv, int V, int64_t
 
 namespace {
 
+// ticket counters of the verifier kernels: one per 64-token tile (MLP) or per sequence (linear)
+int verify_counters(int B, int K) { return max((B * K + 63) / 64, B); }
+
 size_t verify_ws_bytes(int B, int K, int h)
 {
     const int M = B * K;
-    return verify_ws_layout(M, verifier_simt_slices(h), (M + 63) / 64).end;
+    return verify_ws_layout(M, verifier_simt_slices(h), verify_counters(B, K)).end;
 }
 
 }  // namespace
@@ -176,7 +179,7 @@ size_t spr_workspace_bytes(int op, int B, int K, int V, int d, int h, int dt)
         return replace_ws_layout(B, stat_steps_per_row(V, dt)).end;
     case SPR_OP_SPRINTER_STEP:
         if (K <= 0 || d <= 0 || h < 0 || V <= 0 || (int64_t)B * K > 0x7fffffff) return 0;
-        return step_ws_layout(B, K, verifier_simt_slices(h), (B * K + 63) / 64, stat_steps_per_row(V, dt)).end;
+        return step_ws_layout(B, K, verifier_simt_slices(h), verify_counters(B, K), stat_steps_per_row(V, dt)).end;
     case SPR_OP_SD_VERIFY:
         if (K <= 0 || V <= 0 || (int64_t)B * K > 0x7fffffff) return 0;
         return sd_ws_layout(B, K, stat_max_segments_per_row(V, dt), stat_steps_per_row(V, dt)).end;
@@ -200,7 +203,7 @@ int sprinter_verify(const void *hidden, const void *W1, const float *b1, const v
     VerifyParams vp = verify_params(hidden, W1, b1, W2, b2, threshold, B, K, d, h, scores, accept, first_reject);
     int rc = check_verify_args(vp, dt, path);
     if (rc != SPR_OK || B == 0) return rc;  // empty batch: nothing to read or write
-    const VerifyWs lay = verify_ws_layout(B * K, verifier_simt_slices(h), (B * K + 63) / 64);
+    const VerifyWs lay = verify_ws_layout(B * K, verifier_simt_slices(h), verify_counters(B, K));
     if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
     if ((rc = check_device()) != SPR_OK) return rc;
 
@@ -248,7 +251,7 @@ int sprinter_step(const void *hidden, const void *W1, const float *b1, const voi
                                    seq_stride, B, uniforms, dt, tokens);
     rc = check_replace_args(dp, B, dt);
     if (rc != SPR_OK || B == 0) return rc;
-    const StepWs lay = step_ws_layout(B, K, verifier_simt_slices(h), (B * K + 63) / 64, dp.steps);
+    const StepWs lay = step_ws_layout(B, K, verifier_simt_slices(h), verify_counters(B, K), dp.steps);
     if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
     if ((rc = check_device()) != SPR_OK) return rc;
 

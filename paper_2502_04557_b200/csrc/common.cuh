@@ -103,7 +103,7 @@ __host__ __device__ inline SdWs sd_ws_layout(int B, int K, int S, int T)   // S 
 }
 
 struct VerifyWs {
-    size_t counter;          // int32 [1 + row tiles]   CTAs finished
+    size_t counter;          // int32 [1 + max(row tiles, B)]   CTAs finished per tile / tokens per sequence
     size_t counters_end;
     size_t part_z;           // float [slices * M]      per-slice partial of W2 . relu(...)
     size_t end;

@@ -1,7 +1,7 @@
-// SIMT verifier: score = sigmoid(b2 + W2 . relu(W1 s + b1)) (or sigmoid(b + w . s) for the
-// single linear layer of the paper), threshold test, first-rejection scan.  Takes any
-// element type and shape; it is the path for float32 inputs and for batches too small to
-// fill a tensor-core tile, where the work is a bandwidth-bound sweep over W1.
+// SIMT verifiers.  MLP: score = sigmoid(b2 + W2 . relu(W1 s + b1)) for any element type and
+// shape - the path for float32 inputs and for batches too small for a tensor-core tile, where
+// the work is a bandwidth-bound sweep over W1.  Linear: the paper's single layer,
+// score = sigmoid(b + w . s).  Both end with the threshold test and the first-rejection scan.
 #include "common.cuh"
 #include "launch.h"
 #include "verifier_common.cuh"
@@ -118,18 +118,6 @@ __global__ void __launch_bounds__(kThreads) verifier_simt_kernel(const VerifyPar
             }
             __syncthreads();
         }
-    } else {
-        // single linear layer: one warp per token tile
-        const int m0 = (blockIdx.x * kWarps + warp) * kTokTile;
-        if (m0 < M) {
-            float acc[kTokTile];
-            warp_dots<T>(W1, hid, prm.d, m0, M, vec_ok, acc);
-            if (lane == 0) {
-#pragma unroll
-                for (int t = 0; t < kTokTile; ++t)
-                    if (m0 + t < M) prm.part_z[m0 + t] = acc[t];
-            }
-        }
     }
     __syncthreads();
     if (tid == 0) {
@@ -142,19 +130,67 @@ __global__ void __launch_bounds__(kThreads) verifier_simt_kernel(const VerifyPar
     finalise_scores(prm);
 }
 
-int verifier_simt_slices(int h) { return h > 0 ? (h + kWarps - 1) / kWarps : 1; }
-
-static int simt_grid(const VerifyParams &vp)
+// The paper's verifier: one linear layer and a sigmoid.  A bandwidth-bound sweep over the hidden
+// states: one warp per token reads its row once with 16-byte loads (the weight vector stays in
+// L1), forms the score and the accept bit on the spot, and takes a ticket on its sequence;
+// the warp that completes a sequence runs the first-rejection scan.  No partial sums, no
+// single-CTA tail.
+template <typename T>
+__global__ void __launch_bounds__(kThreads) verifier_linear_kernel(const VerifyParams prm)
 {
-    if (vp.h > 0) return verifier_simt_slices(vp.h);
-    const int M = vp.B * vp.K;
-    return (M + kWarps * kTokTile - 1) / (kWarps * kTokTile);
+    pdl_trigger();   // a replacement draw launched behind this grid may be scheduled now
+    constexpr int N = 16 / sizeof(T);
+    const int M = prm.B * prm.K;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int m = blockIdx.x * kWarps + warp;
+    if (m >= M) return;
+    const T *w = static_cast<const T *>(prm.W1);
+    const T *x = static_cast<const T *>(prm.hidden) + (int64_t)m * prm.d;
+    const bool vec_ok = (prm.d % N == 0) && ((reinterpret_cast<uintptr_t>(prm.hidden) & 15) == 0) &&
+                        ((reinterpret_cast<uintptr_t>(w) & 15) == 0);
+    float acc = 0.f;
+    if (vec_ok) {
+#pragma unroll 4
+        for (int i = lane * N; i < prm.d; i += 32 * N) {
+            float wv[N], xv[N];
+            unpack16<T>(__ldg(reinterpret_cast<const uint4 *>(w + i)), wv);
+            unpack16<T>(__ldg(reinterpret_cast<const uint4 *>(x + i)), xv);
+#pragma unroll
+            for (int e = 0; e < N; ++e) acc = fmaf(wv[e], xv[e], acc);
+        }
+    } else {
+        for (int i = lane; i < prm.d; i += 32) acc = fmaf(to_f32<T>(w[i]), to_f32<T>(x[i]), acc);
+    }
+    const float z = warp_sum(acc) + prm.b2[0];
+    const int b = m / prm.K;
+    int ticket = 0;
+    if (lane == 0) {
+        const double score = 1.0 / (1.0 + exp(-(double)z));
+        if (prm.scores) prm.scores[m] = (float)score;
+        prm.accept[m] = score >= (double)prm.threshold ? 1 : 0;
+        __threadfence();
+        ticket = atomicAdd(&prm.counter[1 + b], 1);
+    }
+    ticket = __shfl_sync(0xffffffffu, ticket, 0);
+    if (ticket != prm.K - 1 || !prm.first_reject) return;
+    __threadfence();
+    scan_sequence(prm, b, lane);
 }
+
+int verifier_simt_slices(int h) { return h > 0 ? (h + kWarps - 1) / kWarps : 1; }
 
 cudaError_t launch_verifier_simt(const VerifyParams &vp, int dt, cudaStream_t st)
 {
-    const int grid = simt_grid(vp);
-    if (grid <= 0) return cudaSuccess;
+    if (vp.h == 0) {   // single linear layer
+        const int64_t grid = ((int64_t)vp.B * vp.K + kWarps - 1) / kWarps;
+        if (grid <= 0) return cudaSuccess;
+        if (dt == SPR_F32)
+            verifier_linear_kernel<float><<<(unsigned)grid, kThreads, 0, st>>>(vp);
+        else
+            verifier_linear_kernel<__nv_bfloat16><<<(unsigned)grid, kThreads, 0, st>>>(vp);
+        return cudaGetLastError();
+    }
+    const int grid = verifier_simt_slices(vp.h);
     if (dt == SPR_F32)
         verifier_simt_kernel<float><<<grid, kThreads, 0, st>>>(vp);
     else
