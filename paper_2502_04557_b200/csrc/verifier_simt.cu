@@ -48,7 +48,8 @@ __device__ __forceinline__ void warp_dots(const T *__restrict__ wrow, const T *_
 #pragma unroll
     for (int t = 0; t < kTokTile; ++t) acc[t] = 0.f;
     if (vec_ok) {
-        for (int i = lane * N; i < d; i += 32 * N) {
+#pragma unroll 4
+        for (int i = lane * N; i < d; i += 32 * N) {   // several weight vectors in flight per lane
             float w[N];
             unpack16<T>(__ldg(reinterpret_cast<const uint4 *>(wrow + i)), w);
 #pragma unroll
