@@ -180,11 +180,14 @@ def run_reference(args):
     dt = (time.perf_counter() - t0) / max(args.steps, 1)
     value = sample * wl.K / dt
     desc = f"{sample} sequences ({sample * wl.K} draft tokens) of the workload per step"
+    c = wl.cfg
+    full_label = (f"{c.name}: B={c.B} K={c.K} V={c.V} d={c.d} h={c.h} {str(c.dtype).split('.')[-1]} "
+                  f"(per GPU), Kp={wl.Kp}")
     print(json.dumps({
         "impl": "reference", "metric": "verified_tokens_per_s", "value": value, "unit": "tokens/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": {"workload": workload_label(wl), "sample": desc},
+        "data": "synthetic", "config": {"workload": full_label, "sample": desc},
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": 1, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
