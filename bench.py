@@ -30,10 +30,10 @@ if ROOT not in sys.path:
 # capture summarised under profiles/; reported only while the kernel source is unchanged.
 NCU_TRAFFIC = {
     "sources": ("sd_row_stats.cu", "vocab_common.cuh", "common.cuh"),
-    "sha256": "7a0264a12ad9f730d10325ef514e4549e5abd5e8f0722d8a22f1cce9de696c17",
-    # (262,795,520 read + 3,676,160 written) / 512 tokens in the B = 32 capture; traffic grows
+    "sha256": "305fa9cc1ad14a54eff43ef35244ff5a54f29d60c2e39741ebbf1d4395d0983f",
+    # (262,767,616 read + 3,982,336 written) / 512 tokens in the B = 32 capture; traffic grows
     # in proportion to the tokens, so a full launch is this times B*K
-    "bytes_per_unit": 520452,   # DRAM bytes per verified token at V = 128256, bf16
+    "bytes_per_unit": 520996,   # DRAM bytes per verified token at V = 128256, bf16
 }
 
 
