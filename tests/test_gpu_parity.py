@@ -575,3 +575,39 @@ def test_sd_rows_with_huge_dynamic_range(spr, dtype):
     assert np.all(np.abs(got_q[ok] - ref["q_tok"][ok]) <= RTOL[dtype] * ref["q_tok"][ok])
     # logits of magnitude ~300 carry an absolute fp32 rounding error of ~2e-5 into the exponent
     assert_close_rel(out["residual_mass"], ref["residual_mass"], max(RTOL[dtype], 1e-4), "residual_mass")
+
+
+def test_host_buffer_entry_points(spr):
+    """The *_host calls (host pointers in, host pointers out) give the same bits as the device calls."""
+    wl_cpu = spr.workloads.make("gpt2", "cpu", B=5)
+    wl = to_device(wl_cpu)
+    cfg = wl.cfg
+    B, K, V = wl.B, wl.K, wl.V
+    ws = spr.Workspace.for_problem(B, K, V, cfg.d, cfg.h, spr.BF16)
+    arena = spr.Arena(max(spr.host_arena_bytes(2, B, K, wl.Kp, wl.ldv, 0, 0, spr.BF16),
+                          spr.host_arena_bytes(0, B, K, 0, 0, cfg.d, cfg.h, spr.BF16),
+                          spr.host_arena_bytes(1, B, 0, 0, wl.ldv, 0, 0, spr.BF16)))
+    pin = lambda t: t.contiguous().pin_memory()   # noqa: E731
+    s_h, a_h, fr_h = spr.sprinter_verify_host(pin(wl_cpu.hidden), pin(wl_cpu.W1), pin(wl_cpu.b1), pin(wl_cpu.W2),
+                                              pin(wl_cpu.b2), 0.5, arena, ws)
+    s_d, a_d, fr_d = spr.sprinter_verify(wl.hidden, wl.W1, wl.b1, wl.W2, wl.b2, 0.5, ws)
+    assert torch.equal(s_h, s_d.cpu()) and torch.equal(a_h, a_d.cpu()) and torch.equal(fr_h, fr_d.cpu())
+    t_h = spr.replace_sample_host(pin(wl_cpu.p_logits), V, pin(wl_cpu.u_replace), arena, ws, first_reject=fr_h,
+                                  K=K, seq_stride=wl.Kp)
+    t_d = spr.replace_sample(wl.p_logits, V, wl.u_replace, ws, first_reject=fr_d, K=K, seq_stride=wl.Kp)
+    assert torch.equal(t_h, t_d.cpu())
+    o_h = spr.sd_verify_host(pin(wl_cpu.p_logits), pin(wl_cpu.q_logits), V, pin(wl_cpu.draft_tokens),
+                             pin(wl_cpu.uniforms), arena, ws, extras=True)
+    o_d = spr.sd_verify(wl.p_logits, wl.q_logits, V, wl.draft_tokens, wl.uniforms, ws)
+    for k in o_d:
+        assert torch.equal(o_h[k], o_d[k].cpu()), k
+    # device-detected problems come back as the return status of the host call
+    bad = wl_cpu.draft_tokens.clone()
+    bad[0, 0] = V
+    with pytest.raises(spr.SprinterError) as e:
+        spr.sd_verify_host(pin(wl_cpu.p_logits), pin(wl_cpu.q_logits), V, pin(bad), pin(wl_cpu.uniforms), arena, ws)
+    assert e.value.status == 6
+    rows = torch.tensor([0, 10 ** 6], dtype=torch.int32)
+    with pytest.raises(spr.SprinterError) as e:
+        spr.replace_sample_host(pin(wl_cpu.p_logits), V, pin(wl_cpu.u_replace[:2]), arena, ws, rows=rows)
+    assert e.value.status == 7
