@@ -361,6 +361,38 @@ def main():
                         "sample": f"first {sample} of {B} sequences ({sample * K} draft tokens), one pass, "
                                   f"{dt:.1f} s"}
 
+    # each call on its own, one stream, events around 50 back-to-back launches
+    def time_call(fn, n=50):
+        for _ in range(3):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+
+    fr = ver_out[2]
+    t_ver = time_call(lambda: spr.sprinter_verify(wl.hidden, wl.W1, wl.b1, wl.W2, wl.b2, tau, ws, out=ver_out))
+    t_rep = time_call(lambda: spr.replace_sample(wl.p_logits, V, wl.u_replace, ws, first_reject=fr, K=K,
+                                                 seq_stride=wl.Kp, out=tok_out))
+    t_stp = time_call(lambda: spr.sprinter_step(wl.hidden, wl.W1, wl.b1, wl.W2, wl.b2, tau, wl.p_logits, V,
+                                                wl.u_replace, ws, out=(ver_out[0], ver_out[1], ver_out[2], tok_out)))
+    t_sd = time_call(lambda: spr.sd_verify(wl.p_logits, wl.q_logits, V, wl.draft_tokens, wl.uniforms, ws, out=sd_out))
+    n_rej = int((fr < K).sum())
+    kept = float(fr.float().sum())          # draft tokens the verifier kept
+    calls = {
+        "sprinter_verify": {"ms": t_ver, "verified_tokens_per_s": M / (t_ver * 1e-3)},
+        "replace_sample": {"ms": t_rep, "draws": n_rej},
+        "sprinter_step": {"ms": t_stp, "verified_tokens_per_s": M / (t_stp * 1e-3),
+                          "emitted_tokens_per_s": (kept + n_rej) / (t_stp * 1e-3),
+                          "bytes": int(wl.hidden.numel() * es + wl.W1.numel() * es + n_rej * V * es)},
+        "sd_verify": {"ms": t_sd, "verified_tokens_per_s": M / (t_sd * 1e-3),
+                      "emitted_tokens_per_s": float(sd_out["accepted_len"].float().sum() + B) / (t_sd * 1e-3),
+                      "bytes": int(alg_bytes + int((sd_out["accepted_len"] < K).sum()) * 2 * V * es)},
+    }
+
     simulator = None
     if args.simulator_runs > 0:
         runs = args.simulator_runs
@@ -400,7 +432,7 @@ def main():
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                          "traffic": traffic, "algorithmic_bytes_per_launch": alg_bytes,
                          "avg_launch_ms": stats_ms},
-            "cpu_baseline": cpu_baseline,
+            "cpu_baseline": cpu_baseline, "calls": calls,
             **({"simulator": simulator} if simulator else {}),
         }))
     if world > 1:
