@@ -611,3 +611,50 @@ def test_host_buffer_entry_points(spr):
     with pytest.raises(spr.SprinterError) as e:
         spr.replace_sample_host(pin(wl_cpu.p_logits), V, pin(wl_cpu.u_replace[:2]), arena, ws, rows=rows)
     assert e.value.status == 7
+
+
+def test_calls_replay_from_a_cuda_graph(spr):
+    """sd_verify and sprinter_step enqueue only stream work (a clear and kernels, one of them
+    launched programmatically behind another): captured once, replayed, same bits; and the
+    replay follows the inputs when they change in place."""
+    wl_cpu = spr.workloads.make("gpt2", "cpu", B=6)
+    wl = to_device(wl_cpu)
+    cfg = wl.cfg
+    B, K, V = wl.B, wl.K, wl.V
+    ws = spr.Workspace.for_problem(B, K, V, cfg.d, cfg.h, spr.BF16)
+    out_sd = dict(accepted_len=torch.empty((B,), dtype=torch.int32, device="cuda"),
+                  correction_token=torch.empty((B,), dtype=torch.int32, device="cuda"))
+    out_st = (torch.empty((B, K), device="cuda"), torch.empty((B, K), dtype=torch.uint8, device="cuda"),
+              torch.empty((B,), dtype=torch.int32, device="cuda"), torch.empty((B,), dtype=torch.int32, device="cuda"))
+
+    def step():
+        spr.sd_verify(wl.p_logits, wl.q_logits, V, wl.draft_tokens, wl.uniforms, ws, out=out_sd)
+        spr.sprinter_step(wl.hidden, wl.W1, wl.b1, wl.W2, wl.b2, 0.5, wl.p_logits, V, wl.u_replace, ws, out=out_st)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()                                   # first call outside capture (one-time set-up)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    eager = [t.clone() for t in (*out_sd.values(), *out_st)]
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step()
+    for t in (*out_sd.values(), *out_st):
+        t.fill_(-3)
+    g.replay()
+    torch.cuda.synchronize()
+    for a, b in zip(eager, (*out_sd.values(), *out_st)):
+        assert torch.equal(a, b)
+    # new uniforms in the same buffers: the replay must follow them
+    wl.uniforms.copy_(torch.rand_like(wl.uniforms))
+    wl.u_replace.copy_(torch.rand_like(wl.u_replace))
+    g.replay()
+    torch.cuda.synchronize()
+    replayed = [t.clone() for t in (*out_sd.values(), *out_st)]
+    step()
+    torch.cuda.synchronize()
+    for a, b in zip(replayed, (*out_sd.values(), *out_st)):
+        assert torch.equal(a, b)
+    assert ws.device_status() == 0
