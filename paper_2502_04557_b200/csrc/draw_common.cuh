@@ -1,0 +1,312 @@
+// Inverse-CDF draws from softmax(l) or from the residual norm(max(0, p - q)) of Eq. 1: the
+// device code shared by the draw kernel and by the vocabulary-sharded correction draw.
+#pragma once
+
+#include <limits.h>
+
+#include "vocab_common.cuh"
+
+namespace spr {
+
+enum { MODE_NONE = 0, MODE_SOFTMAX = 1, MODE_RESIDUAL = 2 };
+
+template <typename T>
+struct Job {
+    int mode;
+    const T *p_row;
+    const T *q_row;
+    float cp, cq;  // residual: (max + ln Z) * log2(e) of the p row and of the q row
+    float u;
+};
+
+// residual weights max(0, p_i - q_i) of one vector (probabilities, already normalised)
+template <typename T>
+__device__ __forceinline__ void residual_weights(const uint4 &vp, const uint4 &vq, float cp, float cq,
+                                                 float (&w)[Vec<T>::N])
+{
+    constexpr int N = Vec<T>::N;
+    float fp[N], fq[N];
+    Vec<T>::unpack(vp, fp);
+    Vec<T>::unpack(vq, fq);
+#pragma unroll
+    for (int e = 0; e < N; ++e)
+        w[e] = fmaxf(0.f, ex2(fmaf(fp[e], kLog2e, -cp)) - ex2(fmaf(fq[e], kLog2e, -cq)));
+}
+
+constexpr int kCachedSteps = 512;   // step weights the last CTA of a draw keeps in shared memory
+
+struct DrawSmem {
+    double weight[kCachedSteps];   // weight of each step, relative to the row maximum
+    double base;                   // weight before the crossing step
+    double t_in;
+    double total;
+    float row_max;
+    float ref;
+    int step;
+    int token;
+    int last;
+};
+
+// inclusive prefix sum over the lanes of a warp, in lane order
+__device__ __forceinline__ double warp_scan_f64(double v, int lane)
+{
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += up;
+    }
+    return v;
+}
+
+// like load_step, for a row whose vectors need not be 16-byte aligned at `first`
+template <typename T>
+__device__ __forceinline__ void load_step_any(const T *__restrict__ row, int first, int V, int lane,
+                                              uint4 (&raw)[kUnroll])
+{
+    constexpr int N = Vec<T>::N;
+    if ((reinterpret_cast<uintptr_t>(row + first) & 15) == 0) {
+        load_step<T>(row, first, V, lane, raw);
+    } else {
+#pragma unroll
+        for (int j = 0; j < kUnroll; ++j) raw[j] = load_vec<T>(row, first + (j * 32 + lane) * N, V);
+    }
+}
+
+// lane-local sum of the residual weights of one warp step
+template <typename T>
+__device__ __forceinline__ float residual_step_sum(const uint4 (&rp)[kUnroll], const uint4 (&rq)[kUnroll],
+                                                   float cp, float cq)
+{
+    constexpr int N = Vec<T>::N;
+    float acc[kUnroll];
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) {
+        float w[N];
+        residual_weights<T>(rp[j], rq[j], cp, cq, w);
+        acc[j] = 0.f;
+#pragma unroll
+        for (int e = 0; e < N; ++e) acc[j] += w[e];
+    }
+    return (acc[0] + acc[1]) + (acc[2] + acc[3]);
+}
+
+// (max, sum of exp(x - max)) of one warp step of a softmax draw, in every lane
+template <typename T>
+__device__ __forceinline__ MS softmax_step(const uint4 (&raw)[kUnroll])
+{
+    const MS t = thread_ms<T>(raw);
+    MS r;
+    r.m = warp_max(t.m);
+    const float ref = (r.m == neg_inf()) ? 0.f : r.m;
+    r.s = warp_sum(t.s * ex2((t.m - ref) * kLog2e));
+    return r;
+}
+
+// Step partials (max, weight) of segment c of the job's row(s), written to part[step] for the
+// steps this CTA owns (iters per warp; fewer when there are few draws, so that more CTAs
+// share a row); same step interleaving and prefetch as the row-statistics kernel.
+// Residual draws store (0, sum of max(0, p - q)).
+template <typename T>
+__device__ __forceinline__ void segment_pass(const Job<T> &job, int mode, int V, int c, int steps, int iters,
+                                             float2 *__restrict__ part)
+{
+    constexpr int N = Vec<T>::N;
+    constexpr int kStep = 32 * kUnroll * N;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int step0 = c * kWarps * iters + warp;          // this warp's steps: step0 + it*kWarps
+    const int first = step0 * kStep - row_pad(job.p_row);
+    uint4 rp[kUnroll], rq[kUnroll];
+    if (step0 >= steps) return;
+    load_step<T>(job.p_row, first, V, lane, rp);
+    if (mode == MODE_RESIDUAL) load_step_any<T>(job.q_row, first, V, lane, rq);
+#pragma unroll
+    for (int it = 0; it < kStatIters; ++it) {
+        const int step = step0 + it * kWarps;
+        const int nxt = (it + 1) * kWarps * kStep;
+        const bool more = it + 1 < iters && step + kWarps < steps;
+        MS v;
+        if (mode == MODE_SOFTMAX) {
+            uint4 cur[kUnroll];
+#pragma unroll
+            for (int j = 0; j < kUnroll; ++j) cur[j] = rp[j];
+            if (more) load_step<T>(job.p_row, first + nxt, V, lane, rp);   // in flight during the math
+            v = softmax_step<T>(cur);
+        } else {
+            v.m = 0.f;
+            v.s = warp_sum(residual_step_sum<T>(rp, rq, job.cp, job.cq));
+            if (more) {
+                load_step<T>(job.p_row, first + nxt, V, lane, rp);
+                load_step_any<T>(job.q_row, first + nxt, V, lane, rq);
+            }
+        }
+        if (lane == 0) part[step] = make_float2(v.m, v.s);
+        if (!more) break;
+    }
+    __threadfence();
+}
+
+// Inside step `step` of the row, the first element whose running weight exceeds t_in (softmax
+// weights relative to `ref`); the last positive-weight element of the step if rounding
+// leaves no crossing, -1 if the step has no weight.  One warp; result in every lane.
+template <typename T>
+__device__ int step_locate(const Job<T> &job, int mode, int V, int step, double t_in, float ref)
+{
+    constexpr int N = Vec<T>::N;
+    constexpr int kStep = 32 * kUnroll * N;
+    const int lane = threadIdx.x & 31;
+    const int f0 = step * kStep - row_pad(job.p_row);
+    const float off = -ref * kLog2e;
+    uint4 rp[kUnroll], rq[kUnroll] = {};
+    load_step<T>(job.p_row, f0, V, lane, rp);
+    if (mode == MODE_RESIDUAL) load_step_any<T>(job.q_row, f0, V, lane, rq);
+    double run = 0.0;
+    int tok = -1, lastpos = -1;
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) {
+        float w[N];
+        if (mode == MODE_SOFTMAX) {
+            float f[N];
+            Vec<T>::unpack(rp[j], f);
+#pragma unroll
+            for (int e = 0; e < N; ++e) w[e] = ex2(fmaf(f[e], kLog2e, off));
+        } else {
+            residual_weights<T>(rp[j], rq[j], job.cp, job.cq, w);
+        }
+        const int e0 = f0 + (j * 32 + lane) * N;
+        double ts = 0.0;
+#pragma unroll
+        for (int e = 0; e < N; ++e) {
+            ts += (double)w[e];
+            if (w[e] > 0.f) lastpos = e0 + e;
+        }
+        const double incl = run + warp_scan_f64(ts, lane);
+        const unsigned cross = __ballot_sync(0xffffffffu, incl > t_in);
+        if (tok < 0 && cross != 0u) {
+            const int owner = __ffs(cross) - 1;
+            int mine = -1;
+            if (lane == owner) {
+                double r = incl - ts;
+                int last_e = -1;
+#pragma unroll
+                for (int e = 0; e < N; ++e) {
+                    r += (double)w[e];
+                    if (w[e] > 0.f) last_e = e;
+                    if (mine < 0 && r > t_in && w[e] > 0.f) mine = e;
+                }
+                if (mine < 0) mine = last_e;       // rounding inside the vector
+                if (mine >= 0) mine += e0;
+            }
+            tok = __shfl_sync(0xffffffffu, mine, owner);
+            if (tok < 0) tok = -2;                 // no weight in the crossing vector: fall back
+        }
+        run = __shfl_sync(0xffffffffu, incl, 31);
+    }
+    lastpos = (int)__reduce_max_sync(0xffffffffu, lastpos);
+    return tok >= 0 ? tok : lastpos;
+}
+
+// Warp 0, once every step partial of a draw is in part[0 .. steps): adds the step weights in
+// step order (fp64, relative to the largest step maximum) -> sm.total, sm.row_max; the first
+// kCachedSteps weights stay in sm.weight for steps_cross.
+__device__ __forceinline__ void steps_total(const float2 *part, int steps, DrawSmem &sm)
+{
+    const int lane = threadIdx.x & 31;
+    float M = neg_inf();
+    for (int t = lane; t < steps; t += 32) M = fmaxf(M, __ldcg(&part[t]).x);
+    M = warp_max(M);
+    double carry = 0.0;
+    for (int t0 = 0; t0 < steps; t0 += 32) {
+        const int t = t0 + lane;
+        double S = 0.0;
+        if (t < steps) {
+            const float2 ms = __ldcg(&part[t]);
+            if (ms.y > 0.f) S = (double)ms.y * exp((double)ms.x - (double)M);
+            if (t < kCachedSteps) sm.weight[t] = S;
+        }
+        carry += __shfl_sync(0xffffffffu, warp_scan_f64(S, lane), 31);
+    }
+    if (lane == 0) {
+        sm.total = carry;
+        sm.row_max = M;
+    }
+    __syncwarp();
+}
+
+// Warp 0, after steps_total: the step where the running weight first exceeds `target` (same
+// scale as sm.total) -> sm.step, with sm.t_in = what is left of the target inside that step,
+// relative to that step's own maximum sm.ref.  If rounding (or u >= 1) leaves no crossing:
+// the last step with positive weight and an infinite t_in; sm.step = -1 if there is none.
+__device__ __forceinline__ void steps_cross(const float2 *part, int steps, double target, DrawSmem &sm)
+{
+    const int lane = threadIdx.x & 31;
+    const float M = sm.row_max;
+    double carry = 0.0, before = 0.0;
+    int hit = -1, last_pos = -1;
+    for (int t0 = 0; t0 < steps && hit < 0; t0 += 32) {
+        const int t = t0 + lane;
+        double S = 0.0;
+        if (t < steps) {
+            if (t < kCachedSteps) {
+                S = sm.weight[t];
+            } else {
+                const float2 ms = __ldcg(&part[t]);
+                if (ms.y > 0.f) S = (double)ms.y * exp((double)ms.x - (double)M);
+            }
+        }
+        const double incl = carry + warp_scan_f64(S, lane);
+        const unsigned pos = __ballot_sync(0xffffffffu, S > 0.0);
+        if (pos != 0u) last_pos = t0 + 31 - __clz(pos);
+        const unsigned cross = __ballot_sync(0xffffffffu, incl > target);
+        if (cross != 0u) {
+            const int owner = __ffs(cross) - 1;
+            hit = t0 + owner;
+            before = __shfl_sync(0xffffffffu, incl - S, owner);
+        }
+        carry = __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) {
+        if (hit >= 0) {
+            const float mc = __ldcg(&part[hit]).x;
+            sm.step = hit;
+            sm.ref = mc;
+            sm.t_in = (target - before) * exp((double)M - (double)mc);
+        } else {
+            sm.step = last_pos;
+            sm.ref = last_pos >= 0 ? __ldcg(&part[last_pos]).x : 0.f;
+            sm.t_in = __longlong_as_double(0x7ff0000000000000LL);
+        }
+    }
+    __syncwarp();
+}
+
+// Whole CTA, once every step partial of a draw is in part[0 .. steps): the token where the
+// running weight crosses u * total.  A residual draw whose weights vanish (Eq. 1 undefined)
+// is redone as a draw from p.  The token is returned in warp 0 (other warps get -1);
+// *residual_mass, if given, receives the total residual weight (0 for softmax draws).
+template <typename T>
+__device__ int finish_draw(const Job<T> &job, int mode, int V, int steps, int iters, float2 *part, DrawSmem &sm,
+                           float *residual_mass)
+{
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int C = (steps + kWarps * iters - 1) / (kWarps * iters);
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        if (warp == 0) {
+            steps_total(part, steps, sm);
+            steps_cross(part, steps, (double)job.u * sm.total, sm);
+        }
+        __syncthreads();
+        if (attempt == 0 && tid == 0 && residual_mass) *residual_mass = mode == MODE_RESIDUAL ? (float)sm.total : 0.f;
+        if (mode == MODE_RESIDUAL && !(sm.total > 0.0)) {
+            // max(0, p - q) vanished: Eq. 1 is undefined, draw from p itself (one CTA, rare)
+            mode = MODE_SOFTMAX;
+            for (int cc = 0; cc < C; ++cc) segment_pass<T>(job, mode, V, cc, steps, iters, part);
+            __syncthreads();
+            continue;
+        }
+        break;
+    }
+    if (warp != 0) return -1;
+    return sm.step >= 0 ? step_locate<T>(job, mode, V, sm.step, sm.t_in, sm.ref) : -1;
+}
+
+}  // namespace spr
