@@ -60,7 +60,8 @@ typedef enum {
     SPR_OP_SPRINTER_VERIFY = 0,
     SPR_OP_REPLACE_SAMPLE = 1,
     SPR_OP_SD_VERIFY = 2,
-    SPR_OP_SPRINTER_STEP = 3
+    SPR_OP_SPRINTER_STEP = 3,
+    SPR_OP_SD_SHARD = 4
 } spr_op;
 
 /* Which verifier kernel sprinter_verify() uses.  AUTO picks the tensor-core
@@ -70,7 +71,8 @@ typedef enum { SPR_VERIFIER_AUTO = 0, SPR_VERIFIER_SIMT = 1, SPR_VERIFIER_TENSOR
 /* Bytes of device scratch one call of `op` needs.  For SPR_OP_REPLACE_SAMPLE,
  * B is the number of draws n and K, d, h are ignored; for SPR_OP_SD_VERIFY d
  * and h are ignored; for SPR_OP_SPRINTER_VERIFY V is ignored; SPR_OP_SPRINTER_STEP
- * uses all of them.  Returns 0 for invalid arguments.  A workspace sized for the
+ * uses all of them; for SPR_OP_SD_SHARD V is the width of this GPU's vocabulary
+ * shard and d, h are ignored.  Returns 0 for invalid arguments.  A workspace sized for the
  * largest op serves all of them. */
 size_t spr_workspace_bytes(int op, int B, int K, int V, int d, int h, int dt);
 
@@ -178,6 +180,59 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
               const float *uniforms, int B, int K, int Kp, int V, int dt, int32_t *accepted_len,
               int32_t *correction_token, uint8_t *accept, float *p_tok, float *q_tok,
               float *residual_mass, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * sd_shard_* - sd_verify for logits split along the vocabulary across G GPUs.
+ *
+ * Defined by: the same passages as sd_verify (Section 2, Eq. 1); the paper has no
+ * multi-GPU form.  This is sd_verify for a tensor-parallel LM head: GPU g holds columns
+ * [v0_g, v0_g + Vs_g) of every p and q row (shards in rank order tile [0, V) without gaps).
+ * Results equal sd_verify's on the concatenated rows, on every GPU, except that
+ * correction_token[b] is the token on the one GPU whose shard contains it and -1 on the
+ * others (reduce with max).  The sequence of calls on each GPU, all on one stream and one
+ * workspace of spr_workspace_bytes(SPR_OP_SD_SHARD, B, K, Vs, 0, 0, dt) bytes that nothing
+ * else uses in between:
+ *
+ *   sd_shard_stats    reads the shard once.  stats [B*Kp, 6] f32 per row b*Kp + k:
+ *                     (max, sum exp(l - max)) of the p shard row, the same of the q shard
+ *                     row, and l_p[x], l_q[x] of the draft token x = draft_tokens[b,k] if
+ *                     v0 <= x < v0 + Vs, else -inf (q entries of the bonus row k = K:
+ *                     -inf, 0, -inf).
+ *   -- all-gather stats -> all_stats [G, B*Kp, 6], rank order --
+ *   sd_shard_decide   merges the G records of every row in rank order, then accept,
+ *                     accepted_len, p_tok, q_tok exactly as sd_verify defines them
+ *                     (identical on every GPU); keeps the whole-row statistics in ws.
+ *                     V is the whole vocabulary (draft tokens outside [0,V) are reported
+ *                     as in sd_verify); Vs and dt only size the workspace.
+ *   sd_shard_weights  weights [B, 2] f64 per sequence: this shard's total weight of the
+ *                     correction draw - (0, sum over the shard of max(0, p_i - q_i)) with
+ *                     whole-row probabilities at position accepted_len[b] < K;
+ *                     (shard max, sum exp(l - shard max)) of the bonus row when
+ *                     accepted_len[b] = K and Kp = K+1; (0, 0) when there is no draw.
+ *   -- all-gather weights -> all_weights [G, B, 2], rank order --
+ *   sd_shard_draw     adds the G shard weights in rank order, finds the shard in which
+ *                     uniforms[b,K] * total falls, and on that GPU (rank) locates the token
+ *                     by the inverse CDF of sd_verify, returned as a whole-vocabulary id.
+ *                     residual_mass [B] (optional) is the total over all shards, on every
+ *                     GPU.  If the residual vanishes on every shard the draw is from p at
+ *                     that position, using the shard statistics in all_stats.
+ *
+ * p_shard [B,Kp,ldv] dt and q_shard [B,K,ldv] dt point at column v0 of the first row; ldv
+ * is the row stride in elements (>= Vs).  Errors as for sd_verify; G <= 1024.
+ */
+int sd_shard_stats(const void *p_shard, const void *q_shard, int64_t ldv, int Vs, int v0,
+                   const int32_t *draft_tokens, int B, int K, int Kp, int dt, float *stats, void *ws,
+                   size_t ws_bytes, void *cuda_stream);
+int sd_shard_decide(const float *all_stats, int G, const int32_t *draft_tokens, const float *uniforms, int B,
+                    int K, int Kp, int V, int Vs, int dt, int32_t *accepted_len, uint8_t *accept, float *p_tok,
+                    float *q_tok, void *ws, size_t ws_bytes, void *cuda_stream);
+int sd_shard_weights(const void *p_shard, const void *q_shard, int64_t ldv, int Vs, const int32_t *accepted_len,
+                     const float *uniforms, int B, int K, int Kp, int dt, double *weights, void *ws,
+                     size_t ws_bytes, void *cuda_stream);
+int sd_shard_draw(const void *p_shard, const void *q_shard, int64_t ldv, int Vs, int v0, const double *all_weights,
+                  const float *all_stats, int G, int rank, const int32_t *accepted_len, const float *uniforms,
+                  int B, int K, int Kp, int dt, int32_t *correction_token, float *residual_mass, void *ws,
+                  size_t ws_bytes, void *cuda_stream);
 
 /*
  * sprinter_simulate - run lengths of an i.i.d. verifier (Monte-Carlo of Theorems 2 and 3).

@@ -15,7 +15,7 @@ import torch
 from . import build as _build
 
 F32, BF16 = 0, 1
-OP_SPRINTER_VERIFY, OP_REPLACE_SAMPLE, OP_SD_VERIFY, OP_SPRINTER_STEP = 0, 1, 2, 3
+OP_SPRINTER_VERIFY, OP_REPLACE_SAMPLE, OP_SD_VERIFY, OP_SPRINTER_STEP, OP_SD_SHARD = 0, 1, 2, 3, 4
 PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
 
 EXPORTS = [
@@ -23,6 +23,7 @@ EXPORTS = [
     "spr_device_status", "spr_status_string", "spr_last_cuda_error", "spr_version",
     "spr_host_arena_bytes", "sprinter_verify_host", "replace_sample_host", "sd_verify_host",
     "spr_set_stage_events", "replace_sample_static", "sprinter_step", "sprinter_simulate",
+    "sd_shard_stats", "sd_shard_decide", "sd_shard_weights", "sd_shard_draw",
 ]
 
 
@@ -70,6 +71,15 @@ def lib():
         L.sd_verify.restype = i32
         L.sd_verify.argtypes = [vp, vp, i64, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp,
                                 vp, sz, vp]
+        L.sd_shard_stats.restype = i32
+        L.sd_shard_stats.argtypes = [vp, vp, i64, i32, i32, vp, i32, i32, i32, i32, vp, vp, sz, vp]
+        L.sd_shard_decide.restype = i32
+        L.sd_shard_decide.argtypes = [vp, i32, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+        L.sd_shard_weights.restype = i32
+        L.sd_shard_weights.argtypes = [vp, vp, i64, i32, vp, vp, i32, i32, i32, i32, vp, vp, sz, vp]
+        L.sd_shard_draw.restype = i32
+        L.sd_shard_draw.argtypes = [vp, vp, i64, i32, i32, vp, vp, i32, i32, vp, vp, i32, i32, i32, i32,
+                                    vp, vp, vp, sz, vp]
         L.spr_host_arena_bytes.restype = sz
         L.spr_host_arena_bytes.argtypes = [i32, i32, i32, i32, i64, i32, i32, i32]
         L.sprinter_verify_host.restype = i32
@@ -281,6 +291,104 @@ def sd_verify(p_logits, q_logits, V: int, draft_tokens, uniforms, ws: Workspace,
                          _ptr(out.get("q_tok")), _ptr(out.get("residual_mass")),
                          _ptr(ws.buf), ws.nbytes, _stream())
     _check("sd_verify", rc)
+    return out
+
+
+# ---------------------------------------------------------------------------- vocabulary shards
+
+
+def _shard(t: torch.Tensor, dtype=None, name="tensor"):
+    """A [*, rows, Vs] view whose last dimension is dense; rows may be strided (a column slice
+    of a wider tensor).  Returns the row stride in elements."""
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}")
+    B, R, Vs = t.shape
+    ldv = t.stride(1)
+    if t.stride(2) != 1 or ldv < Vs or (B > 1 and t.stride(0) != R * ldv):
+        raise ValueError(f"{name}: rows must be dense and equally spaced")
+    return ldv
+
+
+def sd_shard_stats(p_shard, q_shard, v0: int, draft_tokens, ws: Workspace, out=None):
+    """Pass 1 of the vocabulary-sharded sd_verify: this shard's row statistics [B*Kp, 6] f32."""
+    ldv = _shard(p_shard, name="p_shard")
+    if _shard(q_shard, p_shard.dtype, "q_shard") != ldv:
+        raise ValueError("p_shard and q_shard must have the same row stride")
+    B, Kp, Vs = p_shard.shape
+    K = q_shard.shape[1]
+    _dev(draft_tokens, torch.int32, "draft_tokens")
+    if out is None:
+        out = torch.empty((B * Kp, 6), dtype=torch.float32, device=p_shard.device)
+    rc = lib().sd_shard_stats(_ptr(p_shard), _ptr(q_shard), ldv, Vs, v0, _ptr(draft_tokens), B, K, Kp,
+                              _dt(p_shard), _ptr(out), _ptr(ws.buf), ws.nbytes, _stream())
+    _check("sd_shard_stats", rc)
+    return out
+
+
+def sd_shard_decide(all_stats, draft_tokens, uniforms, V: int, Vs: int, Kp: int, dt: int, ws: Workspace,
+                    extras: bool = True, out=None):
+    """Pass 2: all_stats [G, B*Kp, 6] (rank order) -> accepted_len (and accept, p_tok, q_tok)."""
+    _dev(all_stats, torch.float32, "all_stats")
+    _dev(draft_tokens, torch.int32, "draft_tokens")
+    _dev(uniforms, torch.float32, "uniforms")
+    B, K = draft_tokens.shape
+    G = all_stats.shape[0]
+    if tuple(all_stats.shape) != (G, B * Kp, 6) or tuple(uniforms.shape) != (B, K + 1):
+        raise ValueError("all_stats must be [G,B*Kp,6] and uniforms [B,K+1]")
+    dev = all_stats.device
+    if out is None:
+        out = dict(accepted_len=torch.empty((B,), dtype=torch.int32, device=dev))
+        if extras:
+            out.update(accept=torch.empty((B, K), dtype=torch.uint8, device=dev),
+                       p_tok=torch.empty((B, K), dtype=torch.float32, device=dev),
+                       q_tok=torch.empty((B, K), dtype=torch.float32, device=dev))
+    rc = lib().sd_shard_decide(_ptr(all_stats), G, _ptr(draft_tokens), _ptr(uniforms), B, K, Kp, V, Vs, dt,
+                               _ptr(out["accepted_len"]), _ptr(out.get("accept")), _ptr(out.get("p_tok")),
+                               _ptr(out.get("q_tok")), _ptr(ws.buf), ws.nbytes, _stream())
+    _check("sd_shard_decide", rc)
+    return out
+
+
+def sd_shard_weights(p_shard, q_shard, accepted_len, uniforms, ws: Workspace, out=None):
+    """Pass 3: this shard's share [B, 2] f64 of every sequence's correction draw."""
+    ldv = _shard(p_shard, name="p_shard")
+    _shard(q_shard, p_shard.dtype, "q_shard")
+    B, Kp, Vs = p_shard.shape
+    K = q_shard.shape[1]
+    _dev(accepted_len, torch.int32, "accepted_len")
+    _dev(uniforms, torch.float32, "uniforms")
+    if out is None:
+        out = torch.empty((B, 2), dtype=torch.float64, device=p_shard.device)
+    rc = lib().sd_shard_weights(_ptr(p_shard), _ptr(q_shard), ldv, Vs, _ptr(accepted_len), _ptr(uniforms),
+                                B, K, Kp, _dt(p_shard), _ptr(out), _ptr(ws.buf), ws.nbytes, _stream())
+    _check("sd_shard_weights", rc)
+    return out
+
+
+def sd_shard_draw(p_shard, q_shard, v0: int, all_weights, all_stats, rank: int, accepted_len, uniforms,
+                  ws: Workspace, extras: bool = True, out=None):
+    """Pass 4: correction_token [B] (-1 unless this shard holds the token) and residual_mass."""
+    ldv = _shard(p_shard, name="p_shard")
+    _shard(q_shard, p_shard.dtype, "q_shard")
+    B, Kp, Vs = p_shard.shape
+    K = q_shard.shape[1]
+    _dev(all_weights, torch.float64, "all_weights")
+    _dev(all_stats, torch.float32, "all_stats")
+    G = all_weights.shape[0]
+    if tuple(all_weights.shape) != (G, B, 2) or tuple(all_stats.shape) != (G, B * Kp, 6):
+        raise ValueError("all_weights must be [G,B,2] and all_stats [G,B*Kp,6]")
+    dev = p_shard.device
+    if out is None:
+        out = dict(correction_token=torch.empty((B,), dtype=torch.int32, device=dev))
+        if extras:
+            out["residual_mass"] = torch.empty((B,), dtype=torch.float32, device=dev)
+    rc = lib().sd_shard_draw(_ptr(p_shard), _ptr(q_shard), ldv, Vs, v0, _ptr(all_weights), _ptr(all_stats),
+                             G, rank, _ptr(accepted_len), _ptr(uniforms), B, K, Kp, _dt(p_shard),
+                             _ptr(out["correction_token"]), _ptr(out.get("residual_mass")),
+                             _ptr(ws.buf), ws.nbytes, _stream())
+    _check("sd_shard_draw", rc)
     return out
 
 

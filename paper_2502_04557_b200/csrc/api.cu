@@ -21,6 +21,12 @@ int cuda_fail(cudaError_t e)
 namespace spr {
 int report_cuda_error(cudaError_t e) { return cuda_fail(e); }
 }  // namespace spr
+namespace {
+int check_device();
+}
+namespace spr {
+int device_supported() { return check_device(); }
+}  // namespace spr
 
 namespace {
 
@@ -183,6 +189,9 @@ size_t spr_workspace_bytes(int op, int B, int K, int V, int d, int h, int dt)
     case SPR_OP_SD_VERIFY:
         if (K <= 0 || V <= 0 || (int64_t)B * K > 0x7fffffff) return 0;
         return sd_ws_layout(B, K, stat_max_segments_per_row(V, dt), stat_steps_per_row(V, dt)).end;
+    case SPR_OP_SD_SHARD:   // V = shard width; sized for a bonus row
+        if (K <= 0 || V <= 0 || (int64_t)B * (K + 1) > 0x7fffffff) return 0;
+        return shard_ws_layout(B, K, K + 1, stat_max_segments_per_row(V, dt), stat_steps_per_row(V, dt)).end;
     default:
         return 0;
     }

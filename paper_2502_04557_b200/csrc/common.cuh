@@ -102,6 +102,31 @@ __host__ __device__ inline SdWs sd_ws_layout(int B, int K, int S, int T)   // S 
     return w;
 }
 
+struct ShardWs {             // vocabulary-sharded sd_verify: the four passes share one workspace
+    size_t row_counters;     // int32 [B*Kp]
+    size_t draw_counters;    // int32 [B]
+    size_t counters_end;
+    size_t acc;              // uint8 [B*K]
+    size_t part;             // float4 [B*Kp*S]
+    size_t rowstats;         // float4 [B*Kp]  whole-row (max_p, ln Z_p, max_q, ln Z_q)
+    size_t draw_part;        // float2 [B*T]
+    size_t end;
+};
+__host__ __device__ inline ShardWs shard_ws_layout(int B, int K, int Kp, int S, int T)
+{
+    const size_t R = (size_t)B * Kp;
+    ShardWs w;
+    w.row_counters = kHeaderBytes;
+    w.draw_counters = w.row_counters + 4 * R;
+    w.counters_end = align_up(w.draw_counters + 4 * (size_t)B, 256);
+    w.acc = w.counters_end;
+    w.part = align_up(w.acc + (size_t)B * K, 256);
+    w.rowstats = align_up(w.part + 16 * R * S, 256);
+    w.draw_part = align_up(w.rowstats + 16 * R, 256);
+    w.end = align_up(w.draw_part + 8 * (size_t)B * T, 256);
+    return w;
+}
+
 struct VerifyWs {
     size_t counter;          // int32 [1 + max(row tiles, B)]   CTAs finished per tile / tokens per sequence
     size_t counters_end;

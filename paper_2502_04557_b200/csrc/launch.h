@@ -54,6 +54,54 @@ struct DrawParams {
     float2 *part;    // [n*steps] (max, weight) of every warp step
 };
 
+// Vocabulary-sharded sd_verify (sd_shard.cu): V is the width of this GPU's shard, v0 its
+// first column; *_all arrays hold one block per rank, in rank order.
+struct ShardStatsParams {
+    const void *p;  // [B,Kp,ldv] shard columns
+    const void *q;  // [B,K,ldv]
+    int64_t ldv;
+    int V, v0, K, Kp, chunks, iters;
+    const int32_t *draft_tokens;  // [B,K] global token ids
+    float *stats;                 // [B*Kp, 6]
+    int *row_counters;            // [B*Kp]
+    float4 *part;                 // [B*Kp*chunks]
+};
+
+struct ShardDecideParams {
+    const float *all_stats;       // [G, B*Kp, 6]
+    int G, K, Kp, V;              // V: the whole vocabulary
+    const int32_t *draft_tokens;
+    const float *uniforms;        // [B,K+1]
+    int32_t *accepted_len;        // [B]
+    uint8_t *accept;              // [B,K] or null
+    float *p_tok, *q_tok;         // [B,K] or null
+    int *status;
+    uint8_t *acc;                 // [B*K]
+    float4 *rowstats;             // [B*Kp] (max_p, ln Z_p, max_q, ln Z_q) of the whole rows
+};
+
+struct ShardDrawParams {
+    const void *p;
+    const void *q;
+    int64_t ldv;
+    int V, v0, K, Kp, chunks, steps, iters;
+    int G, rank;
+    const int32_t *accepted_len;
+    const float *uniforms;
+    const float4 *rowstats;
+    double2 *weights;             // [B] this shard's (max, weight); weights pass only
+    const double2 *all_weights;   // [G, B]; draw pass only
+    const float *all_stats;       // [G, B*Kp, 6]; draw pass only
+    int32_t *tokens;              // [B]
+    float *residual_mass;         // [B] or null
+    int *counters;                // [B]
+    float2 *part;                 // [B*steps]
+};
+cudaError_t launch_shard_stats(const ShardStatsParams &sp, int64_t rows, int dt, cudaStream_t st);
+cudaError_t launch_shard_decide(const ShardDecideParams &dp, int B, cudaStream_t st);
+cudaError_t launch_shard_weights(const ShardDrawParams &dp, int B, int dt, cudaStream_t st);
+cudaError_t launch_shard_draw(const ShardDrawParams &dp, int B, int dt, cudaStream_t st);
+
 struct VerifyParams {
     const void *hidden;  // [M,d]
     const void *W1;      // [h,d] (or [d] when h == 0)
@@ -83,6 +131,7 @@ cudaError_t launch_simulate(const SimParams &sp, cudaStream_t st);
 
 cudaError_t launch_sd_row_stats(const SdParams &sp, int B, int K, int dt, cudaStream_t st);
 int report_cuda_error(cudaError_t e);  // records the text, returns SPR_ERR_CUDA
+int device_supported();                // SPR_OK on a compute-capability-10 device
 void set_stage_events(cudaEvent_t before, cudaEvent_t after);
 // everything of a replacement draw except the scratch pointers (status, counters, part)
 DrawParams replace_params(const void *target_logits, int64_t ldv, int V, int64_t R, const int32_t *rows,

@@ -1,0 +1,190 @@
+"""Vocabulary-sharded sd_verify against the float64 oracle of the unsharded definition.
+
+One GPU stands in for G ranks: every rank is a host thread with its own stream, workspace
+and column slice of the logits, and the collectives are host-side rendezvous (each thread
+synchronises its stream, then a barrier).  No kernel waits on another kernel."""
+import threading
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import MARGIN, RTOL, assert_close_rel, enforce_margins, oracle_sd, to_device, to_np
+from test_gpu_parity import _clear_sd, _rand_problem, eq
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def spr():
+    import paper_2502_04557_b200 as s
+    s.lib()
+    return s
+
+
+class ThreadExchange:
+    """all_gather / all_reduce_max between G host threads."""
+
+    def __init__(self, shared, rank):
+        self.shared, self.rank, self.world = shared, rank, shared["G"]
+
+    def _meet(self):
+        self.shared["barrier"].wait(timeout=120)
+
+    def all_gather(self, t):
+        torch.cuda.current_stream().synchronize()
+        self.shared["slots"][self.rank] = t
+        self._meet()
+        out = torch.stack(self.shared["slots"]).contiguous()
+        torch.cuda.current_stream().synchronize()
+        self._meet()   # nobody overwrites a slot that is still being read
+        return out
+
+    def all_reduce_max(self, t):
+        t.copy_(self.all_gather(t.clone()).amax(dim=0))
+        return t
+
+
+def run_sharded(spr, p, q, V, x, u, G, shards=None, extras=True):
+    """p [B,Kp,ldv], q [B,K,ldv], x, u on the GPU; returns the result dict of every rank."""
+    from paper_2502_04557_b200 import sharded
+    shards = shards or sharded.vocab_shards(V, G, p.element_size())
+    B, Kp, _ = p.shape
+    K = q.shape[1]
+    shared = dict(G=G, barrier=threading.Barrier(G), slots=[None] * G)
+    results, errors = [None] * G, []
+    torch.cuda.synchronize()
+
+    def rank_main(g):
+        try:
+            v0, Vs = shards[g]
+            with torch.cuda.stream(torch.cuda.Stream()):
+                ws = spr.Workspace(spr.workspace_bytes(spr.binding.OP_SD_SHARD, B, K, Vs, 0, 0, spr.binding._dt(p)))
+                results[g] = sharded.sd_verify_sharded(p[:, :, v0:v0 + Vs], q[:, :, v0:v0 + Vs], V, v0, x, u, ws,
+                                                       ThreadExchange(shared, g), extras=extras)
+                results[g]["status"] = ws.device_status()
+        except BaseException as e:   # noqa: BLE001 - release the other threads, then re-raise in the test
+            errors.append(e)
+            shared["barrier"].abort()
+
+    threads = [threading.Thread(target=rank_main, args=(g,)) for g in range(G)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    if errors:
+        raise errors[0]
+    return results
+
+
+def check_against(ref, results, dtype, status=0):
+    for g, out in enumerate(results):
+        assert out["status"] == status, f"rank {g}"
+        eq(out["accept"], ref["accept"], f"rank {g} accept")
+        eq(out["accepted_len"], ref["accepted_len"], f"rank {g} accepted_len")
+        eq(out["correction_token"], ref["correction_token"], f"rank {g} correction_token")
+        assert_close_rel(out["p_tok"], ref["p_tok"], RTOL[dtype], "p_tok")
+        assert_close_rel(out["q_tok"], ref["q_tok"], RTOL[dtype], "q_tok")
+        assert_close_rel(out["residual_mass"], ref["residual_mass"], RTOL[dtype], "residual_mass")
+
+
+@pytest.mark.parametrize("G", [1, 2, 3, 8])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("B,K,V,ldv,Kp", [
+    (3, 1, 64, None, 2), (5, 2, 200, None, 3), (4, 3, 1000, None, 3), (2, 33, 129, 131, 34),
+    (3, 4, 8191, None, 5), (2, 2, 8193, 8200, 2), (2, 5, 16385, None, 6), (1, 40, 50257, None, 40),
+])
+def test_sharded_ragged_shapes(spr, dtype, B, K, V, ldv, Kp, G):
+    p, q, x, u = _rand_problem(B, K, V, dtype, seed=G + B * 1000 + K * 10 + V, ldv=ldv, Kp=Kp)
+    ref = _clear_sd(p, q, V, x, u)
+    results = run_sharded(spr, p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), G)
+    check_against(ref, results, dtype)
+
+
+@pytest.mark.parametrize("name,B,G", [("gpt2", 6, 4), ("llama2", 8, 2), ("llama3", 4, 8), ("sequential", 16, 8)])
+def test_sharded_configs(spr, name, B, G):
+    wl_cpu = spr.workloads.make(name, "cpu", B=B, bonus_row=(name != "sequential"))
+    enforce_margins(wl_cpu)
+    wl = to_device(wl_cpu)
+    ref = oracle_sd(wl_cpu)
+    results = run_sharded(spr, wl.p_logits, wl.q_logits, wl.V, wl.draft_tokens, wl.uniforms, G)
+    check_against(ref, results, wl.q_logits.dtype)
+    # and the same decisions as the single-GPU call
+    ws = spr.Workspace(spr.workspace_bytes(2, wl.B, wl.K, wl.V, 1, 0, spr.binding._dt(wl.p_logits)))
+    one = spr.sd_verify(wl.p_logits, wl.q_logits, wl.V, wl.draft_tokens, wl.uniforms, ws)
+    for k in ("accept", "accepted_len", "correction_token"):
+        assert torch.equal(one[k], results[0][k]), k
+
+
+def test_sharded_uneven_and_misaligned_shards(spr):
+    B, K, V = 3, 4, 5003
+    p, q, x, u = _rand_problem(B, K, V, torch.bfloat16, seed=77)
+    shards = [(0, 1), (1, 2048), (2049, 7), (2056, 2947)]   # widths 1 .. thousands, odd offsets
+    assert sum(s[1] for s in shards) == V
+    for b in range(B):          # draft tokens on both sides of every boundary
+        for k in range(K):
+            v0 = shards[(b * K + k) % 4][0]
+            x[b, k] = max(0, v0 - (k % 2))
+    ref = _clear_sd(p, q, V, x, u)
+    results = run_sharded(spr, p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), 4, shards=shards)
+    check_against(ref, results, torch.bfloat16)
+
+
+def test_sharded_disjoint_supports_and_all_accepted(spr):
+    g = torch.Generator().manual_seed(8)
+    B, K, V, G = 4, 3, 5000, 4
+    ninf = float("-inf")
+    u = torch.rand((B, K + 1), generator=g).clamp_(min=1e-3, max=0.999)
+    # disjoint supports: three of the four p shards carry no mass at all
+    p = torch.full((B, K + 1, V), ninf); p[..., :100] = torch.randn((B, K + 1, 100), generator=g)
+    q = torch.full((B, K, V), ninf); q[..., 100:] = torch.randn((B, K, V - 100), generator=g)
+    x = torch.randint(100, V, (B, K), generator=g, dtype=torch.int32)
+    ref = oracle.sd_verify(to_np(p), to_np(q), V, to_np(x), to_np(u))
+    results = run_sharded(spr, p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), G)
+    for out in results:
+        assert out["status"] == 0
+        assert (out["accept"] == 0).all() and (out["accepted_len"] == 0).all()
+        assert torch.allclose(out["residual_mass"], torch.ones(B, device="cuda"), rtol=1e-5)
+        for b in range(B):
+            m, t = oracle.residual_draw_margin(to_np(p)[b, 0], to_np(q)[b, 0], float(u[b, K]))
+            if m > 1e-5:
+                assert int(out["correction_token"][b]) == t == ref["correction_token"][b]
+    # p == q: everything accepted, bonus token from p at position K
+    q = (torch.randn((B, K, V), generator=g) * 2).to(torch.bfloat16)
+    p = torch.cat([q, q[:, :1]], 1).contiguous()
+    x = torch.randint(0, V, (B, K), generator=g, dtype=torch.int32)
+    ref = oracle.sd_verify(to_np(p), to_np(q), V, to_np(x), to_np(u))
+    results = run_sharded(spr, p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), G)
+    for out in results:
+        assert (out["accept"] == 1).all() and (out["accepted_len"] == K).all()
+        assert (out["residual_mass"] == 0).all()
+        for b in range(B):
+            m, t = oracle.softmax_draw_margin(to_np(p)[b, K], float(u[b, K]))
+            if m > 1e-5:
+                assert int(out["correction_token"][b]) == t == ref["correction_token"][b]
+    # no bonus row: nothing to draw
+    results = run_sharded(spr, p[:, :K].contiguous().cuda(), q.cuda(), V, x.cuda(), u.cuda(), G)
+    for out in results:
+        assert (out["accepted_len"] == K).all() and (out["correction_token"] == -1).all()
+
+
+def test_sharded_bad_token_and_empty_batch(spr):
+    B, K, V, G = 3, 4, 3000, 3
+    p, q, x, u = _rand_problem(B, K, V, torch.float32, seed=5)
+    x[1, 2] = V   # outside the whole vocabulary
+    ref = _clear_sd(p, q, V, x.clamp(max=V - 1), u)
+    results = run_sharded(spr, p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), G)
+    for out in results:
+        assert out["status"] == 6   # SPR_ERR_BAD_TOKEN
+        assert int(out["accepted_len"][1]) == -1 and int(out["correction_token"][1]) == -1
+        assert (out["accept"][1] == 0).all()
+        for b in (0, 2):
+            assert int(out["accepted_len"][b]) == ref["accepted_len"][b]
+            assert int(out["correction_token"][b]) == ref["correction_token"][b]
+    # empty batch: every pass returns without touching a pointer
+    e = torch.empty
+    ws = spr.Workspace(256)
+    st = spr.binding.sd_shard_stats(e((0, K + 1, 8), device="cuda"), e((0, K, 8), device="cuda"), 0,
+                                    e((0, K), dtype=torch.int32, device="cuda"), ws)
+    assert st.shape == (0, 6)
