@@ -188,3 +188,27 @@ def test_sharded_bad_token_and_empty_batch(spr):
     st = spr.binding.sd_shard_stats(e((0, K + 1, 8), device="cuda"), e((0, K, 8), device="cuda"), 0,
                                     e((0, K), dtype=torch.int32, device="cuda"), ws)
     assert st.shape == (0, 6)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_residual_below_fp32_resolution_falls_back_to_p(spr, dtype):
+    """p equals q except for a slightly lower logit at the draft token: the token is rejected
+    (ratio 0.998 against u = 0.9995), but every p_i - q_i elsewhere is about 4e-8 / V, far
+    below what fp32 probabilities resolve, so max(0, p - q) is exactly zero on the GPU.  Both
+    the single-GPU call and the sharded one must then draw from p itself."""
+    B, K, V, G = 3, 2, 50257, 4
+    q = torch.zeros((B, K, V), dtype=dtype)
+    p = torch.zeros((B, K + 1, V), dtype=dtype)
+    x = torch.tensor([[7, 100], [25000, 3], [V - 1, 0]], dtype=torch.int32)
+    u = torch.tensor([[0.9995, 0.5, 0.31], [0.9995, 0.5, 0.77], [0.9995, 0.5, 0.123]], dtype=torch.float32)
+    for b in range(B):
+        p[b, 0, int(x[b, 0])] = -2e-3
+    ws = spr.Workspace(spr.workspace_bytes(2, B, K, V, 1, 0, spr.binding._dt(p)))
+    one = spr.sd_verify(p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), ws)
+    results = run_sharded(spr, p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), G)
+    for out in [one] + results:
+        assert (out["accepted_len"] == 0).all()
+        assert (out["residual_mass"] == 0).all()
+        for b in range(B):
+            m, t = oracle.softmax_draw_margin(to_np(p)[b, 0], float(u[b, K]))
+            assert m > 1e-6 and int(out["correction_token"][b]) == t
