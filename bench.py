@@ -56,6 +56,9 @@ def parse_args():
     ap.add_argument("--threshold", type=float, default=0.5)
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--vocab-shards", type=int, default=8,
+                    help="also time the four passes of the vocabulary-sharded sd_verify on one of this many "
+                         "column shards (0 = skip)")
     ap.add_argument("--simulator-runs", type=int, default=0,
                     help="also time sprinter_simulate on this many runs (r=5, eta_TP=0.9, eta_FP=0.5)")
     return ap.parse_args()
@@ -392,6 +395,34 @@ def main():
                       "emitted_tokens_per_s": float(sd_out["accepted_len"].float().sum() + B) / (t_sd * 1e-3),
                       "bytes": int(alg_bytes + int((sd_out["accepted_len"] < K).sum()) * 2 * V * es)},
     }
+
+    # vocabulary-sharded sd_verify: what one of G GPUs would run on its V/G columns (the two
+    # all-gathers between the passes, 24 B per row and 16 B per sequence per GPU, are not timed)
+    if args.vocab_shards > 0:
+        from paper_2502_04557_b200 import binding as bd, sharded
+        G = args.vocab_shards
+        shards = sharded.vocab_shards(V, G, es)
+        views = [(wl.p_logits[:, :, v0:v0 + vs], wl.q_logits[:, :, v0:v0 + vs]) for v0, vs in shards]
+        wss = [spr.Workspace(spr.workspace_bytes(bd.OP_SD_SHARD, B, K, vs, 0, 0, dt_code), device=dev) for _, vs in shards]
+        all_stats = torch.stack([bd.sd_shard_stats(pv, qv, v0, wl.draft_tokens, w)
+                                 for (pv, qv), (v0, _), w in zip(views, shards, wss)])
+        dec = [bd.sd_shard_decide(all_stats, wl.draft_tokens, wl.uniforms, V, vs, wl.Kp, dt_code, w, extras=False)
+               for (_, vs), w in zip(shards, wss)]
+        all_w = torch.stack([bd.sd_shard_weights(pv, qv, dec[0]["accepted_len"], wl.uniforms, w)
+                             for (pv, qv), w in zip(views, wss)])
+        (pv, qv), (v0, vs), w0, n0 = views[0], shards[0], wss[0], dec[0]["accepted_len"]
+        o_stats, o_w = torch.empty_like(all_stats[0]), torch.empty_like(all_w[0])
+        o_tok = dict(correction_token=torch.empty((B,), dtype=torch.int32, device=dev))
+        t1 = time_call(lambda: bd.sd_shard_stats(pv, qv, v0, wl.draft_tokens, w0, out=o_stats))
+        t2 = time_call(lambda: bd.sd_shard_decide(all_stats, wl.draft_tokens, wl.uniforms, V, vs, wl.Kp, dt_code, w0,
+                                                  out=dec[0]))
+        t3 = time_call(lambda: bd.sd_shard_weights(pv, qv, n0, wl.uniforms, w0, out=o_w))
+        t4 = time_call(lambda: bd.sd_shard_draw(pv, qv, v0, all_w, all_stats, 0, n0, wl.uniforms, w0, out=o_tok))
+        shard_bytes = (2 * M + B * (wl.Kp - K)) * vs * es
+        calls[f"sd_verify_sharded_1_of_{G}"] = {
+            "shard_columns": vs, "stats_ms": t1, "decide_ms": t2, "weights_ms": t3, "draw_ms": t4,
+            "ms": t1 + t2 + t3 + t4, "stats_bytes": int(shard_bytes), "stats_gbs": shard_bytes / (t1 * 1e-3) / 1e9,
+            "exchange_bytes_per_gpu": int(B * wl.Kp * 24 + B * 16 + B * 4)}
 
     simulator = None
     if args.simulator_runs > 0:
