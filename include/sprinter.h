@@ -61,7 +61,9 @@ typedef enum {
     SPR_OP_REPLACE_SAMPLE = 1,
     SPR_OP_SD_VERIFY = 2,
     SPR_OP_SPRINTER_STEP = 3,
-    SPR_OP_SD_SHARD = 4
+    SPR_OP_SD_SHARD = 4,
+    SPR_OP_VERIFIER_LABELS = 5,
+    SPR_OP_VERIFIER_TRAIN = 6
 } spr_op;
 
 /* Which verifier kernel sprinter_verify() uses.  AUTO picks the tensor-core
@@ -72,7 +74,8 @@ typedef enum { SPR_VERIFIER_AUTO = 0, SPR_VERIFIER_SIMT = 1, SPR_VERIFIER_TENSOR
  * B is the number of draws n and K, d, h are ignored; for SPR_OP_SD_VERIFY d
  * and h are ignored; for SPR_OP_SPRINTER_VERIFY V is ignored; SPR_OP_SPRINTER_STEP
  * uses all of them; for SPR_OP_SD_SHARD V is the width of this GPU's vocabulary
- * shard and d, h are ignored.  Returns 0 for invalid arguments.  A workspace sized for the
+ * shard and d, h are ignored; SPR_OP_VERIFIER_LABELS uses B, K, V; SPR_OP_VERIFIER_TRAIN
+ * uses d only.  Returns 0 for invalid arguments.  A workspace sized for the
  * largest op serves all of them. */
 size_t spr_workspace_bytes(int op, int B, int K, int V, int d, int h, int dt);
 
@@ -233,6 +236,52 @@ int sd_shard_draw(const void *p_shard, const void *q_shard, int64_t ldv, int Vs,
                   const float *all_stats, int G, int rank, const int32_t *accepted_len, const float *uniforms,
                   int B, int K, int Kp, int dt, int32_t *correction_token, float *residual_mass, void *ws,
                   size_t ws_bytes, void *cuda_stream);
+
+/*
+ * verifier_labels - training labels of the verifier.
+ *
+ * Defined by: Section 3.2 ("Verifier Training Methodology"): a (prefix, draft token x) pair
+ * is labelled 1 if q(x)/p(x) <= lambda and 0 otherwise; lambda = 1 is the ideal verifier of
+ * Section 3, the appendix on training details uses lambda in {1, 1.2, 1.5}.
+ *
+ * p_logits [B,Kp,ldv] dt (Kp >= K; only the first K rows of a sequence are read),
+ * q_logits [B,K,ldv] dt, draft_tokens [B,K] int32 (device).  lambdas: HOST array of
+ * n_lambda <= 8 thresholds (read during the call).  p, q = softmax of the rows; the ratio
+ * is formed in log space in double precision from fp32 row statistics.
+ *   labels [n_lambda,B,K] uint8 (device): labels[l,b,k] = (q(x)/p(x) <= lambdas[l])
+ *   ratio  [B,K] f32 (device, optional):  q(x)/p(x), +inf where p(x) = 0
+ * Each logits row is read once (2*V*es bytes per token).  Device-detected: draft token
+ * outside [0,V) -> labels 0, ratio -1, SPR_ERR_BAD_TOKEN.
+ * Workspace: spr_workspace_bytes(SPR_OP_VERIFIER_LABELS, B, K, V, 0, 0, dt).
+ */
+int verifier_labels(const void *p_logits, const void *q_logits, int64_t ldv, const int32_t *draft_tokens, int B,
+                    int K, int Kp, int V, int dt, const float *lambdas, int n_lambda, uint8_t *labels, float *ratio,
+                    void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * verifier_train_step - one optimiser step of the single-layer verifier.
+ *
+ * Defined by: Section 3.2 ("Verifier architecture used for evaluation"): V(s) = sigmoid(b +
+ * w.s) on the draft model's last hidden state, trained with Adam on the binary
+ * cross-entropy loss.  One call is one Adam step (Kingma & Ba, Algorithm 1, with bias
+ * correction) on the mean loss over the N samples passed:
+ *   z_i = b + w.s_i,  loss = (1/N) sum_i [ln(1 + e^{z_i}) - y_i z_i],
+ *   g = (1/N) sum_i (sigmoid(z_i) - y_i) (s_i, 1),
+ *   m <- beta1 m + (1-beta1) g,  v <- beta2 v + (1-beta2) g^2,
+ *   theta <- theta - lr (m / (1-beta1^t)) / (sqrt(v / (1-beta2^t)) + eps).
+ * The batch is whatever the caller passes; early stopping is the caller's loop over `loss`.
+ *
+ * hidden [N,d] dt (device, 16-byte aligned, d a multiple of 16/es and at most 4096 for
+ * bf16, 2048 for fp32: otherwise SPR_ERR_UNSUPPORTED), labels [N] uint8 in {0,1} (device),
+ * theta, adam_m, adam_v [d+1] f32 (device; weights then bias; updated in place; start m
+ * and v at zero), t >= 1 the step number, loss [1] f32 (device, optional): the loss BEFORE
+ * the update.  Every hidden state is read once (N*d*es bytes per step); sums have a fixed
+ * order, so a step is reproducible bit for bit.
+ * Workspace: spr_workspace_bytes(SPR_OP_VERIFIER_TRAIN, 0, 0, 0, d, 0, dt).
+ */
+int verifier_train_step(const void *hidden, const uint8_t *labels, int64_t N, int d, int dt, float *theta,
+                        float *adam_m, float *adam_v, int t, float lr, float beta1, float beta2, float eps,
+                        float *loss, void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
  * sprinter_simulate - run lengths of an i.i.d. verifier (Monte-Carlo of Theorems 2 and 3).

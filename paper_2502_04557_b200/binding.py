@@ -16,6 +16,7 @@ from . import build as _build
 
 F32, BF16 = 0, 1
 OP_SPRINTER_VERIFY, OP_REPLACE_SAMPLE, OP_SD_VERIFY, OP_SPRINTER_STEP, OP_SD_SHARD = 0, 1, 2, 3, 4
+OP_VERIFIER_LABELS, OP_VERIFIER_TRAIN = 5, 6
 PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
 
 EXPORTS = [
@@ -24,6 +25,7 @@ EXPORTS = [
     "spr_host_arena_bytes", "sprinter_verify_host", "replace_sample_host", "sd_verify_host",
     "spr_set_stage_events", "replace_sample_static", "sprinter_step", "sprinter_simulate",
     "sd_shard_stats", "sd_shard_decide", "sd_shard_weights", "sd_shard_draw",
+    "verifier_labels", "verifier_train_step",
 ]
 
 
@@ -80,6 +82,10 @@ def lib():
         L.sd_shard_draw.restype = i32
         L.sd_shard_draw.argtypes = [vp, vp, i64, i32, i32, vp, vp, i32, i32, vp, vp, i32, i32, i32, i32,
                                     vp, vp, vp, sz, vp]
+        L.verifier_labels.restype = i32
+        L.verifier_labels.argtypes = [vp, vp, i64, vp, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp, sz, vp]
+        L.verifier_train_step.restype = i32
+        L.verifier_train_step.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, i32, f32, f32, f32, f32, vp, vp, sz, vp]
         L.spr_host_arena_bytes.restype = sz
         L.spr_host_arena_bytes.argtypes = [i32, i32, i32, i32, i64, i32, i32, i32]
         L.sprinter_verify_host.restype = i32
@@ -390,6 +396,53 @@ def sd_shard_draw(p_shard, q_shard, v0: int, all_weights, all_stats, rank: int, 
                              _ptr(ws.buf), ws.nbytes, _stream())
     _check("sd_shard_draw", rc)
     return out
+
+
+# ---------------------------------------------------------------------------- fitting the verifier
+
+
+def verifier_labels(p_logits, q_logits, V: int, draft_tokens, lambdas, ws: Workspace, want_ratio: bool = True):
+    """p_logits [B,Kp,ldv], q_logits [B,K,ldv], draft_tokens i32 [B,K]; lambdas: up to 8 floats.
+
+    Returns (labels u8 [len(lambdas),B,K], ratio f32 [B,K] or None) with ratio = q(x)/p(x)."""
+    _dev(p_logits, name="p_logits")
+    _dev(q_logits, p_logits.dtype, "q_logits")
+    B, Kp, ldv = p_logits.shape
+    K = q_logits.shape[1]
+    _dev(draft_tokens, torch.int32, "draft_tokens")
+    if q_logits.shape[0] != B or q_logits.shape[2] != ldv or tuple(draft_tokens.shape) != (B, K):
+        raise ValueError("shapes of p_logits, q_logits and draft_tokens disagree")
+    lam = (C.c_float * len(lambdas))(*[float(x) for x in lambdas])
+    dev = p_logits.device
+    labels = torch.empty((len(lambdas), B, K), dtype=torch.uint8, device=dev)
+    ratio = torch.empty((B, K), dtype=torch.float32, device=dev) if want_ratio else None
+    rc = lib().verifier_labels(_ptr(p_logits), _ptr(q_logits), ldv, _ptr(draft_tokens), B, K, Kp, V,
+                               _dt(p_logits), C.cast(lam, C.c_void_p), len(lambdas), _ptr(labels), _ptr(ratio),
+                               _ptr(ws.buf), ws.nbytes, _stream())
+    _check("verifier_labels", rc)
+    return labels, ratio
+
+
+def verifier_train_step(hidden, labels, theta, adam_m, adam_v, t: int, lr: float, ws: Workspace,
+                        beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8, loss=None):
+    """One Adam step on the mean BCE loss of sigmoid(b + w.s): hidden [N,d], labels u8 [N], theta /
+    adam_m / adam_v f32 [d+1] (updated in place).  Returns the loss before the step (f32 [1])."""
+    _dev(hidden, name="hidden")
+    N, d = hidden.shape
+    _dev(labels, torch.uint8, "labels")
+    for name, a in (("theta", theta), ("adam_m", adam_m), ("adam_v", adam_v)):
+        _dev(a, torch.float32, name)
+        if a.numel() != d + 1:
+            raise ValueError(f"{name} must have d + 1 entries")
+    if labels.numel() != N:
+        raise ValueError("labels must have one entry per hidden state")
+    if loss is None:
+        loss = torch.empty((1,), dtype=torch.float32, device=hidden.device)
+    rc = lib().verifier_train_step(_ptr(hidden), _ptr(labels), N, d, _dt(hidden), _ptr(theta), _ptr(adam_m),
+                                   _ptr(adam_v), t, lr, beta1, beta2, eps, _ptr(loss), _ptr(ws.buf), ws.nbytes,
+                                   _stream())
+    _check("verifier_train_step", rc)
+    return loss
 
 
 # ---------------------------------------------------------------------------- host buffers

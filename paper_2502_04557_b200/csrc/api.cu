@@ -192,6 +192,12 @@ size_t spr_workspace_bytes(int op, int B, int K, int V, int d, int h, int dt)
     case SPR_OP_SD_SHARD:   // V = shard width; sized for a bonus row
         if (K <= 0 || V <= 0 || (int64_t)B * (K + 1) > 0x7fffffff) return 0;
         return shard_ws_layout(B, K, K + 1, stat_max_segments_per_row(V, dt), stat_steps_per_row(V, dt)).end;
+    case SPR_OP_VERIFIER_LABELS:
+        if (K <= 0 || V <= 0 || (int64_t)B * K > 0x7fffffff) return 0;
+        return label_ws_layout(B, K, stat_max_segments_per_row(V, dt)).end;
+    case SPR_OP_VERIFIER_TRAIN:
+        if (d <= 0) return 0;
+        return train_ws_bytes(d);
     default:
         return 0;
     }

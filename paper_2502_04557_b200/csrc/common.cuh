@@ -127,6 +127,30 @@ __host__ __device__ inline ShardWs shard_ws_layout(int B, int K, int Kp, int S, 
     return w;
 }
 
+struct LabelWs {             // verifier_labels: row records of the statistics pass
+    size_t row_counters;     // int32 [M]
+    size_t part;             // float4 [M*S]
+    size_t stats;            // float [M*6]
+    size_t end;
+};
+__host__ __device__ inline LabelWs label_ws_layout(int B, int K, int S)
+{
+    const size_t M = (size_t)B * K;
+    LabelWs w;
+    w.row_counters = kHeaderBytes;
+    w.part = align_up(w.row_counters + 4 * M, 256);
+    w.stats = align_up(w.part + 16 * M * S, 256);
+    w.end = align_up(w.stats + 24 * M, 256);
+    return w;
+}
+
+// verifier_train_step: per-CTA gradient sums, float [kTrainMaxCtas, d + 2]
+constexpr int kTrainMaxCtas = 592;   // 148 SMs x 4
+__host__ __device__ inline size_t train_ws_bytes(int d)
+{
+    return align_up(kHeaderBytes + 4 * (size_t)kTrainMaxCtas * ((size_t)d + 2), 256);
+}
+
 struct VerifyWs {
     size_t counter;          // int32 [1 + max(row tiles, B)]   CTAs finished per tile / tokens per sequence
     size_t counters_end;

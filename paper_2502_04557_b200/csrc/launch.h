@@ -61,10 +61,11 @@ struct ShardStatsParams {
     const void *q;  // [B,K,ldv]
     int64_t ldv;
     int V, v0, K, Kp, chunks, iters;
+    int Kr;                       // positions per sequence that get a record (Kp, or K without the bonus row)
     const int32_t *draft_tokens;  // [B,K] global token ids
-    float *stats;                 // [B*Kp, 6]
-    int *row_counters;            // [B*Kp]
-    float4 *part;                 // [B*Kp*chunks]
+    float *stats;                 // [B*Kr, 6]
+    int *row_counters;            // [B*Kr]
+    float4 *part;                 // [B*Kr*chunks]
 };
 
 struct ShardDecideParams {

@@ -51,9 +51,10 @@ __device__ __forceinline__ float logit_at(const T *row, int x)
     return __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(row)[x]);
 }
 
-// One CTA per (p row, segment); row r = b*Kp + k pairs with q row b*K + k when k < K (the
-// bonus row k = K has no q row).  The CTA that finishes a row last merges its segments in
-// segment order and writes the row's record.
+// One CTA per (row, segment); row r = b*Kr + k (the first Kr <= Kp positions of every
+// sequence) reads p row b*Kp + k and, when k < K, q row b*K + k (the bonus row k = K has no q
+// row).  The CTA that finishes a row last merges its segments in segment order and writes
+// the row's record.
 template <typename T, int ITERS>
 __global__ void __launch_bounds__(kThreads, 4) shard_stats_kernel(const ShardStatsParams prm)
 {
@@ -62,10 +63,10 @@ __global__ void __launch_bounds__(kThreads, 4) shard_stats_kernel(const ShardSta
     const int C = prm.chunks;
     const int64_t row = blockIdx.x / C;
     const int c = blockIdx.x % C;
-    const int b = (int)(row / prm.Kp), k = (int)(row % prm.Kp);
+    const int b = (int)(row / prm.Kr), k = (int)(row % prm.Kr);
     const bool has_q = k < prm.K;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const T *prow = static_cast<const T *>(prm.p) + row * prm.ldv;
+    const T *prow = static_cast<const T *>(prm.p) + ((int64_t)b * prm.Kp + k) * prm.ldv;
     const T *qrow = has_q ? static_cast<const T *>(prm.q) + ((int64_t)b * prm.K + k) * prm.ldv : prow;
 
     MS mp{neg_inf(), 0.f}, mq{neg_inf(), 0.f};

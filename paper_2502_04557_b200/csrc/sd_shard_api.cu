@@ -69,6 +69,7 @@ int sd_shard_stats(const void *p_shard, const void *q_shard, int64_t ldv, int Vs
     sp.v0 = v0;
     sp.K = K;
     sp.Kp = Kp;
+    sp.Kr = Kp;
     draw_geometry(B * Kp, stat_steps_per_row(Vs, dt), &sp.chunks, &sp.iters);
     sp.draft_tokens = draft_tokens;
     sp.stats = stats;

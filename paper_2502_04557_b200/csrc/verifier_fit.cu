@@ -1,0 +1,311 @@
+// Preparing and fitting the verifier (Section 3.2): training labels 1[q(x)/p(x) <= lambda]
+// from the two models' logits, and optimiser steps (binary cross-entropy + Adam) for the
+// linear-layer + sigmoid verifier on the draft model's hidden states.
+#include <string.h>
+
+#include "launch.h"
+#include "vocab_common.cuh"
+
+namespace spr {
+
+namespace {
+
+constexpr int kStatRecord = 6;       // floats per row from shard_stats_kernel
+constexpr int kMaxLambdas = 8;
+constexpr int kTrainMaxVpl = 16;     // 16-byte vectors per lane: d <= 4096 (bf16) or 2048 (fp32)
+
+// ---------------------------------------------------------------------------- labels
+struct LabelParams {
+    const float *stats;            // [M, 6] whole-row records (one shard covering the vocabulary)
+    int64_t M;
+    int V;
+    const int32_t *draft_tokens;   // [M]
+    int n_lambda;
+    float lambdas[kMaxLambdas];
+    uint8_t *labels;               // [n_lambda, M]
+    float *ratio;                  // [M] or null
+    int *status;
+};
+
+__global__ void __launch_bounds__(256) labels_kernel(const LabelParams prm)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= prm.M) return;
+    const float *rec = prm.stats + i * kStatRecord;
+    const int x = prm.draft_tokens[i];
+    double ratio = -1.0;
+    const bool valid = x >= 0 && x < prm.V;
+    if (valid) {
+        const double logP = (double)rec[4] - (double)rec[0] - log((double)rec[1]);
+        const double logQ = (double)rec[5] - (double)rec[2] - log((double)rec[3]);
+        ratio = exp(logQ - logP);
+    } else {
+        raise_status(prm.status, SPR_ERR_BAD_TOKEN);
+    }
+    for (int l = 0; l < prm.n_lambda; ++l)
+        prm.labels[(int64_t)l * prm.M + i] = (valid && ratio <= (double)prm.lambdas[l]) ? 1 : 0;
+    if (prm.ratio) prm.ratio[i] = (float)ratio;
+}
+
+// ---------------------------------------------------------------------------- training
+struct TrainParams {
+    const void *hidden;      // [N, d]
+    const uint8_t *labels;   // [N]
+    int64_t N;
+    int d;
+    float *theta, *m, *v;    // [d+1]: weights, then the bias
+    int t;
+    float lr, beta1, beta2, eps;
+    float *loss;             // [1] or null
+    float *part;             // [ctas, d+2]: per-CTA sums of the gradient terms, then of the loss
+    int ctas;
+};
+
+// Gradient pass: one warp per sample, samples dealt to warps in a fixed pattern; a lane keeps
+// its columns of the row in registers, so every hidden state is read from HBM exactly once.
+//   z = b + w.s,  r = sigma(z) - y,  grad_w += r s,  grad_b += r,  loss += ln(1 + e^z) - y z
+// The warps of a CTA add their sums in warp order; the CTA's sums go to part[blockIdx.x].
+template <typename T, int VPL>
+__global__ void __launch_bounds__(kThreads, 1) train_grad_kernel(const TrainParams prm)
+{
+    constexpr int N = Vec<T>::N;
+    extern __shared__ float smem[];
+    const int d = prm.d;
+    float *sw = smem;              // [d] weights
+    float *red = smem + d;         // [d + 2] CTA sums
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nv = d / N;          // vectors per row
+    for (int j = tid; j < d; j += kThreads) sw[j] = prm.theta[j];
+    const float bias = prm.theta[d];
+    __syncthreads();
+
+    float acc[VPL * N];
+#pragma unroll
+    for (int e = 0; e < VPL * N; ++e) acc[e] = 0.f;
+    float acc_b = 0.f, acc_loss = 0.f;
+    const T *base = static_cast<const T *>(prm.hidden);
+    for (int64_t row = (int64_t)blockIdx.x * kWarps + warp; row < prm.N; row += (int64_t)gridDim.x * kWarps) {
+        const T *x = base + row * d;
+        uint4 raw[VPL];
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) {
+            const int vi = j * 32 + lane;
+            raw[j] = vi < nv ? ld_stream(reinterpret_cast<const uint4 *>(x) + vi) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        float dot = 0.f;
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) {
+            const int vi = j * 32 + lane;
+            if (vi < nv) {
+                float f[N];
+                Vec<T>::unpack(raw[j], f);
+#pragma unroll
+                for (int e = 0; e < N; ++e) dot = fmaf(f[e], sw[vi * N + e], dot);
+            }
+        }
+        const float z = warp_sum(dot) + bias;
+        const float y = (float)prm.labels[row];
+        const float r = 1.f / (1.f + expf(-z)) - y;
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) {
+            float f[N];
+            Vec<T>::unpack(raw[j], f);     // zero beyond the row
+#pragma unroll
+            for (int e = 0; e < N; ++e) acc[j * N + e] = fmaf(r, f[e], acc[j * N + e]);
+        }
+        acc_b += r;
+        acc_loss += fmaxf(z, 0.f) + log1pf(expf(-fabsf(z))) - y * z;
+    }
+
+    for (int w = 0; w < kWarps; ++w) {     // fixed order: warp 0 stores, the others add
+        if (warp == w) {
+#pragma unroll
+            for (int j = 0; j < VPL; ++j) {
+                const int vi = j * 32 + lane;
+                if (vi < nv) {
+#pragma unroll
+                    for (int e = 0; e < N; ++e) {
+                        float *dst = red + vi * N + e;
+                        *dst = w == 0 ? acc[j * N + e] : *dst + acc[j * N + e];
+                    }
+                }
+            }
+            if (lane == 0) {
+                red[d] = w == 0 ? acc_b : red[d] + acc_b;
+                red[d + 1] = w == 0 ? acc_loss : red[d + 1] + acc_loss;
+            }
+        }
+        __syncthreads();
+    }
+    float *out = prm.part + (int64_t)blockIdx.x * (d + 2);
+    for (int j = tid; j < d + 2; j += kThreads) out[j] = red[j];
+}
+
+// One thread per parameter: sums the CTA partials in CTA order, divides by N, applies the
+// bias-corrected Adam update (arithmetic in double, state kept in float).
+__global__ void __launch_bounds__(256) train_adam_kernel(const TrainParams prm)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    const int d = prm.d;
+    if (j > d + 1) return;
+    double sum = 0.0;
+    for (int c = 0; c < prm.ctas; ++c) sum += (double)prm.part[(int64_t)c * (d + 2) + j];
+    sum /= (double)prm.N;
+    if (j == d + 1) {
+        if (prm.loss) *prm.loss = (float)sum;
+        return;
+    }
+    const double b1 = (double)prm.beta1, b2 = (double)prm.beta2;
+    const double m = b1 * (double)prm.m[j] + (1.0 - b1) * sum;
+    const double v = b2 * (double)prm.v[j] + (1.0 - b2) * sum * sum;
+    const double m_hat = m / (1.0 - pow(b1, (double)prm.t));
+    const double v_hat = v / (1.0 - pow(b2, (double)prm.t));
+    prm.m[j] = (float)m;
+    prm.v[j] = (float)v;
+    prm.theta[j] = (float)((double)prm.theta[j] - (double)prm.lr * m_hat / (sqrt(v_hat) + (double)prm.eps));
+}
+
+template <typename T, int VPL>
+cudaError_t launch_grad(const TrainParams &tp, cudaStream_t st)
+{
+    const size_t smem = sizeof(float) * (2 * (size_t)tp.d + 2);
+    cudaError_t e = cudaFuncSetAttribute(train_grad_kernel<T, VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e != cudaSuccess) return e;
+    train_grad_kernel<T, VPL><<<tp.ctas, kThreads, smem, st>>>(tp);
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_grad_any(const TrainParams &tp, cudaStream_t st)
+{
+    const int vpl = (tp.d / Vec<T>::N + 31) / 32;
+    if (vpl <= 1) return launch_grad<T, 1>(tp, st);
+    if (vpl <= 2) return launch_grad<T, 2>(tp, st);
+    if (vpl <= 3) return launch_grad<T, 3>(tp, st);
+    if (vpl <= 4) return launch_grad<T, 4>(tp, st);
+    if (vpl <= 8) return launch_grad<T, 8>(tp, st);
+    return launch_grad<T, 16>(tp, st);
+}
+
+bool dtype_ok(int dt) { return dt == SPR_F32 || dt == SPR_BF16; }
+bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+template <typename T>
+T *at(void *ws, size_t off)
+{
+    return reinterpret_cast<T *>(static_cast<char *>(ws) + off);
+}
+int finish(cudaError_t e) { return e == cudaSuccess ? SPR_OK : report_cuda_error(e); }
+
+}  // namespace
+
+int train_ctas(int64_t N) { return (int)max((int64_t)1, min((int64_t)kTrainMaxCtas, (N + kWarps - 1) / kWarps)); }
+
+}  // namespace spr
+
+using namespace spr;
+
+extern "C" {
+
+int verifier_labels(const void *p_logits, const void *q_logits, int64_t ldv, const int32_t *draft_tokens, int B,
+                    int K, int Kp, int V, int dt, const float *lambdas, int n_lambda, uint8_t *labels, float *ratio,
+                    void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
+    if (B < 0 || K <= 0 || Kp < K || V <= 0 || V > (1 << 30) || ldv < V || (int64_t)B * K > 0x7fffffff ||
+        n_lambda <= 0 || n_lambda > kMaxLambdas || !lambdas)
+        return SPR_ERR_INVALID_ARG;
+    if (B == 0) return SPR_OK;
+    if (!p_logits || !q_logits || !draft_tokens || !labels) return SPR_ERR_INVALID_ARG;
+    const size_t es = elem_size(dt);
+    if (!aligned(p_logits, es) || !aligned(q_logits, es) || !aligned(draft_tokens, 4) || (ratio && !aligned(ratio, 4)))
+        return SPR_ERR_INVALID_ARG;
+    const LabelWs lay = label_ws_layout(B, K, stat_max_segments_per_row(V, dt));
+    if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
+    int rc = device_supported();
+    if (rc != SPR_OK) return rc;
+
+    const int64_t M = (int64_t)B * K;
+    ShardStatsParams sp;
+    memset(&sp, 0, sizeof sp);
+    sp.p = p_logits;
+    sp.q = q_logits;
+    sp.ldv = ldv;
+    sp.V = V;
+    sp.v0 = 0;
+    sp.K = K;
+    sp.Kp = Kp;
+    sp.Kr = K;   // the bonus row has no draft token
+    draw_geometry((int)M, stat_steps_per_row(V, dt), &sp.chunks, &sp.iters);
+    sp.draft_tokens = draft_tokens;
+    sp.stats = at<float>(ws, lay.stats);
+    sp.row_counters = at<int>(ws, lay.row_counters);
+    sp.part = at<float4>(ws, lay.part);
+    LabelParams lp;
+    memset(&lp, 0, sizeof lp);
+    lp.stats = sp.stats;
+    lp.M = M;
+    lp.V = V;
+    lp.draft_tokens = draft_tokens;
+    lp.n_lambda = n_lambda;
+    for (int l = 0; l < n_lambda; ++l) lp.lambdas[l] = lambdas[l];
+    lp.labels = labels;
+    lp.ratio = ratio;
+    lp.status = at<int>(ws, 0);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaMemsetAsync(sp.row_counters, 0, sizeof(int) * (size_t)M, st);
+    if (e == cudaSuccess) e = launch_shard_stats(sp, M, dt, st);
+    if (e == cudaSuccess) {
+        labels_kernel<<<(unsigned)((M + 255) / 256), 256, 0, st>>>(lp);
+        e = cudaGetLastError();
+    }
+    return finish(e);
+}
+
+int verifier_train_step(const void *hidden, const uint8_t *labels, int64_t N, int d, int dt, float *theta,
+                        float *adam_m, float *adam_v, int t, float lr, float beta1, float beta2, float eps,
+                        float *loss, void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
+    if (N < 0 || d <= 0 || t < 1 || !(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) ||
+        !(eps >= 0.f) || !(lr == lr))
+        return SPR_ERR_INVALID_ARG;
+    const int vec = vec_elems(dt);
+    if (d % vec != 0 || d / vec > 32 * kTrainMaxVpl) return SPR_ERR_UNSUPPORTED;
+    if (N == 0) return SPR_OK;
+    if (!hidden || !labels || !theta || !adam_m || !adam_v) return SPR_ERR_INVALID_ARG;
+    if (!aligned(hidden, 16) || !aligned(theta, 4) || !aligned(adam_m, 4) || !aligned(adam_v, 4) ||
+        (loss && !aligned(loss, 4)))
+        return SPR_ERR_INVALID_ARG;
+    const size_t need = train_ws_bytes(d);
+    if (!ws || !aligned(ws, 256) || ws_bytes < need) return SPR_ERR_WORKSPACE;
+    int rc = device_supported();
+    if (rc != SPR_OK) return rc;
+
+    TrainParams tp;
+    memset(&tp, 0, sizeof tp);
+    tp.hidden = hidden;
+    tp.labels = labels;
+    tp.N = N;
+    tp.d = d;
+    tp.theta = theta;
+    tp.m = adam_m;
+    tp.v = adam_v;
+    tp.t = t;
+    tp.lr = lr;
+    tp.beta1 = beta1;
+    tp.beta2 = beta2;
+    tp.eps = eps;
+    tp.loss = loss;
+    tp.part = at<float>(ws, kHeaderBytes);
+    tp.ctas = train_ctas(N);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = dt == SPR_F32 ? launch_grad_any<float>(tp, st) : launch_grad_any<__nv_bfloat16>(tp, st);
+    if (e == cudaSuccess) {
+        train_adam_kernel<<<(d + 2 + 255) / 256, 256, 0, st>>>(tp);
+        e = cudaGetLastError();
+    }
+    return finish(e);
+}
+
+}  // extern "C"

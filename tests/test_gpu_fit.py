@@ -1,0 +1,183 @@
+"""verifier_labels and verifier_train_step (Section 3.2) against the float64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import RTOL, to_np
+from oracle import training
+from test_gpu_parity import _rand_problem
+
+pytestmark = pytest.mark.gpu
+
+LAMBDAS = [1.0, 1.2, 1.5]          # the thresholds the paper trains with
+LABEL_MARGIN = 1e-4                # labels are compared where |ratio / lambda - 1| exceeds this
+
+
+@pytest.fixture(scope="module")
+def spr():
+    import paper_2502_04557_b200 as s
+    s.lib()
+    return s
+
+
+def bd(spr):
+    return spr.binding
+
+
+def check_labels(spr, p, q, V, x, lambdas, dtype):
+    B, K = x.shape
+    ws = spr.Workspace(spr.workspace_bytes(bd(spr).OP_VERIFIER_LABELS, B, K, V, 0, 0, bd(spr)._dt(p)))
+    labels, ratio = bd(spr).verifier_labels(p.cuda(), q.cuda(), V, x.cuda(), lambdas, ws)
+    status = ws.device_status()
+    want_labels, want_ratio = training.verifier_labels(to_np(p), to_np(q), V, to_np(x), lambdas)
+    got_ratio = ratio.cpu().double().numpy()
+    finite = np.isfinite(want_ratio) & (want_ratio > 0)
+    assert np.array_equal(np.isfinite(got_ratio), np.isfinite(want_ratio))
+    assert np.all(np.abs(got_ratio[finite] / want_ratio[finite] - 1.0) <= RTOL[dtype])
+    assert np.array_equal(got_ratio[want_ratio < 0], want_ratio[want_ratio < 0])      # invalid tokens: -1
+    got = labels.cpu().numpy()
+    skipped = 0
+    for i, lam in enumerate(lambdas):
+        clear = ~finite | (np.abs(want_ratio / float(np.float32(lam)) - 1.0) > LABEL_MARGIN)
+        skipped += int((~clear).sum())
+        assert np.array_equal(got[i][clear], want_labels[i][clear]), f"lambda {lam}"
+    assert skipped <= max(1, x.size // 50)
+    return status, want_labels
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("B,K,V,ldv,Kp", [
+    (3, 1, 2, None, 2), (5, 2, 7, None, 2), (4, 3, 1000, None, 4), (2, 33, 129, 131, 34),
+    (3, 4, 8191, None, 4), (2, 2, 8193, 8200, 3), (2, 5, 32769, None, 6), (1, 40, 50257, None, 40),
+])
+def test_labels_ragged_shapes(spr, dtype, B, K, V, ldv, Kp):
+    p, q, x, _ = _rand_problem(B, K, V, dtype, seed=3 + B * 1000 + K * 10 + V, ldv=ldv, Kp=Kp)
+    status, want = check_labels(spr, p, q, V, x, LAMBDAS, dtype)
+    assert status == 0
+    if V > 100:
+        assert 0 < want.sum() < want.size
+
+
+@pytest.mark.parametrize("name,B", [("tiny", None), ("gpt2", 6), ("llama2", 8), ("llama3", 3)])
+def test_labels_on_the_workload_shapes(spr, name, B):
+    wl = spr.workloads.make(name, "cpu", B=B)
+    status, _ = check_labels(spr, wl.p_logits, wl.q_logits, wl.V, wl.draft_tokens, LAMBDAS + [0.5, 3.0],
+                             wl.q_logits.dtype)
+    assert status == 0
+
+
+def test_labels_invalid_token_zero_probability_and_limits(spr):
+    B, K, V = 2, 3, 600
+    p, q, x, _ = _rand_problem(B, K, V, torch.float32, seed=11)
+    x[0, 1] = -1
+    x[1, 2] = V
+    p[1, 0, int(x[1, 0])] = float("-inf")          # p(x) = 0: ratio +inf, never labelled 1
+    status, want = check_labels(spr, p, q, V, x, [1.0, 1e30], torch.float32)
+    assert status == 6                                 # SPR_ERR_BAD_TOKEN
+    assert want[:, 0, 1].sum() == 0 and want[:, 1, 2].sum() == 0 and want[:, 1, 0].sum() == 0
+    ws = spr.Workspace(spr.workspace_bytes(bd(spr).OP_VERIFIER_LABELS, B, K, V, 0, 0, spr.F32))
+    with pytest.raises(spr.SprinterError) as e:        # more thresholds than one call takes
+        bd(spr).verifier_labels(p.cuda(), q.cuda(), V, x.cuda(), [1.0] * 9, ws)
+    assert e.value.status == 1
+    empty = bd(spr).verifier_labels(torch.empty((0, K, V), device="cuda"), torch.empty((0, K, V), device="cuda"), V,
+                                    torch.empty((0, K), dtype=torch.int32, device="cuda"), [1.0], ws)
+    assert empty[0].shape == (1, 0, K)
+
+
+# ----------------------------------------------------------------------------- training
+def teacher_problem(N, d, dtype, seed, noise=0.5):
+    g = torch.Generator().manual_seed(seed)
+    S = torch.randn((N, d), generator=g).to(dtype)
+    w = torch.randn((d,), generator=g) / d ** 0.5
+    y = ((S.float() @ w + noise * torch.randn((N,), generator=g)) > 0.1).to(torch.uint8)
+    return S, y
+
+
+def run_steps(spr, S, y, steps, lr, theta0=None, **hyper):
+    N, d = S.shape
+    ws = spr.Workspace(spr.workspace_bytes(bd(spr).OP_VERIFIER_TRAIN, 0, 0, 0, d, 0, bd(spr)._dt(S)))
+    Sg, yg = S.cuda(), y.cuda()
+    theta = torch.zeros(d + 1, device="cuda") if theta0 is None else theta0.clone().cuda()
+    m, v = torch.zeros(d + 1, device="cuda"), torch.zeros(d + 1, device="cuda")
+    hist = []
+    for t in range(1, steps + 1):
+        loss = bd(spr).verifier_train_step(Sg, yg, theta, m, v, t, lr, ws, **hyper)
+        hist.append((float(loss), theta.cpu().double().numpy().copy()))
+    return hist, (theta, m, v)
+
+
+@pytest.mark.parametrize("N,d,dtype", [
+    (5000, 768, torch.bfloat16), (1, 768, torch.bfloat16), (7, 64, torch.bfloat16), (20000, 256, torch.bfloat16),
+    (3000, 2048, torch.bfloat16), (2000, 4096, torch.bfloat16), (4001, 1000, torch.bfloat16),
+    (3000, 100, torch.float32), (1500, 2048, torch.float32), (999, 4, torch.float32),
+], ids=lambda v: str(v).replace("torch.", ""))
+def test_train_steps_match_the_oracle(spr, N, d, dtype):
+    """fp32 sums on the GPU against float64: the loss agrees to 2e-5 relative, and since an Adam
+    step is lr * m_hat / sqrt(v_hat) (of order lr whatever the gradient's size), a relative
+    gradient error e moves a parameter by about lr * e per step: bound 1e-3 * lr * t."""
+    S, y = teacher_problem(N, d, dtype, seed=N + d)
+    lr, steps = 0.02, 12
+    hist, _ = run_steps(spr, S, y, steps, lr)
+    Sn, yn = to_np(S), y.numpy()
+    theta, m, v = np.zeros(d + 1), np.zeros(d + 1), np.zeros(d + 1)
+    for t, (loss_gpu, theta_gpu) in enumerate(hist, 1):
+        loss, theta, m, v = training.verifier_train_step(Sn, yn, theta, m, v, t, lr)
+        assert abs(loss_gpu / loss - 1.0) < 2e-5, f"step {t}: loss {loss_gpu} vs {loss}"
+        err = np.abs(theta_gpu - theta).max()
+        assert err <= 1e-3 * lr * t, f"step {t}: max parameter error {err:.3e}"
+    assert hist[0][0] == pytest.approx(np.log(2.0), rel=1e-6)
+
+
+def test_train_other_hyperparameters_and_nonzero_start(spr):
+    S, y = teacher_problem(2500, 768, torch.bfloat16, seed=5)
+    g = torch.Generator().manual_seed(6)
+    theta0 = 0.05 * torch.randn(769, generator=g)
+    hyper = dict(beta1=0.5, beta2=0.9, eps=1e-6)
+    hist, _ = run_steps(spr, S, y, 8, 0.01, theta0=theta0, **hyper)
+    theta, m, v = theta0.double().numpy(), np.zeros(769), np.zeros(769)
+    for t, (loss_gpu, theta_gpu) in enumerate(hist, 1):
+        loss, theta, m, v = training.verifier_train_step(to_np(S), y.numpy(), theta, m, v, t, 0.01, **hyper)
+        assert abs(loss_gpu / loss - 1.0) < 2e-5
+        assert np.abs(theta_gpu - theta).max() <= 1e-3 * 0.01 * t
+
+
+def test_train_is_reproducible_and_rejects_unsupported_widths(spr):
+    S, y = teacher_problem(6000, 768, torch.bfloat16, seed=9)
+    a, sa = run_steps(spr, S, y, 5, 0.02)
+    b, sb = run_steps(spr, S, y, 5, 0.02)
+    assert [h[0] for h in a] == [h[0] for h in b]
+    assert all(torch.equal(x, z) for x, z in zip(sa, sb))
+    for d, dtype in [(770, torch.bfloat16), (8192, torch.bfloat16), (4096, torch.float32), (6, torch.float32)]:
+        ws = spr.Workspace(spr.workspace_bytes(bd(spr).OP_VERIFIER_TRAIN, 0, 0, 0, d, 0, bd(spr)._dt(torch.empty(0, dtype=dtype))))
+        z = torch.zeros(d + 1, device="cuda")
+        with pytest.raises(spr.SprinterError) as e:
+            bd(spr).verifier_train_step(torch.zeros((4, d), dtype=dtype, device="cuda"),
+                                        torch.zeros(4, dtype=torch.uint8, device="cuda"), z, z.clone(), z.clone(), 1,
+                                        0.01, ws)
+        assert e.value.status == 2
+
+
+def test_labels_then_training_then_the_verifier_call(spr):
+    """The preparation chain on the GPU alone: labels from the two models' logits, a linear
+    verifier fitted to hidden states that carry the label, and sprinter_verify using it."""
+    wl = spr.workloads.make("gpt2", "cuda", B=64)
+    B, K, V, d = wl.B, wl.K, wl.V, wl.hidden.shape[-1]
+    ws = spr.Workspace(max(spr.workspace_bytes(bd(spr).OP_VERIFIER_LABELS, B, K, V, 0, 0, spr.BF16),
+                           spr.workspace_bytes(bd(spr).OP_VERIFIER_TRAIN, 0, 0, 0, d, 0, spr.BF16),
+                           spr.workspace_bytes(0, B, K, V, d, 0, spr.BF16)))
+    labels, _ = bd(spr).verifier_labels(wl.p_logits, wl.q_logits, V, wl.draft_tokens, [1.2], ws)
+    y = labels[0].reshape(-1).contiguous()
+    assert 0.05 < y.float().mean() < 0.95
+    g = torch.Generator().manual_seed(1)
+    direction = torch.randn(d, generator=g).cuda() / d ** 0.5
+    hidden = torch.randn((B * K, d), generator=g).cuda()
+    hidden += (y.float() * 2 - 1)[:, None] * 4.0 * direction           # separable along one direction
+    hidden = hidden.to(torch.bfloat16).contiguous()
+    theta = torch.zeros(d + 1, device="cuda")
+    m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+    losses = [float(bd(spr).verifier_train_step(hidden, y, theta, m, v, t, 0.05, ws)) for t in range(1, 101)]
+    assert losses[-1] < 0.2 * losses[0]
+    scores, accept, _ = spr.sprinter_verify(hidden.view(B, K, d), theta[:d].to(torch.bfloat16).contiguous(), None, None,
+                                            theta[d:].contiguous(), 0.5, ws)
+    assert ws.device_status() == 0
+    assert (accept.reshape(-1) == y).float().mean() > 0.97
