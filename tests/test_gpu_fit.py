@@ -41,7 +41,7 @@ def check_labels(spr, p, q, V, x, lambdas, dtype):
         clear = ~finite | (np.abs(want_ratio / float(np.float32(lam)) - 1.0) > LABEL_MARGIN)
         skipped += int((~clear).sum())
         assert np.array_equal(got[i][clear], want_labels[i][clear]), f"lambda {lam}"
-    assert skipped <= max(1, x.size // 50)
+    assert skipped <= max(1, x.numel() // 50)
     return status, want_labels
 
 
