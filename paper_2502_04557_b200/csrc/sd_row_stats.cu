@@ -20,7 +20,6 @@ __global__ void __launch_bounds__(kThreads, 4) sd_row_stats_kernel(const SdParam
     __shared__ float4 s_part[kWarps];
     __shared__ int s_last;
 
-    pdl_trigger();                       // the correction draw may be scheduled behind this grid
     const int C = prm.chunks;            // segments per row
     const int64_t row = blockIdx.x / C;  // = b*K + k
     const int c = blockIdx.x % C;
@@ -48,23 +47,24 @@ __global__ void __launch_bounds__(kThreads, 4) sd_row_stats_kernel(const SdParam
         if (more) load_step<T>(qrow, first_q + nxt, V, lane, rq);
         if (!more) break;
     }
+    pdl_trigger();                       // the correction draw may be scheduled behind this grid
     mp = warp_ms(mp);
     mq = warp_ms(mq);
     if (lane == 0) s_part[warp] = make_float4(mp.m, mp.s, mq.m, mq.s);
     __syncthreads();
-    if (warp == 0) {
-        float4 v = lane < kWarps ? s_part[lane] : make_float4(neg_inf(), 0.f, neg_inf(), 0.f);
+    if (warp != 0) return;               // the other warps leave before the ticket's round trip
+    {
+        const float4 v = lane < kWarps ? s_part[lane] : make_float4(neg_inf(), 0.f, neg_inf(), 0.f);
         mp = warp_ms(MS{v.x, v.y});
         mq = warp_ms(MS{v.z, v.w});
-        if (lane == 0) {
-            prm.part[row * C + c] = make_float4(mp.m, mp.s, mq.m, mq.s);
-            __threadfence();
-            const int ticket = atomicAdd(&prm.row_counters[row], 1);
-            s_last = (ticket == C - 1);
-        }
     }
-    __syncthreads();
-    if (!s_last || warp != 0) return;
+    if (lane == 0) {
+        prm.part[row * C + c] = make_float4(mp.m, mp.s, mq.m, mq.s);
+        __threadfence();
+        s_last = (atomicAdd(&prm.row_counters[row], 1) == C - 1);
+    }
+    __syncwarp();
+    if (!s_last) return;
 
     // ---- this CTA saw the last chunk of the row: merge chunks in chunk order (warp 0)
     __threadfence();
