@@ -30,10 +30,10 @@ if ROOT not in sys.path:
 # capture summarised under profiles/; reported only while the kernel source is unchanged.
 NCU_TRAFFIC = {
     "sources": ("sd_row_stats.cu", "vocab_common.cuh", "common.cuh"),
-    "sha256": "305fa9cc1ad14a54eff43ef35244ff5a54f29d60c2e39741ebbf1d4395d0983f",
-    # (262,767,616 read + 3,982,336 written) / 512 tokens in the B = 32 capture; traffic grows
+    "sha256": "55c54fc662a742d6e0d4b76da7e20c83800f853dea1c3ce4e81f5214cb199761",
+    # (262,802,944 read + 3,682,048 written) / 512 tokens in the B = 32 capture; traffic grows
     # in proportion to the tokens, so a full launch is this times B*K
-    "bytes_per_unit": 520996,   # DRAM bytes per verified token at V = 128256, bf16
+    "bytes_per_unit": 520478,   # DRAM bytes per verified token at V = 128256, bf16
 }
 
 

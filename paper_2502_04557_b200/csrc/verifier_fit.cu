@@ -61,7 +61,8 @@ struct TrainParams {
     int ctas;
 };
 
-// Gradient pass: one warp per sample, samples dealt to warps in a fixed pattern; a lane keeps
+// Gradient pass (one resident wave of CTAs): one warp per sample, samples dealt to warps in a
+// fixed pattern; a lane keeps
 // its columns of the row in registers, so every hidden state is read from HBM exactly once.
 //   z = b + w.s,  r = sigma(z) - y,  grad_w += r s,  grad_b += r,  loss += ln(1 + e^z) - y z
 // The warps of a CTA add their sums in warp order; the CTA's sums go to part[blockIdx.x].
@@ -79,20 +80,32 @@ __global__ void __launch_bounds__(kThreads, 1) train_grad_kernel(const TrainPara
     const float bias = prm.theta[d];
     __syncthreads();
 
-    float acc[VPL * N];
+    uint64_t acc[VPL * N / 2];       // packed pairs of fp32 sums (two columns each)
 #pragma unroll
-    for (int e = 0; e < VPL * N; ++e) acc[e] = 0.f;
+    for (int e = 0; e < VPL * N / 2; ++e) acc[e] = pack2(0.f, 0.f);
     float acc_b = 0.f, acc_loss = 0.f;
     const T *base = static_cast<const T *>(prm.hidden);
-    for (int64_t row = (int64_t)blockIdx.x * kWarps + warp; row < prm.N; row += (int64_t)gridDim.x * kWarps) {
-        const T *x = base + row * d;
-        uint4 raw[VPL];
+    constexpr bool kPrefetch = VPL <= 4;   // short rows: keep the next row in flight as well
+    auto load_row = [&](int64_t row, uint4 (&dst)[VPL], float &y) {
+        const uint4 *x = reinterpret_cast<const uint4 *>(base + row * d);
 #pragma unroll
         for (int j = 0; j < VPL; ++j) {
             const int vi = j * 32 + lane;
-            raw[j] = vi < nv ? ld_stream(reinterpret_cast<const uint4 *>(x) + vi) : make_uint4(0u, 0u, 0u, 0u);
+            dst[j] = vi < nv ? ld_stream(x + vi) : make_uint4(0u, 0u, 0u, 0u);
         }
-        float dot = 0.f;
+        y = (float)prm.labels[row];
+    };
+    const int64_t stride = (int64_t)gridDim.x * kWarps;
+    int64_t row = (int64_t)blockIdx.x * kWarps + warp;
+    uint4 raw[VPL];
+    float y = 0.f;
+    if (row < prm.N) load_row(row, raw, y);
+    for (; row < prm.N; row += stride) {
+        uint4 nxt[VPL];
+        float y_nxt = 0.f;
+        const bool more = row + stride < prm.N;
+        if (kPrefetch && more) load_row(row + stride, nxt, y_nxt);
+        uint64_t dot2 = pack2(0.f, 0.f);   // even and odd columns apart
 #pragma unroll
         for (int j = 0; j < VPL; ++j) {
             const int vi = j * 32 + lane;
@@ -100,21 +113,32 @@ __global__ void __launch_bounds__(kThreads, 1) train_grad_kernel(const TrainPara
                 float f[N];
                 Vec<T>::unpack(raw[j], f);
 #pragma unroll
-                for (int e = 0; e < N; ++e) dot = fmaf(f[e], sw[vi * N + e], dot);
+                for (int e = 0; e < N; e += 2)
+                    dot2 = fma2(pack2(f[e], f[e + 1]), *reinterpret_cast<const uint64_t *>(&sw[vi * N + e]), dot2);
             }
         }
-        const float z = warp_sum(dot) + bias;
-        const float y = (float)prm.labels[row];
+        float d_even, d_odd;
+        unpack2(dot2, d_even, d_odd);
+        const float z = warp_sum(d_even + d_odd) + bias;
         const float r = 1.f / (1.f + expf(-z)) - y;
+        const uint64_t r2 = pack2(r, r);
 #pragma unroll
         for (int j = 0; j < VPL; ++j) {
             float f[N];
             Vec<T>::unpack(raw[j], f);     // zero beyond the row
 #pragma unroll
-            for (int e = 0; e < N; ++e) acc[j * N + e] = fmaf(r, f[e], acc[j * N + e]);
+            for (int e = 0; e < N; e += 2)
+                acc[(j * N + e) / 2] = fma2(r2, pack2(f[e], f[e + 1]), acc[(j * N + e) / 2]);
         }
         acc_b += r;
         acc_loss += fmaxf(z, 0.f) + log1pf(expf(-fabsf(z))) - y * z;
+        if (kPrefetch) {
+#pragma unroll
+            for (int j = 0; j < VPL; ++j) raw[j] = nxt[j];
+            y = y_nxt;
+        } else if (more) {
+            load_row(row + stride, raw, y);
+        }
     }
 
     for (int w = 0; w < kWarps; ++w) {     // fixed order: warp 0 stores, the others add
@@ -124,9 +148,12 @@ __global__ void __launch_bounds__(kThreads, 1) train_grad_kernel(const TrainPara
                 const int vi = j * 32 + lane;
                 if (vi < nv) {
 #pragma unroll
-                    for (int e = 0; e < N; ++e) {
+                    for (int e = 0; e < N; e += 2) {
+                        float lo, hi;
+                        unpack2(acc[(j * N + e) / 2], lo, hi);
                         float *dst = red + vi * N + e;
-                        *dst = w == 0 ? acc[j * N + e] : *dst + acc[j * N + e];
+                        dst[0] = w == 0 ? lo : dst[0] + lo;
+                        dst[1] = w == 0 ? hi : dst[1] + hi;
                     }
                 }
             }
@@ -172,7 +199,17 @@ cudaError_t launch_grad(const TrainParams &tp, cudaStream_t st)
     cudaError_t e = cudaFuncSetAttribute(train_grad_kernel<T, VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)smem);
     if (e != cudaSuccess) return e;
-    train_grad_kernel<T, VPL><<<tp.ctas, kThreads, smem, st>>>(tp);
+    // one full wave: as many CTAs as are resident at once, so that all of them finish together
+    int per_sm = 0, dev = 0, sms = 0;
+    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, train_grad_kernel<T, VPL>, kThreads, smem)) !=
+            cudaSuccess ||
+        (e = cudaGetDevice(&dev)) != cudaSuccess ||
+        (e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+        return e;
+    TrainParams p = tp;
+    p.ctas = (int)max((int64_t)1, min((int64_t)min(kTrainMaxCtas, per_sm * sms), (tp.N + kWarps - 1) / kWarps));
+    train_grad_kernel<T, VPL><<<p.ctas, kThreads, smem, st>>>(p);
+    train_adam_kernel<<<(tp.d + 2 + 255) / 256, 256, 0, st>>>(p);
     return cudaGetLastError();
 }
 
@@ -198,8 +235,6 @@ T *at(void *ws, size_t off)
 int finish(cudaError_t e) { return e == cudaSuccess ? SPR_OK : report_cuda_error(e); }
 
 }  // namespace
-
-int train_ctas(int64_t N) { return (int)max((int64_t)1, min((int64_t)kTrainMaxCtas, (N + kWarps - 1) / kWarps)); }
 
 }  // namespace spr
 
@@ -298,14 +333,8 @@ int verifier_train_step(const void *hidden, const uint8_t *labels, int64_t N, in
     tp.eps = eps;
     tp.loss = loss;
     tp.part = at<float>(ws, kHeaderBytes);
-    tp.ctas = train_ctas(N);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    cudaError_t e = dt == SPR_F32 ? launch_grad_any<float>(tp, st) : launch_grad_any<__nv_bfloat16>(tp, st);
-    if (e == cudaSuccess) {
-        train_adam_kernel<<<(d + 2 + 255) / 256, 256, 0, st>>>(tp);
-        e = cudaGetLastError();
-    }
-    return finish(e);
+    return finish(dt == SPR_F32 ? launch_grad_any<float>(tp, st) : launch_grad_any<__nv_bfloat16>(tp, st));
 }
 
 }  // extern "C"
