@@ -59,80 +59,25 @@ struct TrainParams {
     float *loss;             // [1] or null
     float *part;             // [ctas, d+2]: per-CTA sums of the gradient terms, then of the loss
     int ctas;
-    int stages;              // row buffers per warp in the shared-memory ring
-    int *status;
 };
 
-// ---- shared-memory ring fed by bulk asynchronous copies (one ring per warp)
-constexpr uint32_t kSpinLimit = 1u << 22;   // polls of mbarrier.try_wait before giving up
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
-                 : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// bounded wait: false when the phase did not complete within kSpinLimit polls
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
-{
-    for (uint32_t i = 0; i < kSpinLimit; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-// global -> shared copy of `bytes` (a multiple of 16, both addresses 16-byte aligned) that
-// completes on `bar`
-__device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     smem_u32(dst)),
-                 "l"(src), "r"(bytes), "r"(smem_u32(bar))
-                 : "memory");
-}
-
 // Gradient pass (one resident wave of CTAs): one warp per sample, samples dealt to warps in a
-// fixed pattern.  Every warp owns a ring of `stages` row buffers in shared memory that one
-// of its lanes keeps filled with bulk asynchronous copies, so a whole SM has ~100-200 KB of
-// hidden states in flight and every hidden state is read from HBM exactly once:
+// fixed pattern; a lane keeps
+// its columns of the row in registers, so every hidden state is read from HBM exactly once.
 //   z = b + w.s,  r = sigma(z) - y,  grad_w += r s,  grad_b += r,  loss += ln(1 + e^z) - y z
 // The warps of a CTA add their sums in warp order; the CTA's sums go to part[blockIdx.x].
-// A wait that runs out raises SPR_ERR_TIMEOUT; the warp then stops, waits (bounded) for its
-// copies in flight and joins the reduction, whose result is then meaningless.
 template <typename T, int VPL>
-__global__ void __launch_bounds__(kThreads, VPL <= 8 ? 2 : 1) train_grad_kernel(const TrainParams prm)
+__global__ void __launch_bounds__(kThreads, 1) train_grad_kernel(const TrainParams prm)
 {
     constexpr int N = Vec<T>::N;
-    constexpr int kDots = VPL < 4 ? VPL : 4;   // independent partial dot products
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    const int d = prm.d, S = prm.stages;
-    const uint32_t row_bytes = (uint32_t)d * sizeof(T);
+    extern __shared__ float smem[];
+    const int d = prm.d;
+    float *sw = smem;              // [d] weights
+    float *red = smem + d;         // [d + 2] CTA sums
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    unsigned char *ring = smem_raw + (size_t)warp * S * row_bytes;                      // this warp's stages
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + (size_t)kWarps * S * row_bytes) + warp * S;
-    float *sw = reinterpret_cast<float *>(smem_raw + (size_t)kWarps * S * (row_bytes + 8));   // [d] weights
-    float *red = sw + d;                                                                // [d + 2] CTA sums
     const int nv = d / N;          // vectors per row
     for (int j = tid; j < d; j += kThreads) sw[j] = prm.theta[j];
     const float bias = prm.theta[d];
-    if (lane == 0) {
-        for (int s = 0; s < S; ++s) mbar_init(&bars[s], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
     __syncthreads();
 
     uint64_t acc[VPL * N / 2];       // packed pairs of fp32 sums (two columns each)
@@ -140,82 +85,59 @@ __global__ void __launch_bounds__(kThreads, VPL <= 8 ? 2 : 1) train_grad_kernel(
     for (int e = 0; e < VPL * N / 2; ++e) acc[e] = pack2(0.f, 0.f);
     float acc_b = 0.f, acc_loss = 0.f;
     const T *base = static_cast<const T *>(prm.hidden);
-    const int64_t stride = (int64_t)gridDim.x * kWarps;
-    const int64_t first = (int64_t)blockIdx.x * kWarps + warp;
-    const int64_t n = first < prm.N ? (prm.N - first + stride - 1) / stride : 0;   // this warp's rows
-    int64_t issued = 0;
-    if (lane == 0) {
-        for (; issued < n && issued < S; ++issued) {
-            mbar_expect_tx(&bars[issued], row_bytes);
-            bulk_load(ring + issued * row_bytes, base + (first + issued * stride) * d, row_bytes, &bars[issued]);
-        }
-    }
-    issued = __shfl_sync(0xffffffffu, issued, 0);
-    float y = n > 0 ? (float)prm.labels[first] : 0.f;
-    int s = 0;
-    uint32_t phase = 0;
-    int64_t i = 0;
-    for (; i < n; ++i) {
-        const float y_next = i + 1 < n ? (float)prm.labels[first + (i + 1) * stride] : 0.f;
-        if (!__all_sync(0xffffffffu, mbar_wait(&bars[s], phase))) {
-            if (lane == 0) raise_status(prm.status, SPR_ERR_TIMEOUT);
-            break;
-        }
-        const uint4 *x = reinterpret_cast<const uint4 *>(ring + (size_t)s * row_bytes);
-        uint64_t dot2[kDots];
+    constexpr bool kPrefetch = VPL <= 4;   // short rows: keep the next row in flight as well
+    auto load_row = [&](int64_t row, uint4 (&dst)[VPL], float &y) {
+        const uint4 *x = reinterpret_cast<const uint4 *>(base + row * d);
 #pragma unroll
-        for (int k = 0; k < kDots; ++k) dot2[k] = pack2(0.f, 0.f);
+        for (int j = 0; j < VPL; ++j) {
+            const int vi = j * 32 + lane;
+            dst[j] = vi < nv ? ld_stream(x + vi) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        y = (float)prm.labels[row];
+    };
+    const int64_t stride = (int64_t)gridDim.x * kWarps;
+    int64_t row = (int64_t)blockIdx.x * kWarps + warp;
+    uint4 raw[VPL];
+    float y = 0.f;
+    if (row < prm.N) load_row(row, raw, y);
+    for (; row < prm.N; row += stride) {
+        uint4 nxt[VPL];
+        float y_nxt = 0.f;
+        const bool more = row + stride < prm.N;
+        if (kPrefetch && more) load_row(row + stride, nxt, y_nxt);
+        uint64_t dot2 = pack2(0.f, 0.f);   // even and odd columns apart
 #pragma unroll
         for (int j = 0; j < VPL; ++j) {
             const int vi = j * 32 + lane;
             if (vi < nv) {
                 float f[N];
-                Vec<T>::unpack(x[vi], f);
+                Vec<T>::unpack(raw[j], f);
 #pragma unroll
                 for (int e = 0; e < N; e += 2)
-                    dot2[j % kDots] = fma2(pack2(f[e], f[e + 1]),
-                                           *reinterpret_cast<const uint64_t *>(&sw[vi * N + e]), dot2[j % kDots]);
+                    dot2 = fma2(pack2(f[e], f[e + 1]), *reinterpret_cast<const uint64_t *>(&sw[vi * N + e]), dot2);
             }
         }
-#pragma unroll
-        for (int k = 1; k < kDots; ++k) dot2[0] = add2(dot2[0], dot2[k]);
         float d_even, d_odd;
-        unpack2(dot2[0], d_even, d_odd);
+        unpack2(dot2, d_even, d_odd);
         const float z = warp_sum(d_even + d_odd) + bias;
         const float r = 1.f / (1.f + expf(-z)) - y;
         const uint64_t r2 = pack2(r, r);
 #pragma unroll
         for (int j = 0; j < VPL; ++j) {
-            const int vi = j * 32 + lane;
-            if (vi < nv) {
-                float f[N];
-                Vec<T>::unpack(x[vi], f);
+            float f[N];
+            Vec<T>::unpack(raw[j], f);     // zero beyond the row
 #pragma unroll
-                for (int e = 0; e < N; e += 2)
-                    acc[(j * N + e) / 2] = fma2(r2, pack2(f[e], f[e + 1]), acc[(j * N + e) / 2]);
-            }
+            for (int e = 0; e < N; e += 2)
+                acc[(j * N + e) / 2] = fma2(r2, pack2(f[e], f[e + 1]), acc[(j * N + e) / 2]);
         }
         acc_b += r;
         acc_loss += fmaxf(z, 0.f) + log1pf(expf(-fabsf(z))) - y * z;
-        y = y_next;
-        __syncwarp();               // every lane is done with this stage before it is refilled
-        if (issued < n) {
-            if (lane == 0) {
-                mbar_expect_tx(&bars[s], row_bytes);
-                bulk_load(ring + (size_t)s * row_bytes, base + (first + issued * stride) * d, row_bytes, &bars[s]);
-            }
-            ++issued;
-        }
-        if (++s == S) {
-            s = 0;
-            phase ^= 1u;
-        }
-    }
-    for (; i < issued; ++i) {       // only after a timeout: let the copies in flight land
-        mbar_wait(&bars[s], phase);
-        if (++s == S) {
-            s = 0;
-            phase ^= 1u;
+        if (kPrefetch) {
+#pragma unroll
+            for (int j = 0; j < VPL; ++j) raw[j] = nxt[j];
+            y = y_nxt;
+        } else if (more) {
+            load_row(row + stride, raw, y);
         }
     }
 
@@ -273,12 +195,7 @@ __global__ void __launch_bounds__(256) train_adam_kernel(const TrainParams prm)
 template <typename T, int VPL>
 cudaError_t launch_grad(const TrainParams &tp, cudaStream_t st)
 {
-    TrainParams p = tp;
-    // ring: about 90 KB per CTA where two CTAs share an SM, 196 KB where one CTA has it
-    const size_t row_bytes = (size_t)tp.d * sizeof(T);
-    const size_t budget = VPL <= 8 ? 92 * 1024 : 196 * 1024;
-    p.stages = (int)max((size_t)2, min((size_t)8, budget / (kWarps * row_bytes)));
-    const size_t smem = (size_t)kWarps * p.stages * (row_bytes + 8) + sizeof(float) * (2 * (size_t)tp.d + 2);
+    const size_t smem = sizeof(float) * (2 * (size_t)tp.d + 2);
     cudaError_t e = cudaFuncSetAttribute(train_grad_kernel<T, VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)smem);
     if (e != cudaSuccess) return e;
@@ -289,7 +206,7 @@ cudaError_t launch_grad(const TrainParams &tp, cudaStream_t st)
         (e = cudaGetDevice(&dev)) != cudaSuccess ||
         (e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
         return e;
-    if (per_sm < 1) return cudaErrorInvalidConfiguration;
+    TrainParams p = tp;
     p.ctas = (int)max((int64_t)1, min((int64_t)min(kTrainMaxCtas, per_sm * sms), (tp.N + kWarps - 1) / kWarps));
     train_grad_kernel<T, VPL><<<p.ctas, kThreads, smem, st>>>(p);
     train_adam_kernel<<<(tp.d + 2 + 255) / 256, 256, 0, st>>>(p);
@@ -416,7 +333,6 @@ int verifier_train_step(const void *hidden, const uint8_t *labels, int64_t N, in
     tp.eps = eps;
     tp.loss = loss;
     tp.part = at<float>(ws, kHeaderBytes);
-    tp.status = at<int>(ws, 0);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     return finish(dt == SPR_F32 ? launch_grad_any<float>(tp, st) : launch_grad_any<__nv_bfloat16>(tp, st));
 }
