@@ -424,6 +424,25 @@ def main():
             "ms": t1 + t2 + t3 + t4, "stats_bytes": int(shard_bytes), "stats_gbs": shard_bytes / (t1 * 1e-3) / 1e9,
             "exchange_bytes_per_gpu": int(B * wl.Kp * 24 + B * 16 + B * 4)}
 
+    # preparing and fitting the verifier (Section 3.2): labels from the same logits, one optimiser step of
+    # the single-layer verifier on N = 2^20 hidden states of the draft model's width
+    from paper_2502_04557_b200 import binding as bd
+    ws_fit = spr.Workspace(max(spr.workspace_bytes(bd.OP_VERIFIER_LABELS, B, K, V, 0, 0, dt_code),
+                               spr.workspace_bytes(bd.OP_VERIFIER_TRAIN, 0, 0, 0, cfg.d, 0, dt_code)), device=dev)
+    t_lab = time_call(lambda: bd.verifier_labels(wl.p_logits, wl.q_logits, V, wl.draft_tokens, [1.0, 1.2, 1.5], ws_fit,
+                                                 want_ratio=False), n=20)
+    n_fit = 1 << 20
+    fit_h = torch.randn((n_fit, cfg.d), device=dev).to(wl.hidden.dtype)
+    fit_y = (torch.rand(n_fit, device=dev) < 0.5).to(torch.uint8)
+    fit_state = [torch.zeros(cfg.d + 1, device=dev) for _ in range(3)]
+    fit_loss = torch.empty(1, device=dev)
+    t_fit = time_call(lambda: bd.verifier_train_step(fit_h, fit_y, *fit_state, 1, 1e-3, ws_fit, loss=fit_loss), n=20)
+    calls["verifier_labels"] = {"ms": t_lab, "tokens_per_s": M / (t_lab * 1e-3), "bytes": int(alg_bytes),
+                                "gbs": alg_bytes / (t_lab * 1e-3) / 1e9}
+    calls["verifier_train_step"] = {"ms": t_fit, "samples": n_fit, "d": cfg.d, "samples_per_s": n_fit / (t_fit * 1e-3),
+                                    "bytes": int(fit_h.numel() * es), "gbs": fit_h.numel() * es / (t_fit * 1e-3) / 1e9}
+    del fit_h, fit_y
+
     simulator = None
     if args.simulator_runs > 0:
         runs = args.simulator_runs
