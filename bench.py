@@ -56,6 +56,9 @@ def parse_args():
     ap.add_argument("--threshold", type=float, default=0.5)
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--shard", default="batch", choices=["batch", "vocab"],
+                    help="how --gpus N ranks split the work: every rank its own batch (default), or every "
+                         "rank V/N columns of the same logits (sd_verify only, NCCL exchanges between the passes)")
     ap.add_argument("--vocab-shards", type=int, default=8,
                     help="also time the four passes of the vocabulary-sharded sd_verify on one of this many "
                          "column shards (0 = skip)")
@@ -196,10 +199,104 @@ def run_reference(args):
     }))
 
 
+def run_vocab_sharded(args):
+    """sd_verify with the vocabulary split over the ranks (a tensor-parallel LM head): every rank
+    reads V/N columns of the same rows; two all-gathers and one max-reduce per step over NCCL."""
+    import torch
+    import torch.distributed as dist
+
+    import paper_2502_04557_b200 as spr
+    from paper_2502_04557_b200 import binding as bd, sharded
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29533")
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    spr.lib()
+    wl = spr.workloads.make(args.workload, dev, B=args.batch, sweep=0)     # the same rows on every rank
+    B, K, V, Kp = wl.B, wl.K, wl.V, wl.Kp
+    es = wl.q_logits.element_size()
+    dt_code = spr.BF16 if wl.cfg.dtype == torch.bfloat16 else spr.F32
+    v0, vs = sharded.vocab_shards(V, world, es)[rank]
+    # a rank of a tensor-parallel head owns only its columns: keep a dense copy of them
+    p_sh, q_sh = wl.p_logits[:, :, v0:v0 + vs].contiguous(), wl.q_logits[:, :, v0:v0 + vs].contiguous()
+    x, u = wl.draft_tokens, wl.uniforms
+    del wl.p_logits, wl.q_logits
+    ws = spr.Workspace(spr.workspace_bytes(bd.OP_SD_SHARD, B, K, vs, 0, 0, dt_code), device=dev)
+    ex = sharded.DistExchange()
+
+    def step():
+        return sharded.sd_verify_sharded(p_sh, q_sh, V, v0, x, u, ws, ex, extras=False)
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        out = step()
+    assert ws.device_status() == 0
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.time()
+    start.record()
+    for _ in range(args.steps):
+        out = step()
+    stop.record()
+    dist.barrier()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    t = torch.tensor([start.elapsed_time(stop)], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_per_step = float(t.item()) / args.steps
+    # the pass that moves the bytes, alone on this rank
+    stats = torch.empty((B * Kp, 6), dtype=torch.float32, device=dev)
+    for _ in range(3):
+        bd.sd_shard_stats(p_sh, q_sh, v0, x, ws, out=stats)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(20):
+        bd.sd_shard_stats(p_sh, q_sh, v0, x, ws, out=stats)
+    b.record()
+    torch.cuda.synchronize()
+    stats_ms = a.elapsed_time(b) / 20
+    alg_bytes = float((B * Kp + B * K) * vs * es)
+    peak, peak_kind = peaks()
+    if rank == 0:
+        sampler.stop()
+        print(json.dumps({
+            "metric": "verified_tokens_per_s", "value": B * K / (ms_per_step * 1e-3), "unit": "tokens/s",
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+            "dtype": "bf16" if dt_code == spr.BF16 else "f32", "data": "synthetic",
+            "config": {"workload": f"{args.workload}: B={B} K={K} V={V} Kp={Kp}, vocabulary split over {world} "
+                                   f"rank(s), {vs} columns on rank 0",
+                       "step": "sd_verify_sharded: stats, all-gather, decide, weights, all-gather, draw, max-reduce",
+                       "l2": "a rank's shard is re-read every step; shards under 126 MB stay L2-resident",
+                       "mean_sd_accepted_len": out["accepted_len"].float().mean().item()},
+            "clocks": sampler.summary(t0, t1), "e2e": None, "gpu_launches": 4 * args.steps,
+            "roofline": {"bound": "hbm", "kernel": "shard_stats_kernel", "achieved": alg_bytes / (stats_ms * 1e-3) / 1e9,
+                         "peak": peak, "unit": "GB/s", "frac": alg_bytes / (stats_ms * 1e-3) / 1e9 / peak,
+                         "peak_kind": f"of {peak_kind}", "traffic": None, "algorithmic_bytes_per_launch": alg_bytes,
+                         "avg_launch_ms": stats_ms},
+            "cpu_baseline": None,
+        }))
+    dist.destroy_process_group()
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.shard == "vocab":
+        run_vocab_sharded(args)
         return
 
     import torch
