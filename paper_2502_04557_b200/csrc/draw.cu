@@ -49,8 +49,10 @@ __device__ __forceinline__ Job<T> resolve_job(const DrawParams &prm, int i)
     return job;
 }
 
-template <typename T>
-__global__ void __launch_bounds__(kThreads, 3) draw_kernel(const DrawParams prm)
+// kSoftmaxOnly: replacement draws never take the residual branch; compiled without it the
+// kernel needs fewer registers and four CTAs fit an SM.
+template <typename T, bool kSoftmaxOnly>
+__global__ void __launch_bounds__(kThreads, kSoftmaxOnly ? 4 : 3) draw_kernel(const DrawParams prm)
 {
     __shared__ DrawSmem sm;
     const int C = prm.chunks;   // segments (CTAs) per row, of kWarps * prm.iters steps each
@@ -68,7 +70,7 @@ __global__ void __launch_bounds__(kThreads, 3) draw_kernel(const DrawParams prm)
         }
         return;
     }
-    int mode = job.mode;
+    const int mode = kSoftmaxOnly ? (int)MODE_SOFTMAX : job.mode;
     float2 *part = prm.part + (int64_t)i * steps;
 
     segment_pass<T>(job, mode, prm.V, c, steps, prm.iters, part);
@@ -102,8 +104,11 @@ cudaError_t launch_draw(const DrawParams &dp, int n, int dt, cudaStream_t st, bo
         cfg.attrs = attr;
         cfg.numAttrs = 1;
     }
-    return dt == SPR_F32 ? cudaLaunchKernelEx(&cfg, draw_kernel<float>, dp)
-                         : cudaLaunchKernelEx(&cfg, draw_kernel<__nv_bfloat16>, dp);
+    if (dp.kind == DRAW_REPLACE)
+        return dt == SPR_F32 ? cudaLaunchKernelEx(&cfg, draw_kernel<float, true>, dp)
+                             : cudaLaunchKernelEx(&cfg, draw_kernel<__nv_bfloat16, true>, dp);
+    return dt == SPR_F32 ? cudaLaunchKernelEx(&cfg, draw_kernel<float, false>, dp)
+                         : cudaLaunchKernelEx(&cfg, draw_kernel<__nv_bfloat16, false>, dp);
 }
 
 }  // namespace spr
