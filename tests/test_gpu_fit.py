@@ -181,3 +181,55 @@ def test_labels_then_training_then_the_verifier_call(spr):
                                             theta[d:].contiguous(), 0.5, ws)
     assert ws.device_status() == 0
     assert (accept.reshape(-1) == y).float().mean() > 0.97
+
+
+def test_labels_llama3_full_size_sampled(spr):
+    """The benchmark's workload: the oracle on a sample of sequences, and the link to sd_verify
+    (ratio = q(x)/p(x) of its outputs) on all 4096 tokens."""
+    wl = spr.workloads.make("llama3", "cuda")
+    B, K, V = wl.B, wl.K, wl.V
+    ws = spr.Workspace(max(spr.workspace_bytes(bd(spr).OP_VERIFIER_LABELS, B, K, V, 0, 0, spr.BF16),
+                           spr.workspace_bytes(2, B, K, V, 1, 0, spr.BF16)))
+    labels, ratio = bd(spr).verifier_labels(wl.p_logits, wl.q_logits, V, wl.draft_tokens, LAMBDAS, ws)
+    assert ws.device_status() == 0
+    seqs = [0, 3, 77, 128, 255]
+    idx = torch.tensor(seqs, device="cuda")
+    want_labels, want_ratio = training.verifier_labels(to_np(wl.p_logits[idx]), to_np(wl.q_logits[idx]), V,
+                                                       to_np(wl.draft_tokens[idx]), LAMBDAS)
+    got_ratio = ratio[idx].cpu().double().numpy()
+    assert np.all(np.abs(got_ratio / want_ratio - 1.0) <= 1e-3)
+    got = labels[:, idx].cpu().numpy()
+    for i, lam in enumerate(LAMBDAS):
+        clear = np.abs(want_ratio / lam - 1.0) > LABEL_MARGIN
+        assert clear.mean() > 0.95 and np.array_equal(got[i][clear], want_labels[i][clear])
+    sd = spr.sd_verify(wl.p_logits, wl.q_logits, V, wl.draft_tokens, wl.uniforms, ws)
+    assert torch.allclose(ratio, sd["q_tok"] / sd["p_tok"], rtol=1e-4)
+    lab = labels.cpu().numpy().astype(int)
+    assert np.all(np.diff(lab, axis=0) >= 0)                       # more accepts as lambda grows
+    assert np.array_equal(lab[0] == 1, (ratio <= 1.0).cpu().numpy())
+
+
+def test_train_step_at_the_benchmark_size(spr):
+    """N = 2^20 samples of width 2048 (the configuration bench.py times): the first step has a
+    closed form - loss ln 2 and a move of lr * g / (|g| + eps) with g = mean((1/2 - y) s) - checked
+    against a float64 matrix product; the oracle itself takes one step on a slice that fits."""
+    N, d, lr = 1 << 20, 2048, 0.01
+    g = torch.Generator(device="cuda").manual_seed(12)
+    S = torch.randn((N, d), generator=g, device="cuda").to(torch.bfloat16)
+    y = (torch.rand(N, generator=g, device="cuda") < 0.3).to(torch.uint8)
+    ws = spr.Workspace(spr.workspace_bytes(bd(spr).OP_VERIFIER_TRAIN, 0, 0, 0, d, 0, spr.BF16))
+    theta = torch.zeros(d + 1, device="cuda")
+    m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+    loss = bd(spr).verifier_train_step(S, y, theta, m, v, 1, lr, ws)
+    assert float(loss) == pytest.approx(np.log(2.0), rel=1e-6)
+    r = 0.5 - y.double()
+    grad = torch.cat([(r[None, :] @ S.double()).reshape(-1), r.sum()[None]]) / N
+    want = -lr * grad / (grad.abs() + 1e-8)
+    assert (theta.double() - want).abs().max() <= 1e-3 * lr
+    assert torch.allclose(m.double(), 0.1 * grad, rtol=1e-3, atol=1e-9)
+    n = 1 << 16                                                     # a slice the oracle handles in seconds
+    theta.zero_(); m.zero_(); v.zero_()
+    loss = bd(spr).verifier_train_step(S[:n].contiguous(), y[:n].contiguous(), theta, m, v, 1, lr, ws)
+    l0, t0, _, _ = training.verifier_train_step(to_np(S[:n]), y[:n].cpu().numpy(), np.zeros(d + 1), np.zeros(d + 1),
+                                                np.zeros(d + 1), 1, lr)
+    assert abs(float(loss) / l0 - 1.0) < 2e-5 and np.abs(theta.cpu().double().numpy() - t0).max() <= 1e-3 * lr

@@ -212,3 +212,49 @@ def test_residual_below_fp32_resolution_falls_back_to_p(spr, dtype):
         for b in range(B):
             m, t = oracle.softmax_draw_margin(to_np(p)[b, 0], float(u[b, K]))
             assert m > 1e-6 and int(out["correction_token"][b]) == t
+
+
+def test_sharded_llama3_full_size_sampled(spr):
+    """The benchmark's workload (B=256, K=16, V=128256) cut into 8 column shards: the oracle on a
+    sample of sequences, and agreement with the single-GPU call on everything."""
+    wl = spr.workloads.make("llama3", "cuda")
+    K, V = wl.K, wl.V
+    results = run_sharded(spr, wl.p_logits, wl.q_logits, V, wl.draft_tokens, wl.uniforms, 8)
+    for out in results[1:]:                                   # every rank reports the same
+        for k in ("accept", "accepted_len", "correction_token", "p_tok", "q_tok", "residual_mass"):
+            assert torch.equal(out[k], results[0][k]), k
+    out = results[0]
+    assert out["status"] == 0
+    seqs = [0, 1, 37, 100, 128, 254, 255]
+    idx = torch.tensor(seqs, device="cuda")
+    P, Q = to_np(wl.p_logits[idx]), to_np(wl.q_logits[idx])
+    X, U = to_np(wl.draft_tokens[idx]), to_np(wl.uniforms[idx])
+    ref = oracle.sd_verify(P, Q, V, X, U)
+    clear = np.abs(U[:, :K].astype(np.float64) - ref["p_tok"] / ref["q_tok"]) >= MARGIN
+    assert clear.mean() > 0.99
+    assert np.array_equal(out["accept"][idx].cpu().numpy()[clear], ref["accept"][clear])
+    assert_close_rel(out["p_tok"][idx], ref["p_tok"], 1e-3, "p_tok")
+    assert_close_rel(out["q_tok"][idx], ref["q_tok"], 1e-3, "q_tok")
+    n_tok = 0
+    for j, b in enumerate(seqs):
+        if not clear[j].all():
+            continue
+        nb = int(ref["accepted_len"][j])
+        assert int(out["accepted_len"][b]) == nb
+        u = float(U[j, K])
+        if nb < K:
+            m, t = oracle.residual_draw_margin(P[j, nb, :V], Q[j, nb, :V], u)
+            assert abs(float(out["residual_mass"][b]) / ref["residual_mass"][j] - 1.0) <= 1e-3
+        else:
+            m, t = oracle.softmax_draw_margin(P[j, K, :V], u)
+        if m >= 1e-6:
+            assert int(out["correction_token"][b]) == t
+            n_tok += 1
+    assert n_tok >= len(seqs) // 2
+    # the single-GPU call on the same tensors: different summation order, same decisions up to
+    # the rare tie inside the margin
+    ws = spr.Workspace(spr.workspace_bytes(2, wl.B, K, V, 1, 0, spr.BF16))
+    one = spr.sd_verify(wl.p_logits, wl.q_logits, V, wl.draft_tokens, wl.uniforms, ws)
+    assert (one["accept"] == out["accept"]).float().mean() > 0.999
+    assert (one["correction_token"] == out["correction_token"]).float().mean() > 0.98
+    assert torch.allclose(one["p_tok"], out["p_tok"], rtol=1e-4, atol=1e-30)
