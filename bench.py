@@ -62,6 +62,8 @@ def parse_args():
     ap.add_argument("--vocab-shards", type=int, default=8,
                     help="also time the four passes of the vocabulary-sharded sd_verify on one of this many "
                          "column shards (0 = skip)")
+    ap.add_argument("--fit-samples", type=int, default=1 << 20,
+                    help="hidden states in the timed verifier_train_step call")
     ap.add_argument("--simulator-runs", type=int, default=0,
                     help="also time sprinter_simulate on this many runs (r=5, eta_TP=0.9, eta_FP=0.5)")
     return ap.parse_args()
@@ -528,7 +530,7 @@ def main():
                                spr.workspace_bytes(bd.OP_VERIFIER_TRAIN, 0, 0, 0, cfg.d, 0, dt_code)), device=dev)
     t_lab = time_call(lambda: bd.verifier_labels(wl.p_logits, wl.q_logits, V, wl.draft_tokens, [1.0, 1.2, 1.5], ws_fit,
                                                  want_ratio=False), n=20)
-    n_fit = 1 << 20
+    n_fit = args.fit_samples
     fit_h = torch.randn((n_fit, cfg.d), device=dev).to(wl.hidden.dtype)
     fit_y = (torch.rand(n_fit, device=dev) < 0.5).to(torch.uint8)
     fit_state = [torch.zeros(cfg.d + 1, device=dev) for _ in range(3)]

@@ -83,7 +83,7 @@ __global__ void __launch_bounds__(kThreads, VPL <= 3 ? 3 : (VPL <= 4 ? 2 : 1)) t
     uint64_t acc[VPL * N / 2];       // packed pairs of fp32 sums (two columns each)
 #pragma unroll
     for (int e = 0; e < VPL * N / 2; ++e) acc[e] = pack2(0.f, 0.f);
-    float acc_b = 0.f, acc_loss = 0.f;
+    double acc_b = 0.0, acc_loss = 0.0;   // same-signed addends: fp32 sums would drift
     const T *base = static_cast<const T *>(prm.hidden);
     constexpr bool kPrefetch = VPL <= 4;   // short rows: keep the next row in flight as well
     auto load_row = [&](int64_t row, uint4 (&dst)[VPL], float &y) {
@@ -130,8 +130,8 @@ __global__ void __launch_bounds__(kThreads, VPL <= 3 ? 3 : (VPL <= 4 ? 2 : 1)) t
             for (int e = 0; e < N; e += 2)
                 acc[(j * N + e) / 2] = fma2(r2, pack2(f[e], f[e + 1]), acc[(j * N + e) / 2]);
         }
-        acc_b += r;
-        acc_loss += fmaxf(z, 0.f) + log1pf(expf(-fabsf(z))) - y * z;
+        acc_b += (double)r;
+        acc_loss += (double)(fmaxf(z, 0.f) + log1pf(expf(-fabsf(z))) - y * z);
         if (kPrefetch) {
 #pragma unroll
             for (int j = 0; j < VPL; ++j) raw[j] = nxt[j];
@@ -158,8 +158,8 @@ __global__ void __launch_bounds__(kThreads, VPL <= 3 ? 3 : (VPL <= 4 ? 2 : 1)) t
                 }
             }
             if (lane == 0) {
-                red[d] = w == 0 ? acc_b : red[d] + acc_b;
-                red[d + 1] = w == 0 ? acc_loss : red[d + 1] + acc_loss;
+                red[d] = w == 0 ? (float)acc_b : red[d] + (float)acc_b;
+                red[d + 1] = w == 0 ? (float)acc_loss : red[d + 1] + (float)acc_loss;
             }
         }
         __syncthreads();
