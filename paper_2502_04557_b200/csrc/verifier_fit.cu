@@ -67,7 +67,7 @@ struct TrainParams {
 //   z = b + w.s,  r = sigma(z) - y,  grad_w += r s,  grad_b += r,  loss += ln(1 + e^z) - y z
 // The warps of a CTA add their sums in warp order; the CTA's sums go to part[blockIdx.x].
 template <typename T, int VPL>
-__global__ void __launch_bounds__(kThreads, VPL <= 3 ? 3 : (VPL <= 4 ? 2 : 1)) train_grad_kernel(const TrainParams prm)
+__global__ void __launch_bounds__(kThreads, VPL <= 3 ? 3 : (VPL <= 8 ? 2 : 1)) train_grad_kernel(const TrainParams prm)
 {
     constexpr int N = Vec<T>::N;
     extern __shared__ float smem[];
