@@ -57,7 +57,9 @@ __global__ void __launch_bounds__(kThreads, kSoftmaxOnly ? 4 : 3) draw_kernel(co
     __shared__ DrawSmem sm;
     const int C = prm.chunks;   // segments (CTAs) per row, of kWarps * prm.iters steps each
     const int steps = prm.steps;
-    const int i = blockIdx.x / C;
+    // correction draws go through the sequences last to first: the statistics pass has just
+    // streamed the rows in ascending order, so the highest ones are the ones still in L2
+    const int i = kSoftmaxOnly ? blockIdx.x / C : (int)(gridDim.x / C) - 1 - (int)(blockIdx.x / C);
     const int c = blockIdx.x % C;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
