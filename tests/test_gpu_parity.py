@@ -658,3 +658,68 @@ def test_calls_replay_from_a_cuda_graph(spr):
     for a, b in zip(replayed, (*out_sd.values(), *out_st)):
         assert torch.equal(a, b)
     assert ws.device_status() == 0
+
+
+# ---------------------------------------------------------------------------- K = 1 (rows staged on chip)
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("B,V,ldv", [
+    (3, 8, None), (5, 64, 72), (4, 1000, None), (7, 1024, None), (2, 8200, 8208), (3, 16384, None),
+    (2, 50264, None), (2, 65536, None), (1, 128256, None), (2, 130048, None),
+    (3, 1001, None), (2, 131072, None), (2, 8192, 8195),      # rows the staged kernel does not take
+])
+def test_sd_single_position_shapes(spr, dtype, B, V, ldv):
+    """K = Kp = 1 goes to the kernel that keeps each row pair in shared memory when the rows are
+    16-byte aligned, whole vectors and short enough; every other shape takes the general path.
+    Both must agree with the oracle."""
+    p, q, x, u = _rand_problem(B, 1, V, dtype, seed=17 + B * 1000 + V, ldv=ldv, Kp=1)
+    ref = _clear_sd(p, q, V, x, u)
+    ws = spr.Workspace(spr.workspace_bytes(2, B, 1, V, 1, 0, spr.binding._dt(p)))
+    for _ in range(2):                       # twice on one workspace
+        out = spr.sd_verify(p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), ws)
+        assert ws.device_status() == 0
+        eq(out["accept"], ref["accept"], "accept")
+        eq(out["accepted_len"], ref["accepted_len"], "accepted_len")
+        eq(out["correction_token"], ref["correction_token"], "correction_token")
+        assert_close_rel(out["p_tok"], ref["p_tok"], RTOL[dtype], "p_tok")
+        assert_close_rel(out["q_tok"], ref["q_tok"], RTOL[dtype], "q_tok")
+        assert_close_rel(out["residual_mass"], ref["residual_mass"], RTOL[dtype], "residual_mass")
+    assert (ref["accepted_len"] == 0).any() or B < 3
+
+
+def test_sd_single_position_special_cases(spr):
+    g = torch.Generator().manual_seed(21)
+    B, V = 6, 5000
+    u = torch.rand((B, 2), generator=g).clamp_(min=1e-3, max=0.999)
+    ws = spr.Workspace(spr.workspace_bytes(2, B, 1, V, 1, 0, spr.F32))
+    # p == q: everything accepted, nothing to draw
+    q = torch.randn((B, 1, V), generator=g)
+    x = torch.randint(0, V, (B, 1), generator=g, dtype=torch.int32)
+    out = spr.sd_verify(q.clone().cuda(), q.cuda(), V, x.cuda(), u.cuda(), ws)
+    assert (out["accept"] == 1).all() and (out["accepted_len"] == 1).all()
+    assert (out["correction_token"] == -1).all() and (out["residual_mass"] == 0).all()
+    # disjoint supports: everything rejected, correction token from p's support, residual mass 1
+    ninf = float("-inf")
+    p2 = torch.full((B, 1, V), ninf); p2[..., 4000:4100] = torch.randn((B, 1, 100), generator=g)
+    q2 = torch.full((B, 1, V), ninf); q2[..., :4000] = torch.randn((B, 1, 4000), generator=g)
+    x2 = torch.randint(0, 4000, (B, 1), generator=g, dtype=torch.int32)
+    out = spr.sd_verify(p2.cuda(), q2.cuda(), V, x2.cuda(), u.cuda(), ws)
+    assert (out["accept"] == 0).all() and (out["accepted_len"] == 0).all()
+    assert ((out["correction_token"] >= 4000) & (out["correction_token"] < 4100)).all()
+    assert torch.allclose(out["residual_mass"], torch.ones(B, device="cuda"), rtol=1e-5)
+    for b in range(B):
+        m, t = oracle.residual_draw_margin(to_np(p2)[b, 0], to_np(q2)[b, 0], float(u[b, 1]))
+        if m > 1e-5:
+            assert int(out["correction_token"][b]) == t
+    # a draft token outside the vocabulary
+    x3 = x.clone(); x3[2, 0] = V; x3[4, 0] = -1
+    p3 = q + 0.7 * torch.randn((B, 1, V), generator=g)
+    ref = _clear_sd(p3, q, V, x3.clamp(0, V - 1), u)
+    out = spr.sd_verify(p3.cuda(), q.cuda(), V, x3.cuda(), u.cuda(), ws)
+    assert ws.device_status() == 6
+    for b in range(B):
+        if b in (2, 4):
+            assert int(out["accepted_len"][b]) == -1 and int(out["correction_token"][b]) == -1
+            assert int(out["accept"][b, 0]) == 0 and float(out["p_tok"][b, 0]) == -1.0
+        else:
+            assert int(out["accepted_len"][b]) == ref["accepted_len"][b]
+            assert int(out["correction_token"][b]) == ref["correction_token"][b]
