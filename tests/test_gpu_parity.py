@@ -672,6 +672,7 @@ def test_sd_single_position_shapes(spr, dtype, B, V, ldv):
     16-byte aligned, whole vectors and short enough; every other shape takes the general path.
     Both must agree with the oracle."""
     p, q, x, u = _rand_problem(B, 1, V, dtype, seed=17 + B * 1000 + V, ldv=ldv, Kp=1)
+    u[::2, 0] = 0.9 + 0.09 * u[::2, 0]       # mostly rejections in the even sequences
     ref = _clear_sd(p, q, V, x, u)
     ws = spr.Workspace(spr.workspace_bytes(2, B, 1, V, 1, 0, spr.binding._dt(p)))
     for _ in range(2):                       # twice on one workspace
@@ -683,7 +684,6 @@ def test_sd_single_position_shapes(spr, dtype, B, V, ldv):
         assert_close_rel(out["p_tok"], ref["p_tok"], RTOL[dtype], "p_tok")
         assert_close_rel(out["q_tok"], ref["q_tok"], RTOL[dtype], "q_tok")
         assert_close_rel(out["residual_mass"], ref["residual_mass"], RTOL[dtype], "residual_mass")
-    assert (ref["accepted_len"] == 0).any() or B < 3
 
 
 def test_sd_single_position_special_cases(spr):
