@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libsprinter.so")
-SOURCES = ["api.cu", "host_api.cu", "sd_row_stats.cu", "draw.cu", "verifier_simt.cu", "verifier_tensor.cu", "no_alloc.cu", "simulate.cu", "sd_shard.cu", "sd_shard_api.cu", "verifier_fit.cu", "sd_row1.cu"]
+SOURCES = ["api.cu", "host_api.cu", "sd_row_stats.cu", "draw.cu", "verifier_simt.cu", "verifier_tensor.cu", "no_alloc.cu", "simulate.cu", "sd_shard.cu", "sd_shard_api.cu", "verifier_fit.cu"]
 HEADERS = ["common.cuh", "launch.h", "verifier_common.cuh", "vocab_common.cuh", "draw_common.cuh"]
 
 

@@ -355,10 +355,6 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
     dp.part = at<float2>(ws, lay.draw.part);
 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    if (sd_row1_applies(p_logits, q_logits, ldv, K, Kp, V, dt)) {   // one position per sequence: rows stay on chip
-        const cudaError_t e1 = launch_sd_row1(sp, dp.part, correction_token, residual_mass, B, dt, st);
-        return e1 == cudaSuccess ? SPR_OK : cuda_fail(e1);
-    }
     cudaError_t e = cudaMemsetAsync(sp.row_counters, 0, lay.counters_end - lay.row_counters, st);
     if (e == cudaSuccess) e = launch_sd_row_stats(sp, B, K, dt, st);
     if (e == cudaSuccess) e = launch_draw(dp, B, dt, st, /*after_kernel=*/true);

@@ -131,11 +131,6 @@ struct SimParams {
 cudaError_t launch_simulate(const SimParams &sp, cudaStream_t st);
 
 cudaError_t launch_sd_row_stats(const SdParams &sp, int B, int K, int dt, cudaStream_t st);
-// sd_verify with K = Kp = 1 on rows that can be staged in shared memory (sd_row1.cu): one launch,
-// each row read from HBM once.  `part` is the [B * steps] step-weight scratch of the draw.
-bool sd_row1_applies(const void *p, const void *q, int64_t ldv, int K, int Kp, int V, int dt);
-cudaError_t launch_sd_row1(const SdParams &sp, float2 *part, int32_t *correction_token, float *residual_mass, int B,
-                           int dt, cudaStream_t st);
 int report_cuda_error(cudaError_t e);  // records the text, returns SPR_ERR_CUDA
 int device_supported();                // SPR_OK on a compute-capability-10 device
 void set_stage_events(cudaEvent_t before, cudaEvent_t after);

@@ -660,17 +660,16 @@ def test_calls_replay_from_a_cuda_graph(spr):
     assert ws.device_status() == 0
 
 
-# ---------------------------------------------------------------------------- K = 1 (rows staged on chip)
+# ---------------------------------------------------------------------------- K = 1
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
 @pytest.mark.parametrize("B,V,ldv", [
     (3, 8, None), (5, 64, 72), (4, 1000, None), (7, 1024, None), (2, 8200, 8208), (3, 16384, None),
     (2, 50264, None), (2, 65536, None), (1, 128256, None), (2, 130048, None),
-    (3, 1001, None), (2, 131072, None), (2, 8192, 8195),      # rows the staged kernel does not take
+    (3, 1001, None), (2, 131072, None), (2, 8192, 8195),      # misaligned rows, odd lengths
 ])
 def test_sd_single_position_shapes(spr, dtype, B, V, ldv):
-    """K = Kp = 1 goes to the kernel that keeps each row pair in shared memory when the rows are
-    16-byte aligned, whole vectors and short enough; every other shape takes the general path.
-    Both must agree with the oracle."""
+    """One position per sequence and no bonus row: the keep-or-resample rule of Section 3 on a
+    single token, over aligned and misaligned rows of many lengths."""
     p, q, x, u = _rand_problem(B, 1, V, dtype, seed=17 + B * 1000 + V, ldv=ldv, Kp=1)
     u[::2, 0] = 0.9 + 0.09 * u[::2, 0]       # mostly rejections in the even sequences
     ref = _clear_sd(p, q, V, x, u)
