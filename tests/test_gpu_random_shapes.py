@@ -1,0 +1,122 @@
+"""Seeded random shapes, strides and base alignments for the vocabulary calls, each checked
+against the float64 oracle: batch and position counts, vocabulary sizes around the vector, step
+and segment boundaries, padded rows, and logits that start 0-7 elements past a 16-byte
+boundary."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import MARGIN, RTOL, assert_close_rel, to_np
+from oracle import training
+from test_gpu_parity import _clear_sd, eq
+
+pytestmark = pytest.mark.gpu
+
+EDGES = [1, 2, 7, 8, 9, 511, 512, 513, 1023, 1024, 1025, 4095, 4096, 4097, 8191, 8192, 8193, 16384, 16385,
+         32767, 32768, 32769, 33000]
+
+
+@pytest.fixture(scope="module")
+def spr():
+    import paper_2502_04557_b200 as s
+    s.lib()
+    return s
+
+
+def draw_case(seed):
+    r = np.random.default_rng(seed)
+    dtype = [torch.float32, torch.bfloat16][int(r.integers(2))]
+    V = int(r.choice(EDGES)) if r.random() < 0.7 else int(r.integers(1, 20000))
+    K = int(r.choice([1, 1, 2, 3, 5, 8, 17, 33]))
+    B = int(r.integers(1, max(2, 48 // K)))
+    Kp = K + int(r.integers(2))
+    ldv = V + int(r.choice([0, 0, 1, 3, 8, 13]))
+    off_p, off_q = int(r.integers(8)), int(r.integers(8))
+    return dtype, B, K, Kp, V, ldv, off_p, off_q
+
+
+def offset_tensor(t, off):
+    """The same values in device memory that starts `off` elements past an aligned address."""
+    buf = torch.empty(t.numel() + off + 8, dtype=t.dtype, device="cuda")
+    view = buf[off:off + t.numel()].view(t.shape)
+    view.copy_(t)
+    assert view.is_contiguous() and view.data_ptr() == buf.data_ptr() + off * t.element_size()
+    return view
+
+
+def make_problem(seed, dtype, B, K, Kp, V, ldv):
+    g = torch.Generator().manual_seed(seed)
+    q = torch.randn((B, K, ldv), generator=g) * 2.0
+    p = torch.cat([q, torch.randn((B, Kp - K, ldv), generator=g) * 2.0], 1) + 0.7 * torch.randn((B, Kp, ldv), generator=g)
+    if ldv > V:                       # padding columns must never be read as logits
+        p[..., V:] = 60.0
+        q[..., V:] = 60.0
+    x = torch.randint(0, V, (B, K), generator=g, dtype=torch.int32)
+    u = torch.rand((B, K + 1), generator=g)
+    return p.to(dtype).contiguous(), q.to(dtype).contiguous(), x, u
+
+
+@pytest.mark.parametrize("seed", range(60))
+def test_sd_verify_random_case(spr, seed):
+    dtype, B, K, Kp, V, ldv, off_p, off_q = draw_case(1000 + seed)
+    p, q, x, u = make_problem(seed, dtype, B, K, Kp, V, ldv)
+    ref = _clear_sd(p, q, V, x, u)
+    ws = spr.Workspace(spr.workspace_bytes(2, B, K, V, 1, 0, spr.binding._dt(p)))
+    out = spr.sd_verify(offset_tensor(p, off_p), offset_tensor(q, off_q), V, x.cuda(), u.cuda(), ws)
+    assert ws.device_status() == 0
+    eq(out["accept"], ref["accept"], "accept")
+    eq(out["accepted_len"], ref["accepted_len"], "accepted_len")
+    eq(out["correction_token"], ref["correction_token"], "correction_token")
+    assert_close_rel(out["p_tok"], ref["p_tok"], RTOL[dtype], "p_tok")
+    assert_close_rel(out["q_tok"], ref["q_tok"], RTOL[dtype], "q_tok")
+    assert_close_rel(out["residual_mass"], ref["residual_mass"], RTOL[dtype], "residual_mass")
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_replace_sample_random_case(spr, seed):
+    dtype, B, K, Kp, V, ldv, off_p, _ = draw_case(2000 + seed)
+    p, _, _, _ = make_problem(seed, dtype, B, K, Kp, V, ldv)
+    r = np.random.default_rng(seed)
+    R = B * Kp
+    n = int(r.integers(1, 2 * R + 1))
+    rows = torch.from_numpy(r.integers(0, R, n).astype(np.int32))
+    u = torch.from_numpy(r.random(n).astype(np.float32))
+    P = to_np(p).reshape(R, ldv)
+    want = np.empty(n, np.int64)
+    for i in range(n):                               # keep the uniform away from the edges of its bin
+        for _ in range(50):
+            m, t = oracle.softmax_draw_margin(P[int(rows[i]), :V], float(u[i]))
+            if m >= min(MARGIN, 0.1 / V):
+                break
+            u[i] = float(r.random())
+        want[i] = t
+    ws = spr.Workspace(spr.workspace_bytes(1, n, 1, V, 1, 0, spr.binding._dt(p)))
+    tokens = spr.replace_sample(offset_tensor(p, off_p), V, u.cuda(), ws, rows=rows.cuda())
+    assert ws.device_status() == 0
+    eq(tokens, want.astype(np.int32), "tokens")
+
+
+@pytest.mark.parametrize("seed", range(30))
+def test_sharded_and_labels_random_case(spr, seed):
+    from test_gpu_sharded import check_against, run_sharded
+    dtype, B, K, Kp, V, ldv, _, _ = draw_case(3000 + seed)
+    p, q, x, u = make_problem(seed, dtype, B, K, Kp, V, ldv)
+    ref = _clear_sd(p, q, V, x, u)
+    r = np.random.default_rng(seed)
+    G = int(r.integers(1, min(V, 6) + 1))
+    cuts = sorted(r.choice(np.arange(1, V), size=G - 1, replace=False).tolist()) if G > 1 else []
+    bounds = [0] + cuts + [V]
+    shards = [(bounds[g], bounds[g + 1] - bounds[g]) for g in range(G)]     # arbitrary, unaligned cuts
+    results = run_sharded(spr, p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), G, shards=shards)
+    check_against(ref, results, dtype)
+    lambdas = [1.0, 1.2, 1.5]
+    ws = spr.Workspace(spr.workspace_bytes(spr.binding.OP_VERIFIER_LABELS, B, K, V, 0, 0, spr.binding._dt(p)))
+    labels, ratio = spr.binding.verifier_labels(p.cuda(), q.cuda(), V, x.cuda(), lambdas, ws)
+    assert ws.device_status() == 0
+    want_labels, want_ratio = training.verifier_labels(to_np(p), to_np(q), V, to_np(x), lambdas)
+    assert np.all(np.abs(ratio.cpu().double().numpy() / want_ratio - 1.0) <= RTOL[dtype])
+    got = labels.cpu().numpy()
+    for i, lam in enumerate(lambdas):
+        clear = np.abs(want_ratio / lam - 1.0) > 1e-4
+        assert np.array_equal(got[i][clear], want_labels[i][clear])
