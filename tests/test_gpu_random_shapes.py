@@ -120,3 +120,45 @@ def test_sharded_and_labels_random_case(spr, seed):
     for i, lam in enumerate(lambdas):
         clear = np.abs(want_ratio / lam - 1.0) > 1e-4
         assert np.array_equal(got[i][clear], want_labels[i][clear])
+
+
+@pytest.mark.parametrize("seed", range(50))
+def test_sprinter_verify_random_case(spr, seed):
+    """Random verifier shapes through the automatic kernel choice (tensor-core kernel where its
+    shape and alignment rules hold, SIMT kernels elsewhere), hidden states and weights at random
+    element offsets from an aligned address."""
+    r = np.random.default_rng(4000 + seed)
+    g = torch.Generator().manual_seed(seed)
+    dtype = [torch.float32, torch.bfloat16, torch.bfloat16][int(r.integers(3))]
+    d = int(r.choice([8, 37, 64, 100, 128, 136, 256, 768, 1000, 1024, 2048]))
+    h = int(r.choice([0, 0, 1, 3, 16, 20, 64, 96, 128, 256]))
+    K = int(r.choice([1, 2, 4, 8, 16, 33]))
+    B = int(r.integers(1, max(2, 300 // K)))
+    tau = float(r.choice([0.5, 0.5, 0.3, 0.7]))
+    H = torch.randn((B, K, d), generator=g).to(dtype)
+    if h:
+        W1 = (torch.randn((h, d), generator=g) / d ** 0.5).to(dtype)
+        b1 = torch.randn(h, generator=g) / d ** 0.5
+        W2 = (torch.randn(h, generator=g) / h ** 0.5 * 3).to(dtype)
+    else:
+        W1 = (torch.randn(d, generator=g) / d ** 0.5 * 2).to(dtype)
+        b1 = W2 = None
+    b2 = torch.tensor([float(r.normal() * 0.2)])
+    npo = lambda t: None if t is None else to_np(t)   # noqa: E731
+    for _ in range(20):
+        s_ref, a_ref, fr_ref = oracle.sprinter_verify(to_np(H), to_np(W1), npo(b1), npo(W2), to_np(b2), tau)
+        near = np.argwhere(np.abs(s_ref - float(np.float32(tau))) < MARGIN)
+        if not len(near):
+            break
+        for b, k in near:
+            H[b, k] = torch.randn(d, generator=g).to(dtype)
+    aligned = r.random() < 0.5            # half of the cases keep 16-byte alignment (tensor-core path eligible)
+    off = (lambda: 0) if aligned else (lambda: int(r.integers(8)))
+    ws = spr.Workspace(spr.workspace_bytes(0, B, K, 1, d, h, spr.binding._dt(H)))
+    cu = lambda t: None if t is None else t.cuda()   # noqa: E731
+    scores, accept, fr = spr.sprinter_verify(offset_tensor(H, off()), offset_tensor(W1, off()), cu(b1),
+                                             None if W2 is None else offset_tensor(W2, off()), cu(b2), tau, ws)
+    assert ws.device_status() == 0
+    eq(accept, a_ref, "accept")
+    eq(fr, fr_ref, "first_reject")
+    assert_close_rel(scores, s_ref, RTOL[dtype], "scores")
