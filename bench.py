@@ -175,6 +175,20 @@ def slice_workload(wl, n):
     return type(wl)(**kw)
 
 
+def slice_rows(wl_cpu, lo, hi):
+    """Sequences lo .. hi-1 of a host workload."""
+    import dataclasses
+    import torch
+    kw = {}
+    for f in dataclasses.fields(wl_cpu):
+        v = getattr(wl_cpu, f.name)
+        if isinstance(v, torch.Tensor) and f.name not in ("W1", "b1", "W2", "b2"):
+            v = v[lo:hi].contiguous()
+        kw[f.name] = v
+    kw["B"] = hi - lo
+    return type(wl_cpu)(**kw)
+
+
 def run_reference(args):
     """The oracle as it stands, timed on the host cores: each step is a bounded sample."""
     rank = int(os.environ.get("RANK", "0"))
@@ -475,6 +489,18 @@ def main():
         cpu_baseline = {"value": sample * K / dt, "unit": "tokens/s", "cores": 1, "kind": "oracle",
                         "sample": f"first {sample} of {B} sequences ({sample * K} draft tokens), one pass, "
                                   f"{dt:.1f} s"}
+        # the same oracle, unchanged, on all host cores: sequences dealt to threads (the C calls
+        # release the interpreter lock)
+        from concurrent.futures import ThreadPoolExecutor
+        threads = max(1, min(os.cpu_count() or 1, sample))
+        parts = [slice_rows(wl_cpu, i * sample // threads, (i + 1) * sample // threads) for i in range(threads)]
+        t0 = time.perf_counter()
+        with ThreadPoolExecutor(threads) as pool:
+            list(pool.map(lambda part: oracle_step(part, tau), parts))
+        dt_all = time.perf_counter() - t0
+        cpu_baseline["all_cores"] = {"value": sample * K / dt_all, "unit": "tokens/s", "cores": threads,
+                                     "sample": f"the same {sample} sequences split over {threads} threads, "
+                                               f"{dt_all:.1f} s"}
 
     # each call on its own, one stream, events around 50 back-to-back launches
     def time_call(fn, n=50):
