@@ -59,6 +59,7 @@ struct TrainParams {
     float *loss;             // [1] or null
     float *part;             // [ctas, d+2]: per-CTA sums of the gradient terms, then of the loss
     int ctas;
+    int stages;              // rows a warp keeps in flight (queue variant)
 };
 
 // Gradient pass (one resident wave of CTAs): one warp per sample, samples dealt to warps in a
@@ -168,6 +169,131 @@ __global__ void __launch_bounds__(kThreads, VPL <= 3 ? 3 : (VPL <= 8 ? 2 : 1)) t
     for (int j = tid; j < d + 2; j += kThreads) out[j] = red[j];
 }
 
+// Short rows (at most 4 vectors per lane, d <= 1024 bf16): the same pass, but a warp's next
+// `depth` rows are already on their way into shared memory (cp.async, 16 bytes per lane per
+// copy) while it works on the current one, and the weights stay in registers.  A lane reads back
+// only what it copied itself, so the queue needs no barrier: cp.async.wait_group orders a lane's
+// own copies.  With 16 warps and 8 rows each an SM has ~190 KB of hidden states in flight.
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
+                 "l"(gmem_src)
+                 : "memory");
+}
+
+template <typename T, int VPL>
+__global__ void __launch_bounds__(kThreads, 2) train_grad_queue_kernel(const TrainParams prm)
+{
+    constexpr int N = Vec<T>::N;
+    extern __shared__ __align__(16) unsigned char qsmem[];
+    const int d = prm.d, depth = prm.stages;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nv = d / N;                     // vectors per row
+    const int slot_vecs = VPL * 32;           // vectors per queue slot
+    uint4 *queue = reinterpret_cast<uint4 *>(qsmem) + (size_t)warp * depth * slot_vecs;
+    float *red = reinterpret_cast<float *>(qsmem + (size_t)kWarps * depth * slot_vecs * 16);   // [d + 2] CTA sums
+
+    uint64_t w2[VPL * N / 2];                 // this lane's columns of the weight vector
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) {
+        const int vi = j * 32 + lane;
+#pragma unroll
+        for (int e = 0; e < N; e += 2)
+            w2[(j * N + e) / 2] = vi < nv ? pack2(prm.theta[vi * N + e], prm.theta[vi * N + e + 1]) : pack2(0.f, 0.f);
+    }
+    const float bias = prm.theta[d];
+    uint64_t acc[VPL * N / 2];
+#pragma unroll
+    for (int e = 0; e < VPL * N / 2; ++e) acc[e] = pack2(0.f, 0.f);
+    double acc_b = 0.0, acc_loss = 0.0;
+
+    const T *base = static_cast<const T *>(prm.hidden);
+    const int64_t stride = (int64_t)gridDim.x * kWarps;
+    const int64_t first = (int64_t)blockIdx.x * kWarps + warp;
+    const int64_t n = first < prm.N ? (prm.N - first + stride - 1) / stride : 0;   // this warp's rows
+    auto enqueue = [&](int64_t i, int slot) {       // row i of this warp -> queue slot (one commit group)
+        if (i < n) {
+            const uint4 *x = reinterpret_cast<const uint4 *>(base + (first + i * stride) * d);
+#pragma unroll
+            for (int j = 0; j < VPL; ++j) {
+                const int vi = j * 32 + lane;
+                if (vi < nv) cp_async16(queue + slot * slot_vecs + vi, x + vi);
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    for (int s = 0; s < depth; ++s) enqueue(s, s);
+    float y = n > 0 ? (float)prm.labels[first] : 0.f;
+    int slot = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        const float y_next = i + 1 < n ? (float)prm.labels[first + (i + 1) * stride] : 0.f;
+        // all but the newest depth-1 groups are complete: row i has landed
+        if (depth == 8) asm volatile("cp.async.wait_group 7;" ::: "memory");
+        else if (depth == 4) asm volatile("cp.async.wait_group 3;" ::: "memory");
+        else asm volatile("cp.async.wait_group 0;" ::: "memory");
+        uint4 raw[VPL];
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) {
+            const int vi = j * 32 + lane;
+            raw[j] = vi < nv ? queue[slot * slot_vecs + vi] : make_uint4(0u, 0u, 0u, 0u);
+        }
+        enqueue(i + depth, slot);               // the slot is free again: its values are in registers
+        uint64_t dot2 = pack2(0.f, 0.f);
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) {
+            float f[N];
+            Vec<T>::unpack(raw[j], f);
+#pragma unroll
+            for (int e = 0; e < N; e += 2) dot2 = fma2(pack2(f[e], f[e + 1]), w2[(j * N + e) / 2], dot2);
+        }
+        float d_even, d_odd;
+        unpack2(dot2, d_even, d_odd);
+        const float z = warp_sum(d_even + d_odd) + bias;
+        const float r = 1.f / (1.f + expf(-z)) - y;
+        const uint64_t r2 = pack2(r, r);
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) {
+            float f[N];
+            Vec<T>::unpack(raw[j], f);
+#pragma unroll
+            for (int e = 0; e < N; e += 2)
+                acc[(j * N + e) / 2] = fma2(r2, pack2(f[e], f[e + 1]), acc[(j * N + e) / 2]);
+        }
+        acc_b += (double)r;
+        acc_loss += (double)(fmaxf(z, 0.f) + log1pf(expf(-fabsf(z))) - y * z);
+        y = y_next;
+        if (++slot == depth) slot = 0;
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+
+    for (int w = 0; w < kWarps; ++w) {     // fixed order: warp 0 stores, the others add
+        if (warp == w) {
+#pragma unroll
+            for (int j = 0; j < VPL; ++j) {
+                const int vi = j * 32 + lane;
+                if (vi < nv) {
+#pragma unroll
+                    for (int e = 0; e < N; e += 2) {
+                        float lo, hi;
+                        unpack2(acc[(j * N + e) / 2], lo, hi);
+                        float *dst = red + vi * N + e;
+                        dst[0] = w == 0 ? lo : dst[0] + lo;
+                        dst[1] = w == 0 ? hi : dst[1] + hi;
+                    }
+                }
+            }
+            if (lane == 0) {
+                red[d] = w == 0 ? (float)acc_b : red[d] + (float)acc_b;
+                red[d + 1] = w == 0 ? (float)acc_loss : red[d + 1] + (float)acc_loss;
+            }
+        }
+        __syncthreads();
+    }
+    float *out = prm.part + (int64_t)blockIdx.x * (d + 2);
+    for (int j = tid; j < d + 2; j += kThreads) out[j] = red[j];
+}
+
 // One thread per parameter: sums the CTA partials in CTA order, divides by N, applies the
 // bias-corrected Adam update (arithmetic in double, state kept in float).
 __global__ void __launch_bounds__(256) train_adam_kernel(const TrainParams prm)
@@ -213,14 +339,37 @@ cudaError_t launch_grad(const TrainParams &tp, cudaStream_t st)
     return cudaGetLastError();
 }
 
+template <typename T, int VPL>
+cudaError_t launch_grad_queue(const TrainParams &tp, cudaStream_t st)
+{
+    TrainParams p = tp;
+    const size_t slot_bytes = (size_t)kWarps * VPL * 32 * 16;       // one queue slot of every warp
+    p.stages = slot_bytes * 8 <= 96 * 1024 ? 8 : 4;
+    const size_t smem = slot_bytes * p.stages + sizeof(float) * ((size_t)tp.d + 2);
+    cudaError_t e = cudaFuncSetAttribute(train_grad_queue_kernel<T, VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    int per_sm = 0, dev = 0, sms = 0;
+    if (e != cudaSuccess ||
+        (e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, train_grad_queue_kernel<T, VPL>, kThreads, smem)) !=
+            cudaSuccess ||
+        (e = cudaGetDevice(&dev)) != cudaSuccess ||
+        (e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+        return e;
+    if (per_sm < 1) return cudaErrorInvalidConfiguration;
+    p.ctas = (int)max((int64_t)1, min((int64_t)min(kTrainMaxCtas, per_sm * sms), (tp.N + kWarps - 1) / kWarps));
+    train_grad_queue_kernel<T, VPL><<<p.ctas, kThreads, smem, st>>>(p);
+    train_adam_kernel<<<(tp.d + 2 + 255) / 256, 256, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
 template <typename T>
 cudaError_t launch_grad_any(const TrainParams &tp, cudaStream_t st)
 {
     const int vpl = (tp.d / Vec<T>::N + 31) / 32;
-    if (vpl <= 1) return launch_grad<T, 1>(tp, st);
-    if (vpl <= 2) return launch_grad<T, 2>(tp, st);
-    if (vpl <= 3) return launch_grad<T, 3>(tp, st);
-    if (vpl <= 4) return launch_grad<T, 4>(tp, st);
+    if (vpl <= 1) return launch_grad_queue<T, 1>(tp, st);
+    if (vpl <= 2) return launch_grad_queue<T, 2>(tp, st);
+    if (vpl <= 3) return launch_grad_queue<T, 3>(tp, st);
+    if (vpl <= 4) return launch_grad_queue<T, 4>(tp, st);
     if (vpl <= 8) return launch_grad<T, 8>(tp, st);
     return launch_grad<T, 16>(tp, st);
 }
