@@ -58,6 +58,9 @@ __global__ void __launch_bounds__(kThreads, 4) sd_row_stats_kernel(const SdParam
         mp = warp_ms(MS{v.x, v.y});
         mq = warp_ms(MS{v.z, v.w});
     }
+    float m_p = mp.m, m_q = mq.m;
+    double z_p = mp.s, z_q = mq.s;
+    if (C > 1) {   // (a row that one CTA covers needs no ticket and no trip through global memory)
     if (lane == 0) {
         prm.part[row * C + c] = make_float4(mp.m, mp.s, mq.m, mq.s);
         __threadfence();
@@ -68,7 +71,7 @@ __global__ void __launch_bounds__(kThreads, 4) sd_row_stats_kernel(const SdParam
 
     // ---- this CTA saw the last chunk of the row: merge chunks in chunk order (warp 0)
     __threadfence();
-    float m_p = neg_inf(), m_q = neg_inf();
+    m_p = m_q = neg_inf();
     for (int cc = lane; cc < C; cc += 32) {
         const float4 v = __ldcg(&prm.part[row * C + cc]);
         m_p = fmaxf(m_p, v.x);
@@ -76,7 +79,7 @@ __global__ void __launch_bounds__(kThreads, 4) sd_row_stats_kernel(const SdParam
     }
     m_p = warp_max(m_p);
     m_q = warp_max(m_q);
-    double z_p = 0.0, z_q = 0.0;
+    z_p = z_q = 0.0;
     for (int c0 = 0; c0 < C; c0 += 32) {  // fixed order: chunk groups ascending, butterfly inside
         const int cc = c0 + lane;
         double a = 0.0, bq = 0.0;
@@ -92,6 +95,7 @@ __global__ void __launch_bounds__(kThreads, 4) sd_row_stats_kernel(const SdParam
         }
         z_p += a;
         z_q += bq;
+    }
     }
     int last_row = 0;
     if (lane == 0) {
