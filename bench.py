@@ -30,10 +30,10 @@ if ROOT not in sys.path:
 # capture summarised under profiles/; reported only while the kernel source is unchanged.
 NCU_TRAFFIC = {
     "sources": ("sd_row_stats.cu", "vocab_common.cuh", "common.cuh"),
-    "sha256": "55c54fc662a742d6e0d4b76da7e20c83800f853dea1c3ce4e81f5214cb199761",
-    # (262,802,944 read + 3,682,048 written) / 512 tokens in the B = 32 capture; traffic grows
+    "sha256": "2b0fecb1e12cbf45b8e20129dcea797c15c1934c08bf50e5d56dd7fa7fe3a644",
+    # (262,815,232 read + 3,749,120 written) / 512 tokens in the B = 32 capture; traffic grows
     # in proportion to the tokens, so a full launch is this times B*K
-    "bytes_per_unit": 520478,   # DRAM bytes per verified token at V = 128256, bf16
+    "bytes_per_unit": 520633,   # DRAM bytes per verified token at V = 128256, bf16
 }
 
 
