@@ -555,11 +555,13 @@ def main():
         t2 = time_call(lambda: bd.sd_shard_decide(all_stats, wl.draft_tokens, wl.uniforms, V, vs, wl.Kp, dt_code, w0,
                                                   out=dec[0]))
         t3 = time_call(lambda: bd.sd_shard_weights(pv, qv, n0, wl.uniforms, w0, out=o_w))
+        t23 = time_call(lambda: bd.sd_shard_decide_weights(pv, qv, all_stats, wl.draft_tokens, wl.uniforms, V, w0,
+                                                           extras=False))
         t4 = time_call(lambda: bd.sd_shard_draw(pv, qv, v0, all_w, all_stats, 0, n0, wl.uniforms, w0, out=o_tok))
         shard_bytes = (2 * M + B * (wl.Kp - K)) * vs * es
         calls[f"sd_verify_sharded_1_of_{G}"] = {
-            "shard_columns": vs, "stats_ms": t1, "decide_ms": t2, "weights_ms": t3, "draw_ms": t4,
-            "ms": t1 + t2 + t3 + t4, "stats_bytes": int(shard_bytes), "stats_gbs": shard_bytes / (t1 * 1e-3) / 1e9,
+            "shard_columns": vs, "stats_ms": t1, "decide_ms": t2, "weights_ms": t3, "decide_weights_ms": t23,
+            "draw_ms": t4, "ms": t1 + t23 + t4, "stats_bytes": int(shard_bytes), "stats_gbs": shard_bytes / (t1 * 1e-3) / 1e9,
             "exchange_bytes_per_gpu": int(B * wl.Kp * 24 + B * 16 + B * 4)}
 
     # preparing and fitting the verifier (Section 3.2): labels from the same logits, one optimiser step of

@@ -212,6 +212,8 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
  *                     whole-row probabilities at position accepted_len[b] < K;
  *                     (shard max, sum exp(l - shard max)) of the bonus row when
  *                     accepted_len[b] = K and Kp = K+1; (0, 0) when there is no draw.
+ *   (sd_shard_decide_weights does the two passes above in one launch: it takes the
+ *   arguments of both and gives the results of sd_shard_decide followed by sd_shard_weights.)
  *   -- all-gather weights -> all_weights [G, B, 2], rank order --
  *   sd_shard_draw     adds the G shard weights in rank order, finds the shard in which
  *                     uniforms[b,K] * total falls, and on that GPU (rank) locates the token
@@ -232,6 +234,10 @@ int sd_shard_decide(const float *all_stats, int G, const int32_t *draft_tokens, 
 int sd_shard_weights(const void *p_shard, const void *q_shard, int64_t ldv, int Vs, const int32_t *accepted_len,
                      const float *uniforms, int B, int K, int Kp, int dt, double *weights, void *ws,
                      size_t ws_bytes, void *cuda_stream);
+int sd_shard_decide_weights(const void *p_shard, const void *q_shard, int64_t ldv, int Vs, const float *all_stats,
+                            int G, const int32_t *draft_tokens, const float *uniforms, int B, int K, int Kp, int V,
+                            int dt, int32_t *accepted_len, uint8_t *accept, float *p_tok, float *q_tok,
+                            double *weights, void *ws, size_t ws_bytes, void *cuda_stream);
 int sd_shard_draw(const void *p_shard, const void *q_shard, int64_t ldv, int Vs, int v0, const double *all_weights,
                   const float *all_stats, int G, int rank, const int32_t *accepted_len, const float *uniforms,
                   int B, int K, int Kp, int dt, int32_t *correction_token, float *residual_mass, void *ws,

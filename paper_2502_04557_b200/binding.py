@@ -24,7 +24,7 @@ EXPORTS = [
     "spr_device_status", "spr_status_string", "spr_last_cuda_error", "spr_version",
     "spr_host_arena_bytes", "sprinter_verify_host", "replace_sample_host", "sd_verify_host",
     "spr_set_stage_events", "replace_sample_static", "sprinter_step", "sprinter_simulate",
-    "sd_shard_stats", "sd_shard_decide", "sd_shard_weights", "sd_shard_draw",
+    "sd_shard_stats", "sd_shard_decide", "sd_shard_weights", "sd_shard_draw", "sd_shard_decide_weights",
     "verifier_labels", "verifier_train_step",
 ]
 
@@ -79,6 +79,9 @@ def lib():
         L.sd_shard_decide.argtypes = [vp, i32, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
         L.sd_shard_weights.restype = i32
         L.sd_shard_weights.argtypes = [vp, vp, i64, i32, vp, vp, i32, i32, i32, i32, vp, vp, sz, vp]
+        L.sd_shard_decide_weights.restype = i32
+        L.sd_shard_decide_weights.argtypes = [vp, vp, i64, i32, vp, i32, vp, vp, i32, i32, i32, i32, i32,
+                                              vp, vp, vp, vp, vp, vp, sz, vp]
         L.sd_shard_draw.restype = i32
         L.sd_shard_draw.argtypes = [vp, vp, i64, i32, i32, vp, vp, i32, i32, vp, vp, i32, i32, i32, i32,
                                     vp, vp, vp, sz, vp]
@@ -371,6 +374,35 @@ def sd_shard_weights(p_shard, q_shard, accepted_len, uniforms, ws: Workspace, ou
                                 B, K, Kp, _dt(p_shard), _ptr(out), _ptr(ws.buf), ws.nbytes, _stream())
     _check("sd_shard_weights", rc)
     return out
+
+
+def sd_shard_decide_weights(p_shard, q_shard, all_stats, draft_tokens, uniforms, V: int, ws: Workspace,
+                            extras: bool = True):
+    """Passes 2 and 3 in one launch.  Returns (dict(accepted_len[, accept, p_tok, q_tok]), weights [B,2] f64)."""
+    ldv = _shard(p_shard, name="p_shard")
+    _shard(q_shard, p_shard.dtype, "q_shard")
+    B, Kp, Vs = p_shard.shape
+    K = q_shard.shape[1]
+    _dev(all_stats, torch.float32, "all_stats")
+    _dev(draft_tokens, torch.int32, "draft_tokens")
+    _dev(uniforms, torch.float32, "uniforms")
+    G = all_stats.shape[0]
+    if tuple(all_stats.shape) != (G, B * Kp, 6) or tuple(uniforms.shape) != (B, K + 1) or \
+            tuple(draft_tokens.shape) != (B, K):
+        raise ValueError("all_stats must be [G,B*Kp,6], draft_tokens [B,K] and uniforms [B,K+1]")
+    dev = p_shard.device
+    out = dict(accepted_len=torch.empty((B,), dtype=torch.int32, device=dev))
+    if extras:
+        out.update(accept=torch.empty((B, K), dtype=torch.uint8, device=dev),
+                   p_tok=torch.empty((B, K), dtype=torch.float32, device=dev),
+                   q_tok=torch.empty((B, K), dtype=torch.float32, device=dev))
+    weights = torch.empty((B, 2), dtype=torch.float64, device=dev)
+    rc = lib().sd_shard_decide_weights(_ptr(p_shard), _ptr(q_shard), ldv, Vs, _ptr(all_stats), G, _ptr(draft_tokens),
+                                       _ptr(uniforms), B, K, Kp, V, _dt(p_shard), _ptr(out["accepted_len"]),
+                                       _ptr(out.get("accept")), _ptr(out.get("p_tok")), _ptr(out.get("q_tok")),
+                                       _ptr(weights), _ptr(ws.buf), ws.nbytes, _stream())
+    _check("sd_shard_decide_weights", rc)
+    return out, weights
 
 
 def sd_shard_draw(p_shard, q_shard, v0: int, all_weights, all_stats, rank: int, accepted_len, uniforms,

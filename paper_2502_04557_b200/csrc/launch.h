@@ -100,7 +100,9 @@ struct ShardDrawParams {
 };
 cudaError_t launch_shard_stats(const ShardStatsParams &sp, int64_t rows, int dt, cudaStream_t st);
 cudaError_t launch_shard_decide(const ShardDecideParams &dp, int B, cudaStream_t st);
-cudaError_t launch_shard_weights(const ShardDrawParams &dp, int B, int dt, cudaStream_t st);
+// dec != null: the decision pass runs inside the weights kernel
+cudaError_t launch_shard_weights(const ShardDrawParams &dp, const ShardDecideParams *dec, int B, int dt,
+                                 cudaStream_t st);
 cudaError_t launch_shard_draw(const ShardDrawParams &dp, int B, int dt, cudaStream_t st);
 
 struct VerifyParams {

@@ -174,12 +174,12 @@ __device__ __forceinline__ void merge_shards(const float *all_stats, int64_t row
     lnZ = log(Z);
 }
 
-// One CTA per sequence: threads take the Kp rows, then warp 0 scans the accept bits.
-__global__ void __launch_bounds__(128) shard_decide_kernel(const ShardDecideParams prm)
+// Whole CTA, for sequence b of B: threads take the Kp rows, then warp 0 scans the accept bits.
+// Several CTAs may do this for the same sequence: they write the same values.
+__device__ __forceinline__ void decide_sequence(const ShardDecideParams &prm, int b, int B)
 {
-    const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31;
-    const int64_t rows = (int64_t)gridDim.x * prm.Kp;
+    const int64_t rows = (int64_t)B * prm.Kp;
     for (int k = tid; k < prm.Kp; k += blockDim.x) {
         const int64_t row = (int64_t)b * prm.Kp + k;
         float m_p, m_q = neg_inf();
@@ -233,6 +233,11 @@ __global__ void __launch_bounds__(128) shard_decide_kernel(const ShardDecidePara
     }
 }
 
+__global__ void __launch_bounds__(128) shard_decide_kernel(const ShardDecideParams prm)
+{
+    decide_sequence(prm, blockIdx.x, gridDim.x);
+}
+
 cudaError_t launch_shard_decide(const ShardDecideParams &dp, int B, cudaStream_t st)
 {
     if (B == 0) return cudaSuccess;
@@ -271,14 +276,21 @@ __device__ __forceinline__ Job<T> shard_job(const ShardDrawParams &prm, int b)
 // One CTA per (sequence, segment) writes the step partials; the last CTA of a sequence adds
 // them up: weights[b] = (largest step maximum, total weight relative to it); (0, total) for
 // residual draws, (0, 0) when the sequence has no draw.
-template <typename T>
-__global__ void __launch_bounds__(kThreads, 3) shard_weights_kernel(const ShardDrawParams prm)
+// kDecide: the kernel first takes the decision of its sequence itself (every CTA of a sequence
+// does, with identical results), which saves the separate decision launch.
+template <typename T, bool kDecide>
+__global__ void __launch_bounds__(kThreads, 3) shard_weights_kernel(const ShardDrawParams prm,
+                                                                    const ShardDecideParams dec)
 {
     __shared__ DrawSmem sm;
     const int C = prm.chunks;
     const int b = blockIdx.x / C;
     const int c = blockIdx.x % C;
     const int tid = threadIdx.x;
+    if (kDecide) {
+        decide_sequence(dec, b, (int)(gridDim.x / C));
+        __syncthreads();   // accepted_len[b] and the row statistics this CTA wrote are visible to all its threads
+    }
     const Job<T> job = shard_job<T>(prm, b);
     if (job.mode == MODE_NONE) {
         if (c == 0 && tid == 0) prm.weights[b] = make_double2(0.0, 0.0);
@@ -411,13 +423,20 @@ __global__ void __launch_bounds__(kThreads, 3) shard_draw_kernel(const ShardDraw
     if (tid == 0) prm.tokens[b] = token >= 0 ? token + prm.v0 : -1;
 }
 
-cudaError_t launch_shard_weights(const ShardDrawParams &dp, int B, int dt, cudaStream_t st)
+cudaError_t launch_shard_weights(const ShardDrawParams &dp, const ShardDecideParams *dec, int B, int dt,
+                                 cudaStream_t st)
 {
     const int64_t grid = (int64_t)B * dp.chunks;
     if (grid > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     if (grid == 0) return cudaSuccess;
-    if (dt == SPR_F32) shard_weights_kernel<float><<<(unsigned)grid, kThreads, 0, st>>>(dp);
-    else shard_weights_kernel<__nv_bfloat16><<<(unsigned)grid, kThreads, 0, st>>>(dp);
+    const ShardDecideParams none = {};
+    if (dec) {
+        if (dt == SPR_F32) shard_weights_kernel<float, true><<<(unsigned)grid, kThreads, 0, st>>>(dp, *dec);
+        else shard_weights_kernel<__nv_bfloat16, true><<<(unsigned)grid, kThreads, 0, st>>>(dp, *dec);
+    } else {
+        if (dt == SPR_F32) shard_weights_kernel<float, false><<<(unsigned)grid, kThreads, 0, st>>>(dp, none);
+        else shard_weights_kernel<__nv_bfloat16, false><<<(unsigned)grid, kThreads, 0, st>>>(dp, none);
+    }
     return cudaGetLastError();
 }
 

@@ -81,9 +81,11 @@ int sd_shard_stats(const void *p_shard, const void *q_shard, int64_t ldv, int Vs
     return finish(e);
 }
 
-int sd_shard_decide(const float *all_stats, int G, const int32_t *draft_tokens, const float *uniforms, int B,
-                    int K, int Kp, int V, int Vs, int dt, int32_t *accepted_len, uint8_t *accept, float *p_tok,
-                    float *q_tok, void *ws, size_t ws_bytes, void *cuda_stream)
+namespace {
+// validation and parameters of the decision pass; 1 = proceed, otherwise the status to return
+int decide_params(ShardDecideParams &dp, const float *all_stats, int G, const int32_t *draft_tokens,
+                  const float *uniforms, int B, int K, int Kp, int V, int Vs, int dt, int32_t *accepted_len,
+                  uint8_t *accept, float *p_tok, float *q_tok, void *ws, size_t ws_bytes)
 {
     int rc = check_sizes(B, K, Kp, Vs, Vs, dt);
     if (rc != 1) return rc;
@@ -94,9 +96,6 @@ int sd_shard_decide(const float *all_stats, int G, const int32_t *draft_tokens, 
         return SPR_ERR_INVALID_ARG;
     const ShardWs lay = layout(B, K, Kp, Vs, dt);
     if (!ws_ok(ws, ws_bytes, lay)) return SPR_ERR_WORKSPACE;
-    if ((rc = device_supported()) != SPR_OK) return rc;
-
-    ShardDecideParams dp;
     memset(&dp, 0, sizeof dp);
     dp.all_stats = all_stats;
     dp.G = G;
@@ -112,6 +111,19 @@ int sd_shard_decide(const float *all_stats, int G, const int32_t *draft_tokens, 
     dp.status = at<int>(ws, 0);
     dp.acc = at<uint8_t>(ws, lay.acc);
     dp.rowstats = at<float4>(ws, lay.rowstats);
+    return 1;
+}
+}  // namespace
+
+int sd_shard_decide(const float *all_stats, int G, const int32_t *draft_tokens, const float *uniforms, int B,
+                    int K, int Kp, int V, int Vs, int dt, int32_t *accepted_len, uint8_t *accept, float *p_tok,
+                    float *q_tok, void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    ShardDecideParams dp;
+    int rc = decide_params(dp, all_stats, G, draft_tokens, uniforms, B, K, Kp, V, Vs, dt, accepted_len, accept,
+                           p_tok, q_tok, ws, ws_bytes);
+    if (rc != 1) return rc;
+    if ((rc = device_supported()) != SPR_OK) return rc;
     return finish(launch_shard_decide(dp, B, static_cast<cudaStream_t>(cuda_stream)));
 }
 
@@ -159,7 +171,28 @@ int sd_shard_weights(const void *p_shard, const void *q_shard, int64_t ldv, int 
     dp.weights = reinterpret_cast<double2 *>(weights);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaMemsetAsync(dp.counters, 0, sizeof(int) * (size_t)B, st);
-    if (e == cudaSuccess) e = launch_shard_weights(dp, B, dt, st);
+    if (e == cudaSuccess) e = launch_shard_weights(dp, nullptr, B, dt, st);
+    return finish(e);
+}
+
+int sd_shard_decide_weights(const void *p_shard, const void *q_shard, int64_t ldv, int Vs, const float *all_stats,
+                            int G, const int32_t *draft_tokens, const float *uniforms, int B, int K, int Kp, int V,
+                            int dt, int32_t *accepted_len, uint8_t *accept, float *p_tok, float *q_tok,
+                            double *weights, void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    ShardDecideParams dec;
+    int rc = decide_params(dec, all_stats, G, draft_tokens, uniforms, B, K, Kp, V, Vs, dt, accepted_len, accept,
+                           p_tok, q_tok, ws, ws_bytes);
+    if (rc != 1) return rc;
+    ShardDrawParams dp;
+    rc = draw_params(dp, p_shard, q_shard, ldv, Vs, 0, accepted_len, uniforms, B, K, Kp, dt, ws, ws_bytes);
+    if (rc != 1) return rc;
+    if (!weights || !aligned(weights, 16)) return SPR_ERR_INVALID_ARG;
+    if ((rc = device_supported()) != SPR_OK) return rc;
+    dp.weights = reinterpret_cast<double2 *>(weights);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaMemsetAsync(dp.counters, 0, sizeof(int) * (size_t)B, st);
+    if (e == cudaSuccess) e = launch_shard_weights(dp, &dec, B, dt, st);
     return finish(e);
 }
 

@@ -51,7 +51,7 @@ class DistExchange:
 
 
 def sd_verify_sharded(p_shard, q_shard, V: int, v0: int, draft_tokens, uniforms, ws: _b.Workspace,
-                      exchange, extras: bool = True):
+                      exchange, extras: bool = True, fused: bool = True):
     """p_shard [B,Kp,Vs], q_shard [B,K,Vs] (rows may be strided), draft_tokens i32 [B,K] with
     whole-vocabulary ids, uniforms f32 [B,K+1]; `exchange` has rank, world, all_gather and
     all_reduce_max (a `DistExchange`).  Returns what `sd_verify` returns for the whole rows,
@@ -60,8 +60,12 @@ def sd_verify_sharded(p_shard, q_shard, V: int, v0: int, draft_tokens, uniforms,
     dt = _b._dt(p_shard)
     stats = _b.sd_shard_stats(p_shard, q_shard, v0, draft_tokens, ws)
     all_stats = exchange.all_gather(stats)
-    out = _b.sd_shard_decide(all_stats, draft_tokens, uniforms, V, Vs, Kp, dt, ws, extras=extras)
-    weights = _b.sd_shard_weights(p_shard, q_shard, out["accepted_len"], uniforms, ws)
+    if fused:     # decision and shard weights in one launch
+        out, weights = _b.sd_shard_decide_weights(p_shard, q_shard, all_stats, draft_tokens, uniforms, V, ws,
+                                                  extras=extras)
+    else:
+        out = _b.sd_shard_decide(all_stats, draft_tokens, uniforms, V, Vs, Kp, dt, ws, extras=extras)
+        weights = _b.sd_shard_weights(p_shard, q_shard, out["accepted_len"], uniforms, ws)
     all_weights = exchange.all_gather(weights)
     out.update(_b.sd_shard_draw(p_shard, q_shard, v0, all_weights, all_stats, exchange.rank,
                                 out["accepted_len"], uniforms, ws, extras=extras))

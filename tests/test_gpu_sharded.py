@@ -46,7 +46,7 @@ class ThreadExchange:
         return t
 
 
-def run_sharded(spr, p, q, V, x, u, G, shards=None, extras=True):
+def run_sharded(spr, p, q, V, x, u, G, shards=None, extras=True, fused=True):
     """p [B,Kp,ldv], q [B,K,ldv], x, u on the GPU; returns the result dict of every rank."""
     from paper_2502_04557_b200 import sharded
     shards = shards or sharded.vocab_shards(V, G, p.element_size())
@@ -62,7 +62,7 @@ def run_sharded(spr, p, q, V, x, u, G, shards=None, extras=True):
             with torch.cuda.stream(torch.cuda.Stream()):
                 ws = spr.Workspace(spr.workspace_bytes(spr.binding.OP_SD_SHARD, B, K, Vs, 0, 0, spr.binding._dt(p)))
                 results[g] = sharded.sd_verify_sharded(p[:, :, v0:v0 + Vs], q[:, :, v0:v0 + Vs], V, v0, x, u, ws,
-                                                       ThreadExchange(shared, g), extras=extras)
+                                                       ThreadExchange(shared, g), extras=extras, fused=fused)
                 results[g]["status"] = ws.device_status()
         except BaseException as e:   # noqa: BLE001 - release the other threads, then re-raise in the test
             errors.append(e)
@@ -100,6 +100,10 @@ def test_sharded_ragged_shapes(spr, dtype, B, K, V, ldv, Kp, G):
     ref = _clear_sd(p, q, V, x, u)
     results = run_sharded(spr, p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), G)
     check_against(ref, results, dtype)
+    if G == 3:      # the decision and the weights as separate launches give the same bits
+        split = run_sharded(spr, p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), G, fused=False)
+        for k in ("accept", "accepted_len", "correction_token", "p_tok", "q_tok", "residual_mass"):
+            assert torch.equal(split[0][k], results[0][k]), k
 
 
 @pytest.mark.parametrize("name,B,G", [("gpt2", 6, 4), ("llama2", 8, 2), ("llama3", 4, 8), ("sequential", 16, 8)])

@@ -193,7 +193,7 @@ def _rank_main_vocab(rank, world, port, out_dir):
     binding.sd_shard_weights, binding.sd_shard_draw = passes.weights, passes.draw
     v0, Vs = sharded.vocab_shards(wl.V, world, wl.p_logits.element_size())[rank]
     out = sharded.sd_verify_sharded(wl.p_logits[:, :, v0:v0 + Vs], wl.q_logits[:, :, v0:v0 + Vs], wl.V, v0,
-                                    wl.draft_tokens, wl.uniforms, None, ex)
+                                    wl.draft_tokens, wl.uniforms, None, ex, fused=False)
     full = oracle.sd_verify(to_np(wl.p_logits), to_np(wl.q_logits), wl.V, to_np(wl.draft_tokens),
                             to_np(wl.uniforms))
     ok = [int(np.array_equal(out[k].numpy(), full[k])) for k in ("accept", "accepted_len", "correction_token")]
