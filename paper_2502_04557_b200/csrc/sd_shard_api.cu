@@ -22,14 +22,16 @@ T *at(void *ws, size_t off)
 
 int finish(cudaError_t e) { return e == cudaSuccess ? SPR_OK : report_cuda_error(e); }
 
-// sizes shared by the four passes; 1 = proceed, otherwise the status to return
+constexpr int kProceed = -1;   // not a status: the arguments are fine and there is work to do
+
+// sizes shared by the passes; kProceed, or the status to return
 int check_sizes(int B, int K, int Kp, int Vs, int64_t ldv, int dt)
 {
     if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
     if (B < 0 || K <= 0 || Vs <= 0 || Vs > kMaxVocab || ldv < Vs || (Kp != K && Kp != K + 1) ||
         (int64_t)B * Kp > 0x7fffffff)
         return SPR_ERR_INVALID_ARG;
-    return B == 0 ? SPR_OK : 1;
+    return B == 0 ? SPR_OK : kProceed;
 }
 
 ShardWs layout(int B, int K, int Kp, int Vs, int dt)
@@ -51,7 +53,7 @@ int sd_shard_stats(const void *p_shard, const void *q_shard, int64_t ldv, int Vs
                    size_t ws_bytes, void *cuda_stream)
 {
     int rc = check_sizes(B, K, Kp, Vs, ldv, dt);
-    if (rc != 1) return rc;
+    if (rc != kProceed) return rc;
     if (v0 < 0 || !p_shard || !q_shard || !draft_tokens || !stats) return SPR_ERR_INVALID_ARG;
     const size_t es = elem_size(dt);
     if (!aligned(p_shard, es) || !aligned(q_shard, es) || !aligned(draft_tokens, 4) || !aligned(stats, 4))
@@ -82,13 +84,13 @@ int sd_shard_stats(const void *p_shard, const void *q_shard, int64_t ldv, int Vs
 }
 
 namespace {
-// validation and parameters of the decision pass; 1 = proceed, otherwise the status to return
+// validation and parameters of the decision pass; kProceed, or the status to return
 int decide_params(ShardDecideParams &dp, const float *all_stats, int G, const int32_t *draft_tokens,
                   const float *uniforms, int B, int K, int Kp, int V, int Vs, int dt, int32_t *accepted_len,
                   uint8_t *accept, float *p_tok, float *q_tok, void *ws, size_t ws_bytes)
 {
     int rc = check_sizes(B, K, Kp, Vs, Vs, dt);
-    if (rc != 1) return rc;
+    if (rc != kProceed) return rc;
     if (G <= 0 || G > kMaxRanks || V <= 0 || V > kMaxVocab) return SPR_ERR_INVALID_ARG;
     if (!all_stats || !draft_tokens || !uniforms || !accepted_len) return SPR_ERR_INVALID_ARG;
     if (!aligned(all_stats, 4) || !aligned(draft_tokens, 4) || !aligned(uniforms, 4) || !aligned(accepted_len, 4) ||
@@ -111,7 +113,7 @@ int decide_params(ShardDecideParams &dp, const float *all_stats, int G, const in
     dp.status = at<int>(ws, 0);
     dp.acc = at<uint8_t>(ws, lay.acc);
     dp.rowstats = at<float4>(ws, lay.rowstats);
-    return 1;
+    return kProceed;
 }
 }  // namespace
 
@@ -122,7 +124,7 @@ int sd_shard_decide(const float *all_stats, int G, const int32_t *draft_tokens, 
     ShardDecideParams dp;
     int rc = decide_params(dp, all_stats, G, draft_tokens, uniforms, B, K, Kp, V, Vs, dt, accepted_len, accept,
                            p_tok, q_tok, ws, ws_bytes);
-    if (rc != 1) return rc;
+    if (rc != kProceed) return rc;
     if ((rc = device_supported()) != SPR_OK) return rc;
     return finish(launch_shard_decide(dp, B, static_cast<cudaStream_t>(cuda_stream)));
 }
@@ -133,7 +135,7 @@ int draw_params(ShardDrawParams &dp, const void *p_shard, const void *q_shard, i
                 size_t ws_bytes)
 {
     int rc = check_sizes(B, K, Kp, Vs, ldv, dt);
-    if (rc != 1) return rc;
+    if (rc != kProceed) return rc;
     if (v0 < 0 || !p_shard || !q_shard || !accepted_len || !uniforms) return SPR_ERR_INVALID_ARG;
     const size_t es = elem_size(dt);
     if (!aligned(p_shard, es) || !aligned(q_shard, es) || !aligned(accepted_len, 4) || !aligned(uniforms, 4))
@@ -155,7 +157,7 @@ int draw_params(ShardDrawParams &dp, const void *p_shard, const void *q_shard, i
     dp.rowstats = at<float4>(ws, lay.rowstats);
     dp.counters = at<int>(ws, lay.draw_counters);
     dp.part = at<float2>(ws, lay.draw_part);
-    return 1;
+    return kProceed;
 }
 }  // namespace
 
@@ -165,7 +167,7 @@ int sd_shard_weights(const void *p_shard, const void *q_shard, int64_t ldv, int 
 {
     ShardDrawParams dp;
     int rc = draw_params(dp, p_shard, q_shard, ldv, Vs, 0, accepted_len, uniforms, B, K, Kp, dt, ws, ws_bytes);
-    if (rc != 1) return rc;
+    if (rc != kProceed) return rc;
     if (!weights || !aligned(weights, 16)) return SPR_ERR_INVALID_ARG;
     if ((rc = device_supported()) != SPR_OK) return rc;
     dp.weights = reinterpret_cast<double2 *>(weights);
@@ -183,10 +185,10 @@ int sd_shard_decide_weights(const void *p_shard, const void *q_shard, int64_t ld
     ShardDecideParams dec;
     int rc = decide_params(dec, all_stats, G, draft_tokens, uniforms, B, K, Kp, V, Vs, dt, accepted_len, accept,
                            p_tok, q_tok, ws, ws_bytes);
-    if (rc != 1) return rc;
+    if (rc != kProceed) return rc;
     ShardDrawParams dp;
     rc = draw_params(dp, p_shard, q_shard, ldv, Vs, 0, accepted_len, uniforms, B, K, Kp, dt, ws, ws_bytes);
-    if (rc != 1) return rc;
+    if (rc != kProceed) return rc;
     if (!weights || !aligned(weights, 16)) return SPR_ERR_INVALID_ARG;
     if ((rc = device_supported()) != SPR_OK) return rc;
     dp.weights = reinterpret_cast<double2 *>(weights);
@@ -203,7 +205,7 @@ int sd_shard_draw(const void *p_shard, const void *q_shard, int64_t ldv, int Vs,
 {
     ShardDrawParams dp;
     int rc = draw_params(dp, p_shard, q_shard, ldv, Vs, v0, accepted_len, uniforms, B, K, Kp, dt, ws, ws_bytes);
-    if (rc != 1) return rc;
+    if (rc != kProceed) return rc;
     if (G <= 0 || G > kMaxRanks || rank < 0 || rank >= G || (int64_t)v0 + Vs > kMaxVocab) return SPR_ERR_INVALID_ARG;
     if (!all_weights || !all_stats || !correction_token || !aligned(all_weights, 16) || !aligned(all_stats, 4) ||
         !aligned(correction_token, 4) || (residual_mass && !aligned(residual_mass, 4)))

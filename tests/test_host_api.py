@@ -108,3 +108,42 @@ def test_shard_batch_partitions():
             for (f0, n0), (f1, _) in zip(spans, spans[1:]):
                 assert f0 + n0 == f1
             assert max(n for _, n in spans) - min(n for _, n in spans) <= 1
+
+
+def test_argument_validation_of_the_later_entry_points():
+    """Shards, labels and the training step: sizes and pointers are checked on the host, before any
+    device call (the pointers here are never dereferenced)."""
+    L = spr.lib()
+    buf = (ctypes.c_char * 4096)()
+    addr = (ctypes.addressof(buf) + 255) // 256 * 256
+    p = ctypes.c_void_p(addr)
+    lam = (ctypes.c_float * 3)(1.0, 1.2, 1.5)
+    lamp = ctypes.cast(lam, ctypes.c_void_p)
+    # shard statistics: null tensor, negative offset, Kp not in {K, K+1}, workspace too small
+    assert L.sd_shard_stats(None, p, 8, 8, 0, p, 1, 1, 1, 0, p, p, 1 << 20, None) == 1
+    assert L.sd_shard_stats(p, p, 8, 8, -1, p, 1, 1, 1, 0, p, p, 1 << 20, None) == 1
+    assert L.sd_shard_stats(p, p, 8, 8, 0, p, 1, 1, 3, 0, p, p, 1 << 20, None) == 1
+    assert L.sd_shard_stats(p, p, 8, 8, 0, p, 1, 1, 1, 0, p, p, 16, None) == 3
+    assert L.sd_shard_stats(p, p, 8, 8, 0, p, 0, 1, 1, 0, p, p, 16, None) == 0          # empty batch
+    # decision: no shards, too many shards
+    assert L.sd_shard_decide(p, 0, p, p, 1, 1, 1, 8, 8, 0, p, None, None, None, p, 1 << 20, None) == 1
+    assert L.sd_shard_decide(p, 5000, p, p, 1, 1, 1, 8, 8, 0, p, None, None, None, p, 1 << 20, None) == 1
+    # draw: rank outside [0, G)
+    assert L.sd_shard_draw(p, p, 8, 8, 0, p, p, 2, 2, p, p, 1, 1, 1, 0, p, None, p, 1 << 20, None) == 1
+    # labels: no thresholds, too many, null output
+    assert L.verifier_labels(p, p, 8, p, 1, 1, 1, 8, 0, lamp, 0, p, None, p, 1 << 20, None) == 1
+    assert L.verifier_labels(p, p, 8, p, 1, 1, 1, 8, 0, lamp, 9, p, None, p, 1 << 20, None) == 1
+    assert L.verifier_labels(p, p, 8, p, 1, 1, 1, 8, 0, lamp, 3, None, None, p, 1 << 20, None) == 1
+    assert L.verifier_labels(p, p, 8, p, 1, 1, 1, 8, 7, lamp, 3, p, None, p, 1 << 20, None) == 2
+    # training step: step 0, beta out of range, width not a whole number of vectors / too wide
+    f = ctypes.c_float
+    assert L.verifier_train_step(p, p, 4, 8, 1, p, p, p, 0, f(.01), f(.9), f(.999), f(1e-8), None, p, 1 << 20, None) == 1
+    assert L.verifier_train_step(p, p, 4, 8, 1, p, p, p, 1, f(.01), f(1.0), f(.999), f(1e-8), None, p, 1 << 20, None) == 1
+    assert L.verifier_train_step(p, p, 4, 12, 1, p, p, p, 1, f(.01), f(.9), f(.999), f(1e-8), None, p, 1 << 20, None) == 2
+    assert L.verifier_train_step(p, p, 4, 8192, 1, p, p, p, 1, f(.01), f(.9), f(.999), f(1e-8), None, p, 1 << 26, None) == 2
+    assert L.verifier_train_step(p, p, 0, 8, 1, p, p, p, 1, f(.01), f(.9), f(.999), f(1e-8), None, p, 1 << 20, None) == 0
+    assert L.verifier_train_step(p, p, 4, 8, 1, p, p, p, 1, f(.01), f(.9), f(.999), f(1e-8), None, p, 16, None) == 3
+    wb = spr.workspace_bytes
+    assert wb(binding.OP_SD_SHARD, 4, 2, 1000, 0, 0, spr.BF16) > 0 and wb(binding.OP_SD_SHARD, 4, 0, 1000, 0, 0, spr.BF16) == 0
+    assert wb(binding.OP_VERIFIER_LABELS, 4, 2, 1000, 0, 0, spr.BF16) > 0
+    assert wb(binding.OP_VERIFIER_TRAIN, 0, 0, 0, 768, 0, spr.BF16) >= 592 * 770 * 4
