@@ -147,3 +147,31 @@ def test_argument_validation_of_the_later_entry_points():
     assert wb(binding.OP_SD_SHARD, 4, 2, 1000, 0, 0, spr.BF16) > 0 and wb(binding.OP_SD_SHARD, 4, 0, 1000, 0, 0, spr.BF16) == 0
     assert wb(binding.OP_VERIFIER_LABELS, 4, 2, 1000, 0, 0, spr.BF16) > 0
     assert wb(binding.OP_VERIFIER_TRAIN, 0, 0, 0, 768, 0, spr.BF16) >= 592 * 770 * 4
+
+
+def test_argument_validation_of_the_host_buffer_static_and_simulator_calls():
+    L = spr.lib()
+    buf = (ctypes.c_char * 4096)()
+    addr = (ctypes.addressof(buf) + 255) // 256 * 256
+    p = ctypes.c_void_p(addr)
+    f = ctypes.c_float
+    # host-buffer variants: bad dtype, bad sizes, arena too small
+    assert L.sd_verify_host(p, p, 8, p, p, 1, 1, 1, 8, 9, p, p, None, None, None, None, p, 1 << 20, p, 1 << 20, None) == 2
+    assert L.sd_verify_host(p, p, 4, p, p, 1, 1, 1, 8, 0, p, p, None, None, None, None, p, 1 << 20, p, 1 << 20, None) == 1
+    assert L.sd_verify_host(p, p, 8, p, p, 1, 1, 1, 8, 0, p, p, None, None, None, None, p, 16, p, 1 << 20, None) == 3
+    assert L.sprinter_verify_host(p, p, p, p, p, f(.5), 1, 0, 8, 4, 0, 0, None, p, p, p, 1 << 20, p, 1 << 20, None) == 1
+    assert L.replace_sample_host(p, 8, 0, 1, None, None, 0, 1, 1, p, 0, p, p, 1 << 20, p, 1 << 20, None) == 1
+    assert L.spr_host_arena_bytes(2, 4, 2, 3, 1000, 0, 0, 1) > 2 * 4 * 2 * 1000 * 2
+    assert L.spr_host_arena_bytes(2, 4, 2, 3, 1000, 0, 0, 5) == 0
+    # the call without a workspace: too many draws, too long rows, bad sizes
+    assert L.replace_sample_static(p, 8, 8, 2000, None, None, 0, 1, 2000, p, 0, p, None) == 3
+    assert L.replace_sample_static(p, 8, 0, 1, None, None, 0, 1, 1, p, 0, p, None) == 1
+    assert L.replace_sample_static(None, 8, 8, 0, None, None, 0, 1, 0, None, 0, None, None) == 0
+    # simulator: nothing to write to, rates outside [0, 1], negative counts
+    u64 = ctypes.c_uint64
+    assert L.sprinter_simulate(u64(1), 0, 10, 5, f(.9), f(.5), 16, None, None, None) == 1
+    assert L.sprinter_simulate(u64(1), 0, 10, 5, f(1.5), f(.5), 16, p, None, None) == 1
+    assert L.sprinter_simulate(u64(1), 0, -1, 5, f(.9), f(.5), 16, p, None, None) == 1
+    # the fused step: same checks as its two halves
+    assert L.sprinter_step(p, p, p, p, p, f(.5), 1, 1, 8, 4, p, 4, 8, 1, p, 0, 0, None, p, p, p, p, 1 << 20, None) == 1   # ldv < V
+    assert L.sprinter_step(p, p, p, p, p, f(.5), 1, 1, 8, 4, p, 8, 8, 1, p, 0, 0, None, p, p, p, p, 16, None) == 3
