@@ -162,3 +162,36 @@ def test_sprinter_verify_random_case(spr, seed):
     eq(accept, a_ref, "accept")
     eq(fr, fr_ref, "first_reject")
     assert_close_rel(scores, s_ref, RTOL[dtype], "scores")
+
+
+def test_many_short_rows(spr):
+    """Row counts far above the CTA slots of the GPU (and a grid of 10^5 CTAs): short rows, so the
+    oracle still finishes in seconds."""
+    B, K, V = 50000, 2, 40
+    g = torch.Generator().manual_seed(77)
+    q = torch.randn((B, K, V), generator=g) * 2.0
+    p = torch.cat([q, torch.randn((B, 1, V), generator=g) * 2.0], 1) + 0.7 * torch.randn((B, K + 1, V), generator=g)
+    x = torch.randint(0, V, (B, K), generator=g, dtype=torch.int32)
+    u = torch.rand((B, K + 1), generator=g)
+    ref = oracle.sd_verify(to_np(p), to_np(q), V, to_np(x), to_np(u))
+    ws = spr.Workspace(spr.workspace_bytes(2, B, K, V, 1, 0, spr.F32))
+    out = spr.sd_verify(p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), ws)
+    assert ws.device_status() == 0
+    ratio = ref["p_tok"] / ref["q_tok"]
+    clear = np.abs(u[:, :K].numpy().astype(np.float64) - ratio) >= MARGIN
+    assert clear.mean() > 0.999
+    got = out["accept"].cpu().numpy()
+    assert np.array_equal(got[clear], ref["accept"][clear])
+    seq_clear = clear.all(axis=1)
+    assert np.array_equal(out["accepted_len"].cpu().numpy()[seq_clear], ref["accepted_len"][seq_clear])
+    tok = out["correction_token"].cpu().numpy()
+    agree = (tok == ref["correction_token"])[seq_clear].mean()       # draws are not redrawn here: ties are rare
+    assert agree > 0.999 and ((tok >= 0) & (tok < V)).all()
+    assert_close_rel(out["p_tok"], ref["p_tok"], RTOL[torch.float32], "p_tok")
+    # as many replacement draws, each from its own row
+    rows = torch.arange(B, dtype=torch.int32) * (K + 1)
+    ur = torch.rand(B, generator=g)
+    ws2 = spr.Workspace(spr.workspace_bytes(1, B, 1, V, 1, 0, spr.F32))
+    tokens = spr.replace_sample(p.cuda(), V, ur.cuda(), ws2, rows=rows.cuda()).cpu().numpy()
+    want = oracle.replace_sample(to_np(p).reshape(B * (K + 1), V), V, ur.numpy(), rows=rows.numpy())
+    assert (tokens == want).mean() > 0.999 and ws2.device_status() == 0
