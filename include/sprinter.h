@@ -111,8 +111,8 @@ int sprinter_verify(const void *hidden, const void *W1, const float *b1, const v
 /*
  * replace_sample - the target model's replacement token for a rejected draft.
  *
- * Defined by: Algorithm 2, the lines after the loop ("Run M_p once"): p' <- p,
- * t ~ p'.  The draw is an inverse CDF in vocabulary order driven by a
+ * Defined by: Algorithm 2, the part after the loop (the single call of the target
+ * model): p' <- p, t ~ p'.  The draw is an inverse CDF in vocabulary order driven by a
  * caller-supplied uniform: with e_i = exp(l_i - max l),
  *   t = min{ j : sum_{i<=j} e_i > u * sum_i e_i }
  * (the last index with e_j > 0 if rounding leaves none).

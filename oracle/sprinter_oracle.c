@@ -14,8 +14,8 @@
  *                             sigmoid (Section 3.2, "Verifier architecture"),
  *                             or the synthetic d->h->1 ReLU MLP of the
  *                             workloads.
- *   oracle_replace_sample   - "Run M_p once", p' <- p, t ~ p' (Algorithm 2,
- *                             the lines after the loop, branch c <= n).
+ *   oracle_replace_sample   - the single target-model call: p' <- p, t ~ p'
+ *                             (Algorithm 2, the part after the loop, branch c <= n).
  *   oracle_sd_verify        - accept with probability min(1, p(x)/q(x)), else
  *                             resample from norm(max(0, p - q)) (Section 2 and
  *                             Eq. 1; Algorithm 2, branch c > n).
@@ -399,7 +399,7 @@ double oracle_residual_draw_margin(const void *p_row, const void *q_row, int dt,
 
 /* ---- decode-loop statistics with an i.i.d. verifier (Section 3.1, Theorems 2 and 3) ----
  *
- * Scenario of Fig. "token generation": the draft produces r acceptable tokens followed by
+ * Scenario of the token-generation figure of Section 3.1: the draft produces r acceptable tokens followed by
  * unacceptable ones; the verifier accepts an acceptable token with probability eta_TP and an
  * unacceptable one with probability eta_FP, independently; N = number of consecutive tokens
  * it accepts before its first rejection.  Run i draws its uniforms from the counter-based
