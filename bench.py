@@ -502,17 +502,31 @@ def main():
                                      "sample": f"the same {sample} sequences split over {threads} threads, "
                                                f"{dt_all:.1f} s"}
 
-    # each call on its own, one stream, events around 50 back-to-back launches
-    def time_call(fn, n=50):
-        for _ in range(3):
-            fn()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for _ in range(n):
-            fn()
-        b.record()
-        torch.cuda.synchronize()
-        return a.elapsed_time(b) / n
+    # each call on its own: n back-to-back calls captured into one CUDA graph (no host launch cost
+    # between them), events around a replay, best of three replays -> ms of GPU time per call
+    def time_call(fn, n=20):
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for _ in range(3):
+                fn()
+            side.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for _ in range(n):
+                    fn()
+            graph.replay()
+            side.synchronize()
+            best = float("inf")
+            for _ in range(3):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                graph.replay()
+                b.record()
+                side.synchronize()
+                best = min(best, a.elapsed_time(b) / n)
+        torch.cuda.current_stream().wait_stream(side)
+        return best
 
     fr = ver_out[2]
     t_ver = time_call(lambda: spr.sprinter_verify(wl.hidden, wl.W1, wl.b1, wl.W2, wl.b2, tau, ws, out=ver_out))
@@ -570,13 +584,13 @@ def main():
     ws_fit = spr.Workspace(max(spr.workspace_bytes(bd.OP_VERIFIER_LABELS, B, K, V, 0, 0, dt_code),
                                spr.workspace_bytes(bd.OP_VERIFIER_TRAIN, 0, 0, 0, cfg.d, 0, dt_code)), device=dev)
     t_lab = time_call(lambda: bd.verifier_labels(wl.p_logits, wl.q_logits, V, wl.draft_tokens, [1.0, 1.2, 1.5], ws_fit,
-                                                 want_ratio=False), n=20)
+                                                 want_ratio=False), n=10)
     n_fit = args.fit_samples
     fit_h = torch.randn((n_fit, cfg.d), device=dev).to(wl.hidden.dtype)
     fit_y = (torch.rand(n_fit, device=dev) < 0.5).to(torch.uint8)
     fit_state = [torch.zeros(cfg.d + 1, device=dev) for _ in range(3)]
     fit_loss = torch.empty(1, device=dev)
-    t_fit = time_call(lambda: bd.verifier_train_step(fit_h, fit_y, *fit_state, 1, 1e-3, ws_fit, loss=fit_loss), n=20)
+    t_fit = time_call(lambda: bd.verifier_train_step(fit_h, fit_y, *fit_state, 1, 1e-3, ws_fit, loss=fit_loss), n=10)
     calls["verifier_labels"] = {"ms": t_lab, "tokens_per_s": M / (t_lab * 1e-3), "bytes": int(alg_bytes),
                                 "gbs": alg_bytes / (t_lab * 1e-3) / 1e9}
     calls["verifier_train_step"] = {"ms": t_fit, "samples": n_fit, "d": cfg.d, "samples_per_s": n_fit / (t_fit * 1e-3),
