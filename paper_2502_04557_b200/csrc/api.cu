@@ -48,10 +48,6 @@ int check_device()
 // AUTO hands batches of at least this many tokens to the tensor-core verifier
 constexpr int kTensorMinTokens = 4;
 
-// sd_verify launches the correction draws from the device up to this many sequences (the device
-// runtime keeps at most 2048 launches pending by default)
-constexpr int kMaxDeviceDraws = 1024;
-
 // row indices are 32-bit inside the kernels; leave room for the padding of the last step
 constexpr int kMaxVocab = 1 << 30;
 
@@ -360,17 +356,8 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaMemsetAsync(sp.row_counters, 0, lay.counters_end - lay.row_counters, st);
-    // Device-side launches of the per-sequence draws: not while the stream is being captured, and
-    // not beyond the device runtime's limit of pending launches.
-    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
-    if (e == cudaSuccess) e = cudaStreamIsCapturing(st, &capturing);
-    sp.device_draw = capturing == cudaStreamCaptureStatusNone && B <= kMaxDeviceDraws;
-    if (sp.device_draw) {
-        sp.draw = dp;
-        draw_geometry(1, T, &sp.draw.chunks, &sp.draw.iters);   // one draw per launch: spread it wide
-    }
     if (e == cudaSuccess) e = launch_sd_row_stats(sp, B, K, dt, st);
-    if (e == cudaSuccess && !sp.device_draw) e = launch_draw(dp, B, dt, st, /*after_kernel=*/true);
+    if (e == cudaSuccess) e = launch_draw(dp, B, dt, st, /*after_kernel=*/true);
     return e == cudaSuccess ? SPR_OK : cuda_fail(e);
 }
 

@@ -6,34 +6,6 @@
 
 namespace spr {
 
-enum { DRAW_REPLACE = 0, DRAW_SD = 1 };
-
-struct DrawParams {
-    int kind;
-    const void *p;
-    const void *q;
-    int64_t ldv;
-    int V, chunks, steps;   // segments (CTAs) and warp steps per row
-    int first;              // index of the first draw of this launch (device-side launches: one draw each)
-    int iters;              // warp steps each warp of a CTA takes (1, 2 or 4)
-    // replace_sample
-    int64_t R;
-    const int32_t *rows;
-    const int32_t *gate;
-    int seq_stride;
-    // sd_verify correction draw (K also bounds the gate of replace_sample)
-    int K, Kp;
-    const int32_t *accepted_len;
-    const float4 *rowstats;
-    const float *uniforms;
-    int32_t *tokens;
-    float *residual_mass;
-    // workspace
-    int *status;
-    int *counters;   // [n]
-    float2 *part;    // [n*steps] (max, weight) of every warp step
-};
-
 struct SdParams {
     const void *p;  // [B,Kp,ldv]
     const void *q;  // [B,K,ldv]
@@ -53,11 +25,34 @@ struct SdParams {
     uint8_t *acc;       // [B*K]
     float4 *part;       // [B*K*chunks]
     float4 *rowstats;   // [B*K]
-    // the correction draw of a sequence is launched from the device when that sequence completes
-    int device_draw;
-    DrawParams draw;
 };
 
+enum { DRAW_REPLACE = 0, DRAW_SD = 1 };
+
+struct DrawParams {
+    int kind;
+    const void *p;
+    const void *q;
+    int64_t ldv;
+    int V, chunks, steps;   // segments (CTAs) and warp steps per row
+    int iters;              // warp steps each warp of a CTA takes (1, 2 or 4)
+    // replace_sample
+    int64_t R;
+    const int32_t *rows;
+    const int32_t *gate;
+    int seq_stride;
+    // sd_verify correction draw (K also bounds the gate of replace_sample)
+    int K, Kp;
+    const int32_t *accepted_len;
+    const float4 *rowstats;
+    const float *uniforms;
+    int32_t *tokens;
+    float *residual_mass;
+    // workspace
+    int *status;
+    int *counters;   // [n]
+    float2 *part;    // [n*steps] (max, weight) of every warp step
+};
 
 // Vocabulary-sharded sd_verify (sd_shard.cu): V is the width of this GPU's shard, v0 its
 // first column; *_all arrays hold one block per rank, in rank order.

@@ -2,7 +2,7 @@
 // and the first-rejection scan.  Streams each logits row from HBM exactly once in 16-byte
 // vectors; per-segment partial results go to the last CTA that finishes a row ("last block
 // done" tickets: nothing ever waits on another CTA).
-#include "draw_common.cuh"
+#include "vocab_common.cuh"
 
 namespace spr {
 
@@ -146,24 +146,9 @@ __global__ void __launch_bounds__(kThreads, 4) sd_row_stats_kernel(const SdParam
         if (rej != 0u && first == prm.K) first = k0 + __ffs(rej) - 1;
     }
     if (lane == 0) {
-        const int nb = bad ? -1 : first;
-        prm.accepted_len[b] = nb;
+        prm.accepted_len[b] = bad ? -1 : first;
         if (bad && prm.accept)
             for (int kk = 0; kk < prm.K; ++kk) prm.accept[(int64_t)b * prm.K + kk] = 0;
-        if (prm.device_draw) {
-            // The sequence is complete: its correction draw starts now, as a grid of its own,
-            // while the rows it needs are still in L2 and the rest of this grid keeps streaming.
-            if (nb < 0 || (nb == prm.K && prm.Kp == prm.K)) {
-                prm.draw.tokens[b] = -1;
-                if (prm.draw.residual_mass) prm.draw.residual_mass[b] = 0.f;
-            } else {
-                DrawParams d = prm.draw;
-                d.first = b;
-                __threadfence();
-                draw_kernel<T, false><<<d.chunks, kThreads, 0, cudaStreamFireAndForget>>>(d);
-                if (cudaGetLastError() != cudaSuccess) raise_status(prm.status, SPR_ERR_CUDA);
-            }
-        }
     }
 }
 
