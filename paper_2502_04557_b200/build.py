@@ -10,7 +10,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libsprinter.so")
 SOURCES = ["api.cu", "host_api.cu", "sd_row_stats.cu", "draw.cu", "verifier_simt.cu", "verifier_tensor.cu", "no_alloc.cu", "simulate.cu", "sd_shard.cu", "sd_shard_api.cu", "verifier_fit.cu"]
-HEADERS = ["common.cuh", "launch.h", "verifier_common.cuh", "vocab_common.cuh", "draw_common.cuh"]
+HEADERS = ["common.cuh", "launch.h", "verifier_common.cuh", "vocab_common.cuh", "draw_common.cuh", "host_util.h"]
 
 
 def _nvcc() -> str:

@@ -3,6 +3,7 @@
 #include <string.h>
 
 #include "common.cuh"
+#include "host_util.h"
 #include "launch.h"
 
 using namespace spr;
@@ -51,14 +52,6 @@ constexpr int kTensorMinTokens = 4;
 // row indices are 32-bit inside the kernels; leave room for the padding of the last step
 constexpr int kMaxVocab = 1 << 30;
 
-bool dtype_ok(int dt) { return dt == SPR_F32 || dt == SPR_BF16; }
-bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
-
-template <typename T>
-T *at(void *ws, size_t off)
-{
-    return reinterpret_cast<T *>(static_cast<char *>(ws) + off);
-}
 
 // tensor-core kernel where it applies (or is forced), SIMT kernel otherwise
 int launch_verifier(VerifyParams &vp, int dt, int path, cudaStream_t st)

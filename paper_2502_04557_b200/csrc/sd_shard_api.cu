@@ -2,6 +2,7 @@
 #include <string.h>
 
 #include "common.cuh"
+#include "host_util.h"
 #include "launch.h"
 
 using namespace spr;
@@ -11,16 +12,6 @@ namespace {
 constexpr int kMaxVocab = 1 << 30;
 constexpr int kMaxRanks = 1024;
 
-bool dtype_ok(int dt) { return dt == SPR_F32 || dt == SPR_BF16; }
-bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
-
-template <typename T>
-T *at(void *ws, size_t off)
-{
-    return reinterpret_cast<T *>(static_cast<char *>(ws) + off);
-}
-
-int finish(cudaError_t e) { return e == cudaSuccess ? SPR_OK : report_cuda_error(e); }
 
 constexpr int kProceed = -1;   // not a status: the arguments are fine and there is work to do
 

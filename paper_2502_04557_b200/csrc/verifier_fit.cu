@@ -3,6 +3,7 @@
 // linear-layer + sigmoid verifier on the draft model's hidden states.
 #include <string.h>
 
+#include "host_util.h"
 #include "launch.h"
 #include "vocab_common.cuh"
 
@@ -374,14 +375,6 @@ cudaError_t launch_grad_any(const TrainParams &tp, cudaStream_t st)
     return launch_grad<T, 16>(tp, st);
 }
 
-bool dtype_ok(int dt) { return dt == SPR_F32 || dt == SPR_BF16; }
-bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
-template <typename T>
-T *at(void *ws, size_t off)
-{
-    return reinterpret_cast<T *>(static_cast<char *>(ws) + off);
-}
-int finish(cudaError_t e) { return e == cudaSuccess ? SPR_OK : report_cuda_error(e); }
 
 }  // namespace
 
