@@ -175,3 +175,17 @@ def test_argument_validation_of_the_host_buffer_static_and_simulator_calls():
     # the fused step: same checks as its two halves
     assert L.sprinter_step(p, p, p, p, p, f(.5), 1, 1, 8, 4, p, 4, 8, 1, p, 0, 0, None, p, p, p, p, 1 << 20, None) == 1   # ldv < V
     assert L.sprinter_step(p, p, p, p, p, f(.5), 1, 1, 8, 4, p, 8, 8, 1, p, 0, 0, None, p, p, p, p, 16, None) == 3
+
+
+def test_binding_constants_match_the_header():
+    text = open(os.path.join(ROOT, "include", "sprinter.h")).read()
+    enum = dict((k, int(v)) for k, v in re.findall(r"\b(SPR_[A-Z0-9_]+)\s*=\s*(\d+)", text))
+    assert enum["SPR_F32"] == binding.F32 and enum["SPR_BF16"] == binding.BF16
+    for name in ("SPRINTER_VERIFY", "REPLACE_SAMPLE", "SD_VERIFY", "SPRINTER_STEP", "SD_SHARD", "VERIFIER_LABELS",
+                 "VERIFIER_TRAIN"):
+        assert enum["SPR_OP_" + name] == getattr(binding, "OP_" + name), name
+    assert (enum["SPR_VERIFIER_AUTO"], enum["SPR_VERIFIER_SIMT"], enum["SPR_VERIFIER_TENSOR"]) == \
+        (binding.PATH_AUTO, binding.PATH_SIMT, binding.PATH_TENSOR)
+    L = spr.lib()
+    for code in range(8):                      # every status has a text
+        assert len(L.spr_status_string(code).decode()) > 3
