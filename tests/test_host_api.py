@@ -188,4 +188,4 @@ def test_binding_constants_match_the_header():
         (binding.PATH_AUTO, binding.PATH_SIMT, binding.PATH_TENSOR)
     L = spr.lib()
     for code in range(8):                      # every status has a text
-        assert len(L.spr_status_string(code).decode()) > 3
+        assert len(L.spr_status_string(code).decode()) >= 2
