@@ -147,6 +147,19 @@ def _dev(t: torch.Tensor, dtype=None, name="tensor"):
     return t
 
 
+def _selectors(rows, first_reject, n: int):
+    """The optional int32 [n] row selectors of a replacement draw: the kernel reads n entries of
+    each, as 32-bit integers, so anything else is refused here."""
+    for name, t in (("rows", rows), ("first_reject", first_reject)):
+        if t is None:
+            continue
+        if t.dtype != torch.int32:
+            raise TypeError(f"{name} must be torch.int32, got {t.dtype}")
+        if t.numel() != n:
+            raise ValueError(f"{name} must have one entry per draw ({n}), got {t.numel()}")
+        _dev(t, torch.int32, name)
+
+
 def workspace_bytes(op: int, B: int, K: int = 1, V: int = 1, d: int = 1, h: int = 0, dt: int = BF16) -> int:
     return int(lib().spr_workspace_bytes(op, B, K, V, d, h, dt))
 
@@ -258,11 +271,10 @@ def replace_sample(target_logits, V: int, uniforms, ws: Workspace, rows=None, fi
     R = target_logits.numel() // ldv
     _dev(uniforms, torch.float32, "uniforms")
     n = uniforms.numel()
-    if rows is not None:
-        _dev(rows, torch.int32, "rows")
-    if first_reject is not None:
-        _dev(first_reject, torch.int32, "first_reject")
+    _selectors(rows, first_reject, n)
     tokens = torch.empty((n,), dtype=torch.int32, device=target_logits.device) if out is None else out
+    if tokens.numel() != n:
+        raise ValueError("tokens must have one entry per uniform")
     rc = lib().replace_sample(_ptr(target_logits), ldv, V, R, _ptr(rows), _ptr(first_reject), K,
                               seq_stride, n, _ptr(uniforms), _dt(target_logits), _ptr(tokens),
                               _ptr(ws.buf), ws.nbytes, _stream())
@@ -600,6 +612,7 @@ def replace_sample_static(target_logits, V: int, uniforms, tokens, rows=None, fi
     n = uniforms.numel()
     if tokens.numel() != n:
         raise ValueError("tokens must have one entry per uniform")
+    _selectors(rows, first_reject, n)
     rc = lib().replace_sample_static(_ptr(target_logits), ldv, V, R, _ptr(rows), _ptr(first_reject), K,
                                      seq_stride, n, _ptr(uniforms), _dt(target_logits), _ptr(tokens),
                                      _stream())

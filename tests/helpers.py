@@ -97,6 +97,58 @@ def enforce_margins(wl, thresholds=(0.5,), margin=MARGIN, seed=1234):
     return redraws
 
 
+def slice_seqs(wl, lo, hi):
+    """Sequences lo .. hi-1 of a workload as views: writes go through to the parent tensors."""
+    import dataclasses
+    kw = {}
+    for f in dataclasses.fields(wl):
+        v = getattr(wl, f.name)
+        if isinstance(v, torch.Tensor) and f.name not in ("W1", "b1", "W2", "b2"):
+            v = v[lo:hi]
+            assert v.is_contiguous()
+        kw[f.name] = v
+    kw["B"] = hi - lo
+    return type(wl)(**kw)
+
+
+def seq_parts(wl, threads=None):
+    """The batch cut into one contiguous run of sequences per host thread."""
+    import os
+    threads = max(1, min(threads or os.cpu_count() or 1, wl.B))
+    cuts = [i * wl.B // threads for i in range(threads + 1)]
+    return [slice_seqs(wl, lo, hi) for lo, hi in zip(cuts[:-1], cuts[1:]) if hi > lo]
+
+
+def map_parts(parts, fn):
+    """fn(index, part) for every part, one host thread each (the oracle's C calls release the
+    interpreter lock, so the parts run on separate cores)."""
+    from concurrent.futures import ThreadPoolExecutor
+    with ThreadPoolExecutor(len(parts)) as pool:
+        return list(pool.map(lambda a: fn(*a), enumerate(parts)))
+
+
+def enforce_margins_parallel(wl, thresholds=(0.5,), margin=MARGIN, seed=1234, threads=None):
+    """enforce_margins for full-size batches: the sequences are dealt to the host cores, every
+    part is cleared in place with its own redraw stream.  Returns the number of redraws."""
+    parts = seq_parts(wl, threads)
+    return sum(map_parts(parts, lambda i, part: enforce_margins(part, thresholds, margin, seed + i)))
+
+
+def oracle_step_parallel(wl, tau, threads=None):
+    """Every output of the path from the oracle, over all sequences of a host workload:
+    (sd_verify dict, scores, accept, first_reject, replacement tokens)."""
+    def one(_, part):
+        ref = oracle_sd(part)
+        s, a, fr = oracle_verify(part, tau)
+        P = to_np(part.p_logits).reshape(part.B * part.Kp, part.ldv)
+        t = oracle.replace_sample(P, part.V, to_np(part.u_replace), first_reject=fr, K=part.K,
+                                  seq_stride=part.Kp)
+        return ref, s, a, fr, t
+    res = map_parts(seq_parts(wl, threads), one)
+    ref = {k: np.concatenate([r[0][k] for r in res]) for k in res[0][0]}
+    return (ref,) + tuple(np.concatenate([r[j] for r in res]) for j in range(1, 5))
+
+
 def to_device(wl, device="cuda"):
     import dataclasses
     kw = {}

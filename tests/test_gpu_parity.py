@@ -6,8 +6,8 @@ import pytest
 import torch
 
 import oracle
-from helpers import (MARGIN, RTOL, assert_close_rel, enforce_margins, oracle_sd, oracle_verify,
-                     to_device, to_np)
+from helpers import (MARGIN, RTOL, assert_close_rel, enforce_margins, enforce_margins_parallel,
+                     oracle_sd, oracle_step_parallel, oracle_verify, to_device, to_np)
 
 pytestmark = pytest.mark.gpu
 
@@ -199,6 +199,59 @@ def test_sequential_1024_sampled(spr):
     out, fr, tokens = _sampled_rows_check(spr, wl, list(range(0, 1024, 64)) + [1023])
     rej = (fr.cpu().numpy() == 0).mean()
     assert 0.1 < rej < 0.3
+
+
+FULL_SIZE = [("llama3", 256, True), ("sequential", 256, True), ("sequential", 1024, False)]
+
+
+@pytest.mark.parametrize("name,B,bonus", FULL_SIZE, ids=["llama3", "sequential-256", "sequential-1024"])
+def test_full_size_parity_every_sequence(spr, name, B, bonus):
+    """The configurations the throughput is quoted on, at full size: inputs drawn on the device,
+    cleared of ties on the host with the oracle (all host cores), then EVERY accept bit, accepted
+    length, first-rejection index, correction token and replacement token compared with the
+    oracle, in the launch configuration the benchmark times (sd_verify on one stream, the fused
+    sprinter_step on another, separate workspaces)."""
+    tau = 0.5
+    wl = spr.workloads.make(name, "cuda", B=B, bonus_row=bonus)
+    wl_cpu = to_device(wl, "cpu")
+    redraws = enforce_margins_parallel(wl_cpu, thresholds=(tau,))
+    for k in ("hidden", "uniforms", "u_replace"):     # what the redraws may have touched
+        getattr(wl, k).copy_(getattr(wl_cpu, k))
+    # accept tests and scores are redrawn rarely (about 2e-4 per decision); draw uniforms often,
+    # since a token whose bin is narrower than two margins can never be selected
+    print(f"{name} B={B}: {redraws} redraws for {wl.B * wl.K} tokens, {2 * wl.B} draws")
+    assert redraws < 20 * wl.B
+    cfg = wl.cfg
+    ws1 = spr.Workspace.for_problem(wl.B, wl.K, wl.V, cfg.d, cfg.h, spr.BF16)
+    ws2 = spr.Workspace.for_problem(wl.B, wl.K, wl.V, cfg.d, cfg.h, spr.BF16)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s1):
+        out = spr.sd_verify(wl.p_logits, wl.q_logits, wl.V, wl.draft_tokens, wl.uniforms, ws1)
+    with torch.cuda.stream(s2):
+        scores, accept, fr, tokens = spr.sprinter_step(wl.hidden, wl.W1, wl.b1, wl.W2, wl.b2, tau,
+                                                       wl.p_logits, wl.V, wl.u_replace, ws2)
+    torch.cuda.synchronize()
+    assert ws1.device_status() == 0 and ws2.device_status() == 0
+    ref, s_ref, a_ref, fr_ref, t_ref = oracle_step_parallel(wl_cpu, tau)
+    eq(out["accept"], ref["accept"], "sd accept")
+    eq(out["accepted_len"], ref["accepted_len"], "sd accepted_len")
+    eq(out["correction_token"], ref["correction_token"], "sd correction_token")
+    assert_close_rel(out["p_tok"], ref["p_tok"], 1e-3, "p_tok")
+    assert_close_rel(out["q_tok"], ref["q_tok"], 1e-3, "q_tok")
+    assert_close_rel(out["residual_mass"], ref["residual_mass"], 1e-3, "residual_mass")
+    eq(accept, a_ref, "verifier accept")
+    eq(fr, fr_ref, "first_reject")
+    eq(tokens, t_ref, "replacement tokens")
+    assert_close_rel(scores, s_ref, 1e-3, "scores")
+    # the separate calls give the same bits as the fused one
+    s3, a3, fr3 = spr.sprinter_verify(wl.hidden, wl.W1, wl.b1, wl.W2, wl.b2, tau, ws2)
+    t3 = spr.replace_sample(wl.p_logits, wl.V, wl.u_replace, ws2, first_reject=fr3, K=wl.K, seq_stride=wl.Kp)
+    assert torch.equal(a3, accept) and torch.equal(fr3, fr) and torch.equal(t3, tokens)
+    if name == "sequential":
+        assert 0.1 < (fr_ref == 0).mean() < 0.3       # "roughly 20 % rejected"
+    else:
+        assert (ref["accepted_len"] < wl.K).mean() > 0.9 and (fr_ref < wl.K).any()
 
 
 # ---------------------------------------------------------------------------- edge cases

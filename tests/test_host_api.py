@@ -80,6 +80,27 @@ def test_binding_rejects_host_tensors():
         binding._dt(torch.zeros(4, dtype=torch.float16))
 
 
+def test_binding_checks_row_selectors_before_any_launch():
+    """rows / first_reject are read by the kernel as n 32-bit integers: int64 tensors (torch's
+    default integer type) and selectors shorter than the number of draws are refused."""
+    good = torch.zeros(5, dtype=torch.int32)
+    with pytest.raises(TypeError):
+        binding._selectors(torch.zeros(5, dtype=torch.int64), None, 5)
+    with pytest.raises(TypeError):
+        binding._selectors(None, torch.zeros(5, dtype=torch.int64), 5)
+    with pytest.raises(ValueError, match="one entry per draw"):
+        binding._selectors(torch.zeros(4, dtype=torch.int32), None, 5)
+    with pytest.raises(ValueError, match="one entry per draw"):
+        binding._selectors(None, torch.zeros(3, dtype=torch.int32), 5)
+    with pytest.raises(ValueError, match="CUDA"):      # right type and length, but a host tensor
+        binding._selectors(good, None, 5)
+    binding._selectors(None, None, 5)
+    # both wrappers go through the same check before they touch the library
+    import inspect
+    for fn in (binding.replace_sample, binding.replace_sample_static):
+        assert "_selectors(rows, first_reject, n)" in inspect.getsource(fn)
+
+
 def test_workloads_are_seeded_and_shaped():
     a = workloads.make("tiny", "cpu")
     b = workloads.make("tiny", "cpu")

@@ -266,6 +266,34 @@ def test_cdf_margin_by_hand():
     assert t == 1 and m == pytest.approx(0.05)
 
 
+def test_residual_draw_margin_by_hand():
+    """Eq. 1 worked by hand; every case fails if the p and q rows are swapped inside the margin
+    helper (the swapped residual lives on the other tokens)."""
+    # p - q = (0.3, -0.2, -0.1): the residual is all on token 0, whatever u
+    p, q = np.log(np.array([0.5, 0.3, 0.2])), np.log(np.array([0.2, 0.5, 0.3]))
+    for u in (0.0, 0.1, 0.5, 0.93):
+        m, t = oracle.residual_draw_margin(p, q, u)
+        assert t == 0 and m == pytest.approx(min(u, 1.0 - u), abs=1e-12)
+    # p - q = (-0.4, 0.1, 0.3, 0): residual (0, 1/4, 3/4, 0), bins [0, 1/4) and [1/4, 1)
+    p, q = np.log(np.array([0.1, 0.3, 0.4, 0.2])), np.log(np.array([0.5, 0.2, 0.1, 0.2]))
+    m, t = oracle.residual_draw_margin(p, q, 0.2)
+    assert t == 1 and m == pytest.approx(0.05, abs=1e-12)
+    m, t = oracle.residual_draw_margin(p, q, 0.3)
+    assert t == 2 and m == pytest.approx(0.05, abs=1e-12)
+    m, t = oracle.residual_draw_margin(p, q, 0.9)
+    assert t == 2 and m == pytest.approx(0.1, abs=1e-12)
+    # shifted logits (unnormalised rows) give the same draw
+    m, t = oracle.residual_draw_margin(p + 3.0, q - 2.0, 0.2)
+    assert t == 1 and m == pytest.approx(0.05, abs=1e-12)
+    # p = q: Eq. 1 is undefined, the draw comes from p itself (bins of p: 0.1, 0.4, 0.8, 1)
+    m, t = oracle.residual_draw_margin(p, p.copy(), 0.45)
+    assert t == 2 and m == pytest.approx(0.05, abs=1e-12)
+    # the token agrees with the correction token of the full check when the draft token is rejected
+    out = oracle.sd_verify(p[None, None], q[None, None], 4, np.array([[0]], np.int32),
+                           np.array([[0.9, 0.2]], np.float32))
+    assert out["accepted_len"][0] == 0 and out["correction_token"][0] == 1
+
+
 # ----------------------------------------------------------------------------- O3 SD verify
 
 
