@@ -124,8 +124,10 @@ int sprinter_verify(const void *hidden, const void *W1, const float *b1, const v
  * given and first_reject[i] >= K (the verifier kept every draft token, so the
  * target is not called).  Passing sprinter_verify's first_reject output here
  * chains the two calls on one stream with no host synchronisation.
- * uniforms [n] f32, tokens [n] int32.
- * Device-detected: row outside [0,R) -> tokens[i] = -1, SPR_ERR_BAD_ROW.
+ * uniforms [n] f32, tokens [n] int32.  With first_reject and without rows, seq_stride >= K
+ * (otherwise neighbouring sequences would share rows: SPR_ERR_INVALID_ARG).
+ * Device-detected: row outside [0,R), or first_reject[i] < 0 -> tokens[i] = -1,
+ * SPR_ERR_BAD_ROW.
  */
 int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, const int32_t *rows,
                    const int32_t *first_reject, int K, int seq_stride, int n, const float *uniforms,
@@ -352,11 +354,14 @@ int sd_verify_host(const void *p_logits, const void *q_logits, int64_t ldv, cons
  *
  * Limits: n <= SPR_STATIC_MAX_DRAWS and n * steps <= SPR_STATIC_MAX_DRAW_STEPS, where
  * steps = ceil((V + 7) / 1024) for bf16 and ceil((V + 3) / 512) for f32 (126 for
- * V = 128256 bf16, so up to 520 draws per call; 1024 draws up to V = 65536 bf16).  Larger requests return
+ * V = 128256 bf16, so up to 520 draws per call; 1024 draws up to V = 65529 bf16, 1008 draws at
+ * V = 65536, where steps = 65).  Larger requests return
  * SPR_ERR_WORKSPACE and launch nothing; split them or use replace_sample().
  *
- * First call on a device: looks up the device address of the array (the device must be
- * current).  Make that first call before starting any stream capture.
+ * The device that owns the tensors must be the current device of the calling thread: the
+ * scratch used is the current device's copy of the array.
+ * First call on a device: looks up the device address of the array.  Make that first call
+ * before starting any stream capture.
  * Sharing: every call on a GPU uses the same array.  Calls that can overlap on that GPU
  * (two streams, two host threads) race on it and give wrong tokens; issue them on one
  * stream or serialise them.  The array keeps the previous call's contents; the call clears

@@ -234,7 +234,8 @@ int oracle_replace_sample(const void *target_logits, int64_t ldv, int V, int64_t
         int64_t row = rows ? (int64_t)rows[i] : (int64_t)i * seq_stride;
         if (first_reject)
             row += first_reject[i];
-        if (row < 0 || row >= R) {
+        /* Algorithm 2's r counts accepted tokens: a negative first_reject selects no row */
+        if ((first_reject && first_reject[i] < 0) || row < 0 || row >= R) {
             tokens[i] = -1;
             rc = ORC_ERR_ROW;
             continue;

@@ -116,6 +116,8 @@ int check_replace_args(const DrawParams &dp, int n, int dt)
     if (n == 0) return SPR_OK;
     if (!dp.p || !dp.uniforms || !dp.tokens || dp.R == 0) return SPR_ERR_INVALID_ARG;
     if (dp.gate && dp.K <= 0) return SPR_ERR_INVALID_ARG;
+    // rows i*seq_stride + first_reject[i] of neighbouring sequences must not overlap
+    if (dp.gate && !dp.rows && n > 1 && dp.seq_stride < dp.K) return SPR_ERR_INVALID_ARG;
     if (!aligned(dp.p, elem_size(dt)) || !aligned(dp.uniforms, 4) || !aligned(dp.tokens, 4) ||
         (dp.rows && !aligned(dp.rows, 4)) || (dp.gate && !aligned(dp.gate, 4)))
         return SPR_ERR_INVALID_ARG;
@@ -143,10 +145,8 @@ DrawParams replace_params(const void *target_logits, int64_t ldv, int V, int64_t
     dp.K = K;
     dp.uniforms = uniforms;
     dp.tokens = tokens;
-    if (V > 0 && n >= 0 && dtype_ok(dt)) {
-        dp.steps = stat_steps_per_row(V, dt);
-        draw_geometry(n, dp.steps, &dp.chunks, &dp.iters);
-    }
+    dp.n = n;
+    if (V > 0 && dtype_ok(dt)) dp.steps = stat_steps_per_row(V, dt);
     return dp;
 }
 }  // namespace spr
@@ -156,11 +156,8 @@ namespace {
 // ticket counters of the verifier kernels: one per 64-token tile (MLP) or per sequence (linear)
 int verify_counters(int B, int K) { return max((B * K + 63) / 64, B); }
 
-size_t verify_ws_bytes(int B, int K, int h)
-{
-    const int M = B * K;
-    return verify_ws_layout(M, verifier_simt_slices(h), verify_counters(B, K)).end;
-}
+// number of partial sums per token any of the verifier kernels may write for this shape
+int verify_slices(int h) { return verifier_simt_slices(h); }
 
 }  // namespace
 
@@ -172,25 +169,31 @@ size_t spr_workspace_bytes(int op, int B, int K, int V, int d, int h, int dt)
     switch (op) {
     case SPR_OP_SPRINTER_VERIFY:
         if (K <= 0 || d <= 0 || h < 0 || (int64_t)B * K > 0x7fffffff) return 0;
-        return verify_ws_bytes(B, K, h);
+        return ws_bytes_of([&](Carver &c) { verify_ws_layout(c, B * K, verify_slices(h), verify_counters(B, K)); });
     case SPR_OP_REPLACE_SAMPLE:
         if (V <= 0) return 0;
-        return replace_ws_layout(B, stat_steps_per_row(V, dt)).end;
+        return ws_bytes_of([&](Carver &c) { draw_ws_layout(c, B, stat_steps_per_row(V, dt)); });
     case SPR_OP_SPRINTER_STEP:
         if (K <= 0 || d <= 0 || h < 0 || V <= 0 || (int64_t)B * K > 0x7fffffff) return 0;
-        return step_ws_layout(B, K, verifier_simt_slices(h), verify_counters(B, K), stat_steps_per_row(V, dt)).end;
+        return ws_bytes_of([&](Carver &c) {
+            step_ws_layout(c, B, K, verify_slices(h), verify_counters(B, K), stat_steps_per_row(V, dt));
+        });
     case SPR_OP_SD_VERIFY:
         if (K <= 0 || V <= 0 || (int64_t)B * K > 0x7fffffff) return 0;
-        return sd_ws_layout(B, K, stat_max_segments_per_row(V, dt), stat_steps_per_row(V, dt)).end;
+        return ws_bytes_of([&](Carver &c) {
+            sd_ws_layout(c, B, K, stat_max_segments_per_row(V, dt), stat_steps_per_row(V, dt));
+        });
     case SPR_OP_SD_SHARD:   // V = shard width; sized for a bonus row
         if (K <= 0 || V <= 0 || (int64_t)B * (K + 1) > 0x7fffffff) return 0;
-        return shard_ws_layout(B, K, K + 1, stat_max_segments_per_row(V, dt), stat_steps_per_row(V, dt)).end;
+        return ws_bytes_of([&](Carver &c) {
+            shard_ws_layout(c, B, K, K + 1, stat_max_segments_per_row(V, dt), stat_steps_per_row(V, dt));
+        });
     case SPR_OP_VERIFIER_LABELS:
         if (K <= 0 || V <= 0 || (int64_t)B * K > 0x7fffffff) return 0;
-        return label_ws_layout(B, K, stat_max_segments_per_row(V, dt)).end;
+        return ws_bytes_of([&](Carver &c) { label_ws_layout(c, B, K, stat_max_segments_per_row(V, dt)); });
     case SPR_OP_VERIFIER_TRAIN:
         if (d <= 0) return 0;
-        return train_ws_bytes(d);
+        return ws_bytes_of([&](Carver &c) { train_ws_layout(c, d); });
     default:
         return 0;
     }
@@ -211,17 +214,15 @@ int sprinter_verify(const void *hidden, const void *W1, const float *b1, const v
     VerifyParams vp = verify_params(hidden, W1, b1, W2, b2, threshold, B, K, d, h, scores, accept, first_reject);
     int rc = check_verify_args(vp, dt, path);
     if (rc != SPR_OK || B == 0) return rc;  // empty batch: nothing to read or write
-    const VerifyWs lay = verify_ws_layout(B * K, verifier_simt_slices(h), verify_counters(B, K));
-    if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
+    Carver cv = carve(ws_bytes);
+    const VerifyWs lay = verify_ws_layout(cv, B * K, verify_slices(h), verify_counters(B, K));
+    if (!ws || !aligned(ws, 256) || !cv.fits()) return SPR_ERR_WORKSPACE;
     if ((rc = check_device()) != SPR_OK) return rc;
 
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     vp.status = at<int>(ws, 0);
     vp.counter = at<int>(ws, lay.counter);
     vp.part_z = at<float>(ws, lay.part_z);
-    cudaError_t e = cudaMemsetAsync(vp.counter, 0, lay.counters_end - lay.counter, st);
-    if (e != cudaSuccess) return cuda_fail(e);
-    return launch_verifier(vp, dt, path, st);
+    return launch_verifier(vp, dt, path, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, const int32_t *rows,
@@ -232,16 +233,15 @@ int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, con
                                    tokens);
     int rc = check_replace_args(dp, n, dt);
     if (rc != SPR_OK || n == 0) return rc;  // no draws: pointers may be null
-    const DrawWs lay = replace_ws_layout(n, dp.steps);
-    if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
+    Carver cv = carve(ws_bytes);
+    const DrawWs lay = draw_ws_layout(cv, n, dp.steps);
+    if (!ws || !aligned(ws, 256) || !cv.fits()) return SPR_ERR_WORKSPACE;
     if ((rc = check_device()) != SPR_OK) return rc;
 
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     dp.status = at<int>(ws, 0);
     dp.counters = at<int>(ws, lay.counters);
     dp.part = at<float2>(ws, lay.part);
-    cudaError_t e = cudaMemsetAsync(dp.counters, 0, sizeof(int) * (size_t)n, st);
-    if (e == cudaSuccess) e = launch_draw(dp, n, dt, st);
+    const cudaError_t e = launch_draw(dp, dt, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? SPR_OK : cuda_fail(e);
 }
 
@@ -259,21 +259,20 @@ int sprinter_step(const void *hidden, const void *W1, const float *b1, const voi
                                    seq_stride, B, uniforms, dt, tokens);
     rc = check_replace_args(dp, B, dt);
     if (rc != SPR_OK || B == 0) return rc;
-    const StepWs lay = step_ws_layout(B, K, verifier_simt_slices(h), verify_counters(B, K), dp.steps);
-    if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
+    Carver cv = carve(ws_bytes);
+    const StepWs lay = step_ws_layout(cv, B, K, verify_slices(h), verify_counters(B, K), dp.steps);
+    if (!ws || !aligned(ws, 256) || !cv.fits()) return SPR_ERR_WORKSPACE;
     if ((rc = check_device()) != SPR_OK) return rc;
 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     vp.status = dp.status = at<int>(ws, 0);
-    vp.counter = at<int>(ws, lay.verify_counter);
-    vp.part_z = at<float>(ws, lay.part_z);
+    vp.counter = at<int>(ws, lay.verify.counter);
+    vp.part_z = at<float>(ws, lay.verify.part_z);
     dp.counters = at<int>(ws, lay.draw.counters);
     dp.part = at<float2>(ws, lay.draw.part);
-    // one clear for both kernels' tickets, then the draw is launched behind the verifier
-    cudaError_t e = cudaMemsetAsync(vp.counter, 0, lay.counters_end - lay.verify_counter, st);
-    if (e != cudaSuccess) return cuda_fail(e);
+    // the draw is launched behind the verifier
     if ((rc = launch_verifier(vp, dt, path, st)) != SPR_OK) return rc;
-    e = launch_draw(dp, B, dt, st, /*after_kernel=*/true);
+    const cudaError_t e = launch_draw(dp, dt, st, /*after_kernel=*/true);
     return e == cudaSuccess ? SPR_OK : cuda_fail(e);
 }
 
@@ -298,8 +297,9 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
     const int T = stat_steps_per_row(V, dt);
     int C, stat_iters;
     draw_geometry(B * K, T, &C, &stat_iters);   // same rule for the row-statistics pass, over B*K rows
-    const SdWs lay = sd_ws_layout(B, K, stat_max_segments_per_row(V, dt), T);
-    if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
+    Carver cv = carve(ws_bytes);
+    const SdWs lay = sd_ws_layout(cv, B, K, stat_max_segments_per_row(V, dt), T);
+    if (!ws || !aligned(ws, 256) || !cv.fits()) return SPR_ERR_WORKSPACE;
     int rc = check_device();
     if (rc != SPR_OK) return rc;
     if (B == 0) return SPR_OK;
@@ -325,7 +325,7 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
     sp.seq_counters = at<int>(ws, lay.seq_counters);
     sp.acc = at<uint8_t>(ws, lay.acc);
     sp.part = at<float4>(ws, lay.part);
-    sp.rowstats = at<float4>(ws, lay.rowstats);
+    sp.rowstats = at<double2>(ws, lay.rowstats);
 
     DrawParams dp;
     memset(&dp, 0, sizeof dp);
@@ -334,7 +334,7 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
     dp.q = q_logits;
     dp.ldv = ldv;
     dp.V = V;
-    draw_geometry(B, T, &dp.chunks, &dp.iters);
+    dp.n = B;
     dp.K = K;
     dp.Kp = Kp;
     dp.accepted_len = accepted_len;
@@ -348,9 +348,8 @@ int sd_verify(const void *p_logits, const void *q_logits, int64_t ldv, const int
     dp.part = at<float2>(ws, lay.draw.part);
 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    cudaError_t e = cudaMemsetAsync(sp.row_counters, 0, lay.counters_end - lay.row_counters, st);
-    if (e == cudaSuccess) e = launch_sd_row_stats(sp, B, K, dt, st);
-    if (e == cudaSuccess) e = launch_draw(dp, B, dt, st, /*after_kernel=*/true);
+    cudaError_t e = launch_sd_row_stats(sp, B, K, dt, st);
+    if (e == cudaSuccess) e = launch_draw(dp, dt, st, /*after_kernel=*/true);
     return e == cudaSuccess ? SPR_OK : cuda_fail(e);
 }
 

@@ -53,138 +53,162 @@ inline void draw_geometry(int n, int steps, int *segments, int *iters)
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // ---------------------------------------------------------------- workspace layouts
-// All offsets are multiples of 256 bytes from the start of the workspace.  Every layout
-// puts its ticket counters in one contiguous zone right after the header; the entry point
-// clears that zone on the stream before its first kernel, so a workspace may be shared by
-// calls of different ops and shapes.
-struct DrawWs {              // replace_sample, and the correction draw of sd_verify
-    size_t counters;         // int32 [n]      segments finished per draw
-    size_t part;             // float2 [n*T]   (max, weight) of every warp step
-    size_t end;
+// A workspace of ws_bytes bytes is cut at a point that depends on ws_bytes alone:
+//   [0, 256)                   header; word 0 is the sticky status
+//   [256, 256 + Z)             ticket zone, Z = ticket_zone_bytes(ws_bytes): int32 counters only
+//   [256 + Z, ws_bytes)        data zone: partial results, flags, everything else
+// The kernels of sprinter_verify, replace_sample, sprinter_step and sd_verify take tickets from
+// the ticket zone, and whoever takes the last ticket of a counter sets it back to zero
+// (take_ticket below).  The zone is zero after spr_workspace_init and no call ever writes
+// anything but tickets into it, so it is zero again whenever no call is in flight: these calls
+// need no clearing pass, whatever ops and shapes the workspace served before.  The remaining
+// ops keep their counters in the data zone and clear them on the stream at every call.
+__host__ __device__ inline size_t ticket_zone_bytes(size_t ws_bytes)
+{
+    return ws_bytes <= (size_t)kHeaderBytes ? 0 : (ws_bytes - kHeaderBytes) / 4 / 256 * 256;
+}
+__host__ __device__ inline size_t data_zone_start(size_t ws_bytes) { return kHeaderBytes + ticket_zone_bytes(ws_bytes); }
+// smallest workspace whose zones hold `tickets` bytes of counters and `data` bytes of the rest
+__host__ __device__ inline size_t ws_bytes_for(size_t tickets, size_t data)
+{
+    const size_t a = align_up(tickets, 256), b = align_up((align_up(data, 256) + 2) / 3, 256);
+    return kHeaderBytes + 4 * (a > b ? a : b);
+}
+
+// Cursor over the two zones.  Offsets are from the start of the workspace.
+struct Carver {
+    size_t tickets, data;        // next free byte of each zone
+    size_t tickets_end, data_end;
+    __host__ __device__ size_t take_tickets(size_t n)   // n int32 counters
+    {
+        const size_t o = tickets;
+        tickets += 4 * n;
+        return o;
+    }
+    __host__ __device__ size_t take_data(size_t bytes)  // 256-byte aligned block
+    {
+        const size_t o = data;
+        data = align_up(data + bytes, 256);
+        return o;
+    }
+    __host__ __device__ bool fits() const { return tickets <= tickets_end && data <= data_end; }
 };
-__host__ __device__ inline DrawWs draw_ws_layout(size_t counters, size_t scratch, int n, int T)
+__host__ __device__ inline Carver carve(size_t ws_bytes)
+{
+    Carver c;
+    c.tickets = kHeaderBytes;
+    c.tickets_end = c.data = data_zone_start(ws_bytes);
+    c.data_end = ws_bytes;
+    return c;
+}
+// workspace size a layout needs: carve an unbounded workspace, measure both zones
+template <typename F>
+inline size_t ws_bytes_of(F layout)
+{
+    Carver c;
+    c.tickets = c.data = 0;
+    c.tickets_end = c.data_end = ~(size_t)0;
+    layout(c);
+    return ws_bytes_for(c.tickets, c.data);
+}
+
+struct DrawWs {              // replace_sample, and the correction draw of sd_verify
+    size_t counters;         // int32 [n]      warp steps finished per draw (ticket zone)
+    size_t part;             // float2 [n*T]   (max, weight) of every warp step
+};
+__host__ __device__ inline DrawWs draw_ws_layout(Carver &c, int n, int T)
 {
     DrawWs w;
-    w.counters = counters;
-    w.part = align_up(scratch, 256);
-    w.end = align_up(w.part + 8 * (size_t)n * T, 256);
+    w.counters = c.take_tickets((size_t)n);
+    w.part = c.take_data(8 * (size_t)n * T);
     return w;
-}
-// replace_sample alone: counters [n] directly after the header
-__host__ __device__ inline DrawWs replace_ws_layout(int n, int T)
-{
-    return draw_ws_layout(kHeaderBytes, kHeaderBytes + align_up(sizeof(int32_t) * (size_t)n, 256), n, T);
 }
 
 struct SdWs {
-    size_t row_counters;     // int32 [M]      segments finished per row
-    size_t seq_counters;     // int32 [B]      rows finished per sequence
-    size_t counters_end;     // end of the zone cleared per call (includes the draw counters)
+    size_t row_counters;     // int32 [M]      segments finished per row (ticket zone)
+    size_t seq_counters;     // int32 [B]      rows finished per sequence (ticket zone)
     size_t acc;              // uint8 [M]      0 reject, 1 accept, 2 invalid token
     size_t part;             // float4 [M*S]   (max_p, sum_p, max_q, sum_q) per row segment
-    size_t rowstats;         // float4 [M]     (max_p, ln Z_p, max_q, ln Z_q)
+    size_t rowstats;         // double2 [M]    (max + ln Z) of the p row and of the q row
     DrawWs draw;             // correction draw, n = B
-    size_t end;
 };
-__host__ __device__ inline SdWs sd_ws_layout(int B, int K, int S, int T)   // S segments, T steps per row
+__host__ __device__ inline SdWs sd_ws_layout(Carver &c, int B, int K, int S, int T)   // S segments, T steps per row
 {
     const size_t M = (size_t)B * K;
     SdWs w;
-    w.row_counters = kHeaderBytes;
-    w.seq_counters = w.row_counters + 4 * M;
-    const size_t draw_counters = w.seq_counters + 4 * (size_t)B;
-    w.counters_end = align_up(draw_counters + 4 * (size_t)B, 256);
-    w.acc = w.counters_end;
-    w.part = align_up(w.acc + M, 256);
-    w.rowstats = align_up(w.part + 16 * M * S, 256);
-    w.draw = draw_ws_layout(draw_counters, align_up(w.rowstats + 16 * M, 256), B, T);
-    w.end = w.draw.end;
+    w.row_counters = c.take_tickets(M);
+    w.seq_counters = c.take_tickets((size_t)B);
+    w.acc = c.take_data(M);
+    w.part = c.take_data(16 * M * S);
+    w.rowstats = c.take_data(16 * M);
+    w.draw = draw_ws_layout(c, B, T);
     return w;
 }
 
 struct ShardWs {             // vocabulary-sharded sd_verify: the four passes share one workspace
-    size_t row_counters;     // int32 [B*Kp]
-    size_t draw_counters;    // int32 [B]
-    size_t counters_end;
+    size_t row_counters;     // int32 [B*Kp]   (data zone, cleared per call)
+    size_t draw_counters;    // int32 [B]      (data zone, cleared per call)
     size_t acc;              // uint8 [B*K]
     size_t part;             // float4 [B*Kp*S]
-    size_t rowstats;         // float4 [B*Kp]  whole-row (max_p, ln Z_p, max_q, ln Z_q)
+    size_t rowstats;         // double2 [B*Kp] whole-row (max + ln Z) of p and of q
     size_t draw_part;        // float2 [B*T]
-    size_t end;
 };
-__host__ __device__ inline ShardWs shard_ws_layout(int B, int K, int Kp, int S, int T)
+__host__ __device__ inline ShardWs shard_ws_layout(Carver &c, int B, int K, int Kp, int S, int T)
 {
     const size_t R = (size_t)B * Kp;
     ShardWs w;
-    w.row_counters = kHeaderBytes;
-    w.draw_counters = w.row_counters + 4 * R;
-    w.counters_end = align_up(w.draw_counters + 4 * (size_t)B, 256);
-    w.acc = w.counters_end;
-    w.part = align_up(w.acc + (size_t)B * K, 256);
-    w.rowstats = align_up(w.part + 16 * R * S, 256);
-    w.draw_part = align_up(w.rowstats + 16 * R, 256);
-    w.end = align_up(w.draw_part + 8 * (size_t)B * T, 256);
+    w.row_counters = c.take_data(4 * R);
+    w.draw_counters = c.take_data(4 * (size_t)B);
+    w.acc = c.take_data((size_t)B * K);
+    w.part = c.take_data(16 * R * S);
+    w.rowstats = c.take_data(16 * R);
+    w.draw_part = c.take_data(8 * (size_t)B * T);
     return w;
 }
 
 struct LabelWs {             // verifier_labels: row records of the statistics pass
-    size_t row_counters;     // int32 [M]
+    size_t row_counters;     // int32 [M]      (data zone, cleared per call)
     size_t part;             // float4 [M*S]
     size_t stats;            // float [M*6]
-    size_t end;
 };
-__host__ __device__ inline LabelWs label_ws_layout(int B, int K, int S)
+__host__ __device__ inline LabelWs label_ws_layout(Carver &c, int B, int K, int S)
 {
     const size_t M = (size_t)B * K;
     LabelWs w;
-    w.row_counters = kHeaderBytes;
-    w.part = align_up(w.row_counters + 4 * M, 256);
-    w.stats = align_up(w.part + 16 * M * S, 256);
-    w.end = align_up(w.stats + 24 * M, 256);
+    w.row_counters = c.take_data(4 * M);
+    w.part = c.take_data(16 * M * S);
+    w.stats = c.take_data(24 * M);
     return w;
 }
 
-// verifier_train_step: per-CTA gradient sums, float [kTrainMaxCtas, d + 2]
+// verifier_train_step: per-CTA gradient sums, float [kTrainMaxCtas, d + 2] (data zone)
 constexpr int kTrainMaxCtas = 592;   // 148 SMs x 4
-__host__ __device__ inline size_t train_ws_bytes(int d)
+__host__ __device__ inline size_t train_ws_layout(Carver &c, int d)
 {
-    return align_up(kHeaderBytes + 4 * (size_t)kTrainMaxCtas * ((size_t)d + 2), 256);
+    return c.take_data(4 * (size_t)kTrainMaxCtas * ((size_t)d + 2));
 }
 
 struct VerifyWs {
-    size_t counter;          // int32 [1 + max(row tiles, B)]   CTAs finished per tile / tokens per sequence
-    size_t counters_end;
-    size_t part_z;           // float [slices * M]      per-slice partial of W2 . relu(...)
-    size_t end;
+    size_t counter;          // int32 [1 + tickets]   (ticket zone) see verify_tickets()
+    size_t part_z;           // float [slices * M]    per-slice partial of W2 . relu(...)
 };
-__host__ __device__ inline VerifyWs verify_ws_layout(int M, int slices, int tiles)
+__host__ __device__ inline VerifyWs verify_ws_layout(Carver &c, int M, int slices, int tickets)
 {
     VerifyWs w;
-    w.counter = kHeaderBytes;
-    w.counters_end = align_up(w.counter + 4 * (size_t)(1 + tiles), 256);
-    w.part_z = w.counters_end;
-    w.end = align_up(w.part_z + 4 * (size_t)slices * M, 256);
+    w.counter = c.take_tickets(1 + (size_t)tickets);
+    w.part_z = c.take_data(4 * (size_t)slices * M);
     return w;
 }
 
 struct StepWs {              // sprinter_step: verifier and replacement draw in one call
-    size_t verify_counter;   // int32 [1 + row tiles]
-    size_t draw_counters;    // int32 [B]
-    size_t counters_end;
-    size_t part_z;           // float [slices * M]
+    VerifyWs verify;
     DrawWs draw;
-    size_t end;
 };
-__host__ __device__ inline StepWs step_ws_layout(int B, int K, int slices, int tiles, int T)
+__host__ __device__ inline StepWs step_ws_layout(Carver &c, int B, int K, int slices, int tickets, int T)
 {
-    const size_t M = (size_t)B * K;
     StepWs w;
-    w.verify_counter = kHeaderBytes;
-    w.draw_counters = w.verify_counter + 4 * (size_t)(1 + tiles);
-    w.counters_end = align_up(w.draw_counters + 4 * (size_t)B, 256);
-    w.part_z = w.counters_end;
-    w.draw = draw_ws_layout(w.draw_counters, align_up(w.part_z + 4 * (size_t)slices * M, 256), B, T);
-    w.end = w.draw.end;
+    w.verify = verify_ws_layout(c, B * K, slices, tickets);
+    w.draw = draw_ws_layout(c, B, T);
     return w;
 }
 
@@ -206,6 +230,17 @@ __device__ __forceinline__ float ex2(float x)
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+
+// One ticket of a counter that `total` parties take; true for whoever takes the last one, who
+// also sets the counter back to zero so that the next launch finds it clean.  The caller orders
+// its earlier global writes before the ticket (__threadfence) and its later reads after it.
+__device__ __forceinline__ bool take_ticket(int *counter, int total, int n = 1)
+{
+    const int old = atomicAdd(counter, n);
+    if (old + n != total) return false;
+    *reinterpret_cast<volatile int *>(counter) = 0;
+    return true;
 }
 
 // first error wins; the word stays set until the host clears it

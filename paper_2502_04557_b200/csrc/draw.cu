@@ -1,10 +1,35 @@
 // Inverse-CDF draws from softmax(l) (replacement token, bonus token) or from the residual
 // norm(max(0, p - q)) of Eq. 1 (correction token).  One read of the row(s); probabilities live
-// in registers only; per-step partial weights go to the last CTA that finishes a draw, which
-// finds the crossing step and re-reads just that step (2 KB) to pick the token.
+// in registers only.
+//
+// The unit of work is one warp step (2 KB of one row, 4 KB of a row pair).  Every CTA first
+// finds out which draws are live (a draw gated off by first_reject, or a sequence without a
+// correction token, costs nothing), then the live draws' steps, laid end to end, are cut into
+// equal contiguous runs, one per warp of a grid sized to the GPU: no CTA is launched for a dead
+// draw and every warp streams the same number of bytes, with the loads of its next steps in
+// flight while it works on the current one.  A warp writes one (max, weight) pair per step and
+// takes tickets on the draw for the steps it did; the warp that takes the last ticket adds the
+// step weights in step order, finds the step where the running sum crosses u * total and
+// re-reads just that step to pick the token.  Warps never wait for each other.
 #include "draw_common.cuh"
 
 namespace spr {
+
+namespace {
+
+constexpr int kMaxCompact = 4096;   // draws whose live list a CTA builds in shared memory
+// CTAs per SM: what the registers of the streaming loops (three steps of one row, or two steps
+// of a row pair, in flight per warp) leave room for
+constexpr int kDrawCtasSoftmax = 3, kDrawCtasResidual = 2;
+using WarpSmem = DrawSmemT<128>;    // per-warp scratch of a finishing warp
+
+// does draw i need any work?  (a negative first_reject is live: it is reported as a bad row)
+__device__ __forceinline__ bool draw_is_live(const DrawParams &prm, int i)
+{
+    if (prm.kind == DRAW_REPLACE) return !prm.gate || prm.gate[i] < prm.K;
+    const int nb = prm.accepted_len[i];
+    return nb >= 0 && (nb < prm.K || prm.Kp == prm.K + 1);
+}
 
 template <typename T>
 __device__ __forceinline__ Job<T> resolve_job(const DrawParams &prm, int i)
@@ -12,8 +37,8 @@ __device__ __forceinline__ Job<T> resolve_job(const DrawParams &prm, int i)
     Job<T> job;
     job.mode = MODE_NONE;
     job.p_row = job.q_row = nullptr;
-    job.cp = job.cq = 0.f;
-    // the uniform does not depend on the row choice: fetch it alongside the gate
+    job.cp = job.cq = job.dc = 0.f;
+    job.sp = job.sq = 1.f;
     job.u = prm.kind == DRAW_REPLACE ? prm.uniforms[i] : prm.uniforms[(int64_t)i * (prm.K + 1) + prm.K];
     const T *p = static_cast<const T *>(prm.p);
     if (prm.kind == DRAW_REPLACE) {
@@ -23,7 +48,7 @@ __device__ __forceinline__ Job<T> resolve_job(const DrawParams &prm, int i)
             if (off >= prm.K) return job;  // verifier kept every token: the target is not called
         }
         const int64_t row = (prm.rows ? (int64_t)prm.rows[i] : (int64_t)i * prm.seq_stride) + off;
-        if (row < 0 || row >= prm.R) {
+        if (off < 0 || row < 0 || row >= prm.R) {
             raise_status(prm.status, SPR_ERR_BAD_ROW);
             return job;
         }
@@ -33,70 +58,196 @@ __device__ __forceinline__ Job<T> resolve_job(const DrawParams &prm, int i)
         const int nb = prm.accepted_len[i];
         if (nb < 0) return job;  // invalid draft token in this sequence
         if (nb < prm.K) {
-            const float4 st = prm.rowstats[(int64_t)i * prm.K + nb];
             job.mode = MODE_RESIDUAL;
             job.p_row = p + ((int64_t)i * prm.Kp + nb) * prm.ldv;
             job.q_row = static_cast<const T *>(prm.q) + ((int64_t)i * prm.K + nb) * prm.ldv;
-            job.cp = (st.x + st.y) * kLog2e;
-            job.cq = (st.z + st.w) * kLog2e;
+            set_residual_scales(job, prm.rowstats[(int64_t)i * prm.K + nb]);
         } else if (prm.Kp == prm.K + 1) {
             job.mode = MODE_SOFTMAX;
             job.p_row = p + ((int64_t)i * prm.Kp + prm.K) * prm.ldv;
-        } else {
-            return job;
         }
     }
     return job;
 }
 
-// kSoftmaxOnly: replacement draws never take the residual branch; compiled without it the
-// kernel needs fewer registers and four CTAs fit an SM.
+// One warp: (max, weight) of steps [s0, s1) of the job's row(s) -> part[step]; the loads of
+// the following step(s) are issued before the current step is consumed.
 template <typename T, bool kSoftmaxOnly>
-__global__ void __launch_bounds__(kThreads, kSoftmaxOnly ? 4 : 3) draw_kernel(const DrawParams prm)
+__device__ __forceinline__ void warp_steps(const Job<T> &job, int mode, int V, int s0, int s1,
+                                           float2 *__restrict__ part)
 {
-    __shared__ DrawSmem sm;
-    const int C = prm.chunks;   // segments (CTAs) per row, of kWarps * prm.iters steps each
-    const int steps = prm.steps;
-    // correction draws go through the sequences last to first: the statistics pass has just
-    // streamed the rows in ascending order, so the highest ones are the ones still in L2
-    const int i = kSoftmaxOnly ? blockIdx.x / C : (int)(gridDim.x / C) - 1 - (int)(blockIdx.x / C);
-    const int c = blockIdx.x % C;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-
-    pdl_wait();   // the kernel before this one may still be writing first_reject / accepted_len
-    Job<T> job = resolve_job<T>(prm, i);
-    if (job.mode == MODE_NONE) {
-        if (c == 0 && tid == 0) {
-            prm.tokens[i] = -1;
-            if (prm.residual_mass) prm.residual_mass[i] = 0.f;
+    constexpr int N = Vec<T>::N;
+    constexpr int kStep = 32 * kUnroll * N;
+    const int lane = threadIdx.x & 31;
+    const int pad = row_pad(job.p_row);
+    if (kSoftmaxOnly || mode == MODE_SOFTMAX) {
+        // two steps in flight behind the one being summed
+        uint4 a[kUnroll], b[kUnroll], c[kUnroll];
+        load_step<T>(job.p_row, s0 * kStep - pad, V, lane, a);
+        if (s0 + 1 < s1) load_step<T>(job.p_row, (s0 + 1) * kStep - pad, V, lane, b);
+        for (int s = s0; s < s1; ++s) {
+            if (s + 2 < s1) load_step<T>(job.p_row, (s + 2) * kStep - pad, V, lane, c);
+            const MS v = softmax_step<T>(a);
+            if (lane == 0) part[s] = make_float2(v.m, v.s);
+#pragma unroll
+            for (int j = 0; j < kUnroll; ++j) {
+                a[j] = b[j];
+                b[j] = c[j];
+            }
         }
-        return;
+    } else {
+        uint4 rp[kUnroll], rq[kUnroll], np[kUnroll], nq[kUnroll];
+        load_step<T>(job.p_row, s0 * kStep - pad, V, lane, rp);
+        load_step_any<T>(job.q_row, s0 * kStep - pad, V, lane, rq);
+        for (int s = s0; s < s1; ++s) {
+            if (s + 1 < s1) {
+                load_step<T>(job.p_row, (s + 1) * kStep - pad, V, lane, np);
+                load_step_any<T>(job.q_row, (s + 1) * kStep - pad, V, lane, nq);
+            }
+            const float w = warp_sum(residual_step_sum<T>(rp, rq, job));
+            if (lane == 0) part[s] = make_float2(0.f, w);
+#pragma unroll
+            for (int j = 0; j < kUnroll; ++j) {
+                rp[j] = np[j];
+                rq[j] = nq[j];
+            }
+        }
     }
-    const int mode = kSoftmaxOnly ? (int)MODE_SOFTMAX : job.mode;
-    float2 *part = prm.part + (int64_t)i * steps;
-
-    segment_pass<T>(job, mode, prm.V, c, steps, prm.iters, part);
-    __syncthreads();
-    if (tid == 0) {
-        __threadfence();
-        sm.last = (atomicAdd(&prm.counters[i], 1) == C - 1);
-    }
-    __syncthreads();
-    if (!sm.last) return;
-    __threadfence();
-
-    const int token = finish_draw<T>(job, mode, prm.V, steps, prm.iters, part, sm,
-                                     prm.kind == DRAW_SD && prm.residual_mass ? prm.residual_mass + i : nullptr);
-    if (warp == 0 && lane == 0) prm.tokens[i] = token;
 }
 
-cudaError_t launch_draw(const DrawParams &dp, int n, int dt, cudaStream_t st, bool after_kernel)
+// One warp: softmax partials of every step of the row, one step at a time (the rare redo of a
+// residual draw whose weights vanished; kept small on purpose)
+template <typename T>
+__device__ __noinline__ void warp_softmax_row(const T *row, int V, int steps, float2 *part)
 {
-    const int64_t grid = (int64_t)n * dp.chunks;
-    if (grid > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    if (grid == 0) return cudaSuccess;
+    constexpr int kStep = 32 * kUnroll * Vec<T>::N;
+    const int lane = threadIdx.x & 31;
+    const int pad = row_pad(row);
+    for (int s = 0; s < steps; ++s) {
+        uint4 a[kUnroll];
+        load_step<T>(row, s * kStep - pad, V, lane, a);
+        const MS v = softmax_step<T>(a);
+        if (lane == 0) part[s] = make_float2(v.m, v.s);
+    }
+    __syncwarp();   // lane 0's partials are read by the other lanes next
+}
+
+// One warp, once every step partial of the draw is in part[0 .. steps): the token where the
+// running weight crosses u * total.  A residual draw whose weights vanish (Eq. 1 undefined) is
+// redone by this warp as a draw from p.  *residual_mass, if given, receives the total residual
+// weight (0 for softmax draws).
+template <typename T, bool kSoftmaxOnly>
+__device__ __noinline__ int warp_finish(const Job<T> &job, int mode, int V, int steps, float2 *part, WarpSmem &sm,
+                                        float *residual_mass)
+{
+    const int lane = threadIdx.x & 31;
+    steps_total(part, steps, sm);
+    if (lane == 0 && residual_mass) *residual_mass = mode == MODE_RESIDUAL ? (float)sm.total : 0.f;
+    if (!kSoftmaxOnly && mode == MODE_RESIDUAL && !(sm.total > 0.0)) {
+        mode = MODE_SOFTMAX;
+        warp_softmax_row<T>(job.p_row, V, steps, part);
+        steps_total(part, steps, sm);
+    }
+    steps_cross(part, steps, (double)job.u * sm.total, sm);
+    return sm.step >= 0 ? step_locate<T>(job, mode, V, sm.step, sm.t_in, sm.ref) : -1;
+}
+
+// kSoftmaxOnly: replacement draws never take the residual branch; compiled without it the
+// kernel needs fewer registers.
+template <typename T, bool kSoftmaxOnly>
+__global__ void __launch_bounds__(kThreads, kSoftmaxOnly ? kDrawCtasSoftmax : kDrawCtasResidual)
+draw_kernel(const DrawParams prm)
+{
+    __shared__ unsigned short s_live[kMaxCompact];
+    __shared__ int s_count[kWarps];
+    __shared__ WarpSmem s_fin[kWarps];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n = prm.n, steps = prm.steps;
+
+    pdl_wait();   // the kernel before this one may still be writing first_reject / accepted_len
+
+    // ---- which draws are live?  Every CTA builds the same list (ascending draw index).
+    const bool compact = n <= kMaxCompact;
+    int nlive = n;
+    if (compact) {
+        nlive = 0;
+        for (int base = 0; base < n; base += kThreads) {
+            const int i = base + tid;
+            const bool live = i < n && draw_is_live(prm, i);
+            if (i < n && !live && blockIdx.x == 0) {
+                prm.tokens[i] = -1;
+                if (prm.residual_mass) prm.residual_mass[i] = 0.f;
+            }
+            const unsigned mask = __ballot_sync(0xffffffffu, live);
+            if (lane == 0) s_count[warp] = __popc(mask);
+            __syncthreads();
+            int before = nlive, all = nlive;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                if (w < warp) before += s_count[w];
+                all += s_count[w];
+            }
+            if (live) s_live[before + __popc(mask & ((1u << lane) - 1u))] = (unsigned short)i;
+            nlive = all;
+            __syncthreads();
+        }
+    }
+
+    // ---- this warp's run of the live draws' steps
+    const int64_t total = (int64_t)nlive * steps;
+    const int64_t warps = (int64_t)gridDim.x * kWarps, gw = (int64_t)blockIdx.x * kWarps + warp;
+    int64_t u = total / warps * gw + min(gw, total % warps);          // runs differ by one step at most
+    const int64_t u_end = u + total / warps + (gw < total % warps ? 1 : 0);
+    while (u < u_end) {
+        int64_t j = u / steps;
+        const int s0 = (int)(u - j * steps);
+        const int s1 = (int)min((int64_t)steps, s0 + (u_end - u));
+        u += s1 - s0;
+        // correction draws go through the sequences last to first: the statistics pass has just
+        // streamed the rows in ascending order, so the highest ones are the ones still in L2
+        if (!kSoftmaxOnly) j = nlive - 1 - j;
+        const int i = compact ? (int)s_live[j] : (int)j;
+        const Job<T> job = resolve_job<T>(prm, i);
+        if (job.mode == MODE_NONE) {   // gated off (when no list was built), or a bad row
+            if (s0 == 0 && lane == 0) {
+                prm.tokens[i] = -1;
+                if (prm.residual_mass) prm.residual_mass[i] = 0.f;
+            }
+            continue;
+        }
+        const int mode = kSoftmaxOnly ? (int)MODE_SOFTMAX : job.mode;
+        float2 *part = prm.part + (int64_t)i * steps;
+        warp_steps<T, kSoftmaxOnly>(job, mode, prm.V, s0, s1, part);
+        int last = 0;
+        if (lane == 0) {
+            __threadfence();
+            last = take_ticket(&prm.counters[i], steps, s1 - s0);
+        }
+        if (!__shfl_sync(0xffffffffu, last, 0)) continue;
+        __threadfence();
+        const int token = warp_finish<T, kSoftmaxOnly>(job, mode, prm.V, steps, part, s_fin[warp],
+                                                       prm.kind == DRAW_SD && prm.residual_mass
+                                                           ? prm.residual_mass + i : nullptr);
+        if (lane == 0) prm.tokens[i] = token;
+    }
+}
+
+}  // namespace
+
+// CTAs of a launch: enough warps for one step each, at most what the GPU holds at once
+int draw_grid(int n, int steps, bool softmax_only)
+{
+    const int64_t units = (int64_t)n * steps;
+    const int64_t resident = 148 * (softmax_only ? kDrawCtasSoftmax : kDrawCtasResidual);
+    const int64_t ctas = (units + kWarps - 1) / kWarps;
+    return (int)(ctas < resident ? ctas : resident);
+}
+
+cudaError_t launch_draw(const DrawParams &dp, int dt, cudaStream_t st, bool after_kernel)
+{
+    if (dp.n == 0) return cudaSuccess;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)grid);
+    cfg.gridDim = dim3((unsigned)draw_grid(dp.n, dp.steps, dp.kind == DRAW_REPLACE));
     cfg.blockDim = dim3(kThreads);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];

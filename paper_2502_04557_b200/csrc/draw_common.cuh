@@ -15,28 +15,62 @@ struct Job {
     int mode;
     const T *p_row;
     const T *q_row;
-    float cp, cq;  // residual: (max + ln Z) * log2(e) of the p row and of the q row
+    float cp, cq;  // residual: (max + ln Z) * log2(e) of the p row and of the q row, rounded
+    float sp, sq;  // residual: 2^-(what the rounding of cp, cq dropped), factors next to 1
+    float dc;      // residual: cq - cp, formed in double precision before rounding
     float u;
 };
 
-// residual weights max(0, p_i - q_i) of one vector (probabilities, already normalised)
+// Normalisers of both rows of a residual draw from the row statistics st = (max + ln Z of the p
+// row, the same of the q row).  A probability is 2^(l * log2(e) - c) with c = (max + ln Z) *
+// log2(e) of order 10..30: rounded to float c is off by up to 1e-6, a common factor on every
+// probability of the row that would show in the residual mass; the factor is kept beside it.
 template <typename T>
-__device__ __forceinline__ void residual_weights(const uint4 &vp, const uint4 &vq, float cp, float cq,
+__device__ __forceinline__ void set_residual_scales(Job<T> &job, const double2 &st)
+{
+    constexpr double kL = 1.4426950408889634;
+    const double cp = st.x * kL, cq = st.y * kL;
+    job.cp = (float)cp;
+    job.cq = (float)cq;
+    job.sp = (float)exp2((double)job.cp - cp);
+    job.sq = (float)exp2((double)job.cq - cq);
+    job.dc = (float)(cq - cp);
+}
+
+// Residual weights max(0, p_i - q_i) of one vector (probabilities, already normalised).
+// Where p_i and q_i nearly agree the difference of two rounded exponentials would be mostly
+// rounding noise (or exactly zero), so there it is formed as q_i * (2^D - 1) with
+// D = log2(p_i / q_i) = (lp_i - lq_i) * log2(e) + (cq - cp): the logit difference is exact and the
+// normaliser difference comes from double precision, so D keeps its relative accuracy however
+// small it is, and 2^D - 1 is a short series.  From ratio 2^(1/4) on the plain difference is used.
+template <typename T>
+__device__ __forceinline__ void residual_weights(const uint4 &vp, const uint4 &vq, const Job<T> &job,
                                                  float (&w)[Vec<T>::N])
 {
     constexpr int N = Vec<T>::N;
+    constexpr float kLn2 = 0.6931471805599453f;
     float fp[N], fq[N];
     Vec<T>::unpack(vp, fp);
     Vec<T>::unpack(vq, fq);
 #pragma unroll
-    for (int e = 0; e < N; ++e)
-        w[e] = fmaxf(0.f, ex2(fmaf(fp[e], kLog2e, -cp)) - ex2(fmaf(fq[e], kLog2e, -cq)));
+    for (int e = 0; e < N; ++e) {
+        const float qv = ex2(fmaf(fq[e], kLog2e, -job.cq)) * job.sq;
+        const float direct = fmaf(ex2(fmaf(fp[e], kLog2e, -job.cp)), job.sp, -qv);
+        const float D = fmaf(fp[e] - fq[e], kLog2e, job.dc);   // NaN where both logits are -inf
+        const float x = D * kLn2;
+        // e^x - 1 for 0 < x < ln(2)/4: relative error below x^5/720 < 3e-7
+        const float em1 = x * fmaf(x, fmaf(x, fmaf(x, fmaf(x, 1.f / 120.f, 1.f / 24.f), 1.f / 6.f), 0.5f), 1.f);
+        const float r = D < 0.25f ? qv * em1 : direct;
+        w[e] = D > 0.f ? r : 0.f;
+    }
 }
 
-constexpr int kCachedSteps = 512;   // step weights the last CTA of a draw keeps in shared memory
-
-struct DrawSmem {
-    double weight[kCachedSteps];   // weight of each step, relative to the row maximum
+// Scratch of whoever finishes a draw (a CTA in the sharded kernels, one warp in draw_kernel);
+// CACHED = how many step weights it keeps in shared memory between the two passes over them.
+template <int CACHED>
+struct DrawSmemT {
+    static constexpr int kCached = CACHED;
+    double weight[CACHED];         // weight of each step, relative to the row maximum
     double base;                   // weight before the crossing step
     double t_in;
     double total;
@@ -46,6 +80,7 @@ struct DrawSmem {
     int token;
     int last;
 };
+using DrawSmem = DrawSmemT<512>;
 
 // inclusive prefix sum over the lanes of a warp, in lane order
 __device__ __forceinline__ double warp_scan_f64(double v, int lane)
@@ -75,14 +110,14 @@ __device__ __forceinline__ void load_step_any(const T *__restrict__ row, int fir
 // lane-local sum of the residual weights of one warp step
 template <typename T>
 __device__ __forceinline__ float residual_step_sum(const uint4 (&rp)[kUnroll], const uint4 (&rq)[kUnroll],
-                                                   float cp, float cq)
+                                                   const Job<T> &job)
 {
     constexpr int N = Vec<T>::N;
     float acc[kUnroll];
 #pragma unroll
     for (int j = 0; j < kUnroll; ++j) {
         float w[N];
-        residual_weights<T>(rp[j], rq[j], cp, cq, w);
+        residual_weights<T>(rp[j], rq[j], job, w);
         acc[j] = 0.f;
 #pragma unroll
         for (int e = 0; e < N; ++e) acc[j] += w[e];
@@ -133,7 +168,7 @@ __device__ __forceinline__ void segment_pass(const Job<T> &job, int mode, int V,
             v = softmax_step<T>(cur);
         } else {
             v.m = 0.f;
-            v.s = warp_sum(residual_step_sum<T>(rp, rq, job.cp, job.cq));
+            v.s = warp_sum(residual_step_sum<T>(rp, rq, job));
             if (more) {
                 load_step<T>(job.p_row, first + nxt, V, lane, rp);
                 load_step_any<T>(job.q_row, first + nxt, V, lane, rq);
@@ -170,7 +205,7 @@ __device__ int step_locate(const Job<T> &job, int mode, int V, int step, double 
 #pragma unroll
             for (int e = 0; e < N; ++e) w[e] = ex2(fmaf(f[e], kLog2e, off));
         } else {
-            residual_weights<T>(rp[j], rq[j], job.cp, job.cq, w);
+            residual_weights<T>(rp[j], rq[j], job, w);
         }
         const int e0 = f0 + (j * 32 + lane) * N;
         double ts = 0.0;
@@ -205,23 +240,34 @@ __device__ int step_locate(const Job<T> &job, int mode, int V, int step, double 
     return tok >= 0 ? tok : lastpos;
 }
 
-// Warp 0, once every step partial of a draw is in part[0 .. steps): adds the step weights in
-// step order (fp64, relative to the largest step maximum) -> sm.total, sm.row_max; the first
-// kCachedSteps weights stay in sm.weight for steps_cross.
-__device__ __forceinline__ void steps_total(const float2 *part, int steps, DrawSmem &sm)
+// weight of a step relative to the row maximum M: its own sum, rescaled from its own maximum
+__device__ __forceinline__ double step_weight(float2 ms, float M)
+{
+    return ms.y > 0.f ? (double)(ms.y * ex2((ms.x - M) * kLog2e)) : 0.0;
+}
+
+// One warp, once every step partial of a draw is in part[0 .. steps): adds the step weights in
+// step order (fp64 sums of fp32 weights relative to the largest step maximum) -> sm.total,
+// sm.row_max; the first CACHED weights stay in sm.weight for steps_cross.
+template <int CACHED>
+__device__ __forceinline__ void steps_total(const float2 *part, int steps, DrawSmemT<CACHED> &sm)
 {
     const int lane = threadIdx.x & 31;
+    float2 *raw = reinterpret_cast<float2 *>(sm.weight);   // one trip to L2: the pairs wait here
     float M = neg_inf();
-    for (int t = lane; t < steps; t += 32) M = fmaxf(M, __ldcg(&part[t]).x);
+    for (int t = lane; t < steps; t += 32) {
+        const float2 ms = __ldcg(&part[t]);
+        if (t < CACHED) raw[t] = ms;
+        M = fmaxf(M, ms.x);
+    }
     M = warp_max(M);
     double carry = 0.0;
     for (int t0 = 0; t0 < steps; t0 += 32) {
         const int t = t0 + lane;
         double S = 0.0;
         if (t < steps) {
-            const float2 ms = __ldcg(&part[t]);
-            if (ms.y > 0.f) S = (double)ms.y * exp((double)ms.x - (double)M);
-            if (t < kCachedSteps) sm.weight[t] = S;
+            S = step_weight(t < CACHED ? raw[t] : __ldcg(&part[t]), M);
+            if (t < CACHED) sm.weight[t] = S;   // same lane, same slot: the pair is no longer needed
         }
         carry += __shfl_sync(0xffffffffu, warp_scan_f64(S, lane), 31);
     }
@@ -236,7 +282,8 @@ __device__ __forceinline__ void steps_total(const float2 *part, int steps, DrawS
 // scale as sm.total) -> sm.step, with sm.t_in = what is left of the target inside that step,
 // relative to that step's own maximum sm.ref.  If rounding (or u >= 1) leaves no crossing:
 // the last step with positive weight and an infinite t_in; sm.step = -1 if there is none.
-__device__ __forceinline__ void steps_cross(const float2 *part, int steps, double target, DrawSmem &sm)
+template <int CACHED>
+__device__ __forceinline__ void steps_cross(const float2 *part, int steps, double target, DrawSmemT<CACHED> &sm)
 {
     const int lane = threadIdx.x & 31;
     const float M = sm.row_max;
@@ -246,11 +293,10 @@ __device__ __forceinline__ void steps_cross(const float2 *part, int steps, doubl
         const int t = t0 + lane;
         double S = 0.0;
         if (t < steps) {
-            if (t < kCachedSteps) {
+            if (t < CACHED) {
                 S = sm.weight[t];
             } else {
-                const float2 ms = __ldcg(&part[t]);
-                if (ms.y > 0.f) S = (double)ms.y * exp((double)ms.x - (double)M);
+                S = step_weight(__ldcg(&part[t]), M);
             }
         }
         const double incl = carry + warp_scan_f64(S, lane);

@@ -177,6 +177,7 @@ int replace_sample_host(const void *target_logits, int64_t ldv, int V, int64_t R
     if (n == 0) return SPR_OK;
     if (!target_logits || !uniforms || !tokens || R == 0 || (first_reject && K <= 0))
         return SPR_ERR_INVALID_ARG;
+    if (first_reject && !rows && n > 1 && seq_stride < K) return SPR_ERR_INVALID_ARG;
     if (!arena || arena_bytes < spr_host_arena_bytes(SPR_OP_REPLACE_SAMPLE, n, 0, 0, ldv, 0, 0, dt))
         return SPR_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -190,7 +191,7 @@ int replace_sample_host(const void *target_logits, int64_t ldv, int V, int64_t R
         if (first_reject && first_reject[i] >= K) continue;
         const int64_t row = (rows ? (int64_t)rows[i] : (int64_t)i * seq_stride) +
                             (first_reject ? first_reject[i] : 0);
-        if (row < 0 || row >= R) {
+        if ((first_reject && first_reject[i] < 0) || row < 0 || row >= R) {
             bad_row = 1;
             continue;
         }

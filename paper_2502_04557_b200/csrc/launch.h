@@ -24,7 +24,7 @@ struct SdParams {
     int *seq_counters;  // [B]
     uint8_t *acc;       // [B*K]
     float4 *part;       // [B*K*chunks]
-    float4 *rowstats;   // [B*K]
+    double2 *rowstats;  // [B*K] (max + ln Z) of the p row and of the q row
 };
 
 enum { DRAW_REPLACE = 0, DRAW_SD = 1 };
@@ -34,8 +34,8 @@ struct DrawParams {
     const void *p;
     const void *q;
     int64_t ldv;
-    int V, chunks, steps;   // segments (CTAs) and warp steps per row
-    int iters;              // warp steps each warp of a CTA takes (1, 2 or 4)
+    int V, steps;           // warp steps per row
+    int n;                  // draws
     // replace_sample
     int64_t R;
     const int32_t *rows;
@@ -44,13 +44,13 @@ struct DrawParams {
     // sd_verify correction draw (K also bounds the gate of replace_sample)
     int K, Kp;
     const int32_t *accepted_len;
-    const float4 *rowstats;
+    const double2 *rowstats;
     const float *uniforms;
     int32_t *tokens;
     float *residual_mass;
     // workspace
     int *status;
-    int *counters;   // [n]
+    int *counters;   // [n] warp steps finished per draw; zero before and after the launch
     float2 *part;    // [n*steps] (max, weight) of every warp step
 };
 
@@ -78,7 +78,7 @@ struct ShardDecideParams {
     float *p_tok, *q_tok;         // [B,K] or null
     int *status;
     uint8_t *acc;                 // [B*K]
-    float4 *rowstats;             // [B*Kp] (max_p, ln Z_p, max_q, ln Z_q) of the whole rows
+    double2 *rowstats;            // [B*Kp] (max + ln Z) of the whole p row and q row
 };
 
 struct ShardDrawParams {
@@ -89,7 +89,7 @@ struct ShardDrawParams {
     int G, rank;
     const int32_t *accepted_len;
     const float *uniforms;
-    const float4 *rowstats;
+    const double2 *rowstats;
     double2 *weights;             // [B] this shard's (max, weight); weights pass only
     const double2 *all_weights;   // [G, B]; draw pass only
     const float *all_stats;       // [G, B*Kp, 6]; draw pass only
@@ -142,7 +142,7 @@ DrawParams replace_params(const void *target_logits, int64_t ldv, int V, int64_t
                           int dt, int32_t *tokens);
 // after_kernel: the launch directly follows, in the same stream, the kernel whose output
 // selects the rows (programmatic dependent launch)
-cudaError_t launch_draw(const DrawParams &dp, int n, int dt, cudaStream_t st, bool after_kernel = false);
+cudaError_t launch_draw(const DrawParams &dp, int dt, cudaStream_t st, bool after_kernel = false);
 
 // SIMT verifier: any dtype and shape.  `slices` must equal verifier_simt_slices(h).
 int verifier_simt_slices(int h);

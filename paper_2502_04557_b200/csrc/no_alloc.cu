@@ -2,6 +2,8 @@
 // a fixed array that is part of the library image on every GPU that loads it.
 #include <string.h>
 
+#include <atomic>
+
 #include "common.cuh"
 #include "launch.h"
 
@@ -23,8 +25,10 @@ static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
 // Device address of g_static_scratch per device ordinal.  In host code the array's name is
 // only a handle for the runtime, never something a kernel may dereference; the address a
 // kernel needs comes from cudaGetSymbolAddress, asked once per device while it is current.
+// Host threads that make their first call on a device at the same time all look the address
+// up and store the same value; the atomic only keeps that free of a data race.
 constexpr int kMaxDevices = 64;
-void *g_scratch_addr[kMaxDevices];
+std::atomic<void *> g_scratch_addr[kMaxDevices];
 
 int scratch_for_current_device(void **out)
 {
@@ -32,14 +36,14 @@ int scratch_for_current_device(void **out)
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return report_cuda_error(e);
     if (dev < 0 || dev >= kMaxDevices) return SPR_ERR_UNSUPPORTED;
-    if (!g_scratch_addr[dev]) {
-        void *ptr = nullptr;
+    void *ptr = g_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!ptr) {
         e = cudaGetSymbolAddress(&ptr, g_static_scratch);
         if (e != cudaSuccess) return report_cuda_error(e);
         if (!ptr) return SPR_ERR_CUDA;
-        g_scratch_addr[dev] = ptr;
+        g_scratch_addr[dev].store(ptr, std::memory_order_release);
     }
-    *out = g_scratch_addr[dev];
+    *out = ptr;
     return SPR_OK;
 }
 
@@ -55,6 +59,7 @@ extern "C" int replace_sample_static(const void *target_logits, int64_t ldv, int
     if (n == 0) return SPR_OK;
     if (!target_logits || !uniforms || !tokens || R == 0) return SPR_ERR_INVALID_ARG;
     if (first_reject && K <= 0) return SPR_ERR_INVALID_ARG;
+    if (first_reject && !rows && n > 1 && seq_stride < K) return SPR_ERR_INVALID_ARG;
     const size_t es = elem_size(dt);
     if (reinterpret_cast<uintptr_t>(target_logits) % es || reinterpret_cast<uintptr_t>(uniforms) % 4 ||
         reinterpret_cast<uintptr_t>(tokens) % 4 || (rows && reinterpret_cast<uintptr_t>(rows) % 4) ||
@@ -83,6 +88,6 @@ extern "C" int replace_sample_static(const void *target_logits, int64_t ldv, int
     // partials are always written before they are read, and the status word is not reported).
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     e = cudaMemsetAsync(dp.counters, 0, sizeof(int32_t) * (size_t)n, st);
-    if (e == cudaSuccess) e = launch_draw(dp, n, dt, st);
+    if (e == cudaSuccess) e = launch_draw(dp, dt, st);
     return e == cudaSuccess ? SPR_OK : report_cuda_error(e);
 }

@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(kThreads, 4) sd_row_stats_kernel(const SdParam
     if (lane == 0) {
         prm.part[row * C + c] = make_float4(mp.m, mp.s, mq.m, mq.s);
         __threadfence();
-        s_last = (atomicAdd(&prm.row_counters[row], 1) == C - 1);
+        s_last = take_ticket(&prm.row_counters[row], C);
     }
     __syncwarp();
     if (!s_last) return;
@@ -127,9 +127,9 @@ __global__ void __launch_bounds__(kThreads, 4) sd_row_stats_kernel(const SdParam
         if (prm.accept) prm.accept[row] = acc == 1 ? 1 : 0;
         if (prm.p_tok) prm.p_tok[row] = P;
         if (prm.q_tok) prm.q_tok[row] = Q;
-        prm.rowstats[row] = make_float4(m_p, (float)lnz_p, m_q, (float)lnz_q);
+        prm.rowstats[row] = make_double2((double)m_p + lnz_p, (double)m_q + lnz_q);
         __threadfence();
-        last_row = (atomicAdd(&prm.seq_counters[b], 1) == prm.K - 1);
+        last_row = take_ticket(&prm.seq_counters[b], prm.K);
     }
     last_row = __shfl_sync(0xffffffffu, last_row, 0);
     if (!last_row) return;

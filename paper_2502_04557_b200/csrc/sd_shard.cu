@@ -186,7 +186,7 @@ __device__ __forceinline__ void decide_sequence(const ShardDecideParams &prm, in
         double lnz_p, lnz_q = 0.0;
         merge_shards(prm.all_stats, rows, prm.G, row, 0, m_p, lnz_p);
         if (k < prm.K) merge_shards(prm.all_stats, rows, prm.G, row, 2, m_q, lnz_q);
-        prm.rowstats[row] = make_float4(m_p, (float)lnz_p, m_q, (float)lnz_q);
+        prm.rowstats[row] = make_double2((double)m_p + lnz_p, (double)m_q + lnz_q);
         if (k >= prm.K) continue;
         const int64_t tok = (int64_t)b * prm.K + k;
         const int x = prm.draft_tokens[tok];
@@ -255,17 +255,17 @@ __device__ __forceinline__ Job<T> shard_job(const ShardDrawParams &prm, int b)
     Job<T> job;
     job.mode = MODE_NONE;
     job.p_row = job.q_row = nullptr;
-    job.cp = job.cq = 0.f;
+    job.cp = job.cq = job.dc = 0.f;
+    job.sp = job.sq = 1.f;
     job.u = prm.uniforms[(int64_t)b * (prm.K + 1) + prm.K];
     const int nb = prm.accepted_len[b];
     const T *p = static_cast<const T *>(prm.p);
     if (nb >= 0 && nb < prm.K) {
-        const float4 rs = prm.rowstats[(int64_t)b * prm.Kp + nb];
+        const double2 rs = prm.rowstats[(int64_t)b * prm.Kp + nb];
         job.mode = MODE_RESIDUAL;
         job.p_row = p + ((int64_t)b * prm.Kp + nb) * prm.ldv;
         job.q_row = static_cast<const T *>(prm.q) + ((int64_t)b * prm.K + nb) * prm.ldv;
-        job.cp = (rs.x + rs.y) * kLog2e;
-        job.cq = (rs.z + rs.w) * kLog2e;
+        set_residual_scales(job, rs);
     } else if (nb == prm.K && prm.Kp == prm.K + 1) {
         job.mode = MODE_SOFTMAX;
         job.p_row = p + ((int64_t)b * prm.Kp + prm.K) * prm.ldv;

@@ -25,15 +25,16 @@ int check_sizes(int B, int K, int Kp, int Vs, int64_t ldv, int dt)
     return B == 0 ? SPR_OK : kProceed;
 }
 
-ShardWs layout(int B, int K, int Kp, int Vs, int dt)
+// the layout inside a workspace of ws_bytes bytes; *fits tells whether it has room
+ShardWs layout(int B, int K, int Kp, int Vs, int dt, size_t ws_bytes, bool *fits)
 {
-    return shard_ws_layout(B, K, Kp, stat_max_segments_per_row(Vs, dt), stat_steps_per_row(Vs, dt));
+    Carver cv = carve(ws_bytes);
+    const ShardWs lay = shard_ws_layout(cv, B, K, Kp, stat_max_segments_per_row(Vs, dt), stat_steps_per_row(Vs, dt));
+    *fits = cv.fits();
+    return lay;
 }
 
-bool ws_ok(const void *ws, size_t ws_bytes, const ShardWs &lay)
-{
-    return ws && aligned(ws, 256) && ws_bytes >= lay.end;
-}
+bool ws_ok(const void *ws, bool fits) { return ws && aligned(ws, 256) && fits; }
 
 }  // namespace
 
@@ -49,8 +50,9 @@ int sd_shard_stats(const void *p_shard, const void *q_shard, int64_t ldv, int Vs
     const size_t es = elem_size(dt);
     if (!aligned(p_shard, es) || !aligned(q_shard, es) || !aligned(draft_tokens, 4) || !aligned(stats, 4))
         return SPR_ERR_INVALID_ARG;
-    const ShardWs lay = layout(B, K, Kp, Vs, dt);
-    if (!ws_ok(ws, ws_bytes, lay)) return SPR_ERR_WORKSPACE;
+    bool fits;
+    const ShardWs lay = layout(B, K, Kp, Vs, dt, ws_bytes, &fits);
+    if (!ws_ok(ws, fits)) return SPR_ERR_WORKSPACE;
     if ((rc = device_supported()) != SPR_OK) return rc;
 
     ShardStatsParams sp;
@@ -87,8 +89,9 @@ int decide_params(ShardDecideParams &dp, const float *all_stats, int G, const in
     if (!aligned(all_stats, 4) || !aligned(draft_tokens, 4) || !aligned(uniforms, 4) || !aligned(accepted_len, 4) ||
         (p_tok && !aligned(p_tok, 4)) || (q_tok && !aligned(q_tok, 4)))
         return SPR_ERR_INVALID_ARG;
-    const ShardWs lay = layout(B, K, Kp, Vs, dt);
-    if (!ws_ok(ws, ws_bytes, lay)) return SPR_ERR_WORKSPACE;
+    bool fits;
+    const ShardWs lay = layout(B, K, Kp, Vs, dt, ws_bytes, &fits);
+    if (!ws_ok(ws, fits)) return SPR_ERR_WORKSPACE;
     memset(&dp, 0, sizeof dp);
     dp.all_stats = all_stats;
     dp.G = G;
@@ -103,7 +106,7 @@ int decide_params(ShardDecideParams &dp, const float *all_stats, int G, const in
     dp.q_tok = q_tok;
     dp.status = at<int>(ws, 0);
     dp.acc = at<uint8_t>(ws, lay.acc);
-    dp.rowstats = at<float4>(ws, lay.rowstats);
+    dp.rowstats = at<double2>(ws, lay.rowstats);
     return kProceed;
 }
 }  // namespace
@@ -131,8 +134,9 @@ int draw_params(ShardDrawParams &dp, const void *p_shard, const void *q_shard, i
     const size_t es = elem_size(dt);
     if (!aligned(p_shard, es) || !aligned(q_shard, es) || !aligned(accepted_len, 4) || !aligned(uniforms, 4))
         return SPR_ERR_INVALID_ARG;
-    const ShardWs lay = layout(B, K, Kp, Vs, dt);
-    if (!ws_ok(ws, ws_bytes, lay)) return SPR_ERR_WORKSPACE;
+    bool fits;
+    const ShardWs lay = layout(B, K, Kp, Vs, dt, ws_bytes, &fits);
+    if (!ws_ok(ws, fits)) return SPR_ERR_WORKSPACE;
     memset(&dp, 0, sizeof dp);
     dp.p = p_shard;
     dp.q = q_shard;
@@ -145,7 +149,7 @@ int draw_params(ShardDrawParams &dp, const void *p_shard, const void *q_shard, i
     draw_geometry(B, dp.steps, &dp.chunks, &dp.iters);
     dp.accepted_len = accepted_len;
     dp.uniforms = uniforms;
-    dp.rowstats = at<float4>(ws, lay.rowstats);
+    dp.rowstats = at<double2>(ws, lay.rowstats);
     dp.counters = at<int>(ws, lay.draw_counters);
     dp.part = at<float2>(ws, lay.draw_part);
     return kProceed;

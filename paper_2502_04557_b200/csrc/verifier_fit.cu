@@ -397,8 +397,9 @@ int verifier_labels(const void *p_logits, const void *q_logits, int64_t ldv, con
     const size_t es = elem_size(dt);
     if (!aligned(p_logits, es) || !aligned(q_logits, es) || !aligned(draft_tokens, 4) || (ratio && !aligned(ratio, 4)))
         return SPR_ERR_INVALID_ARG;
-    const LabelWs lay = label_ws_layout(B, K, stat_max_segments_per_row(V, dt));
-    if (!ws || !aligned(ws, 256) || ws_bytes < lay.end) return SPR_ERR_WORKSPACE;
+    Carver cv = carve(ws_bytes);
+    const LabelWs lay = label_ws_layout(cv, B, K, stat_max_segments_per_row(V, dt));
+    if (!ws || !aligned(ws, 256) || !cv.fits()) return SPR_ERR_WORKSPACE;
     int rc = device_supported();
     if (rc != SPR_OK) return rc;
 
@@ -454,8 +455,9 @@ int verifier_train_step(const void *hidden, const uint8_t *labels, int64_t N, in
     if (!aligned(hidden, 16) || !aligned(theta, 4) || !aligned(adam_m, 4) || !aligned(adam_v, 4) ||
         (loss && !aligned(loss, 4)))
         return SPR_ERR_INVALID_ARG;
-    const size_t need = train_ws_bytes(d);
-    if (!ws || !aligned(ws, 256) || ws_bytes < need) return SPR_ERR_WORKSPACE;
+    Carver cv = carve(ws_bytes);
+    const size_t part_off = train_ws_layout(cv, d);
+    if (!ws || !aligned(ws, 256) || !cv.fits()) return SPR_ERR_WORKSPACE;
     int rc = device_supported();
     if (rc != SPR_OK) return rc;
 
@@ -474,7 +476,7 @@ int verifier_train_step(const void *hidden, const uint8_t *labels, int64_t N, in
     tp.beta2 = beta2;
     tp.eps = eps;
     tp.loss = loss;
-    tp.part = at<float>(ws, kHeaderBytes);
+    tp.part = at<float>(ws, part_off);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     return finish(dt == SPR_F32 ? launch_grad_any<float>(tp, st) : launch_grad_any<__nv_bfloat16>(tp, st));
 }

@@ -123,7 +123,7 @@ __global__ void __launch_bounds__(kThreads) verifier_simt_kernel(const VerifyPar
     __syncthreads();
     if (tid == 0) {
         __threadfence();
-        s_last = (atomicAdd(prm.counter, 1) == (int)gridDim.x - 1);
+        s_last = take_ticket(prm.counter, (int)gridDim.x);
     }
     __syncthreads();
     if (!s_last) return;
@@ -170,10 +170,10 @@ __global__ void __launch_bounds__(kThreads) verifier_linear_kernel(const VerifyP
         if (prm.scores) prm.scores[m] = (float)score;
         prm.accept[m] = score >= (double)prm.threshold ? 1 : 0;
         __threadfence();
-        ticket = atomicAdd(&prm.counter[1 + b], 1);
+        ticket = take_ticket(&prm.counter[1 + b], prm.K);
     }
     ticket = __shfl_sync(0xffffffffu, ticket, 0);
-    if (ticket != prm.K - 1 || !prm.first_reject) return;
+    if (!ticket || !prm.first_reject) return;
     __threadfence();
     scan_sequence(prm, b, lane);
 }

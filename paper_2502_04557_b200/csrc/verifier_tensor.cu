@@ -276,7 +276,7 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
     // cut by a tile boundary wait for the CTA that completes the last tile.
     if (tid == 0) {
         __threadfence();
-        ctl->last = (atomicAdd(&prm.counter[1 + blockIdx.y], 1) == (int)gridDim.x - 1);
+        ctl->last = take_ticket(&prm.counter[1 + blockIdx.y], (int)gridDim.x);
     }
     __syncthreads();
     if (!ctl->last) return;
@@ -286,7 +286,7 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
     __syncthreads();
     if (tid == 0) {
         __threadfence();
-        ctl->last = (atomicAdd(&prm.counter[0], 1) == (int)gridDim.y - 1);
+        ctl->last = take_ticket(&prm.counter[0], (int)gridDim.y);
     }
     __syncthreads();
     if (!ctl->last) return;

@@ -162,3 +162,12 @@ def assert_close_rel(got: torch.Tensor, want: np.ndarray, rtol: float, what: str
     got = got.detach().cpu().double().numpy()
     err = np.abs(got - want) / np.maximum(np.abs(want), 1e-300)
     assert np.all(err <= rtol), f"{what}: max rel err {err.max():.3e} > {rtol}"
+
+
+def assert_mass_close(got: torch.Tensor, want: np.ndarray, rtol: float, what: str = "residual_mass"):
+    """Residual mass R = sum over {p_i > q_i} of p_i - q_i: a difference of two partial masses of
+    order one, each known to the relative accuracy of the probabilities, so the error scales
+    with those masses and not with R.  Relative to R where R is large, to 0.1 where it is small."""
+    got = got.detach().cpu().double().numpy()
+    err = np.abs(got - want) / np.maximum(np.abs(want), 0.1)
+    assert np.all(err <= rtol), f"{what}: max err {err.max():.3e} (relative to max(R, 0.1)) > {rtol}"

@@ -6,7 +6,7 @@ import pytest
 import torch
 
 import oracle
-from helpers import (MARGIN, RTOL, assert_close_rel, enforce_margins, enforce_margins_parallel,
+from helpers import (MARGIN, RTOL, assert_close_rel, assert_mass_close, enforce_margins, enforce_margins_parallel,
                      oracle_sd, oracle_step_parallel, oracle_verify, to_device, to_np)
 
 pytestmark = pytest.mark.gpu
@@ -315,7 +315,7 @@ def test_sd_ragged_shapes(spr, dtype, B, K, V, ldv, Kp):
     eq(out["accepted_len"], ref["accepted_len"], "accepted_len")
     eq(out["correction_token"], ref["correction_token"], "correction_token")
     assert_close_rel(out["p_tok"], ref["p_tok"], RTOL[dtype], "p_tok")
-    assert_close_rel(out["residual_mass"], ref["residual_mass"], RTOL[dtype], "residual_mass")
+    assert_mass_close(out["residual_mass"], ref["residual_mass"], RTOL[dtype])
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
@@ -428,6 +428,19 @@ def test_device_detected_errors(spr):
     assert ws.device_status() == 7
     t = tok.cpu().tolist()
     assert t[1] == -1 and t[2] == -1 and t[0] >= 0 and t[3] >= 0
+    # a negative first_reject is refused even where row i*seq_stride + first_reject exists
+    fr = torch.tensor([1, -1, 0, 2], dtype=torch.int32)
+    un = torch.full((4,), 0.37)
+    tl8 = torch.randn(8, 300)
+    tok = spr.replace_sample(tl8.cuda(), 300, un.cuda(), ws, first_reject=fr.cuda(), K=2, seq_stride=2)
+    assert ws.device_status() == 7
+    want, rc = oracle.replace_sample(to_np(tl8), 300, un.numpy(), first_reject=fr.numpy(), K=2, seq_stride=2,
+                                     return_status=True)
+    assert rc == oracle.ERR_ROW and want[1] == -1 and want[3] == -1
+    eq(tok, want, "tokens with a negative first_reject")
+    # neighbouring sequences may not share rows: seq_stride < K is refused on the host
+    with pytest.raises(spr.binding.SprinterError):
+        spr.replace_sample(tl8.cuda(), 300, un.cuda(), ws, first_reject=fr.cuda(), K=2, seq_stride=1)
     # the workspace still works afterwards
     x[1, 1] = 0
     out = spr.sd_verify(p.cuda(), q.cuda(), 300, x.cuda(), u.cuda(), ws)
@@ -735,7 +748,7 @@ def test_sd_single_position_shapes(spr, dtype, B, V, ldv):
         eq(out["correction_token"], ref["correction_token"], "correction_token")
         assert_close_rel(out["p_tok"], ref["p_tok"], RTOL[dtype], "p_tok")
         assert_close_rel(out["q_tok"], ref["q_tok"], RTOL[dtype], "q_tok")
-        assert_close_rel(out["residual_mass"], ref["residual_mass"], RTOL[dtype], "residual_mass")
+        assert_mass_close(out["residual_mass"], ref["residual_mass"], RTOL[dtype])
 
 
 def test_sd_single_position_special_cases(spr):

@@ -7,7 +7,7 @@ import pytest
 import torch
 
 import oracle
-from helpers import MARGIN, RTOL, assert_close_rel, to_np
+from helpers import MARGIN, RTOL, assert_close_rel, assert_mass_close, to_np
 from oracle import training
 from test_gpu_parity import _clear_sd, eq
 
@@ -70,7 +70,7 @@ def test_sd_verify_random_case(spr, seed):
     eq(out["correction_token"], ref["correction_token"], "correction_token")
     assert_close_rel(out["p_tok"], ref["p_tok"], RTOL[dtype], "p_tok")
     assert_close_rel(out["q_tok"], ref["q_tok"], RTOL[dtype], "q_tok")
-    assert_close_rel(out["residual_mass"], ref["residual_mass"], RTOL[dtype], "residual_mass")
+    assert_mass_close(out["residual_mass"], ref["residual_mass"], RTOL[dtype])
 
 
 @pytest.mark.parametrize("seed", range(40))

@@ -10,7 +10,7 @@ import pytest
 import torch
 
 import oracle
-from helpers import MARGIN, RTOL, assert_close_rel, enforce_margins, oracle_sd, to_device, to_np
+from helpers import MARGIN, RTOL, assert_close_rel, assert_mass_close, enforce_margins, oracle_sd, to_device, to_np
 from test_gpu_parity import _clear_sd, _rand_problem, eq
 
 pytestmark = pytest.mark.gpu
@@ -86,7 +86,7 @@ def check_against(ref, results, dtype, status=0):
         eq(out["correction_token"], ref["correction_token"], f"rank {g} correction_token")
         assert_close_rel(out["p_tok"], ref["p_tok"], RTOL[dtype], "p_tok")
         assert_close_rel(out["q_tok"], ref["q_tok"], RTOL[dtype], "q_tok")
-        assert_close_rel(out["residual_mass"], ref["residual_mass"], RTOL[dtype], "residual_mass")
+        assert_mass_close(out["residual_mass"], ref["residual_mass"], RTOL[dtype])
 
 
 @pytest.mark.parametrize("G", [1, 2, 3, 8])
@@ -194,28 +194,89 @@ def test_sharded_bad_token_and_empty_batch(spr):
     assert st.shape == (0, 6)
 
 
+@pytest.mark.parametrize("rows", ["uniform", "random"])
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
-def test_residual_below_fp32_resolution_falls_back_to_p(spr, dtype):
-    """p equals q except for a slightly lower logit at the draft token: the token is rejected
-    (ratio 0.998 against u = 0.9995), but every p_i - q_i elsewhere is about 4e-8 / V, far
-    below what fp32 probabilities resolve, so max(0, p - q) is exactly zero on the GPU.  Both
-    the single-GPU call and the sharded one must then draw from p itself."""
+def test_residual_of_vanishing_mass(spr, dtype, rows):
+    """p equals q except for a slightly lower logit at the draft token, which has probability of
+    order 1/V: the token is rejected (ratio 0.998 against u = 0.9995) and Eq. 1's residual is
+    q_i * (Z_q/Z_p - 1) on every other token, with a total mass of a few 1e-8 - far below what a
+    difference of two float32 probabilities resolves.  With uniform rows the row sums are exact
+    and the ratio form of the weights recovers the residual itself; with random rows the
+    normalisers differ by less than their own rounding, and the kernels then either still see
+    a positive ratio (weights proportional to q) or none (the guard for an undefined Eq. 1:
+    draw from p).  All of these are the same distribution to 1e-8, so the token must be the
+    oracle's in every case, on the single-GPU call and on the sharded one."""
     B, K, V, G = 3, 2, 50257, 4
-    q = torch.zeros((B, K, V), dtype=dtype)
-    p = torch.zeros((B, K + 1, V), dtype=dtype)
+    g = torch.Generator().manual_seed(31)
+    if rows == "uniform":
+        q = torch.zeros((B, K, V), dtype=dtype)
+    else:
+        q = (torch.randn((B, K, V), generator=g) * 2).to(dtype)
+    p = torch.cat([q, q[:, :1]], 1).clone()
     x = torch.tensor([[7, 100], [25000, 3], [V - 1, 0]], dtype=torch.int32)
     u = torch.tensor([[0.9995, 0.5, 0.31], [0.9995, 0.5, 0.77], [0.9995, 0.5, 0.123]], dtype=torch.float32)
     for b in range(B):
+        q[b, 0, int(x[b, 0])] = 0.0
         p[b, 0, int(x[b, 0])] = -2e-3
+    P, Q = to_np(p), to_np(q)
+    floor = 8e-6 if rows == "uniform" else 1e-5      # a uniform row's bins are 2e-5 wide
+    for b in range(B):
+        for _ in range(200):
+            m, t = oracle.residual_draw_margin(P[b, 0], Q[b, 0], float(u[b, K]))
+            m2, t2 = oracle.softmax_draw_margin(P[b, 0], float(u[b, K]))
+            if m >= floor and (rows == "uniform" or (m2 >= floor and t2 == t)):
+                break
+            u[b, K] = torch.rand((), generator=g)
+        assert m >= floor
+    ref = oracle.sd_verify(P, Q, V, to_np(x), to_np(u))
+    assert (ref["accepted_len"] == 0).all() and (ref["residual_mass"] < 1e-6).all()
     ws = spr.Workspace(spr.workspace_bytes(2, B, K, V, 1, 0, spr.binding._dt(p)))
     one = spr.sd_verify(p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), ws)
     results = run_sharded(spr, p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), G)
     for out in [one] + results:
-        assert (out["accepted_len"] == 0).all()
-        assert (out["residual_mass"] == 0).all()
-        for b in range(B):
-            m, t = oracle.softmax_draw_margin(to_np(p)[b, 0], float(u[b, K]))
-            assert m > 1e-6 and int(out["correction_token"][b]) == t
+        eq(out["accepted_len"], ref["accepted_len"], "accepted_len")
+        eq(out["correction_token"], ref["correction_token"], "correction_token")
+        rm = out["residual_mass"].cpu().numpy()
+        assert (np.abs(rm - ref["residual_mass"]) < 1e-6).all()
+        if rows == "uniform":            # exact row sums: the mass itself comes out to a few per cent
+            assert (np.abs(rm / ref["residual_mass"] - 1.0) < 0.05).all()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_residual_far_below_the_resolution_of_the_probabilities(spr, dtype):
+    """p equals q except for a logit lowered by 1/32 at a draft token of probability ~4e-4: the
+    token is rejected, and Eq. 1's residual (total mass ~1e-5) is q_i * (Z_q/Z_p - 1) on every
+    other token - a relative difference of 1e-5, of which a difference of two float32
+    probabilities keeps one or two digits.  The ratio form of the weights keeps the residual
+    proportional to q, so both the single-GPU call and the sharded one pick the oracle's token."""
+    B, K, V, G = 6, 2, 50257, 4
+    g = torch.Generator().manual_seed(4242)
+    q = (torch.randn((B, K, V), generator=g) * 2).to(dtype)
+    p = torch.cat([q, (torch.randn((B, 1, V), generator=g) * 2).to(dtype)], 1).clone()
+    x = torch.randint(0, V, (B, K), generator=g, dtype=torch.int32)
+    u = torch.rand((B, K + 1), generator=g)
+    for b in range(B):
+        q[b, 0, int(x[b, 0])] = 5.0
+        p[b, 0, int(x[b, 0])] = 4.96875           # representable in bfloat16
+        u[b, 0] = 0.99                            # above the ratio ~0.969: rejected at position 0
+    P, Q = to_np(p), to_np(q)
+    for b in range(B):
+        for _ in range(50):
+            m, t = oracle.residual_draw_margin(P[b, 0], Q[b, 0], float(u[b, K]))
+            if m >= MARGIN:
+                break
+            u[b, K] = torch.rand((), generator=g)
+        assert m >= MARGIN and t != int(x[b, 0])
+    ref = oracle.sd_verify(P, Q, V, to_np(x), to_np(u))
+    assert (ref["accepted_len"] == 0).all() and (ref["residual_mass"] < 3e-5).all() and (ref["residual_mass"] > 3e-6).all()
+    ws = spr.Workspace(spr.workspace_bytes(2, B, K, V, 1, 0, spr.binding._dt(p)))
+    one = spr.sd_verify(p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), ws)
+    results = run_sharded(spr, p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), G)
+    for out in [one] + results:
+        eq(out["accepted_len"], ref["accepted_len"], "accepted_len")
+        eq(out["correction_token"], ref["correction_token"], "correction_token")
+        # the mass itself is a difference of two row normalisers kept in float32: absolute 1e-6
+        assert np.abs(out["residual_mass"].cpu().numpy() - ref["residual_mass"]).max() < 1e-6
 
 
 def test_sharded_llama3_full_size_sampled(spr):

@@ -254,6 +254,13 @@ def test_replace_sample_row_selection_and_gate():
     # out-of-range row -> -1 and a status
     t, rc = oracle.replace_sample(tl, V, u, rows=np.array([0, 12, -1, 1], np.int32), return_status=True)
     assert rc == oracle.ERR_ROW and t[1] == -1 and t[2] == -1 and t[0] >= 0
+    # a negative first_reject is not a position (Algorithm 2's r counts accepted tokens): the
+    # draw is refused even though row i*K + first_reject would exist
+    fr = np.array([2, -1, 0, 1], np.int32)
+    t, rc = oracle.replace_sample(tl, V, u, first_reject=fr, K=K, seq_stride=K, return_status=True)
+    assert rc == oracle.ERR_ROW and t[1] == -1
+    for i in (0, 2, 3):
+        assert t[i] == oracle.sample_softmax_row(tl[i * K + fr[i], :V], u[i])
 
 
 def test_cdf_margin_by_hand():
