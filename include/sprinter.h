@@ -19,10 +19,15 @@
  *     non-zero return nothing was launched.
  *   - `ws` is caller-owned device scratch of at least spr_workspace_bytes()
  *     bytes, 256-byte aligned, cleared once with spr_workspace_init() after
- *     allocation (this zeroes the status word).  Each call clears the counters
- *     it needs on the stream before its kernels, so one workspace serves calls
- *     of any op and shape it is large enough for, one after the other.  Calls
- *     that may overlap on the GPU (different streams) need separate workspaces.
+ *     allocation (this zeroes the status word and the ticket counters).  The
+ *     kernels leave every counter they use at zero again (or the call clears
+ *     it on the stream first), so one workspace serves calls of any op and
+ *     shape it is large enough for, one after the other.  Calls that may
+ *     overlap on the GPU (different streams) need separate workspaces.
+ *   - The library allocates nothing.  Its only state is per-process caches of
+ *     device properties and kernel attributes, the calling thread's
+ *     timing-event pair (spr_set_stage_events) and the fixed scratch array of
+ *     replace_sample_static.
  *   - Problems a kernel detects (a draft token id outside [0,V), a row index
  *     outside the logits tensor, a bounded wait that ran out) never trap: the
  *     affected outputs are set to -1, a sticky status word in `ws` records the
@@ -379,6 +384,27 @@ int replace_sample_static(const void *target_logits, int64_t ldv, int V, int64_t
  * host thread record `before` / `after` on their stream around the row-statistics
  * kernel, the launch that reads the 2*B*K*V logits.  Pass NULL, NULL to stop. */
 void spr_set_stage_events(void *before, void *after);
+
+/*
+ * spr_test_sprinter_verify - test hook, not part of the stable interface.
+ *
+ * The paper has no counterpart.  sprinter_verify on the tensor-core kernel (bf16 MLP, the
+ * shapes SPR_VERIFIER_TENSOR takes) with the launch shape chosen by the caller instead of by
+ * the library, so that tests reach every shape on small inputs: bm, bn in {64, 128} tokens x
+ * hidden units per tile, splits in {1, 2, 4, 8} CTAs sharing a tile along d, cluster_n = 1
+ * (finish through the workspace) or -1 (a tile's CTAs form one cluster; needs
+ * splits * ceil(h / bn) <= 8); 0 leaves a value to the library.  A combination the problem
+ * does not allow returns SPR_ERR_UNSUPPORTED.
+ * flags bit 0: the kernel's copy engine producer issues nothing, so that the first bounded
+ * wait of every CTA runs out after spin_limit polls (0 = the library's limit): the call
+ * returns SPR_OK, the status word reads SPR_ERR_TIMEOUT, scores are -1, accept bits 0 and
+ * first_reject -1, nothing is left in flight and the workspace stays usable.
+ */
+int spr_test_sprinter_verify(const void *hidden, const void *W1, const float *b1, const void *W2,
+                             const float *b2, float threshold, int B, int K, int d, int h, int dt,
+                             float *scores, uint8_t *accept, int32_t *first_reject, void *ws, size_t ws_bytes,
+                             void *cuda_stream, int bm, int bn, int splits, int cluster_n, int flags,
+                             unsigned spin_limit);
 
 /* Synchronises the stream, returns the sticky device status word of `ws`
  * (SPR_OK if nothing was detected) and clears it. */

@@ -25,7 +25,7 @@ EXPORTS = [
     "spr_host_arena_bytes", "sprinter_verify_host", "replace_sample_host", "sd_verify_host",
     "spr_set_stage_events", "replace_sample_static", "sprinter_step", "sprinter_simulate",
     "sd_shard_stats", "sd_shard_decide", "sd_shard_weights", "sd_shard_draw", "sd_shard_decide_weights",
-    "verifier_labels", "verifier_train_step",
+    "verifier_labels", "verifier_train_step", "spr_test_sprinter_verify",
 ]
 
 
@@ -63,6 +63,9 @@ def lib():
         L.sprinter_verify.restype = i32
         L.sprinter_verify.argtypes = [vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32,
                                       vp, vp, vp, vp, sz, vp]
+        L.spr_test_sprinter_verify.restype = i32
+        L.spr_test_sprinter_verify.argtypes = [vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32,
+                                               vp, vp, vp, vp, sz, vp, i32, i32, i32, i32, i32, C.c_uint]
         L.sprinter_step.restype = i32
         L.sprinter_step.argtypes = [vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, vp, i64, i32, i32, vp,
                                     i32, i32, vp, vp, vp, vp, vp, sz, vp]
@@ -220,6 +223,31 @@ def sprinter_verify(hidden, W1, b1, W2, b2, threshold: float, ws: Workspace, pat
                                B, K, d, h, dt, path, _ptr(scores), _ptr(accept), _ptr(first_reject),
                                _ptr(ws.buf), ws.nbytes, _stream())
     _check("sprinter_verify", rc)
+    return scores, accept, first_reject
+
+
+def sprinter_verify_shaped(hidden, W1, b1, W2, b2, threshold: float, ws: Workspace, bm: int = 0, bn: int = 0,
+                           splits: int = 0, cluster_n: int = 0, flags: int = 0, spin_limit: int = 0, out=None):
+    """Test hook (spr_test_sprinter_verify): the tensor-core verifier with a forced launch shape."""
+    _dev(hidden, torch.bfloat16, "hidden")
+    B, K, d = hidden.shape
+    h = W1.shape[0]
+    for t, ty, nm in ((W1, torch.bfloat16, "W1"), (b1, torch.float32, "b1"), (W2, torch.bfloat16, "W2"),
+                      (b2, torch.float32, "b2")):
+        _dev(t, ty, nm)
+    if W1.shape[-1] != d or b1.numel() != h or W2.numel() != h:
+        raise ValueError("W1 must be [h, d]; b1 and W2 must have h entries")
+    if out is None:
+        scores = torch.empty((B, K), dtype=torch.float32, device=hidden.device)
+        accept = torch.empty((B, K), dtype=torch.uint8, device=hidden.device)
+        first_reject = torch.empty((B,), dtype=torch.int32, device=hidden.device)
+    else:
+        scores, accept, first_reject = out
+    rc = lib().spr_test_sprinter_verify(_ptr(hidden), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), float(threshold),
+                                        B, K, d, h, BF16, _ptr(scores), _ptr(accept), _ptr(first_reject),
+                                        _ptr(ws.buf), ws.nbytes, _stream(), bm, bn, splits, cluster_n, flags,
+                                        spin_limit)
+    _check("spr_test_sprinter_verify", rc)
     return scores, accept, first_reject
 
 

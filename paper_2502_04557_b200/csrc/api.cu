@@ -46,19 +46,20 @@ int check_device()
     return major == 10 ? SPR_OK : SPR_ERR_UNSUPPORTED;
 }
 
-// AUTO hands batches of at least this many tokens to the tensor-core verifier
-constexpr int kTensorMinTokens = 4;
+// AUTO hands batches of at least this many tokens to the tensor-core verifier: with d split
+// over the CTAs of a cluster it is the faster kernel even for a single token
+constexpr int kTensorMinTokens = 1;
 
 // row indices are 32-bit inside the kernels; leave room for the padding of the last step
 constexpr int kMaxVocab = 1 << 30;
 
 
 // tensor-core kernel where it applies (or is forced), SIMT kernel otherwise
-int launch_verifier(VerifyParams &vp, int dt, int path, cudaStream_t st)
+int launch_verifier(VerifyParams &vp, int dt, int path, cudaStream_t st, const VerifierTune *tune = nullptr)
 {
     if (path != SPR_VERIFIER_SIMT) {
         const int min_tokens = path == SPR_VERIFIER_TENSOR ? 1 : kTensorMinTokens;
-        const int tensor_rc = launch_verifier_tensor(vp, dt, min_tokens, st);  // < 0: shape not taken
+        const int tensor_rc = launch_verifier_tensor(vp, dt, min_tokens, tune, st);  // < 0: shape not taken
         if (tensor_rc == 0) return SPR_OK;
         if (tensor_rc > 0) return cuda_fail((cudaError_t)tensor_rc);
         if (path == SPR_VERIFIER_TENSOR) return SPR_ERR_UNSUPPORTED;
@@ -157,7 +158,7 @@ namespace {
 int verify_counters(int B, int K) { return max((B * K + 63) / 64, B); }
 
 // number of partial sums per token any of the verifier kernels may write for this shape
-int verify_slices(int h) { return verifier_simt_slices(h); }
+int verify_slices(int h) { return max(verifier_simt_slices(h), verifier_tensor_max_slices(h)); }
 
 }  // namespace
 
@@ -223,6 +224,26 @@ int sprinter_verify(const void *hidden, const void *W1, const float *b1, const v
     vp.counter = at<int>(ws, lay.counter);
     vp.part_z = at<float>(ws, lay.part_z);
     return launch_verifier(vp, dt, path, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int spr_test_sprinter_verify(const void *hidden, const void *W1, const float *b1, const void *W2,
+                             const float *b2, float threshold, int B, int K, int d, int h, int dt,
+                             float *scores, uint8_t *accept, int32_t *first_reject, void *ws, size_t ws_bytes,
+                             void *cuda_stream, int bm, int bn, int splits, int cluster_n, int flags,
+                             unsigned spin_limit)
+{
+    VerifyParams vp = verify_params(hidden, W1, b1, W2, b2, threshold, B, K, d, h, scores, accept, first_reject);
+    int rc = check_verify_args(vp, dt, SPR_VERIFIER_TENSOR);
+    if (rc != SPR_OK || B == 0) return rc;
+    Carver cv = carve(ws_bytes);
+    const VerifyWs lay = verify_ws_layout(cv, B * K, verify_slices(h), verify_counters(B, K));
+    if (!ws || !aligned(ws, 256) || !cv.fits()) return SPR_ERR_WORKSPACE;
+    if ((rc = check_device()) != SPR_OK) return rc;
+    VerifierTune tune = {bm, bn, splits, cluster_n, flags, spin_limit};
+    vp.status = at<int>(ws, 0);
+    vp.counter = at<int>(ws, lay.counter);
+    vp.part_z = at<float>(ws, lay.part_z);
+    return launch_verifier(vp, dt, SPR_VERIFIER_TENSOR, static_cast<cudaStream_t>(cuda_stream), &tune);
 }
 
 int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, const int32_t *rows,

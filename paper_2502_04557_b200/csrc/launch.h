@@ -120,6 +120,25 @@ struct VerifyParams {
     int *counter;
     float *part_z;  // [slices*M]
     int slices;
+    // tensor-core kernel only
+    int kb_per;             // 64-element blocks of d each of the CTAs that share a tile takes
+    int a_box_rows;         // rows of hidden states one copy fetches (the tile height, or fewer for a small batch)
+    int cluster_n;          // hidden-unit slices of one token tile per cluster (1, or all of them)
+    int final_in_cluster;   // the CTAs of a token tile form one cluster: no tickets, no part_z
+    uint32_t spin_limit;    // polls after which a bounded wait gives up
+    int test_flags;         // VERIFIER_TEST_*
+};
+
+// test_flags: the TMA producer issues no copy, so that the first bounded wait runs out
+enum { VERIFIER_TEST_NO_LOADS = 1 };
+
+// Tile shape of the tensor-core verifier; zeros = chosen from the problem size.
+struct VerifierTune {
+    int bm, bn;         // tokens x hidden units per tile: 64 or 128 each
+    int splits;         // CTAs sharing a tile along d: 1, 2, 4 or 8
+    int cluster_n;      // 0: automatic; 1: one slice per cluster; -1: all slices of a tile in one cluster
+    int test_flags;
+    uint32_t spin_limit;   // 0: default
 };
 
 struct SimParams {
@@ -151,7 +170,11 @@ cudaError_t launch_verifier_simt(const VerifyParams &vp, int dt, cudaStream_t st
 // Tensor-core (tcgen05) verifier for bf16 MLPs.  Returns 0 when launched, a negative
 // value when it does not take this shape or dtype (nothing launched), or a positive
 // cudaError_t.  It sets the slice count itself.  Batches of fewer than min_tokens tokens
-// are left to the SIMT kernel.
-int launch_verifier_tensor(const VerifyParams &vp, int dt, int min_tokens, cudaStream_t st);
+// are left to the SIMT kernel.  tune (may be null) forces the tile shape: a shape that cannot
+// be used for this problem gives a negative value.
+int launch_verifier_tensor(const VerifyParams &vp, int dt, int min_tokens, const VerifierTune *tune,
+                           cudaStream_t st);
+// most partial sums per token the tensor-core kernel may write for h hidden units
+int verifier_tensor_max_slices(int h);
 
 }  // namespace spr

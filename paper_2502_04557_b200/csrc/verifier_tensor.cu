@@ -3,21 +3,29 @@
 //   A = relu(H W1^T + b1)   -> tcgen05.mma (bf16 x bf16 -> fp32 in TMEM), operands staged in
 //                              shared memory by TMA with the 128-byte swizzle
 //   z = A W2                -> fused epilogue: each epilogue thread owns one token (one TMEM
-//                              lane), reads its accumulator row with tcgen05.ld and folds
-//                              bias, ReLU and the W2 dot product in registers; A never
-//                              reaches HBM
-// One CTA computes a BM-token x BN-hidden-unit tile (BM, BN in {64, 128}) and writes one
-// partial z per token.
-// The CTA that completes a token tile adds its partials in slice order, applies the sigmoid
-// and the threshold and scans the sequences inside the tile (same tail as the SIMT kernel).
+//                              lane) and folds bias, ReLU and the W2 dot product in registers;
+//                              A never reaches HBM
+//
+// Grid (S, slices, tiles): a CTA computes a BM-token x BN-hidden-unit tile over one of S equal
+// ranges of d.  The S CTAs of a tile form a cluster (along x) and add their accumulators
+// through distributed shared memory BEFORE the ReLU: CTA r receives, from every CTA of the
+// tile, the BN/S accumulator columns it owns, adds them in CTA order and applies bias, ReLU
+// and W2 to those columns.  Small batches thereby spread the sweep over W1 (the only real
+// traffic they have) over many SMs.
+// Where S x slices <= 8 the cluster also spans the hidden-unit slices of the tile (along y):
+// every CTA sends its per-token partial z to the cluster's first CTA, which adds them in
+// rank order, applies sigmoid and threshold and scans the sequences inside the tile out of
+// shared memory - no trip through global memory.  Otherwise the partial z go to the
+// workspace and the CTA that takes the tile's last ticket finishes it.
 //
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
 // warps 2..5 = epilogue (warp w reads TMEM lanes 32*(w%4) .. +31).
 // Every wait on an mbarrier is bounded: when a wait runs out the kernel records
-// SPR_ERR_TIMEOUT in the status word, all roles leave their loops, TMEM is released and
-// the CTA exits.
+// SPR_ERR_TIMEOUT in the status word, all roles leave their loops, the CTA still goes through
+// every cluster barrier (so its peers never wait for it), hands on NaN instead of its partial
+// results (the tile's tokens then report score -1, accept 0, first_reject -1), waits - again
+// bounded - for what it has in flight, releases TMEM and exits.
 #include <cuda.h>
-#include <stdlib.h>
 
 #include "common.cuh"
 #include "launch.h"
@@ -25,41 +33,61 @@
 
 namespace spr {
 
+// Development aid (compiled only with -DSPR_VERIFIER_STAMPS): SM-clock stamps of the phases of
+// the first CTAs of a launch, read back with spr_debug_verifier_stamps().
+#ifdef SPR_VERIFIER_STAMPS
+__device__ long long g_stamps[512][64];
+#define SPR_STAMP(i)                                                                                     \
+    do {                                                                                                 \
+        const unsigned cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);            \
+        if (cta_ < 512) g_stamps[cta_][i] = clock64();                                                   \
+    } while (0)
+#else
+#define SPR_STAMP(i)
+#endif
+
 namespace {
 
-constexpr int kAtomK = 64;      // bf16 elements of one 128-byte swizzle row (one TMA box)
-constexpr int kAtoms = 2;       // swizzle atoms per pipeline stage
-constexpr int kBK = kAtomK * kAtoms;   // bf16 elements per k-block (pipeline stage)
+constexpr int kAtomK = 64;      // bf16 elements of one 128-byte swizzle row: one TMA box, one "atom" of d
 constexpr int kUmmaK = 16;      // K of one tcgen05.mma for 16-bit operands
 constexpr int kTcThreads = 192;
-constexpr int kMaxStages = 12;
+constexpr int kMaxStages = 4;
+constexpr int kMaxClusterCtas = 8;          // portable cluster size
 constexpr uint32_t kSpinLimit = 1u << 24;   // polls of mbarrier.try_wait before giving up
 
-template <int BM, int BN>
-struct TileCfg {
-    static constexpr int kBytesA = BM * kBK * 2;
-    static constexpr int kBytesB = BN * kBK * 2;
-    static constexpr int kStageBytes = kBytesA + kBytesB;
-    // The k-loop is bound by the time a stage takes to come round again (MMA done -> commit ->
-    // producer -> TMA -> full, about 2 us), so throughput is stages / that time: use all the
-    // shared memory there is (one CTA per SM either way).
-    static constexpr int kStages = (220 * 1024) / kStageBytes < kMaxStages ? (220 * 1024) / kStageBytes : kMaxStages;
-    static constexpr int kTmemCols = BN < 32 ? 32 : BN;
-    // stages, slack to align them to 1024 bytes, control block
-    static constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 + 3072;
-};
-
-struct Control {                 // lives behind the stages in dynamic shared memory
+struct Control {                 // lives behind the ring in dynamic shared memory
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
     uint64_t tmem_full;
+    uint64_t drain;
     uint32_t tmem_base;
     int abort;
     int last;
+    int consumed;                // stages whose operands the MMA issuer saw arrive
     float b1[128];
     float w2[128];
+    float zbuf[kMaxClusterCtas][128];   // first CTA of a cluster: partial z of every CTA, per token
+    unsigned char codes[128];           // accept codes of the tile, for the scan
 };
-static_assert(sizeof(Control) <= 3072, "control block must fit its reservation");
+
+template <int BM, int BN>
+struct TileCfg {
+    static constexpr int kBytesA = BM * kAtomK * 2;     // one atom of the hidden-state tile
+    static constexpr int kBytesB = BN * kAtomK * 2;     // one atom of the W1 tile
+    // A pipeline stage costs the two threads that run it (producer, MMA issuer) about 0.25 us
+    // of barrier and issue latency whatever it holds, so a stage holds several atoms: 48-64 KB.
+    static constexpr int kAtoms = (BM + BN == 128) ? 4 : 2;
+    static constexpr int kStageBytes = kAtoms * (kBytesA + kBytesB);
+    static constexpr int kStages = (200 * 1024) / kStageBytes;
+    static_assert(kStages >= 2 && kStages <= kMaxStages, "stage count");
+    static constexpr int kRingBytes = kStages * kStageBytes;
+    // after the k-loop the ring is reused for the accumulator columns received from the
+    // other CTAs of the tile: [S][BN/S/4][BM] float4
+    static_assert(BM * BN * 4 <= kRingBytes, "ring must hold the exchanged accumulator columns");
+    static constexpr int kTmemCols = BN < 32 ? 32 : BN;
+    // ring, slack to align it to 1024 bytes, control block
+    static constexpr size_t kSmemBytes = (size_t)kRingBytes + 1024 + ((sizeof(Control) + 255) / 256) * 256;
+};
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -86,22 +114,28 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 }
 // Bounded wait.  Returns false (and flags the CTA) if the phase never completes or another
 // role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, Control *ctl, int *status)
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, Control *ctl, int *status, uint32_t limit)
 {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 1023u) == 1023u && *reinterpret_cast<volatile int *>(&ctl->abort)) return false;
+        if ((i & 255u) == 255u && *reinterpret_cast<volatile int *>(&ctl->abort)) return false;
     }
     *reinterpret_cast<volatile int *>(&ctl->abort) = 1;
     raise_status(status, SPR_ERR_TIMEOUT);
     return false;
 }
+// the same without side effects: used on the way out, when the CTA has already given up
+__device__ __forceinline__ void mbar_wait_quiet(uint64_t *bar, uint32_t parity, uint32_t limit)
+{
+    for (uint32_t i = 0; i < limit; ++i)
+        if (mbar_try_wait(bar, parity)) return;
+}
 
-__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c0, int c1, uint64_t *bar)
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint64_t *bar)
 {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(smem_u32(bar))
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(smem_u32(bar))
         : "memory");
 }
 
@@ -139,17 +173,98 @@ __device__ __forceinline__ void umma_commit(uint64_t *bar)
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                  : "memory");
 }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
+// 32 accumulator columns of this thread's TMEM lane; the registers are valid after tmem_ld_wait()
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
 {
-    uint32_t r[16];
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// ---- thread-block cluster: barrier over all threads of all CTAs, shared memory of a peer CTA
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.aligned;" ::: "memory"); }   // release
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.aligned;" ::: "memory"); }       // acquire
+__device__ __forceinline__ void cluster_sync()
+{
+    cluster_arrive();
+    cluster_wait();
+}
+// address, in the cluster's shared window, of this CTA's shared address `saddr` in CTA `rank`
+__device__ __forceinline__ uint32_t peer_smem(uint32_t saddr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v)
+{
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void st_cluster_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d)
+                 : "memory");
+}
+
+// One epilogue thread (= accumulator row r_in): its BN accumulator columns, four at a time, to
+// the CTAs that own them.  Receiver layout: recv4[source split][group of 4 owned columns][row].
+template <int BM, int BN, int S>
+__device__ __forceinline__ void send_columns(uint32_t lane_base, const float4 *recv4, int split, uint32_t row_rank0,
+                                             int r_in, bool live_row)
+{
+    constexpr int kColsPer = BN / S, kGroups = kColsPer / 4;
+    static_assert(kColsPer >= 8 && kColsPer % 4 == 0, "columns per owner");
+    uint32_t base[S];    // where this CTA's block of rows starts in every owner's buffer
 #pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+    for (int o = 0; o < S; ++o)
+        base[o] = peer_smem(smem_u32(recv4 + ((size_t)split * kGroups * BM + r_in)), row_rank0 + (uint32_t)o);
+#pragma unroll
+    for (int c0 = 0; c0 < BN; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(lane_base + (uint32_t)c0, r);
+        tmem_ld_wait();
+        if (live_row) {
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+                const int c = c0 + 4 * g;
+                const int owner = c / kColsPer, cg = (c % kColsPer) / 4;
+                st_cluster_v4(base[owner] + (uint32_t)(cg * BM * 16), r[4 * g], r[4 * g + 1], r[4 * g + 2], r[4 * g + 3]);
+            }
+        }
+    }
+}
+
+// the same thread, after the exchange: sum over the source CTAs (in order), bias, ReLU and W2
+// for the columns this CTA owns
+template <int BM, int BN, int S>
+__device__ __forceinline__ float owned_columns_z(const float4 *recv4, const Control *ctl, int split, int r_in)
+{
+    constexpr int kColsPer = BN / S, kGroups = kColsPer / 4;
+    float z = 0.f;
+#pragma unroll
+    for (int cg = 0; cg < kGroups; ++cg) {
+        float4 a = recv4[(size_t)cg * BM + r_in];
+#pragma unroll
+        for (int s = 1; s < S; ++s) {
+            const float4 b = recv4[((size_t)s * kGroups + cg) * BM + r_in];
+            a.x += b.x;
+            a.y += b.y;
+            a.z += b.z;
+            a.w += b.w;
+        }
+        const int c = split * kColsPer + 4 * cg;
+        z = fmaf(ctl->w2[c], fmaxf(a.x + ctl->b1[c], 0.f), z);
+        z = fmaf(ctl->w2[c + 1], fmaxf(a.y + ctl->b1[c + 1], 0.f), z);
+        z = fmaf(ctl->w2[c + 2], fmaxf(a.z + ctl->b1[c + 2], 0.f), z);
+        z = fmaf(ctl->w2[c + 3], fmaxf(a.w + ctl->b1[c + 3], 0.f), z);
+    }
+    return z;
 }
 
 template <int BM, int BN>
@@ -159,16 +274,26 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
 {
     using Cfg = TileCfg<BM, BN>;
     extern __shared__ unsigned char smem_raw[];
-    unsigned char *stages = reinterpret_cast<unsigned char *>(
+    unsigned char *ring = reinterpret_cast<unsigned char *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    Control *ctl = reinterpret_cast<Control *>(stages + (size_t)Cfg::kStages * Cfg::kStageBytes);
+    Control *ctl = reinterpret_cast<Control *>(ring + Cfg::kRingBytes);
 
     pdl_trigger();   // a replacement draw launched behind this grid may be scheduled now
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) SPR_STAMP(0);
     const int M = prm.B * prm.K;
-    const int n0 = blockIdx.x * BN;      // first hidden unit of this slice
-    const int m0 = blockIdx.y * BM;      // first token of this tile
-    const int num_kb = (prm.d + kBK - 1) / kBK;
+    const int S = (int)gridDim.x, split = (int)blockIdx.x;   // CTAs sharing this tile along d
+    const int n0 = blockIdx.y * BN;      // first hidden unit of this slice
+    const int m0 = blockIdx.z * BM;      // first token of this tile
+    const int atom0 = split * prm.kb_per;                                          // first atom of d of this CTA
+    const int num_atoms = min(prm.kb_per, (prm.d + kAtomK - 1) / kAtomK - atom0);  // >= 1: the host sees to it
+    const int num_stages = (num_atoms + Cfg::kAtoms - 1) / Cfg::kAtoms;
+    const int cluster_ctas = S * prm.cluster_n;
+    const bool clustered = cluster_ctas > 1;
+    // rank inside the cluster (x runs fastest) and the rank of the tile's CTA with split 0
+    const uint32_t my_rank = (uint32_t)split + (blockIdx.y % (unsigned)prm.cluster_n) * (uint32_t)S;
+    const uint32_t row_rank0 = my_rank - (uint32_t)split;
+    const uint32_t limit = prm.spin_limit;
 
     if (tid == 0) {
         for (int s = 0; s < Cfg::kStages; ++s) {
@@ -176,15 +301,14 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
             mbar_init(&ctl->empty[s], 1);
         }
         mbar_init(&ctl->tmem_full, 1);
+        mbar_init(&ctl->drain, 1);
         ctl->abort = 0;
         ctl->last = 0;
+        ctl->consumed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int j = tid; j < BN; j += kTcThreads) {
-        const int n = n0 + j;
-        ctl->b1[j] = n < prm.h ? prm.b1[n] : 0.f;
-        ctl->w2[j] = n < prm.h ? __bfloat162float(static_cast<const __nv_bfloat16 *>(prm.W2)[n]) : 0.f;
-    }
+    if (warp == 0 && lane < 2)   // descriptor fetch off the critical path of the first copy
+        asm volatile("prefetch.tensormap [%0];" ::"l"(lane == 0 ? &map_h : &map_w) : "memory");
     if (warp == 1) {   // TMEM: BN fp32 accumulator columns x 128 lanes
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
                      "r"((uint32_t)Cfg::kTmemCols)
@@ -195,98 +319,215 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_acc = ctl->tmem_base;
+    if (tid == 0) SPR_STAMP(1);
+    // A peer's shared memory may be written once that CTA has started.  Without a split of d
+    // nothing else has to be waited for, so each thread says "started" here and checks for
+    // everybody's word only where the first remote store is made.
+    const bool early_arrive = clustered && S == 1;
+    if (early_arrive) cluster_arrive();
 
+    int issued = 0;       // producer: stages whose copies are on their way
+    bool ok = true;       // epilogue: the accumulator is complete
     if (warp == 0) {
-        // ---------------- TMA producer
-        if (lane == 0) {
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % Cfg::kStages;
-                const uint32_t round = (uint32_t)(kb / Cfg::kStages);
-                if (!mbar_wait(&ctl->empty[s], (round & 1u) ^ 1u, ctl, prm.status)) break;
-                unsigned char *a_dst = stages + (size_t)s * Cfg::kStageBytes;
-                unsigned char *b_dst = a_dst + Cfg::kBytesA;
-                mbar_expect_tx(&ctl->full[s], (uint32_t)Cfg::kStageBytes);
-#pragma unroll
-                for (int a = 0; a < kAtoms; ++a) {   // one box per 64-wide swizzle atom
-                    tma_load_2d(a_dst + a * (Cfg::kBytesA / kAtoms), &map_h, kb * kBK + a * kAtomK, m0, &ctl->full[s]);
-                    tma_load_2d(b_dst + a * (Cfg::kBytesB / kAtoms), &map_w, kb * kBK + a * kAtomK, n0, &ctl->full[s]);
-                }
+        // ---------------- TMA producer: one lane per box of a stage (even lanes: hidden-state
+        // atoms, odd lanes: W1 atoms), so one instruction issues all copies of a stage
+        if (lane < 2 * Cfg::kAtoms && !(prm.test_flags & VERIFIER_TEST_NO_LOADS)) {
+            const int atom = lane >> 1;
+            const bool is_w = lane & 1;
+            const CUtensorMap *map = is_w ? &map_w : &map_h;
+            const int row0 = is_w ? n0 : m0;
+            const uint32_t off = is_w ? (uint32_t)(Cfg::kAtoms * Cfg::kBytesA + atom * Cfg::kBytesB)
+                                      : (uint32_t)(atom * Cfg::kBytesA);
+            const uint32_t atom_bytes = (uint32_t)prm.a_box_rows * (kAtomK * 2) + (uint32_t)Cfg::kBytesB;
+            for (int st = 0; st < num_stages; ++st) {
+                const int s = st % Cfg::kStages;
+                const uint32_t round = (uint32_t)(st / Cfg::kStages);
+                const int n_at = min(Cfg::kAtoms, num_atoms - st * Cfg::kAtoms);
+                if (!mbar_wait(&ctl->empty[s], (round & 1u) ^ 1u, ctl, prm.status, limit)) break;
+                if (lane == 0) mbar_expect_tx(&ctl->full[s], (uint32_t)n_at * atom_bytes);
+                if (atom < n_at)
+                    tma_load_2d(smem_u32(ring + (size_t)s * Cfg::kStageBytes) + off, map,
+                                (atom0 + st * Cfg::kAtoms + atom) * kAtomK, row0, &ctl->full[s]);
+                issued = st + 1;
+                if (st == 0) SPR_STAMP(2);
+                if (st < 24 && lane == 0) SPR_STAMP(40 + st);
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = umma_instr_desc<BM, BN>();
-            bool ok = true;
-            for (int kb = 0; kb < num_kb && ok; ++kb) {
-                const int s = kb % Cfg::kStages;
-                const uint32_t round = (uint32_t)(kb / Cfg::kStages);
-                ok = mbar_wait(&ctl->full[s], round & 1u, ctl, prm.status);
-                if (!ok) break;
+            bool fed = true;
+            int st = 0;
+            for (; st < num_stages; ++st) {
+                const int s = st % Cfg::kStages;
+                const uint32_t round = (uint32_t)(st / Cfg::kStages);
+                const int n_at = min(Cfg::kAtoms, num_atoms - st * Cfg::kAtoms);
+                fed = mbar_wait(&ctl->full[s], round & 1u, ctl, prm.status, limit);
+                if (!fed) break;
+                if (st == 0) SPR_STAMP(3);
+                if (st < 24) SPR_STAMP(16 + st);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a_addr = smem_u32(stages + (size_t)s * Cfg::kStageBytes);
-                const uint32_t b_addr = a_addr + Cfg::kBytesA;
+                const uint32_t a_addr = smem_u32(ring + (size_t)s * Cfg::kStageBytes);
+                const uint32_t b_addr = a_addr + Cfg::kAtoms * Cfg::kBytesA;
 #pragma unroll
-                for (int a = 0; a < kAtoms; ++a) {
-                    const uint64_t da = umma_smem_desc(a_addr + a * (Cfg::kBytesA / kAtoms));
-                    const uint64_t db = umma_smem_desc(b_addr + a * (Cfg::kBytesB / kAtoms));
+                for (int a = 0; a < Cfg::kAtoms; ++a) {
+                    if (a < n_at) {
+                        const uint64_t da = umma_smem_desc(a_addr + a * Cfg::kBytesA);
+                        const uint64_t db = umma_smem_desc(b_addr + a * Cfg::kBytesB);
 #pragma unroll
-                    for (int k = 0; k < kAtomK / kUmmaK; ++k) {
-                        // next 16 elements along K: 32 bytes further inside the swizzle row
-                        const uint64_t adv = (uint64_t)((k * kUmmaK * 2) >> 4);
-                        umma_bf16(tmem_acc, da + adv, db + adv, idesc, (kb | a | k) != 0 ? 1u : 0u);
+                        for (int k = 0; k < kAtomK / kUmmaK; ++k) {
+                            // next 16 elements along K: 32 bytes further inside the swizzle row
+                            const uint64_t adv = (uint64_t)((k * kUmmaK * 2) >> 4);
+                            umma_bf16(tmem_acc, da + adv, db + adv, idesc, (st | a | k) != 0 ? 1u : 0u);
+                        }
                     }
                 }
                 umma_commit(&ctl->empty[s]);       // stage is free once these MMAs have read it
             }
-            if (ok) umma_commit(&ctl->tmem_full);  // accumulator complete
+            ctl->consumed = st;
+            SPR_STAMP(4);
+            if (fed) {
+                umma_commit(&ctl->tmem_full);      // accumulator complete
+            } else {
+                umma_commit(&ctl->drain);          // what was issued is waited for on the way out
+            }
         }
     } else {
-        // ---------------- epilogue: thread = token, TMEM lane = 32*(warp%4) + lane
-        // BM = 128: accumulator row r lives in TMEM lane r.  BM = 64: the 64 rows use lanes
-        // 0-15 of each 32-lane quarter (row r in lane 32*(r/16) + r%16).
-        const int quarter = warp & 3;
-        const bool has_row = BM == 128 || lane < 16;
-        const int row = m0 + (BM == 128 ? quarter * 32 + lane : quarter * 16 + lane);
-        const bool ok = __all_sync(0xffffffffu, mbar_wait(&ctl->tmem_full, 0, ctl, prm.status));
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (ok) {
-            float z = 0.f;
-#pragma unroll
-            for (int c0 = 0; c0 < BN; c0 += 16) {
-                float v[16];
-                tmem_ld16(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, v);
-#pragma unroll
-                for (int j = 0; j < 16; ++j) z = fmaf(ctl->w2[c0 + j], fmaxf(v[j] + ctl->b1[c0 + j], 0.f), z);
-            }
-            if (has_row && row < M) prm.part_z[(int64_t)blockIdx.x * M + row] = z;
+        // ---------------- epilogue threads: layer-2 constants of this slice into shared memory
+        // (read again only after a barrier below), then wait for the accumulator
+        for (int j = tid - 64; j < BN; j += kTcThreads - 64) {
+            const int n = n0 + j;
+            ctl->b1[j] = n < prm.h ? prm.b1[n] : 0.f;
+            ctl->w2[j] = n < prm.h ? __bfloat162float(static_cast<const __nv_bfloat16 *>(prm.W2)[n]) : 0.f;
         }
+        asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps
+        ok = mbar_wait(&ctl->tmem_full, 0, ctl, prm.status, limit);
+        if (tid == 64) SPR_STAMP(5);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    }
+    __syncwarp();
+
+    // thread = token: TMEM lane 32*(warp%4) + lane.  BM = 128: accumulator row r lives in TMEM
+    // lane r.  BM = 64: the 64 rows use lanes 0-15 of each 32-lane quarter.
+    const int quarter = warp & 3;
+    const int r_in = BM == 128 ? quarter * 32 + lane : quarter * 16 + (lane & 15);   // row inside the tile
+    const int row = m0 + r_in;
+    const bool live_row = warp >= 2 && (BM == 128 || lane < 16) && row < M;
+    const uint32_t lane_base = tmem_acc + ((uint32_t)(quarter * 32) << 16);
+    const float4 *recv4 = reinterpret_cast<const float4 *>(ring);
+
+    // With a split of d: every CTA of the cluster is past its k-loop (its ring is free to
+    // receive) and has started.
+    if (clustered && !early_arrive) cluster_sync();
+    if (tid == 64) SPR_STAMP(6);
+
+    if (S > 1) {
+        // ---------------- accumulator columns to their owners
+        if (warp >= 2) {
+            if (S == 2) send_columns<BM, BN, 2>(lane_base, recv4, split, row_rank0, r_in, live_row);
+            if (S == 4) send_columns<BM, BN, 4>(lane_base, recv4, split, row_rank0, r_in, live_row);
+            if (S == 8) send_columns<BM, BN, 8>(lane_base, recv4, split, row_rank0, r_in, live_row);
+        }
+        cluster_sync();
+    }
+    if (tid == 64) SPR_STAMP(7);
+
+    // ---------------- bias, ReLU, W2 over the columns this CTA owns
+    float z = 0.f;
+    if (warp >= 2) {
+        if (S == 1) {
+#pragma unroll
+            for (int c0 = 0; c0 < BN; c0 += 64) {
+                uint32_t v[2][32];
+                tmem_ld32(lane_base + (uint32_t)c0, v[0]);
+                tmem_ld32(lane_base + (uint32_t)(c0 + 32), v[1]);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 64; ++j)
+                    z = fmaf(ctl->w2[c0 + j], fmaxf(__uint_as_float(v[j >> 5][j & 31]) + ctl->b1[c0 + j], 0.f), z);
+            }
+        } else if (live_row) {
+            if (S == 2) z = owned_columns_z<BM, BN, 2>(recv4, ctl, split, r_in);
+            if (S == 4) z = owned_columns_z<BM, BN, 4>(recv4, ctl, split, r_in);
+            if (S == 8) z = owned_columns_z<BM, BN, 8>(recv4, ctl, split, r_in);
+        }
+        if (!ok || *reinterpret_cast<volatile int *>(&ctl->abort)) z = poisoned_z();
+    }
+    if (tid == 64) SPR_STAMP(8);
+
+    if (early_arrive) cluster_wait();
+    if (prm.final_in_cluster) {
+        if (live_row) {
+            const uint32_t dst = smem_u32(&ctl->zbuf[my_rank][r_in]);
+            st_cluster_f32(clustered ? peer_smem(dst, 0) : dst, z);
+        }
+    } else if (live_row) {
+        prm.part_z[((int64_t)blockIdx.y * S + split) * M + row] = z;
     }
 
-    // ---------------- teardown: release TMEM, then the ticket for the final reduction
+    // ---------------- teardown: nothing in flight, release TMEM
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
+    if (clustered && prm.final_in_cluster) {
+        cluster_sync();      // the partial z of every CTA have arrived; peers may exit
+    } else {
+        __syncthreads();
+    }
+    if (*reinterpret_cast<volatile int *>(&ctl->abort)) {   // the same for every thread by now
+        if (warp == 0) {   // copies issued but never consumed
+            int last = issued;     // a lane may be one stage ahead of lane 0
+#pragma unroll
+            for (int o = 1; o < 8; o <<= 1) last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
+            if (lane == 0) {
+                for (int st = ctl->consumed; st < last; ++st)
+                    mbar_wait_quiet(&ctl->full[st % Cfg::kStages], (uint32_t)(st / Cfg::kStages) & 1u, limit);
+            }
+        }
+        if (warp == 1 && lane == 0 && ctl->consumed < num_stages) mbar_wait_quiet(&ctl->drain, 0, limit);
+        __syncthreads();
+    }
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"((uint32_t)Cfg::kTmemCols)
                      : "memory");
     }
-    // Tickets: the CTA that completes a token tile (all slices written) turns its 128 partial
-    // sums into scores, accept bits and the scan of the sequences inside the tile; sequences
-    // cut by a tile boundary wait for the CTA that completes the last tile.
-    if (tid == 0) {
+
+    if (tid == 64) SPR_STAMP(9);
+    const int m_hi = min(m0 + BM, M);
+    if (prm.final_in_cluster) {
+        // ---------------- the cluster's first CTA finishes the tile out of shared memory
+        if (my_rank != 0) return;
+        const float b2 = prm.b2[0];
+        for (int t = tid; t < m_hi - m0; t += kTcThreads) {
+            float zt = b2;
+            for (int i = 0; i < cluster_ctas; ++i) zt += ctl->zbuf[i][t];
+            ctl->codes[t] = (unsigned char)classify_token(prm, zt, m0 + t);
+        }
+        __syncthreads();
+        if (!prm.first_reject) return;
+        const int b_lo = (m0 + prm.K - 1) / prm.K, b_hi = m_hi / prm.K;
+        for (int b = b_lo + warp; b < b_hi; b += kTcThreads / 32)
+            scan_sequence_smem(prm, b, ctl->codes + (b * prm.K - m0), lane);
+        if (tid == 64) SPR_STAMP(10);
+    } else {
+        // Tickets: the CTA that completes a token tile (all partial sums written) turns them
+        // into scores, accept bits and the scan of the sequences inside the tile.
+        if (tid == 0) {
+            __threadfence();
+            ctl->last = take_ticket(&prm.counter[1 + blockIdx.z], (int)(gridDim.x * gridDim.y));
+        }
+        __syncthreads();
+        if (!ctl->last) return;
         __threadfence();
-        ctl->last = take_ticket(&prm.counter[1 + blockIdx.y], (int)gridDim.x);
+        finalise_tile(prm, m0, m_hi, ctl->codes);
+        if (tid == 64) SPR_STAMP(10);
     }
-    __syncthreads();
-    if (!ctl->last) return;
-    __threadfence();
-    finalise_tile(prm, m0, min(m0 + BM, M));
-    if (BM % prm.K == 0) return;   // no sequence straddles a tile boundary
+    // sequences cut by a tile boundary wait for the CTA that completes the last tile
+    if (BM % prm.K == 0 || gridDim.z == 1) return;
     __syncthreads();
     if (tid == 0) {
         __threadfence();
-        ctl->last = take_ticket(&prm.counter[0], (int)gridDim.y);
+        ctl->last = take_ticket(&prm.counter[0], (int)gridDim.z);
     }
     __syncthreads();
     if (!ctl->last) return;
@@ -330,8 +571,91 @@ bool make_map(CUtensorMap *map, const void *base, int rows, int cols, int box_ro
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+struct Shape {
+    int bm, bn, splits, cluster_n;
+};
+
+int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
+
+// k-blocks per CTA when d is cut S ways, or 0 if some CTA would get none
+int kb_per_split(int d, int S)
+{
+    const int kb_all = ceil_div(d, kAtomK), per = ceil_div(kb_all, S);
+    return (int64_t)(S - 1) * per < kb_all ? per : 0;
+}
+
+bool shape_usable(const Shape &s, int64_t M, int d, int h)
+{
+    if ((s.bm != 64 && s.bm != 128) || (s.bn != 64 && s.bn != 128)) return false;
+    if (s.splits != 1 && s.splits != 2 && s.splits != 4 && s.splits != 8) return false;
+    if (s.bn / s.splits < 8 || kb_per_split(d, s.splits) == 0) return false;
+    const int slices = ceil_div(h, s.bn);
+    if (s.cluster_n != 1 && s.cluster_n != slices) return false;
+    if (s.splits * s.cluster_n > kMaxClusterCtas) return false;
+    if (slices > 65535 || ceil_div(M, s.bm) > 65535) return false;
+    return true;
+}
+
+// Estimated microseconds of a launch with this shape: a model with a handful of constants
+// fitted to CUDA-graph timings of every usable shape on the library's workload sizes (B200).
+//   per CTA: set-up and first data; the k-loop, whose stages each cost the larger of a fixed
+//            barrier/issue latency, the rows they fetch (one 128-byte row per ~2 clocks) and
+//            their tensor-pipe time; the exchange of accumulator columns when d is split;
+//            the epilogue
+//   per launch: waves of clusters (a cluster of c CTAs fits the GPU 148, 74, 33, 15 times for
+//            c = 1, 2, 4, 8) and the finish - cheap inside a cluster, two trips through
+//            global memory otherwise.
+double shape_cost(const Shape &s, int64_t M, int d, int h)
+{
+    const int slices = ceil_div(h, s.bn), tiles = ceil_div(M, s.bm);
+    const int cluster_ctas = s.splits * s.cluster_n;
+    const int64_t clusters = (int64_t)tiles * slices * s.splits / cluster_ctas;
+    const int capacity = cluster_ctas == 1 ? 148 : cluster_ctas == 2 ? 74 : cluster_ctas <= 4 ? 33 : 15;
+    const double waves = (double)((clusters + capacity - 1) / capacity);
+    const int atoms_per_stage = s.bm + s.bn == 128 ? 4 : 2;
+    const int stages = ceil_div(kb_per_split(d, s.splits), atoms_per_stage);
+    const double rows_a = tiles == 1 ? (double)((M + 7) / 8 * 8) : (double)s.bm;
+    const double rows = rows_a + (double)(h < s.bn ? h : s.bn);
+    const double feed = rows * atoms_per_stage * 0.00127;
+    const double mma = (double)s.bm * s.bn * atoms_per_stage * kAtomK / 8192.0 / 1965.0;
+    double stage = 0.364;
+    if (feed > stage) stage = feed;
+    if (mma > stage) stage = mma;
+    const double rows_live = (double)(M < s.bm ? M : s.bm);
+    const double exchange = s.splits > 1 ? 2 * 0.615 + rows_live * s.bn * 4 / 1024.0 * 0.0054 : 0.0;
+    const double finish = s.cluster_n == slices ? 0.615 : 3.22;
+    return waves * (2.48 + stages * stage + exchange + 1.93) + finish;
+}
+
+Shape choose_shape(int64_t M, int d, int h)
+{
+    Shape best = {64, 64, 1, 1};
+    double best_cost = -1.0;
+    for (int bm = 64; bm <= 128; bm += 64) {
+        if (bm == 128 && M <= 64) continue;
+        for (int bn = 64; bn <= 128; bn += 64) {
+            if (bn == 128 && h <= 64) continue;
+            for (int S = 1; S <= 8; S *= 2) {
+                const int slices = ceil_div(h, bn);
+                for (int all = 0; all < 2; ++all) {
+                    const Shape s = {bm, bn, S, all ? slices : 1};
+                    if (all && slices == 1) continue;
+                    if (!shape_usable(s, M, d, h)) continue;
+                    const double c = shape_cost(s, M, d, h);
+                    if (best_cost < 0.0 || c < best_cost) {
+                        best_cost = c;
+                        best = s;
+                    }
+                }
+            }
+        }
+    }
+    return best;
+}
+
 template <int BM, int BN>
-int launch_tile(const CUtensorMap &mh, const CUtensorMap &mw, VerifyParams vp, int tiles_m, cudaStream_t st)
+int launch_tile(const CUtensorMap &mh, const CUtensorMap &mw, VerifyParams vp, const Shape &s, int tiles_m,
+                cudaStream_t st)
 {
     using Cfg = TileCfg<BM, BN>;
     static bool attr_set[64];
@@ -343,51 +667,88 @@ int launch_tile(const CUtensorMap &mh, const CUtensorMap &mw, VerifyParams vp, i
         if (e != cudaSuccess) return (int)e;
         attr_set[dev] = true;
     }
-    vp.slices = (vp.h + BN - 1) / BN;
-    dim3 grid((unsigned)vp.slices, (unsigned)tiles_m);
-    verifier_tcgen05_kernel<BM, BN><<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(mh, mw, vp);
-    return (int)cudaGetLastError();
+    const int slices = ceil_div(vp.h, BN);
+    vp.slices = slices * s.splits;
+    vp.kb_per = kb_per_split(vp.d, s.splits);
+    vp.cluster_n = s.cluster_n;
+    vp.final_in_cluster = s.cluster_n == slices ? 1 : 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)s.splits, (unsigned)slices, (unsigned)tiles_m);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    if (s.splits * s.cluster_n > 1) {
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)s.splits;
+        attr[0].val.clusterDim.y = (unsigned)s.cluster_n;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    return (int)cudaLaunchKernelEx(&cfg, verifier_tcgen05_kernel<BM, BN>, mh, mw, vp);
 }
 
 }  // namespace
 
-int launch_verifier_tensor(const VerifyParams &vp, int dt, int min_tokens, cudaStream_t st)
+#ifdef SPR_VERIFIER_STAMPS
+extern "C" int spr_debug_max_clusters(int cx, int cy)   // co-resident clusters of the 64 x 128 kernel
 {
+    using Cfg = TileCfg<64, 128>;
+    cudaFuncSetAttribute(verifier_tcgen05_kernel<64, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmemBytes);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(cx * 16, cy * 16, 1);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cx;
+    attr[0].val.clusterDim.y = cy;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = -1;
+    cudaError_t e = cudaOccupancyMaxActiveClusters(&n, verifier_tcgen05_kernel<64, 128>, &cfg);
+    return e == cudaSuccess ? n : -(int)e;
+}
+extern "C" int spr_debug_verifier_stamps(long long *host_out)   // [512][64]
+{
+    return (int)cudaMemcpyFromSymbol(host_out, g_stamps, sizeof(long long) * 512 * 64);
+}
+#endif
+
+int verifier_tensor_max_slices(int h) { return ceil_div(h > 0 ? h : 1, 128) * 16; }
+
+int launch_verifier_tensor(const VerifyParams &vp_in, int dt, int min_tokens, const VerifierTune *tune,
+                           cudaStream_t st)
+{
+    VerifyParams vp = vp_in;
     const int64_t M = (int64_t)vp.B * vp.K;
     if (dt != SPR_BF16 || vp.h <= 0 || vp.d % 8 != 0 || M < min_tokens) return -1;
     if ((reinterpret_cast<uintptr_t>(vp.hidden) & 15) || (reinterpret_cast<uintptr_t>(vp.W1) & 15)) return -1;
-    // Measured on B200: a CTA's k-loop costs about the same per tcgen05.mma (140-250 cycles)
-    // whatever the tile shape up to 128 x 128, so time is set by the d/16 instructions each CTA
-    // issues in a row and by how many CTAs run at once.  Take the largest of the four tile
-    // shapes that still gives the GPU about a wave of CTAs; 64 x 64 if none does, 128 x 128
-    // once even that exceeds a wave.
-    auto ctas = [&](int m, int n) { return ((M + m - 1) / m) * (int64_t)((vp.h + n - 1) / n); };
-    static const int kShapes[4][2] = {{128, 128}, {64, 128}, {128, 64}, {64, 64}};
-    int bm = 64, bn = 64;
-    for (const auto &sh : kShapes) {
-        if (ctas(sh[0], sh[1]) >= 96) {
-            bm = sh[0];
-            bn = sh[1];
-            break;
-        }
+    Shape s = choose_shape(M, vp.d, vp.h);
+    vp.spin_limit = kSpinLimit;
+    vp.test_flags = 0;
+    if (tune) {
+        if (tune->bm) s.bm = tune->bm;
+        if (tune->bn) s.bn = tune->bn;
+        if (tune->splits) s.splits = tune->splits;
+        const int slices = ceil_div(vp.h, s.bn);
+        if (tune->cluster_n) s.cluster_n = tune->cluster_n < 0 ? slices : 1;
+        else if (tune->bm || tune->bn || tune->splits) s.cluster_n = s.splits * slices <= kMaxClusterCtas ? slices : 1;
+        if (tune->spin_limit) vp.spin_limit = tune->spin_limit;
+        vp.test_flags = tune->test_flags;
     }
-    // tuning aids: SPR_VERIFIER_BM=64|128, SPR_VERIFIER_BN=64|128
-    if (const char *env = getenv("SPR_VERIFIER_BM")) {
-        const int v = atoi(env);
-        if (v == 64 || v == 128) bm = v;
-    }
-    if (const char *env = getenv("SPR_VERIFIER_BN")) {
-        const int v = atoi(env);
-        if (v == 64 || v == 128) bn = v;
-    }
-    const int64_t tiles64 = (M + bm - 1) / bm;
-    if (tiles64 > 65535) return -1;
-    const int tiles_m = (int)tiles64;
+    if (!shape_usable(s, M, vp.d, vp.h)) return -1;
+    const int tiles_m = ceil_div(M, s.bm);
+    // a batch that fills only part of its one tile fetches only the rows it has (the rest of
+    // the operand tile stays as it is: accumulator rows that are never read)
+    vp.a_box_rows = tiles_m == 1 ? (int)((M + 7) / 8 * 8) : s.bm;
     CUtensorMap mh, mw;
-    if (!make_map(&mh, vp.hidden, (int)M, vp.d, bm)) return -1;
-    if (!make_map(&mw, vp.W1, vp.h, vp.d, bn)) return -1;
+    if (!make_map(&mh, vp.hidden, (int)M, vp.d, vp.a_box_rows)) return -1;
+    if (!make_map(&mw, vp.W1, vp.h, vp.d, s.bn)) return -1;
 #define SPR_TILE(BM_, BN_) \
-    if (bm == BM_ && bn == BN_) return launch_tile<BM_, BN_>(mh, mw, vp, tiles_m, st)
+    if (s.bm == BM_ && s.bn == BN_) return launch_tile<BM_, BN_>(mh, mw, vp, s, tiles_m, st)
     SPR_TILE(64, 64);
     SPR_TILE(64, 128);
     SPR_TILE(128, 64);
