@@ -59,6 +59,9 @@ def parse_args():
     ap.add_argument("--rotate", type=int, default=1,
                     help="1: rotate small workloads through copies that together exceed L2 four times; 0: reuse "
                          "one copy (L2-warm numbers)")
+    ap.add_argument("--graph", default="auto", choices=["auto", "0", "1"],
+                    help="1: the timed steps are replays of CUDA graphs of the step (no host launch cost between "
+                         "kernels); auto: only when a step takes the GPU less time than the host needs to issue it")
     ap.add_argument("--shard", default="batch", choices=["batch", "vocab"],
                     help="how --gpus N ranks split the work: every rank its own batch (default), or every "
                          "rank V/N columns of the same logits (sd_verify only, NCCL exchanges between the passes)")
@@ -79,6 +82,34 @@ def peaks():
             p = json.load(f)
         return float(p["hbm_gbs"]), "measured"
     return 6650.0, "fallback"
+
+
+def tensor_peak():
+    """Dense bf16 TFLOP/s of a kernel timed alone (the burst figure)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["bf16_tflops"]), "measured"
+    return 1590.0, "fallback"
+
+
+# sm__pipe_tensor_cycles_active of verifier_tcgen05_kernel from the ncu capture summarised under
+# profiles/ (a counter that only a profiler gives); reported while the kernel source is unchanged
+NCU_VERIFIER = {
+    "sources": ("verifier_tensor.cu", "verifier_common.cuh"),
+    "sha256": None,
+    "tensor_pipe_pct_while_active": None,
+    "profile": "profiles/draw_kernel_and_verifier_llama3.md",
+}
+
+
+def sources_sha(names):
+    h = hashlib.sha256()
+    for name in names:
+        with open(os.path.join(ROOT, "paper_2502_04557_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
 
 
 class ClockSampler:
@@ -470,24 +501,82 @@ def main():
     assert ws.device_status() == 0 and ws_sd.device_status() == 0
 
     nsteps = args.steps
-    stage = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(nsteps)]
+    # Does the host keep up?  A short eager probe: if a step takes the GPU less time than the
+    # host needs to issue its two calls, the timed steps are replays of CUDA graphs of the step,
+    # so that the number is about the kernels and not about the Python interpreter.
+    use_graph = args.graph == "1"
+    if args.graph == "auto":
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        a.record()
+        fork()
+        for _ in range(20):
+            step()
+        join()
+        b.record()
+        host_ms = (time.perf_counter() - t0) * 1e3 / 20     # time the host took to issue a step
+        torch.cuda.synchronize()
+        use_graph = a.elapsed_time(b) / 20 < 1.3 * host_ms
+
+    def capture(n):
+        """n consecutive steps (both streams forked once, joined once) as one CUDA graph."""
+        cap = torch.cuda.Stream(device=dev)
+        cap.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=cap):
+            fork()
+            for _ in range(n):
+                step()
+            join()
+        torch.cuda.current_stream().wait_stream(cap)
+        return graph
+
+    stage = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+             for _ in range(min(nsteps, 50) if use_graph else nsteps)]
     for a, b in stage:          # create the handles
         a.record()
         b.record()
+    graphs = []
+    if use_graph:
+        per_graph = n_copies if n_copies > 1 else min(nsteps, 20)
+        turn[0] = 0
+        if nsteps // per_graph:
+            graphs.append((capture(per_graph), nsteps // per_graph))
+        if nsteps % per_graph:
+            graphs.append((capture(nsteps % per_graph), 1))
+        for g, _ in graphs:
+            g.replay()
+        torch.cuda.synchronize()
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     t_wall0 = time.time()
     start.record()
-    fork()
-    for i in range(nsteps):
-        spr.set_stage_events(*stage[i])
-        step()
-    join()
+    if use_graph:
+        for g, times in graphs:
+            for _ in range(times):
+                g.replay()
+    else:
+        fork()
+        for i in range(nsteps):
+            spr.set_stage_events(*stage[i])
+            step()
+        join()
     stop.record()
     spr.set_stage_events(None, None)
     barrier()
     t_wall1 = time.time()
     elapsed_ms = start.elapsed_time(stop)
+    if use_graph:
+        # event pairs cannot be read back from inside a graph: the launch time of the dominant
+        # kernel comes from an eager pass over the same rotation of inputs right after
+        fork()
+        for i in range(len(stage)):
+            spr.set_stage_events(*stage[i])
+            step()
+        join()
+        spr.set_stage_events(None, None)
+        torch.cuda.synchronize()
     if world > 1:
         t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -611,9 +700,14 @@ def main():
     t_sd = time_call(lambda: spr.sd_verify(wl.p_logits, wl.q_logits, V, wl.draft_tokens, wl.uniforms, ws, out=sd_out))
     n_rej = int((fr < K).sum())
     kept = float(fr.float().sum())          # draft tokens the verifier kept
+    ver_flops = 2.0 * M * cfg.d * cfg.h if cfg.h else 2.0 * M * cfg.d
     calls = {
-        "sprinter_verify": {"ms": t_ver, "verified_tokens_per_s": M / (t_ver * 1e-3)},
-        "replace_sample": {"ms": t_rep, "draws": n_rej},
+        "sprinter_verify": {"ms": t_ver, "verified_tokens_per_s": M / (t_ver * 1e-3), "flops": ver_flops,
+                            "tflops": ver_flops / (t_ver * 1e-3) / 1e12,
+                            "bytes": int((wl.hidden.numel() + wl.W1.numel()) * es),
+                            "gbs": (wl.hidden.numel() + wl.W1.numel()) * es / (t_ver * 1e-3) / 1e9},
+        "replace_sample": {"ms": t_rep, "draws": n_rej, "bytes": int(n_rej * V * es),
+                           "gbs": n_rej * V * es / (t_rep * 1e-3) / 1e9},
         "sprinter_step": {"ms": t_stp, "verified_tokens_per_s": M / (t_stp * 1e-3),
                           "emitted_tokens_per_s": (kept + n_rej) / (t_stp * 1e-3),
                           "bytes": int(wl.hidden.numel() * es + wl.W1.numel() * es + n_rej * V * es)},
@@ -692,6 +786,23 @@ def main():
                      "roofline": {"bound": "alu", "achieved": int_ops / (ms * 1e-3) / 1e12, "peak": alu_peak / 1e12,
                                   "unit": "Tlane-op/s", "frac": int_ops / (ms * 1e-3) / alu_peak}}
 
+    # the two other kernels of the path against their rooflines (each timed alone: graph replays above)
+    tpeak, tpeak_kind = tensor_peak()
+    pipe_pct = None
+    if NCU_VERIFIER["sha256"] == sources_sha(NCU_VERIFIER["sources"]):
+        pipe_pct = NCU_VERIFIER["tensor_pipe_pct_while_active"]
+    roofline_verifier = {
+        "bound": "tensor", "kernel": "verifier_tcgen05_kernel" if dt_code == spr.BF16 and cfg.h else "verifier (SIMT)",
+        "achieved": calls["sprinter_verify"]["tflops"], "peak": tpeak, "unit": "TFLOP/s",
+        "frac": calls["sprinter_verify"]["tflops"] / tpeak, "peak_kind": f"of {tpeak_kind} (burst: kernel timed alone)",
+        "flops_per_launch": ver_flops, "avg_launch_ms": t_ver, "timing": "CUDA-graph replay of 20 calls, inputs L2-warm",
+        "tensor_pipe_pct_while_active": pipe_pct, "tensor_pipe_source": NCU_VERIFIER["profile"] if pipe_pct else None}
+    roofline_draw = {
+        "bound": "hbm", "kernel": "draw_kernel (replacement draws)", "achieved": calls["replace_sample"]["gbs"], "peak": peak,
+        "unit": "GB/s", "frac": calls["replace_sample"]["gbs"] / peak, "peak_kind": f"of {peak_kind}",
+        "algorithmic_bytes_per_launch": calls["replace_sample"]["bytes"], "avg_launch_ms": t_rep, "draws": n_rej,
+        "timing": "CUDA-graph replay of 20 calls" + ("" if n_rej * V * es > 126 << 20 else ", rows L2-warm")}
+
     inputs_sha = None
     if rank == 0:
         h = hashlib.sha256()     # the realised tensors are the inputs, not the generator
@@ -709,6 +820,9 @@ def main():
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16"
             if cfg.dtype == torch.bfloat16 else "f32", "data": "synthetic",
             "config": {"workload": workload_label(wl), "step": "sd_verify (stream 1) || sprinter_step = sprinter_verify + gated replace_sample (stream 2)",
+                       "timed_region": (f"CUDA-graph replays of the step ({'+'.join(str(t) for _, t in graphs)} replays); "
+                                        "row-statistics launch time from an eager pass after it") if use_graph else
+                                       "eager calls",
                        "l2": (f"inputs per step ({(alg_bytes + wl.p_logits[:, K:].numel() * es) / 1e9:.2f} GB of logits) "
                               "exceed the 126 MB L2; no flush needed") if n_copies == 1 and step_bytes > 126 << 20 else
                              (f"steps rotate through {n_copies} copies of the inputs ({n_copies * step_bytes / 1e6:.0f} MB "
@@ -720,6 +834,11 @@ def main():
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                          "traffic": traffic, "algorithmic_bytes_per_launch": alg_bytes,
                          "avg_launch_ms": stats_ms},
+            "roofline_verifier": roofline_verifier, "roofline_draw": roofline_draw,
+            "sprinter_step_tokens_per_s": calls["sprinter_step"]["verified_tokens_per_s"],
+            "sd_verify_tokens_per_s": calls["sd_verify"]["verified_tokens_per_s"],
+            "value_is": "draft tokens per second through one step = sd_verify and sprinter_step of the same tokens, "
+                        "run side by side; each path alone is in sprinter_step_tokens_per_s / sd_verify_tokens_per_s",
             "cpu_baseline": cpu_baseline, "calls": calls,
             **({"simulator": simulator} if simulator else {}),
         }))

@@ -170,7 +170,7 @@ size_t spr_workspace_bytes(int op, int B, int K, int V, int d, int h, int dt)
     switch (op) {
     case SPR_OP_SPRINTER_VERIFY:
         if (K <= 0 || d <= 0 || h < 0 || (int64_t)B * K > 0x7fffffff) return 0;
-        return ws_bytes_of([&](Carver &c) { verify_ws_layout(c, B * K, verify_slices(h), verify_counters(B, K)); });
+        return ws_bytes_of([&](Carver &c) { verify_ws_layout(c, B * K, K, verify_slices(h), verify_counters(B, K)); });
     case SPR_OP_REPLACE_SAMPLE:
         if (V <= 0) return 0;
         return ws_bytes_of([&](Carver &c) { draw_ws_layout(c, B, stat_steps_per_row(V, dt)); });
@@ -216,13 +216,14 @@ int sprinter_verify(const void *hidden, const void *W1, const float *b1, const v
     int rc = check_verify_args(vp, dt, path);
     if (rc != SPR_OK || B == 0) return rc;  // empty batch: nothing to read or write
     Carver cv = carve(ws_bytes);
-    const VerifyWs lay = verify_ws_layout(cv, B * K, verify_slices(h), verify_counters(B, K));
+    const VerifyWs lay = verify_ws_layout(cv, B * K, K, verify_slices(h), verify_counters(B, K));
     if (!ws || !aligned(ws, 256) || !cv.fits()) return SPR_ERR_WORKSPACE;
     if ((rc = check_device()) != SPR_OK) return rc;
 
     vp.status = at<int>(ws, 0);
     vp.counter = at<int>(ws, lay.counter);
     vp.part_z = at<float>(ws, lay.part_z);
+    vp.zacc = K == 1 ? at<unsigned long long>(ws, lay.zacc) : nullptr;
     return launch_verifier(vp, dt, path, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -236,13 +237,14 @@ int spr_test_sprinter_verify(const void *hidden, const void *W1, const float *b1
     int rc = check_verify_args(vp, dt, SPR_VERIFIER_TENSOR);
     if (rc != SPR_OK || B == 0) return rc;
     Carver cv = carve(ws_bytes);
-    const VerifyWs lay = verify_ws_layout(cv, B * K, verify_slices(h), verify_counters(B, K));
+    const VerifyWs lay = verify_ws_layout(cv, B * K, K, verify_slices(h), verify_counters(B, K));
     if (!ws || !aligned(ws, 256) || !cv.fits()) return SPR_ERR_WORKSPACE;
     if ((rc = check_device()) != SPR_OK) return rc;
     VerifierTune tune = {bm, bn, splits, cluster_n, flags, spin_limit};
     vp.status = at<int>(ws, 0);
     vp.counter = at<int>(ws, lay.counter);
     vp.part_z = at<float>(ws, lay.part_z);
+    vp.zacc = K == 1 ? at<unsigned long long>(ws, lay.zacc) : nullptr;
     return launch_verifier(vp, dt, SPR_VERIFIER_TENSOR, static_cast<cudaStream_t>(cuda_stream), &tune);
 }
 
@@ -289,6 +291,7 @@ int sprinter_step(const void *hidden, const void *W1, const float *b1, const voi
     vp.status = dp.status = at<int>(ws, 0);
     vp.counter = at<int>(ws, lay.verify.counter);
     vp.part_z = at<float>(ws, lay.verify.part_z);
+    vp.zacc = K == 1 ? at<unsigned long long>(ws, lay.verify.zacc) : nullptr;
     dp.counters = at<int>(ws, lay.draw.counters);
     dp.part = at<float2>(ws, lay.draw.part);
     // the draw is launched behind the verifier

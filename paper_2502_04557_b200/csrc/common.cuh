@@ -189,12 +189,15 @@ __host__ __device__ inline size_t train_ws_layout(Carver &c, int d)
 }
 
 struct VerifyWs {
+    size_t zacc;             // uint64 [M], K = 1 only (ticket zone, first: 8-byte aligned): per-token sum of
+                             //   partial logits in fixed point with an arrival count; zero between launches
     size_t counter;          // int32 [1 + tickets]   (ticket zone) see verify_tickets()
     size_t part_z;           // float [slices * M]    per-slice partial of W2 . relu(...)
 };
-__host__ __device__ inline VerifyWs verify_ws_layout(Carver &c, int M, int slices, int tickets)
+__host__ __device__ inline VerifyWs verify_ws_layout(Carver &c, int M, int K, int slices, int tickets)
 {
     VerifyWs w;
+    w.zacc = K == 1 ? c.take_tickets(2 * (size_t)M) : 0;
     w.counter = c.take_tickets(1 + (size_t)tickets);
     w.part_z = c.take_data(4 * (size_t)slices * M);
     return w;
@@ -207,7 +210,7 @@ struct StepWs {              // sprinter_step: verifier and replacement draw in 
 __host__ __device__ inline StepWs step_ws_layout(Carver &c, int B, int K, int slices, int tickets, int T)
 {
     StepWs w;
-    w.verify = verify_ws_layout(c, B * K, slices, tickets);
+    w.verify = verify_ws_layout(c, B * K, K, slices, tickets);
     w.draw = draw_ws_layout(c, B, T);
     return w;
 }

@@ -119,12 +119,16 @@ struct VerifyParams {
     int *status;
     int *counter;
     float *part_z;  // [slices*M]
+    unsigned long long *zacc;   // [M] when K == 1, else null (see VerifyWs)
     int slices;
     // tensor-core kernel only
     int kb_per;             // 64-element blocks of d each of the CTAs that share a tile takes
+    int ring_stages;        // pipeline stages in use
+    int recv_dedicated;     // the exchanged accumulator columns have room of their own beside the ring
     int a_box_rows;         // rows of hidden states one copy fetches (the tile height, or fewer for a small batch)
     int cluster_n;          // hidden-unit slices of one token tile per cluster (1, or all of them)
     int final_in_cluster;   // the CTAs of a token tile form one cluster: no tickets, no part_z
+    int atomic_finish;      // K = 1, finish through zacc: one 64-bit atomic per token and slice
     uint32_t spin_limit;    // polls after which a bounded wait gives up
     int test_flags;         // VERIFIER_TEST_*
 };

@@ -9,14 +9,19 @@
 // Grid (S, slices, tiles): a CTA computes a BM-token x BN-hidden-unit tile over one of S equal
 // ranges of d.  The S CTAs of a tile form a cluster (along x) and add their accumulators
 // through distributed shared memory BEFORE the ReLU: CTA r receives, from every CTA of the
-// tile, the BN/S accumulator columns it owns, adds them in CTA order and applies bias, ReLU
-// and W2 to those columns.  Small batches thereby spread the sweep over W1 (the only real
-// traffic they have) over many SMs.
+// tile, the BN/S accumulator columns it owns (asynchronous remote stores that count bytes on
+// the receiver's mbarrier), adds them in CTA order and applies bias, ReLU and W2 to those
+// columns.  Small batches thereby spread the sweep over W1 (the only real traffic they
+// have) over many SMs.  The per-token partial z of the S CTAs go, the same way, to the CTA
+// with split 0, which adds them in order.
 // Where S x slices <= 8 the cluster also spans the hidden-unit slices of the tile (along y):
-// every CTA sends its per-token partial z to the cluster's first CTA, which adds them in
-// rank order, applies sigmoid and threshold and scans the sequences inside the tile out of
-// shared memory - no trip through global memory.  Otherwise the partial z go to the
-// workspace and the CTA that takes the tile's last ticket finishes it.
+// every CTA sends its partial z to the cluster's first CTA, which adds them in rank order,
+// applies sigmoid and threshold and scans the sequences inside the tile out of shared memory
+// - no trip through global memory.  Otherwise one partial z per slice goes to the workspace
+// and the CTA that takes the tile's last ticket finishes it.
+// Cluster barriers are used only as handshakes whose two halves lie far apart: "started"
+// (arrive at the start, wait before the first remote store) and "done with my peers" (arrive
+// when nothing more is sent or expected, wait before exit), so nobody stands at one.
 //
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
 // warps 2..5 = epilogue (warp w reads TMEM lanes 32*(w%4) .. +31).
@@ -60,6 +65,8 @@ struct Control {                 // lives behind the ring in dynamic shared memo
     uint64_t empty[kMaxStages];
     uint64_t tmem_full;
     uint64_t drain;
+    uint64_t xchg;               // counts the bytes of accumulator columns received from the tile's CTAs
+    uint64_t zgather;            // counts the bytes of partial z received (receiving CTA only)
     uint32_t tmem_base;
     int abort;
     int last;
@@ -202,28 +209,34 @@ __device__ __forceinline__ uint32_t peer_smem(uint32_t saddr, uint32_t rank)
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v)
+// Asynchronous stores into a peer's shared memory; each adds its size to the transaction count
+// of the mbarrier `bar` (an address in the same peer), whose waiters then see the data.
+__device__ __forceinline__ void st_async_b32(uint32_t addr, uint32_t v, uint32_t bar)
 {
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(addr), "r"(v), "r"(bar)
+                 : "memory");
 }
-__device__ __forceinline__ void st_cluster_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+__device__ __forceinline__ void st_async_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t bar)
 {
-    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d)
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(addr),
+                 "r"(a), "r"(b), "r"(c), "r"(d), "r"(bar)
                  : "memory");
 }
 
 // One epilogue thread (= accumulator row r_in): its BN accumulator columns, four at a time, to
 // the CTAs that own them.  Receiver layout: recv4[source split][group of 4 owned columns][row].
 template <int BM, int BN, int S>
-__device__ __forceinline__ void send_columns(uint32_t lane_base, const float4 *recv4, int split, uint32_t row_rank0,
-                                             int r_in, bool live_row)
+__device__ __forceinline__ void send_columns(uint32_t lane_base, const float4 *recv4, uint64_t *xchg, int split,
+                                             uint32_t row_rank0, int r_in, bool live_row)
 {
     constexpr int kColsPer = BN / S, kGroups = kColsPer / 4;
     static_assert(kColsPer >= 8 && kColsPer % 4 == 0, "columns per owner");
-    uint32_t base[S];    // where this CTA's block of rows starts in every owner's buffer
+    uint32_t base[S], bar[S];    // where this CTA's block of rows starts in every owner's buffer; its mbarrier
 #pragma unroll
-    for (int o = 0; o < S; ++o)
+    for (int o = 0; o < S; ++o) {
         base[o] = peer_smem(smem_u32(recv4 + ((size_t)split * kGroups * BM + r_in)), row_rank0 + (uint32_t)o);
+        bar[o] = peer_smem(smem_u32(xchg), row_rank0 + (uint32_t)o);
+    }
 #pragma unroll
     for (int c0 = 0; c0 < BN; c0 += 32) {
         uint32_t r[32];
@@ -234,7 +247,8 @@ __device__ __forceinline__ void send_columns(uint32_t lane_base, const float4 *r
             for (int g = 0; g < 8; ++g) {
                 const int c = c0 + 4 * g;
                 const int owner = c / kColsPer, cg = (c % kColsPer) / 4;
-                st_cluster_v4(base[owner] + (uint32_t)(cg * BM * 16), r[4 * g], r[4 * g + 1], r[4 * g + 2], r[4 * g + 3]);
+                st_async_v4(base[owner] + (uint32_t)(cg * BM * 16), r[4 * g], r[4 * g + 1], r[4 * g + 2], r[4 * g + 3],
+                            bar[owner]);
             }
         }
     }
@@ -267,6 +281,28 @@ __device__ __forceinline__ float owned_columns_z(const float4 *recv4, const Cont
     return z;
 }
 
+// K = 1 (one token per sequence, so a token can be finished on its own): a slice's partial
+// logit is added to the token's 64-bit word with ONE atomic - bits 0-7 count the slices that
+// have arrived, bits 8-15 those that arrived poisoned, bits 16-63 hold the sum in fixed point
+// (2^-24; a partial is clamped to +-32768, far beyond where the sigmoid saturates).  Integer
+// addition commutes, so the sum does not depend on who comes first; the thread whose addition
+// completes the count holds the whole sum in its register, finishes the token and sets the
+// word back to zero.  No fence, no ticket, no second trip to read partial sums.
+__device__ __forceinline__ void add_partial_and_finish(const VerifyParams &prm, float z, int m, int slices)
+{
+    const bool bad = !(z == z);
+    const float zc = fminf(fmaxf(bad ? 0.f : z, -32768.f), 32768.f);
+    const long long fix = __double2ll_rn((double)zc * 16777216.0);
+    const unsigned long long add = ((unsigned long long)fix << 16) + (bad ? 0x101ull : 0x1ull);
+    const unsigned long long now = atomicAdd(&prm.zacc[m], add) + add;
+    if ((int)(now & 0xffull) != slices) return;
+    *reinterpret_cast<volatile unsigned long long *>(&prm.zacc[m]) = 0ull;
+    const bool poisoned = ((now >> 8) & 0xffull) != 0ull;
+    const double zsum = (double)((long long)now >> 16) * (1.0 / 16777216.0) + (double)prm.b2[0];
+    const int a = classify_token(prm, poisoned ? poisoned_z() : (float)zsum, m);
+    if (prm.first_reject) prm.first_reject[m] = a == ACC_INVALID ? -1 : (a == ACC_ACCEPT ? 1 : 0);
+}
+
 template <int BM, int BN>
 __global__ void __launch_bounds__(kTcThreads, 1)
 verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w,
@@ -294,6 +330,13 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
     const uint32_t my_rank = (uint32_t)split + (blockIdx.y % (unsigned)prm.cluster_n) * (uint32_t)S;
     const uint32_t row_rank0 = my_rank - (uint32_t)split;
     const uint32_t limit = prm.spin_limit;
+    const int ring_stages = prm.ring_stages;     // the last stage's room may be lent to the exchange
+    const int live_rows = min(BM, M - m0);       // tokens of this tile
+    // which CTA adds up partial z: the cluster's first CTA when the cluster holds the whole
+    // tile, else the tile's CTA with split 0 (nobody when d is not split)
+    const bool gather_z = clustered;
+    const uint32_t z_rank = prm.final_in_cluster ? 0u : row_rank0;
+    const int z_sources = prm.final_in_cluster ? cluster_ctas : S;
 
     if (tid == 0) {
         for (int s = 0; s < Cfg::kStages; ++s) {
@@ -302,6 +345,11 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
         }
         mbar_init(&ctl->tmem_full, 1);
         mbar_init(&ctl->drain, 1);
+        mbar_init(&ctl->xchg, 1);
+        mbar_init(&ctl->zgather, 1);
+        // what this CTA is going to receive from its peers (and from itself)
+        if (S > 1) mbar_expect_tx(&ctl->xchg, (uint32_t)(live_rows * BN * 4));
+        if (gather_z && my_rank == z_rank) mbar_expect_tx(&ctl->zgather, (uint32_t)(z_sources * live_rows * 4));
         ctl->abort = 0;
         ctl->last = 0;
         ctl->consumed = 0;
@@ -320,10 +368,11 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_acc = ctl->tmem_base;
     if (tid == 0) SPR_STAMP(1);
-    // A peer's shared memory may be written once that CTA has started.  Without a split of d
-    // nothing else has to be waited for, so each thread says "started" here and checks for
-    // everybody's word only where the first remote store is made.
-    const bool early_arrive = clustered && S == 1;
+    // A peer's shared memory may be written once that CTA has started and set up its
+    // barriers: each thread says so here and checks for everybody's word only where the first
+    // remote store is made.  Where the exchange buffer overlays the ring, the peers must be
+    // through their k-loops as well: that handshake is made in one piece after the loop.
+    const bool early_arrive = clustered && (S == 1 || prm.recv_dedicated);
     if (early_arrive) cluster_arrive();
 
     int issued = 0;       // producer: stages whose copies are on their way
@@ -340,8 +389,8 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
                                       : (uint32_t)(atom * Cfg::kBytesA);
             const uint32_t atom_bytes = (uint32_t)prm.a_box_rows * (kAtomK * 2) + (uint32_t)Cfg::kBytesB;
             for (int st = 0; st < num_stages; ++st) {
-                const int s = st % Cfg::kStages;
-                const uint32_t round = (uint32_t)(st / Cfg::kStages);
+                const int s = st % ring_stages;
+                const uint32_t round = (uint32_t)(st / ring_stages);
                 const int n_at = min(Cfg::kAtoms, num_atoms - st * Cfg::kAtoms);
                 if (!mbar_wait(&ctl->empty[s], (round & 1u) ^ 1u, ctl, prm.status, limit)) break;
                 if (lane == 0) mbar_expect_tx(&ctl->full[s], (uint32_t)n_at * atom_bytes);
@@ -360,8 +409,8 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
             bool fed = true;
             int st = 0;
             for (; st < num_stages; ++st) {
-                const int s = st % Cfg::kStages;
-                const uint32_t round = (uint32_t)(st / Cfg::kStages);
+                const int s = st % ring_stages;
+                const uint32_t round = (uint32_t)(st / ring_stages);
                 const int n_at = min(Cfg::kAtoms, num_atoms - st * Cfg::kAtoms);
                 fed = mbar_wait(&ctl->full[s], round & 1u, ctl, prm.status, limit);
                 if (!fed) break;
@@ -415,21 +464,21 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
     const int row = m0 + r_in;
     const bool live_row = warp >= 2 && (BM == 128 || lane < 16) && row < M;
     const uint32_t lane_base = tmem_acc + ((uint32_t)(quarter * 32) << 16);
-    const float4 *recv4 = reinterpret_cast<const float4 *>(ring);
+    const float4 *recv4 = reinterpret_cast<const float4 *>(
+        ring + (prm.recv_dedicated ? (size_t)ring_stages * Cfg::kStageBytes : 0));
 
-    // With a split of d: every CTA of the cluster is past its k-loop (its ring is free to
-    // receive) and has started.
-    if (clustered && !early_arrive) cluster_sync();
+    if (clustered) {
+        if (early_arrive) cluster_wait();
+        else cluster_sync();
+    }
     if (tid == 64) SPR_STAMP(6);
 
-    if (S > 1) {
-        // ---------------- accumulator columns to their owners
-        if (warp >= 2) {
-            if (S == 2) send_columns<BM, BN, 2>(lane_base, recv4, split, row_rank0, r_in, live_row);
-            if (S == 4) send_columns<BM, BN, 4>(lane_base, recv4, split, row_rank0, r_in, live_row);
-            if (S == 8) send_columns<BM, BN, 8>(lane_base, recv4, split, row_rank0, r_in, live_row);
-        }
-        cluster_sync();
+    if (S > 1 && warp >= 2) {
+        // ---------------- accumulator columns to their owners; then wait for the columns owned here
+        if (S == 2) send_columns<BM, BN, 2>(lane_base, recv4, &ctl->xchg, split, row_rank0, r_in, live_row);
+        if (S == 4) send_columns<BM, BN, 4>(lane_base, recv4, &ctl->xchg, split, row_rank0, r_in, live_row);
+        if (S == 8) send_columns<BM, BN, 8>(lane_base, recv4, &ctl->xchg, split, row_rank0, r_in, live_row);
+        ok &= mbar_wait(&ctl->xchg, 0, ctl, prm.status, limit);
     }
     if (tid == 64) SPR_STAMP(7);
 
@@ -456,23 +505,39 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
     }
     if (tid == 64) SPR_STAMP(8);
 
-    if (early_arrive) cluster_wait();
-    if (prm.final_in_cluster) {
+    // ---------------- partial z to whoever adds them up
+    const bool z_receiver = my_rank == z_rank;
+    if (gather_z) {
         if (live_row) {
-            const uint32_t dst = smem_u32(&ctl->zbuf[my_rank][r_in]);
-            st_cluster_f32(clustered ? peer_smem(dst, 0) : dst, z);
+            const int src = prm.final_in_cluster ? (int)my_rank : split;
+            st_async_b32(peer_smem(smem_u32(&ctl->zbuf[src][r_in]), z_rank), __float_as_uint(z),
+                         peer_smem(smem_u32(&ctl->zgather), z_rank));
         }
+        if (z_receiver && warp >= 2) {
+            const bool got = mbar_wait(&ctl->zgather, 0, ctl, prm.status, limit);
+            if (!prm.final_in_cluster && live_row) {   // one partial per slice leaves the cluster
+                float zs = 0.f;
+                for (int i = 0; i < z_sources; ++i) zs += ctl->zbuf[i][r_in];
+                if (!got) zs = poisoned_z();
+                if (prm.atomic_finish) add_partial_and_finish(prm, zs, row, (int)gridDim.y);
+                else prm.part_z[(int64_t)blockIdx.y * M + row] = zs;
+            } else if (!got && live_row) {
+                ctl->zbuf[0][r_in] = poisoned_z();
+            }
+        }
+    } else if (prm.final_in_cluster) {      // a tile with a single CTA
+        if (live_row) ctl->zbuf[0][r_in] = z;
     } else if (live_row) {
-        prm.part_z[((int64_t)blockIdx.y * S + split) * M + row] = z;
+        if (prm.atomic_finish) add_partial_and_finish(prm, z, row, (int)gridDim.y);
+        else prm.part_z[(int64_t)blockIdx.y * M + row] = z;
     }
+    __syncwarp();
+    // this CTA sends nothing more and expects nothing more: its peers may leave
+    if (clustered) cluster_arrive();
 
     // ---------------- teardown: nothing in flight, release TMEM
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    if (clustered && prm.final_in_cluster) {
-        cluster_sync();      // the partial z of every CTA have arrived; peers may exit
-    } else {
-        __syncthreads();
-    }
+    __syncthreads();
     if (*reinterpret_cast<volatile int *>(&ctl->abort)) {   // the same for every thread by now
         if (warp == 0) {   // copies issued but never consumed
             int last = issued;     // a lane may be one stage ahead of lane 0
@@ -480,7 +545,7 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
             for (int o = 1; o < 8; o <<= 1) last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
             if (lane == 0) {
                 for (int st = ctl->consumed; st < last; ++st)
-                    mbar_wait_quiet(&ctl->full[st % Cfg::kStages], (uint32_t)(st / Cfg::kStages) & 1u, limit);
+                    mbar_wait_quiet(&ctl->full[st % ring_stages], (uint32_t)(st / ring_stages) & 1u, limit);
             }
         }
         if (warp == 1 && lane == 0 && ctl->consumed < num_stages) mbar_wait_quiet(&ctl->drain, 0, limit);
@@ -491,48 +556,55 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"((uint32_t)Cfg::kTmemCols)
                      : "memory");
     }
-
     if (tid == 64) SPR_STAMP(9);
+
+    // ---------------- finish: the receiver of the partial z when the cluster holds the whole
+    // tile, else whoever takes the tile's last ticket (one ticket per slice)
     const int m_hi = min(m0 + BM, M);
+    bool finisher = false;
     if (prm.final_in_cluster) {
-        // ---------------- the cluster's first CTA finishes the tile out of shared memory
-        if (my_rank != 0) return;
-        const float b2 = prm.b2[0];
-        for (int t = tid; t < m_hi - m0; t += kTcThreads) {
-            float zt = b2;
-            for (int i = 0; i < cluster_ctas; ++i) zt += ctl->zbuf[i][t];
-            ctl->codes[t] = (unsigned char)classify_token(prm, zt, m0 + t);
+        finisher = z_receiver;
+        if (finisher) {
+            const float b2 = prm.b2[0];
+            for (int t = tid; t < m_hi - m0; t += kTcThreads) {
+                float zt = b2;
+                for (int i = 0; i < z_sources; ++i) zt += ctl->zbuf[i][t];
+                ctl->codes[t] = (unsigned char)classify_token(prm, zt, m0 + t);
+            }
+            __syncthreads();
+            if (prm.first_reject) {
+                const int b_lo = (m0 + prm.K - 1) / prm.K, b_hi = m_hi / prm.K;
+                for (int b = b_lo + warp; b < b_hi; b += kTcThreads / 32)
+                    scan_sequence_smem(prm, b, ctl->codes + (b * prm.K - m0), lane);
+            }
         }
-        __syncthreads();
-        if (!prm.first_reject) return;
-        const int b_lo = (m0 + prm.K - 1) / prm.K, b_hi = m_hi / prm.K;
-        for (int b = b_lo + warp; b < b_hi; b += kTcThreads / 32)
-            scan_sequence_smem(prm, b, ctl->codes + (b * prm.K - m0), lane);
-        if (tid == 64) SPR_STAMP(10);
-    } else {
-        // Tickets: the CTA that completes a token tile (all partial sums written) turns them
-        // into scores, accept bits and the scan of the sequences inside the tile.
+    } else if (!prm.atomic_finish && (!gather_z || z_receiver)) {
         if (tid == 0) {
             __threadfence();
-            ctl->last = take_ticket(&prm.counter[1 + blockIdx.z], (int)(gridDim.x * gridDim.y));
+            ctl->last = take_ticket(&prm.counter[1 + blockIdx.z], (int)gridDim.y);
         }
         __syncthreads();
-        if (!ctl->last) return;
-        __threadfence();
-        finalise_tile(prm, m0, m_hi, ctl->codes);
-        if (tid == 64) SPR_STAMP(10);
+        finisher = ctl->last != 0;
+        if (finisher) {
+            __threadfence();
+            finalise_tile(prm, m0, m_hi, ctl->codes);
+        }
     }
+    if (tid == 64) SPR_STAMP(10);
     // sequences cut by a tile boundary wait for the CTA that completes the last tile
-    if (BM % prm.K == 0 || gridDim.z == 1) return;
-    __syncthreads();
-    if (tid == 0) {
-        __threadfence();
-        ctl->last = take_ticket(&prm.counter[0], (int)gridDim.z);
+    if (finisher && BM % prm.K != 0 && gridDim.z > 1) {
+        __syncthreads();
+        if (tid == 0) {
+            __threadfence();
+            ctl->last = take_ticket(&prm.counter[0], (int)gridDim.z);
+        }
+        __syncthreads();
+        if (ctl->last) {
+            __threadfence();
+            finalise_straddlers(prm, BM);
+        }
     }
-    __syncthreads();
-    if (!ctl->last) return;
-    __threadfence();
-    finalise_straddlers(prm, BM);
+    if (clustered) cluster_wait();   // no peer is still sending to this CTA
 }
 
 // ---------------------------------------------------------------- host side
@@ -605,7 +677,7 @@ bool shape_usable(const Shape &s, int64_t M, int d, int h)
 //   per launch: waves of clusters (a cluster of c CTAs fits the GPU 148, 74, 33, 15 times for
 //            c = 1, 2, 4, 8) and the finish - cheap inside a cluster, two trips through
 //            global memory otherwise.
-double shape_cost(const Shape &s, int64_t M, int d, int h)
+double shape_cost(const Shape &s, int64_t M, int K, int d, int h)
 {
     const int slices = ceil_div(h, s.bn), tiles = ceil_div(M, s.bm);
     const int cluster_ctas = s.splits * s.cluster_n;
@@ -613,21 +685,29 @@ double shape_cost(const Shape &s, int64_t M, int d, int h)
     const int capacity = cluster_ctas == 1 ? 148 : cluster_ctas == 2 ? 74 : cluster_ctas <= 4 ? 33 : 15;
     const double waves = (double)((clusters + capacity - 1) / capacity);
     const int atoms_per_stage = s.bm + s.bn == 128 ? 4 : 2;
+    const int stage_bytes = atoms_per_stage * (s.bm + s.bn) * kAtomK * 2;
+    const int ring = (200 * 1024) / stage_bytes;
     const int stages = ceil_div(kb_per_split(d, s.splits), atoms_per_stage);
     const double rows_a = tiles == 1 ? (double)((M + 7) / 8 * 8) : (double)s.bm;
     const double rows = rows_a + (double)(h < s.bn ? h : s.bn);
-    const double feed = rows * atoms_per_stage * 0.00127;
+    const double feed = rows * atoms_per_stage * 0.00135;
     const double mma = (double)s.bm * s.bn * atoms_per_stage * kAtomK / 8192.0 / 1965.0;
-    double stage = 0.364;
+    double stage = 0.483;
     if (feed > stage) stage = feed;
     if (mma > stage) stage = mma;
-    const double rows_live = (double)(M < s.bm ? M : s.bm);
-    const double exchange = s.splits > 1 ? 2 * 0.615 + rows_live * s.bn * 4 / 1024.0 * 0.0054 : 0.0;
-    const double finish = s.cluster_n == slices ? 0.615 : 3.22;
-    return waves * (2.48 + stages * stage + exchange + 1.93) + finish;
+    double loop = stages * stage, exchange = 0.0;
+    if (s.splits > 1) {
+        const double rows_live = (double)(M < s.bm ? M : s.bm);
+        exchange = 2 * 0.314 + rows_live * s.bn * 4 / 1000.0 * 0.0124;
+        const bool dedicated = s.bm * s.bn * 4 <= stage_bytes && ring - 1 >= (stages < 3 ? stages : 3);
+        if (!dedicated) exchange += 1.32;           // the hand-shake after the k-loop
+        else if (stages > ring - 1) loop += 0.83;   // one stage fewer in flight
+    }
+    const double finish = s.cluster_n == slices ? 0.314 : (K == 1 && slices <= 255 ? 0.0 : 1.94);
+    return 1.12 + waves * (2.15 + loop + exchange + 2.03) + finish;
 }
 
-Shape choose_shape(int64_t M, int d, int h)
+Shape choose_shape(int64_t M, int K, int d, int h)
 {
     Shape best = {64, 64, 1, 1};
     double best_cost = -1.0;
@@ -641,7 +721,7 @@ Shape choose_shape(int64_t M, int d, int h)
                     const Shape s = {bm, bn, S, all ? slices : 1};
                     if (all && slices == 1) continue;
                     if (!shape_usable(s, M, d, h)) continue;
-                    const double c = shape_cost(s, M, d, h);
+                    const double c = shape_cost(s, M, K, d, h);
                     if (best_cost < 0.0 || c < best_cost) {
                         best_cost = c;
                         best = s;
@@ -668,10 +748,17 @@ int launch_tile(const CUtensorMap &mh, const CUtensorMap &mw, VerifyParams vp, c
         attr_set[dev] = true;
     }
     const int slices = ceil_div(vp.h, BN);
-    vp.slices = slices * s.splits;
+    vp.slices = slices;
     vp.kb_per = kb_per_split(vp.d, s.splits);
+    // With d split, the accumulator columns that arrive from the other CTAs get the room of
+    // the last pipeline stage if enough stages remain; else they overlay the ring after the k-loop.
+    const int stages_needed = ceil_div(vp.kb_per, Cfg::kAtoms);
+    const int spare = Cfg::kStages - 1;
+    vp.recv_dedicated = s.splits > 1 && BM * BN * 4 <= Cfg::kStageBytes && spare >= (stages_needed < 3 ? stages_needed : 3);
+    vp.ring_stages = vp.recv_dedicated ? spare : Cfg::kStages;
     vp.cluster_n = s.cluster_n;
     vp.final_in_cluster = s.cluster_n == slices ? 1 : 0;
+    vp.atomic_finish = !vp.final_in_cluster && vp.K == 1 && vp.zacc && slices <= 255;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)s.splits, (unsigned)slices, (unsigned)tiles_m);
     cfg.blockDim = dim3(kTcThreads);
@@ -726,7 +813,7 @@ int launch_verifier_tensor(const VerifyParams &vp_in, int dt, int min_tokens, co
     const int64_t M = (int64_t)vp.B * vp.K;
     if (dt != SPR_BF16 || vp.h <= 0 || vp.d % 8 != 0 || M < min_tokens) return -1;
     if ((reinterpret_cast<uintptr_t>(vp.hidden) & 15) || (reinterpret_cast<uintptr_t>(vp.W1) & 15)) return -1;
-    Shape s = choose_shape(M, vp.d, vp.h);
+    Shape s = choose_shape(M, vp.K, vp.d, vp.h);
     vp.spin_limit = kSpinLimit;
     vp.test_flags = 0;
     if (tune) {

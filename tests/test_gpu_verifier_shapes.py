@@ -116,8 +116,10 @@ def test_forced_shape_that_does_not_fit_is_refused(spr):
                                         ((8, 4, 256, 64), (64, 64, 2, -1)),      # cluster of 2 along d
                                         ((40, 8, 512, 256), (128, 128, 2, -1)),  # cluster 2 x 2
                                         ((40, 8, 512, 256), (64, 64, 4, 1)),     # split of d, tickets
-                                        ((40, 8, 512, 256), (128, 64, 1, 1))],   # tickets only
-                         ids=["single", "split2", "cluster2x2", "split4-tickets", "tickets"])
+                                        ((40, 8, 512, 256), (128, 64, 1, 1)),    # tickets only
+                                        ((70, 1, 512, 256), (64, 64, 4, 1)),     # K = 1: per-token atomic finish
+                                        ((70, 1, 512, 256), (64, 128, 1, 1))],
+                         ids=["single", "split2", "cluster2x2", "split4-tickets", "tickets", "k1-split4", "k1"])
 def test_bounded_wait_runs_out_and_the_workspace_survives(spr, dims, shape):
     """Nothing feeds the kernel's pipeline (test flag): every CTA's first wait expires after a
     few thousand polls, the launch ends by itself, reports SPR_ERR_TIMEOUT and marks its outputs;
