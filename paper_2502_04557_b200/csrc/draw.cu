@@ -15,6 +15,26 @@
 
 namespace spr {
 
+// Development aid (compiled only with -DSPR_DRAW_STAMPS): SM-clock stamps of the phases of the
+// first CTAs of a launch, read back with spr_debug_draw_stamps().
+#ifdef SPR_DRAW_STAMPS
+__device__ long long g_draw_stamps[1024][8];
+#define SPR_DSTAMP(i)                                                         \
+    do {                                                                      \
+        if (blockIdx.x < 1024) g_draw_stamps[blockIdx.x][i] = clock64();      \
+    } while (0)
+extern "C" int spr_debug_draw_stamps(long long *host_out)   // reads the stamps and clears them
+{
+    cudaError_t e = cudaMemcpyFromSymbol(host_out, g_draw_stamps, sizeof(long long) * 1024 * 8);
+    void *p = nullptr;
+    if (e == cudaSuccess) e = cudaGetSymbolAddress(&p, g_draw_stamps);
+    if (e == cudaSuccess) e = cudaMemset(p, 0, sizeof(long long) * 1024 * 8);
+    return (int)e;
+}
+#else
+#define SPR_DSTAMP(i)
+#endif
+
 namespace {
 
 constexpr int kMaxCompact = 4096;   // draws whose live list a CTA builds in shared memory
@@ -141,6 +161,16 @@ __device__ __noinline__ int warp_finish(const Job<T> &job, int mode, int V, int 
                                         float *residual_mass)
 {
     const int lane = threadIdx.x & 31;
+    if (steps <= kFastSteps) {     // the short chain: everything in registers
+        Crossing c = warp_crossing(part, steps, job.u);
+        if (lane == 0 && residual_mass) *residual_mass = mode == MODE_RESIDUAL ? (float)c.total : 0.f;
+        if (!kSoftmaxOnly && mode == MODE_RESIDUAL && !(c.total > 0.0)) {
+            mode = MODE_SOFTMAX;
+            warp_softmax_row<T>(job.p_row, V, steps, part);
+            c = warp_crossing(part, steps, job.u);
+        }
+        return c.step >= 0 ? warp_locate<T>(job, mode, V, c.step, c.t_in, c.ref) : -1;
+    }
     steps_total(part, steps, sm);
     if (lane == 0 && residual_mass) *residual_mass = mode == MODE_RESIDUAL ? (float)sm.total : 0.f;
     if (!kSoftmaxOnly && mode == MODE_RESIDUAL && !(sm.total > 0.0)) {
@@ -163,23 +193,38 @@ draw_kernel(const DrawParams prm)
     __shared__ WarpSmem s_fin[kWarps];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = prm.n, steps = prm.steps;
+    if (tid == 0) SPR_DSTAMP(0);
 
     pdl_wait();   // the kernel before this one may still be writing first_reject / accepted_len
+    if (tid == 0) SPR_DSTAMP(1);
 
     // ---- which draws are live?  Every CTA builds the same list (ascending draw index).
     const bool compact = n <= kMaxCompact;
     int nlive = n;
     if (compact) {
+        // Rounds of 1024 draws: warp w looks at draws w*128 .. w*128+127 of the round, four per
+        // lane with their loads in flight together, so a round costs one trip to memory.
         nlive = 0;
-        for (int base = 0; base < n; base += kThreads) {
-            const int i = base + tid;
-            const bool live = i < n && draw_is_live(prm, i);
-            if (i < n && !live && blockIdx.x == 0) {
-                prm.tokens[i] = -1;
-                if (prm.residual_mass) prm.residual_mass[i] = 0.f;
+        for (int base = 0; base < n; base += kWarps * 128) {
+            bool live[4];
+            unsigned mask[4];
+            int mine = 0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int i = base + warp * 128 + j * 32 + lane;
+                live[j] = i < n && draw_is_live(prm, i);
             }
-            const unsigned mask = __ballot_sync(0xffffffffu, live);
-            if (lane == 0) s_count[warp] = __popc(mask);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int i = base + warp * 128 + j * 32 + lane;
+                if (i < n && !live[j] && blockIdx.x == 0) {
+                    prm.tokens[i] = -1;
+                    if (prm.residual_mass) prm.residual_mass[i] = 0.f;
+                }
+                mask[j] = __ballot_sync(0xffffffffu, live[j]);
+                mine += __popc(mask[j]);
+            }
+            if (lane == 0) s_count[warp] = mine;
             __syncthreads();
             int before = nlive, all = nlive;
 #pragma unroll
@@ -187,12 +232,19 @@ draw_kernel(const DrawParams prm)
                 if (w < warp) before += s_count[w];
                 all += s_count[w];
             }
-            if (live) s_live[before + __popc(mask & ((1u << lane) - 1u))] = (unsigned short)i;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (live[j])
+                    s_live[before + __popc(mask[j] & ((1u << lane) - 1u))] =
+                        (unsigned short)(base + warp * 128 + j * 32 + lane);
+                before += __popc(mask[j]);
+            }
             nlive = all;
             __syncthreads();
         }
     }
 
+    if (tid == 0) SPR_DSTAMP(2);
     // ---- this warp's run of the live draws' steps
     const int64_t total = (int64_t)nlive * steps;
     const int64_t warps = (int64_t)gridDim.x * kWarps, gw = (int64_t)blockIdx.x * kWarps + warp;
@@ -218,18 +270,22 @@ draw_kernel(const DrawParams prm)
         const int mode = kSoftmaxOnly ? (int)MODE_SOFTMAX : job.mode;
         float2 *part = prm.part + (int64_t)i * steps;
         warp_steps<T, kSoftmaxOnly>(job, mode, prm.V, s0, s1, part);
+        if (tid == 0) SPR_DSTAMP(3);
         int last = 0;
         if (lane == 0) {
             __threadfence();
             last = take_ticket(&prm.counters[i], steps, s1 - s0);
         }
+        if (tid == 0) SPR_DSTAMP(4);
         if (!__shfl_sync(0xffffffffu, last, 0)) continue;
         __threadfence();
         const int token = warp_finish<T, kSoftmaxOnly>(job, mode, prm.V, steps, part, s_fin[warp],
                                                        prm.kind == DRAW_SD && prm.residual_mass
                                                            ? prm.residual_mass + i : nullptr);
         if (lane == 0) prm.tokens[i] = token;
+        if (lane == 0) SPR_DSTAMP(5);
     }
+    if (tid == 0) SPR_DSTAMP(6);
 }
 
 }  // namespace

@@ -325,6 +325,166 @@ __device__ __forceinline__ void steps_cross(const float2 *part, int steps, doubl
     __syncwarp();
 }
 
+// ---------------------------------------------------------------- one-warp finish, short chain
+// The finish of a draw is a chain of dependent steps on one warp while everybody else is done:
+// the versions below keep it short for rows of at most kFastSteps warp steps.  Lane l owns
+// steps 4l .. 4l+3 (and, inside the crossing step, vectors 4l .. 4l+3), so a lane adds its own
+// items serially and ONE warp scan joins the lanes, where the general routines above scan once
+// per 32 items; nothing is read twice.
+constexpr int kFastSteps = 128;
+
+struct Crossing {
+    double total;     // weight of the row, relative to its maximum
+    double t_in;      // what is left of the target inside the crossing step, in that step's own scale
+    float ref;        // maximum of the crossing step
+    int step;         // crossing step; the last step with weight if rounding leaves none; -1: no weight
+};
+
+// steps <= kFastSteps step partials -> where u * total falls.  Same arithmetic per item as
+// step_weight / steps_total / steps_cross; the scale between the row's units and the crossing
+// step's is the very factor its weight was formed with.
+__device__ __forceinline__ Crossing warp_crossing(const float2 *part, int steps, float u)
+{
+    const int lane = threadIdx.x & 31;
+    float2 ms[4];
+    float M = neg_inf();
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int t = 4 * lane + k;
+        ms[k] = t < steps ? __ldcg(&part[t]) : make_float2(neg_inf(), 0.f);
+        M = fmaxf(M, ms[k].x);
+    }
+    M = warp_max(M);
+    float f[4];
+    double incl[4];
+    double run = 0.0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        f[k] = ms[k].y > 0.f ? ex2((ms[k].x - M) * kLog2e) : 0.f;
+        run += ms[k].y > 0.f ? (double)(ms[k].y * f[k]) : 0.0;
+        incl[k] = run;
+    }
+    const double lanes = warp_scan_f64(run, lane);    // inclusive over the lanes
+    const double before_lane = lanes - run;
+    Crossing c;
+    c.total = __shfl_sync(0xffffffffu, lanes, 31);
+    const double target = (double)u * c.total;
+    // first own step whose running weight passes the target, last own step with weight
+    // (selected without indexing the register arrays by a run-time value)
+    int kfirst = 4, klast = -1;
+    double before_first = 0.0;
+    float f_first = 1.f, ref_first = 0.f, ref_last = 0.f;
+#pragma unroll
+    for (int k = 3; k >= 0; --k) {
+        const bool has = ms[k].y > 0.f && f[k] > 0.f;
+        if (has && before_lane + incl[k] > target) {
+            kfirst = k;
+            before_first = before_lane + (k > 0 ? incl[k > 0 ? k - 1 : 0] : 0.0);
+            f_first = f[k];
+            ref_first = ms[k].x;
+        }
+        if (has && klast < 0) {
+            klast = k;
+            ref_last = ms[k].x;
+        }
+    }
+    const unsigned cross = __ballot_sync(0xffffffffu, kfirst < 4);
+    const unsigned pos = __ballot_sync(0xffffffffu, klast >= 0);
+    if (cross != 0u) {
+        const int owner = __ffs(cross) - 1;
+        c.step = __shfl_sync(0xffffffffu, 4 * lane + kfirst, owner);
+        c.t_in = __shfl_sync(0xffffffffu, (target - before_first) / (double)f_first, owner);
+        c.ref = __shfl_sync(0xffffffffu, ref_first, owner);
+    } else if (pos != 0u) {
+        const int owner = 31 - __clz(pos);
+        c.step = __shfl_sync(0xffffffffu, 4 * lane + klast, owner);
+        c.ref = __shfl_sync(0xffffffffu, ref_last, owner);
+        c.t_in = __longlong_as_double(0x7ff0000000000000LL);
+    } else {
+        c.step = -1;
+        c.ref = 0.f;
+        c.t_in = 0.0;
+    }
+    return c;
+}
+
+// Inside step `step`: the first element whose running weight exceeds t_in, as step_locate
+// finds it, with the step's 128 vectors dealt to the lanes four in a row.
+template <typename T>
+__device__ __forceinline__ int warp_locate(const Job<T> &job, int mode, int V, int step, double t_in, float ref)
+{
+    constexpr int N = Vec<T>::N;
+    constexpr int kStep = 32 * kUnroll * N;
+    static_assert(kUnroll == 4, "four vectors per lane");
+    const int lane = threadIdx.x & 31;
+    const int f0 = step * kStep - row_pad(job.p_row) + 4 * lane * N;    // this lane's first element
+    const float off = -ref * kLog2e;
+    uint4 rp[4], rq[4] = {};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) rp[j] = load_vec<T>(job.p_row, f0 + j * N, V);
+    if (mode == MODE_RESIDUAL) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) rq[j] = load_vec<T>(job.q_row, f0 + j * N, V);
+    }
+    // weights of vector j (recomputed where needed rather than kept: registers are scarce here)
+    auto weights = [&](int j, float (&w)[N]) {
+        if (mode == MODE_SOFTMAX) {
+            float f[N];
+            Vec<T>::unpack(rp[j], f);
+#pragma unroll
+            for (int e = 0; e < N; ++e) w[e] = ex2(fmaf(f[e], kLog2e, off));
+        } else {
+            residual_weights<T>(rp[j], rq[j], job, w);
+        }
+    };
+    double vs[4];      // weight of each of the lane's vectors
+    int lastpos = -1;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        float w[N];
+        weights(j, w);
+        double ts = 0.0;
+#pragma unroll
+        for (int e = 0; e < N; ++e) {
+            ts += (double)w[e];
+            if (w[e] > 0.f) lastpos = f0 + j * N + e;
+        }
+        vs[j] = ts;
+    }
+    const double mine = (vs[0] + vs[1]) + (vs[2] + vs[3]);
+    const double incl = warp_scan_f64(mine, lane);
+    const unsigned cross = __ballot_sync(0xffffffffu, incl > t_in);
+    int tok = -1;
+    if (cross != 0u) {
+        const int owner = __ffs(cross) - 1;
+        int found = -1;
+        if (lane == owner) {
+            double r = incl - mine;
+            int last_e = -1;       // last element with weight up to and including the crossing vector
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (found == -1) {
+                    float w[N];
+                    weights(j, w);
+                    const bool here = r + vs[j] > t_in;
+                    double rr = r;
+#pragma unroll
+                    for (int e = 0; e < N; ++e) {
+                        rr += (double)w[e];
+                        if (w[e] > 0.f) last_e = f0 + j * N + e;
+                        if (here && found < 0 && rr > t_in && w[e] > 0.f) found = f0 + j * N + e;
+                    }
+                    if (here && found < 0) found = last_e >= 0 ? last_e : -2;   // rounding inside the vector
+                    r += vs[j];
+                }
+            }
+        }
+        tok = __shfl_sync(0xffffffffu, found, owner);
+    }
+    lastpos = (int)__reduce_max_sync(0xffffffffu, lastpos);
+    return tok >= 0 ? tok : lastpos;
+}
+
 // Whole CTA, once every step partial of a draw is in part[0 .. steps): the token where the
 // running weight crosses u * total.  A residual draw whose weights vanish (Eq. 1 undefined)
 // is redone as a draw from p.  The token is returned in warp 0 (other warps get -1);
