@@ -2,6 +2,8 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <atomic>
+
 #include "common.cuh"
 #include "host_util.h"
 #include "launch.h"
@@ -34,15 +36,18 @@ namespace {
 // compute capability 10.x only; the answer is cached per device ordinal
 int check_device()
 {
-    static int cached[64];  // 0 unknown, 1 ok, 2 unsupported
+    static std::atomic<int> cached[64];  // 0 unknown, 1 ok, 2 unsupported (racing threads store the same value)
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_fail(e);
-    if (dev >= 0 && dev < 64 && cached[dev]) return cached[dev] == 1 ? SPR_OK : SPR_ERR_UNSUPPORTED;
+    if (dev >= 0 && dev < 64) {
+        const int known = cached[dev].load(std::memory_order_relaxed);
+        if (known) return known == 1 ? SPR_OK : SPR_ERR_UNSUPPORTED;
+    }
     int major = 0;
     e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
     if (e != cudaSuccess) return cuda_fail(e);
-    if (dev >= 0 && dev < 64) cached[dev] = major == 10 ? 1 : 2;
+    if (dev >= 0 && dev < 64) cached[dev].store(major == 10 ? 1 : 2, std::memory_order_relaxed);
     return major == 10 ? SPR_OK : SPR_ERR_UNSUPPORTED;
 }
 

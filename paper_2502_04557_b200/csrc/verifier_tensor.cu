@@ -32,6 +32,8 @@
 // bounded - for what it has in flight, releases TMEM and exits.
 #include <cuda.h>
 
+#include <atomic>
+
 #include "common.cuh"
 #include "launch.h"
 #include "verifier_common.cuh"
@@ -607,6 +609,302 @@ verifier_tcgen05_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_
     if (clustered) cluster_wait();   // no peer is still sending to this CTA
 }
 
+// ---------------------------------------------------------------- CTA pairs (large batches)
+// With many tokens the k-loop is bound by how fast one SM takes operands in (about one 128-byte
+// row per two clocks).  Two CTAs of a cluster then share one 256-token x 128-hidden-unit tile:
+// each stages its own 128 token rows but only HALF of the W1 tile (64 rows), and one thread of
+// the even CTA issues tcgen05.mma.cta_group::2, which reads both CTAs' shared memory and writes
+// both CTAs' TMEM - a quarter fewer operand bytes per SM and per FLOP.  The copies of both CTAs
+// count on the even CTA's "full" barriers; its commits free the stage in both CTAs.  Every
+// CTA then runs the same epilogue as above on its own 128 accumulator rows.  The cluster is
+// (2, n, 1): the pair along x, and along y all slices of the token tiles when they fit (finish
+// out of shared memory, one receiver per token tile), else one slice (tickets).
+constexpr int kPairBM = 128, kPairBN = 128;
+constexpr uint32_t kPeerBitMask = 0xFEFFFFFFu;   // clears the bit that tells the two CTAs of a pair apart
+
+struct PairCfg {
+    static constexpr int kBytesA = kPairBM * kAtomK * 2;          // 128 token rows of one atom
+    static constexpr int kBytesB = (kPairBN / 2) * kAtomK * 2;    // this CTA's 64 W1 rows of one atom
+    static constexpr int kAtoms = 2;
+    static constexpr int kStageBytes = kAtoms * (kBytesA + kBytesB);
+    static constexpr int kStages = 4;
+    static constexpr int kRingBytes = kStages * kStageBytes;
+    static constexpr int kTmemCols = kPairBN;
+    static constexpr size_t kSmemBytes = (size_t)kRingBytes + 1024 + ((sizeof(Control) + 255) / 256) * 256;
+};
+
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(acc), "r"(0u)
+        : "memory");
+}
+// arrives, once the MMAs issued so far are complete, on the barrier at this address in every CTA of `mask`
+__device__ __forceinline__ void umma_commit_pair(uint64_t *bar, uint16_t mask)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"(mask)
+                 : "memory");
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+verifier_pair_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w,
+                     const VerifyParams prm)
+{
+    using Cfg = PairCfg;
+    constexpr int BM = kPairBM, BN = kPairBN;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *ring = reinterpret_cast<unsigned char *>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    Control *ctl = reinterpret_cast<Control *>(ring + Cfg::kRingBytes);
+
+    pdl_trigger();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) SPR_STAMP(0);
+    const int M = prm.B * prm.K;
+    const int half = (int)blockIdx.x;                  // 0: the CTA that issues the MMAs, 1: its peer
+    const int n0 = blockIdx.y * BN;
+    const int tile = (int)blockIdx.z * 2 + half;       // token tile of this CTA
+    const int m0 = tile * BM;
+    const int num_atoms = (prm.d + kAtomK - 1) / kAtomK;
+    const int num_stages = (num_atoms + Cfg::kAtoms - 1) / Cfg::kAtoms;
+    const uint32_t cy = blockIdx.y % (unsigned)prm.cluster_n;
+    const uint32_t my_rank = (uint32_t)half + 2u * cy;             // x runs fastest inside the cluster
+    const uint32_t limit = prm.spin_limit;
+    const int live_rows = max(0, min(BM, M - m0));                 // the odd tile may lie past the batch
+    const bool z_receiver = prm.final_in_cluster && cy == 0;       // one per token tile
+
+    if (tid == 0) {
+        for (int s = 0; s < Cfg::kStages; ++s) {
+            mbar_init(&ctl->full[s], 1);
+            mbar_init(&ctl->empty[s], 1);
+        }
+        mbar_init(&ctl->tmem_full, 1);
+        mbar_init(&ctl->drain, 1);
+        mbar_init(&ctl->zgather, 1);
+        if (z_receiver && live_rows > 0) mbar_expect_tx(&ctl->zgather, (uint32_t)(prm.cluster_n * live_rows * 4));
+        ctl->abort = 0;
+        ctl->last = 0;
+        ctl->consumed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0 && lane < 2)
+        asm volatile("prefetch.tensormap [%0];" ::"l"(lane == 0 ? &map_h : &map_w) : "memory");
+    if (warp == 1) {   // both CTAs of the pair allocate the same columns
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
+                     "r"((uint32_t)Cfg::kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_acc = ctl->tmem_base;
+    // "started, barriers set up": the peer's copies count on the even CTA's barriers and its
+    // commits arrive on the peer's, so both sides check for this word before their loops
+    cluster_arrive();
+    if (tid == 0) SPR_STAMP(1);
+
+    int issued = 0;
+    bool ok = true;
+    if (warp == 0) {
+        // ---------------- TMA producer (both CTAs): even lanes hidden-state atoms, odd lanes W1 atoms
+        cluster_wait();
+        if (lane < 2 * Cfg::kAtoms && !(prm.test_flags & VERIFIER_TEST_NO_LOADS)) {
+            const int atom = lane >> 1;
+            const bool is_w = lane & 1;
+            const CUtensorMap *map = is_w ? &map_w : &map_h;
+            const int row0 = is_w ? n0 + half * (BN / 2) : m0;
+            const uint32_t off = is_w ? (uint32_t)(Cfg::kAtoms * Cfg::kBytesA + atom * Cfg::kBytesB)
+                                      : (uint32_t)(atom * Cfg::kBytesA);
+            for (int st = 0; st < num_stages; ++st) {
+                const int s = st % Cfg::kStages;
+                const uint32_t round = (uint32_t)(st / Cfg::kStages);
+                const int n_at = min(Cfg::kAtoms, num_atoms - st * Cfg::kAtoms);
+                if (!mbar_wait(&ctl->empty[s], (round & 1u) ^ 1u, ctl, prm.status, limit)) break;
+                // the even CTA expects the bytes of both
+                if (lane == 0 && half == 0)
+                    mbar_expect_tx(&ctl->full[s], (uint32_t)(2 * n_at * (Cfg::kBytesA + Cfg::kBytesB)));
+                if (atom < n_at)
+                    tma_load_2d_pair(smem_u32(ring + (size_t)s * Cfg::kStageBytes) + off, map,
+                                     (st * Cfg::kAtoms + atom) * kAtomK, row0, smem_u32(&ctl->full[s]) & kPeerBitMask);
+                issued = st + 1;
+                if (st == 0) SPR_STAMP(2);
+                if (st < 24 && lane == 0) SPR_STAMP(40 + st);
+            }
+        }
+    } else if (warp == 1) {
+        cluster_wait();
+        // ---------------- MMA issuer: one thread of the even CTA, for both
+        if (lane == 0 && half == 0) {
+            constexpr uint32_t idesc = umma_instr_desc<2 * BM, BN>();
+            const uint16_t both = (uint16_t)(3u << my_rank);
+            bool fed = true;
+            int st = 0;
+            for (; st < num_stages; ++st) {
+                const int s = st % Cfg::kStages;
+                const uint32_t round = (uint32_t)(st / Cfg::kStages);
+                const int n_at = min(Cfg::kAtoms, num_atoms - st * Cfg::kAtoms);
+                fed = mbar_wait(&ctl->full[s], round & 1u, ctl, prm.status, limit);
+                if (!fed) break;
+                if (st == 0) SPR_STAMP(3);
+                if (st < 24) SPR_STAMP(16 + st);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a_addr = smem_u32(ring + (size_t)s * Cfg::kStageBytes);
+                const uint32_t b_addr = a_addr + Cfg::kAtoms * Cfg::kBytesA;
+#pragma unroll
+                for (int a = 0; a < Cfg::kAtoms; ++a) {
+                    if (a < n_at) {
+                        const uint64_t da = umma_smem_desc(a_addr + a * Cfg::kBytesA);
+                        const uint64_t db = umma_smem_desc(b_addr + a * Cfg::kBytesB);
+#pragma unroll
+                        for (int k = 0; k < kAtomK / kUmmaK; ++k) {
+                            const uint64_t adv = (uint64_t)((k * kUmmaK * 2) >> 4);
+                            umma_bf16_pair(tmem_acc, da + adv, db + adv, idesc, (st | a | k) != 0 ? 1u : 0u);
+                        }
+                    }
+                }
+                umma_commit_pair(&ctl->empty[s], both);     // the stage is free in both CTAs
+            }
+            ctl->consumed = st;
+            SPR_STAMP(4);
+            if (fed) umma_commit_pair(&ctl->tmem_full, both);   // both epilogues may read
+            else umma_commit_pair(&ctl->drain, (uint16_t)(1u << my_rank));
+        }
+    } else {
+        for (int j = tid - 64; j < BN; j += kTcThreads - 64) {
+            const int n = n0 + j;
+            ctl->b1[j] = n < prm.h ? prm.b1[n] : 0.f;
+            ctl->w2[j] = n < prm.h ? __bfloat162float(static_cast<const __nv_bfloat16 *>(prm.W2)[n]) : 0.f;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        cluster_wait();
+        ok = mbar_wait(&ctl->tmem_full, 0, ctl, prm.status, limit);
+        if (tid == 64) SPR_STAMP(5);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    }
+    __syncwarp();
+
+    const int quarter = warp & 3;
+    const int r_in = quarter * 32 + lane;
+    const int row = m0 + r_in;
+    const bool live_row = warp >= 2 && row < M;
+    const uint32_t lane_base = tmem_acc + ((uint32_t)(quarter * 32) << 16);
+
+    float z = 0.f;
+    if (warp >= 2) {
+#pragma unroll
+        for (int c0 = 0; c0 < BN; c0 += 64) {
+            uint32_t v[2][32];
+            tmem_ld32(lane_base + (uint32_t)c0, v[0]);
+            tmem_ld32(lane_base + (uint32_t)(c0 + 32), v[1]);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 64; ++j)
+                z = fmaf(ctl->w2[c0 + j], fmaxf(__uint_as_float(v[j >> 5][j & 31]) + ctl->b1[c0 + j], 0.f), z);
+        }
+        if (!ok || *reinterpret_cast<volatile int *>(&ctl->abort)) z = poisoned_z();
+        if (prm.final_in_cluster) {
+            // to the CTA that finishes this token tile: same half of the pair, first slice
+            if (live_row)
+                st_async_b32(peer_smem(smem_u32(&ctl->zbuf[cy][r_in]), (uint32_t)half), __float_as_uint(z),
+                             peer_smem(smem_u32(&ctl->zgather), (uint32_t)half));
+            if (z_receiver && live_rows > 0) {
+                const bool got = mbar_wait(&ctl->zgather, 0, ctl, prm.status, limit);
+                if (!got && live_row) ctl->zbuf[0][r_in] = poisoned_z();
+            }
+        } else if (live_row) {
+            prm.part_z[(int64_t)blockIdx.y * M + row] = z;
+        }
+    }
+    __syncwarp();
+    if (tid == 64) SPR_STAMP(8);
+    cluster_arrive();   // done with the peers: TMEM read, nothing more sent or expected
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (*reinterpret_cast<volatile int *>(&ctl->abort)) {
+        if (warp == 0) {
+            int last = issued;
+#pragma unroll
+            for (int o = 1; o < 8; o <<= 1) last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
+            // the copies of both CTAs count on the even CTA's barriers: it waits for them
+            if (lane == 0 && half == 0) {
+                for (int st = ctl->consumed; st < last; ++st)
+                    mbar_wait_quiet(&ctl->full[st % Cfg::kStages], (uint32_t)(st / Cfg::kStages) & 1u, limit);
+            }
+        }
+        if (warp == 1 && lane == 0 && half == 0 && ctl->consumed < num_stages) mbar_wait_quiet(&ctl->drain, 0, limit);
+        __syncthreads();
+    }
+
+    if (tid == 64) SPR_STAMP(9);
+    // ---------------- finish (as in the single-CTA kernel)
+    const int m_hi = min(m0 + BM, M);
+    bool finisher = false;
+    if (live_rows > 0) {
+        if (prm.final_in_cluster) {
+            finisher = z_receiver;
+            if (finisher) {
+                const float b2 = prm.b2[0];
+                for (int t = tid; t < m_hi - m0; t += kTcThreads) {
+                    float zt = b2;
+                    for (int i = 0; i < prm.cluster_n; ++i) zt += ctl->zbuf[i][t];
+                    ctl->codes[t] = (unsigned char)classify_token(prm, zt, m0 + t);
+                }
+                __syncthreads();
+                if (prm.first_reject) {
+                    const int b_lo = (m0 + prm.K - 1) / prm.K, b_hi = m_hi / prm.K;
+                    for (int b = b_lo + warp; b < b_hi; b += kTcThreads / 32)
+                        scan_sequence_smem(prm, b, ctl->codes + (b * prm.K - m0), lane);
+                }
+            }
+        } else {
+            if (tid == 0) {
+                __threadfence();
+                ctl->last = take_ticket(&prm.counter[1 + tile], (int)gridDim.y);
+            }
+            __syncthreads();
+            finisher = ctl->last != 0;
+            if (finisher) {
+                __threadfence();
+                finalise_tile(prm, m0, m_hi, ctl->codes);
+            }
+        }
+    }
+    // sequences cut by a tile boundary wait for the CTA that completes the last tile
+    if (finisher && BM % prm.K != 0 && M > BM) {
+        __syncthreads();
+        if (tid == 0) {
+            __threadfence();
+            ctl->last = take_ticket(&prm.counter[0], (M + BM - 1) / BM);
+        }
+        __syncthreads();
+        if (ctl->last) {
+            __threadfence();
+            finalise_straddlers(prm, BM);
+        }
+    }
+    if (tid == 64) SPR_STAMP(10);
+    // Both CTAs are through with the accumulator (and nobody is still sending here): release it
+    cluster_wait();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"((uint32_t)Cfg::kTmemCols)
+                     : "memory");
+    }
+}
+
 // ---------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
@@ -615,16 +913,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 
 EncodeTiledFn encode_fn()
 {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
+    static const EncodeTiledFn fn = [] {   // initialised once, thread-safe
         void *p = nullptr;
         cudaDriverEntryPointQueryResult q;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
             q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
+            return reinterpret_cast<EncodeTiledFn>(p);
+        return static_cast<EncodeTiledFn>(nullptr);
+    }();
     return fn;
 }
 
@@ -658,6 +954,11 @@ int kb_per_split(int d, int S)
 
 bool shape_usable(const Shape &s, int64_t M, int d, int h)
 {
+    if (s.bm == 2 * kPairBM) {   // a pair of CTAs per 256 x 128 tile
+        const int slices = ceil_div(h, kPairBN);
+        return s.bn == kPairBN && s.splits == 1 && (s.cluster_n == 1 || (s.cluster_n == slices && 2 * slices <= kMaxClusterCtas)) &&
+               slices <= 65535 && ceil_div(M, 2 * kPairBM) <= 65535;
+    }
     if ((s.bm != 64 && s.bm != 128) || (s.bn != 64 && s.bn != 128)) return false;
     if (s.splits != 1 && s.splits != 2 && s.splits != 4 && s.splits != 8) return false;
     if (s.bn / s.splits < 8 || kb_per_split(d, s.splits) == 0) return false;
@@ -679,19 +980,21 @@ bool shape_usable(const Shape &s, int64_t M, int d, int h)
 //            global memory otherwise.
 double shape_cost(const Shape &s, int64_t M, int K, int d, int h)
 {
+    const bool pair = s.bm == 2 * kPairBM;
     const int slices = ceil_div(h, s.bn), tiles = ceil_div(M, s.bm);
-    const int cluster_ctas = s.splits * s.cluster_n;
-    const int64_t clusters = (int64_t)tiles * slices * s.splits / cluster_ctas;
+    const int cluster_ctas = (pair ? 2 : s.splits) * s.cluster_n;
+    const int64_t clusters = (int64_t)tiles * slices * (pair ? 2 : s.splits) / cluster_ctas;
     const int capacity = cluster_ctas == 1 ? 148 : cluster_ctas == 2 ? 74 : cluster_ctas <= 4 ? 33 : 15;
     const double waves = (double)((clusters + capacity - 1) / capacity);
     const int atoms_per_stage = s.bm + s.bn == 128 ? 4 : 2;
-    const int stage_bytes = atoms_per_stage * (s.bm + s.bn) * kAtomK * 2;
+    const int stage_bytes = atoms_per_stage * (pair ? kPairBM + kPairBN / 2 : s.bm + s.bn) * kAtomK * 2;
     const int ring = (200 * 1024) / stage_bytes;
     const int stages = ceil_div(kb_per_split(d, s.splits), atoms_per_stage);
-    const double rows_a = tiles == 1 ? (double)((M + 7) / 8 * 8) : (double)s.bm;
-    const double rows = rows_a + (double)(h < s.bn ? h : s.bn);
-    const double feed = rows * atoms_per_stage * 0.00135;
-    const double mma = (double)s.bm * s.bn * atoms_per_stage * kAtomK / 8192.0 / 1965.0;
+    const double rows_a = pair ? (double)kPairBM : tiles == 1 ? (double)((M + 7) / 8 * 8) : (double)s.bm;
+    const double rows = rows_a + (pair ? (double)(kPairBN / 2) : (double)(h < s.bn ? h : s.bn));
+    // (all SMs together take about 13 TB/s from L2: a pair fetches fewer rows, each a little slower)
+    const double feed = rows * atoms_per_stage * (pair ? 0.00153 : 0.00135);
+    const double mma = (double)(pair ? kPairBM : s.bm) * s.bn * atoms_per_stage * kAtomK / 8192.0 / 1965.0;
     double stage = 0.483;
     if (feed > stage) stage = feed;
     if (mma > stage) stage = mma;
@@ -704,7 +1007,7 @@ double shape_cost(const Shape &s, int64_t M, int K, int d, int h)
         else if (stages > ring - 1) loop += 0.83;   // one stage fewer in flight
     }
     const double finish = s.cluster_n == slices ? 0.314 : (K == 1 && slices <= 255 ? 0.0 : 1.94);
-    return 1.12 + waves * (2.15 + loop + exchange + 2.03) + finish;
+    return 1.12 + waves * ((pair ? 2.6 : 2.15) + loop + exchange + 2.03) + finish;
 }
 
 Shape choose_shape(int64_t M, int K, int d, int h)
@@ -730,7 +1033,52 @@ Shape choose_shape(int64_t M, int K, int d, int h)
             }
         }
     }
+    // CTA pairs: once the batch has at least two 128-token tiles per pair of SMs
+    if (M >= 512 && h > 64) {
+        const int slices = ceil_div(h, kPairBN);
+        for (int all = 0; all < 2; ++all) {
+            const Shape s = {2 * kPairBM, kPairBN, 1, all ? slices : 1};
+            if ((all && slices == 1) || !shape_usable(s, M, d, h)) continue;
+            const double c = shape_cost(s, M, K, d, h);
+            if (c < best_cost) {
+                best_cost = c;
+                best = s;
+            }
+        }
+    }
     return best;
+}
+
+int launch_pair(const CUtensorMap &mh, const CUtensorMap &mw, VerifyParams vp, const Shape &s, cudaStream_t st)
+{
+    static std::atomic<bool> attr_set[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_set[dev].load(std::memory_order_acquire)) {
+        cudaError_t e = cudaFuncSetAttribute(verifier_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)PairCfg::kSmemBytes);
+        if (e != cudaSuccess) return (int)e;
+        attr_set[dev].store(true, std::memory_order_release);
+    }
+    const int slices = ceil_div(vp.h, kPairBN);
+    const int64_t M = (int64_t)vp.B * vp.K;
+    vp.slices = slices;
+    vp.cluster_n = s.cluster_n;
+    vp.final_in_cluster = s.cluster_n == slices ? 1 : 0;
+    vp.atomic_finish = 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2u, (unsigned)slices, (unsigned)ceil_div(M, 2 * kPairBM));
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = PairCfg::kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = (unsigned)s.cluster_n;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return (int)cudaLaunchKernelEx(&cfg, verifier_pair_kernel, mh, mw, vp);
 }
 
 template <int BM, int BN>
@@ -738,14 +1086,14 @@ int launch_tile(const CUtensorMap &mh, const CUtensorMap &mw, VerifyParams vp, c
                 cudaStream_t st)
 {
     using Cfg = TileCfg<BM, BN>;
-    static bool attr_set[64];
+    static std::atomic<bool> attr_set[64];   // host threads may race to set it: all of them store `true`
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+    if (dev >= 0 && dev < 64 && !attr_set[dev].load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(verifier_tcgen05_kernel<BM, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)Cfg::kSmemBytes);
         if (e != cudaSuccess) return (int)e;
-        attr_set[dev] = true;
+        attr_set[dev].store(true, std::memory_order_release);
     }
     const int slices = ceil_div(vp.h, BN);
     vp.slices = slices;
@@ -822,11 +1170,18 @@ int launch_verifier_tensor(const VerifyParams &vp_in, int dt, int min_tokens, co
         if (tune->splits) s.splits = tune->splits;
         const int slices = ceil_div(vp.h, s.bn);
         if (tune->cluster_n) s.cluster_n = tune->cluster_n < 0 ? slices : 1;
-        else if (tune->bm || tune->bn || tune->splits) s.cluster_n = s.splits * slices <= kMaxClusterCtas ? slices : 1;
+        else if (tune->bm || tune->bn || tune->splits)
+            s.cluster_n = (s.bm == 2 * kPairBM ? 2 : s.splits) * slices <= kMaxClusterCtas ? slices : 1;
         if (tune->spin_limit) vp.spin_limit = tune->spin_limit;
         vp.test_flags = tune->test_flags;
     }
     if (!shape_usable(s, M, vp.d, vp.h)) return -1;
+    if (s.bm == 2 * kPairBM) {
+        CUtensorMap mh, mw;
+        if (!make_map(&mh, vp.hidden, (int)M, vp.d, kPairBM)) return -1;
+        if (!make_map(&mw, vp.W1, vp.h, vp.d, kPairBN / 2)) return -1;
+        return launch_pair(mh, mw, vp, s, st);
+    }
     const int tiles_m = ceil_div(M, s.bm);
     // a batch that fills only part of its one tile fetches only the rows it has (the rest of
     // the operand tile stays as it is: accumulator rows that are never read)

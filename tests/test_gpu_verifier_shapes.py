@@ -77,6 +77,13 @@ SHAPES = [
     ((130, 3, 136, 20), (128, 64, 1, 1)),
     ((32, 8, 768, 256), (64, 64, 2, -1)),
     ((32, 8, 768, 256), (128, 128, 4, -1)),
+    # bm = 256: two CTAs share a 256 x 128 tile (each stages half of the W1 tile)
+    ((100, 16, 2048, 512), (256, 128, 1, -1)),
+    ((100, 16, 2048, 512), (256, 128, 1, 1)),
+    ((36, 8, 256, 96), (256, 128, 1, -1)),       # three token tiles: the last pair's second tile is empty
+    ((130, 3, 136, 20), (256, 128, 1, 1)),
+    ((20, 33, 64, 16), (256, 128, 1, -1)),       # sequences cut by tile boundaries
+    ((300, 1, 4096, 1024), (256, 128, 1, 1)),    # eight slices: tickets
 ]
 
 
@@ -118,8 +125,11 @@ def test_forced_shape_that_does_not_fit_is_refused(spr):
                                         ((40, 8, 512, 256), (64, 64, 4, 1)),     # split of d, tickets
                                         ((40, 8, 512, 256), (128, 64, 1, 1)),    # tickets only
                                         ((70, 1, 512, 256), (64, 64, 4, 1)),     # K = 1: per-token atomic finish
-                                        ((70, 1, 512, 256), (64, 128, 1, 1))],
-                         ids=["single", "split2", "cluster2x2", "split4-tickets", "tickets", "k1-split4", "k1"])
+                                        ((70, 1, 512, 256), (64, 128, 1, 1)),
+                                        ((40, 8, 512, 256), (256, 128, 1, -1)),  # CTA pairs, finish in the cluster
+                                        ((40, 8, 512, 256), (256, 128, 1, 1))],  # CTA pairs, tickets
+                         ids=["single", "split2", "cluster2x2", "split4-tickets", "tickets", "k1-split4", "k1",
+                              "pairs", "pairs-tickets"])
 def test_bounded_wait_runs_out_and_the_workspace_survives(spr, dims, shape):
     """Nothing feeds the kernel's pipeline (test flag): every CTA's first wait expires after a
     few thousand polls, the launch ends by itself, reports SPR_ERR_TIMEOUT and marks its outputs;
