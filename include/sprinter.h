@@ -393,8 +393,9 @@ void spr_set_stage_events(void *before, void *after);
  * the library, so that tests reach every shape on small inputs: bm, bn in {64, 128} tokens x
  * hidden units per tile, splits in {1, 2, 4, 8} CTAs sharing a tile along d, cluster_n = 1
  * (finish through the workspace) or -1 (a tile's CTAs form one cluster; needs
- * splits * ceil(h / bn) <= 8); 0 leaves a value to the library.  A combination the problem
- * does not allow returns SPR_ERR_UNSUPPORTED.
+ * splits * ceil(h / bn) <= 8); 0 leaves a value to the library.  bm = 256 (with bn = 128,
+ * splits = 1) selects the kernel in which two CTAs share a 256 x 128 tile.  A combination
+ * the problem does not allow returns SPR_ERR_UNSUPPORTED.
  * flags bit 0: the kernel's copy engine producer issues nothing, so that the first bounded
  * wait of every CTA runs out after spin_limit polls (0 = the library's limit): the call
  * returns SPR_OK, the status word reads SPR_ERR_TIMEOUT, scores are -1, accept bits 0 and

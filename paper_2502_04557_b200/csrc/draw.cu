@@ -78,7 +78,7 @@ __device__ __forceinline__ Job<T> resolve_job(const DrawParams &prm, int i)
         const int nb = prm.accepted_len[i];
         if (nb < 0) return job;  // invalid draft token in this sequence
         if (nb < prm.K) {
-            job.mode = MODE_RESIDUAL;
+            job.mode = MODE_RESIDUAL_FAST;
             job.p_row = p + ((int64_t)i * prm.Kp + nb) * prm.ldv;
             job.q_row = static_cast<const T *>(prm.q) + ((int64_t)i * prm.K + nb) * prm.ldv;
             set_residual_scales(job, prm.rowstats[(int64_t)i * prm.K + nb]);
@@ -124,7 +124,7 @@ __device__ __forceinline__ void warp_steps(const Job<T> &job, int mode, int V, i
                 load_step<T>(job.p_row, (s + 1) * kStep - pad, V, lane, np);
                 load_step_any<T>(job.q_row, (s + 1) * kStep - pad, V, lane, nq);
             }
-            const float w = warp_sum(residual_step_sum<T>(rp, rq, job));
+            const float w = warp_sum(residual_step_sum_fast<T>(rp, rq, job));
             if (lane == 0) part[s] = make_float2(0.f, w);
 #pragma unroll
             for (int j = 0; j < kUnroll; ++j) {
@@ -152,8 +152,27 @@ __device__ __noinline__ void warp_softmax_row(const T *row, int V, int steps, fl
     __syncwarp();   // lane 0's partials are read by the other lanes next
 }
 
+// One warp: the residual partials of every step of a row pair in the ratio form (the rare redo
+// of a draw whose residual mass is too small for plain differences; kept small on purpose)
+template <typename T>
+__device__ __noinline__ void warp_residual_row(const Job<T> &job, int V, int steps, float2 *part)
+{
+    constexpr int kStep = 32 * kUnroll * Vec<T>::N;
+    const int lane = threadIdx.x & 31;
+    const int pad = row_pad(job.p_row);
+    for (int s = 0; s < steps; ++s) {
+        uint4 rp[kUnroll], rq[kUnroll];
+        load_step<T>(job.p_row, s * kStep - pad, V, lane, rp);
+        load_step_any<T>(job.q_row, s * kStep - pad, V, lane, rq);
+        const float w = warp_sum(residual_step_sum<T>(rp, rq, job));
+        if (lane == 0) part[s] = make_float2(0.f, w);
+    }
+    __syncwarp();
+}
+
 // One warp, once every step partial of the draw is in part[0 .. steps): the token where the
-// running weight crosses u * total.  A residual draw whose weights vanish (Eq. 1 undefined) is
+// running weight crosses u * total.  A residual draw whose mass (from plain differences) is
+// below kResidualRedo is first redone by this warp in the ratio form.  A residual draw whose weights vanish (Eq. 1 undefined) is
 // redone by this warp as a draw from p.  *residual_mass, if given, receives the total residual
 // weight (0 for softmax draws).
 template <typename T, bool kSoftmaxOnly>
@@ -161,23 +180,29 @@ __device__ __noinline__ int warp_finish(const Job<T> &job, int mode, int V, int 
                                         float *residual_mass)
 {
     const int lane = threadIdx.x & 31;
-    if (steps <= kFastSteps) {     // the short chain: everything in registers
-        Crossing c = warp_crossing(part, steps, job.u);
-        if (lane == 0 && residual_mass) *residual_mass = mode == MODE_RESIDUAL ? (float)c.total : 0.f;
-        if (!kSoftmaxOnly && mode == MODE_RESIDUAL && !(c.total > 0.0)) {
-            mode = MODE_SOFTMAX;
-            warp_softmax_row<T>(job.p_row, V, steps, part);
+    const bool fast = steps <= kFastSteps;     // the short chain: everything in registers
+    Crossing c;
+    auto cross = [&]() {
+        if (fast) {
             c = warp_crossing(part, steps, job.u);
+        } else {
+            steps_total(part, steps, sm);
+            c.total = sm.total;
         }
-        return c.step >= 0 ? warp_locate<T>(job, mode, V, c.step, c.t_in, c.ref) : -1;
+    };
+    cross();
+    if (!kSoftmaxOnly && mode == MODE_RESIDUAL_FAST && !(c.total >= (double)kResidualRedo)) {
+        mode = MODE_RESIDUAL;
+        warp_residual_row<T>(job, V, steps, part);
+        cross();
     }
-    steps_total(part, steps, sm);
-    if (lane == 0 && residual_mass) *residual_mass = mode == MODE_RESIDUAL ? (float)sm.total : 0.f;
-    if (!kSoftmaxOnly && mode == MODE_RESIDUAL && !(sm.total > 0.0)) {
+    if (lane == 0 && residual_mass) *residual_mass = mode == MODE_SOFTMAX ? 0.f : (float)c.total;
+    if (!kSoftmaxOnly && mode != MODE_SOFTMAX && !(c.total > 0.0)) {
         mode = MODE_SOFTMAX;
         warp_softmax_row<T>(job.p_row, V, steps, part);
-        steps_total(part, steps, sm);
+        cross();
     }
+    if (fast) return c.step >= 0 ? warp_locate<T, kSoftmaxOnly>(job, mode, V, c.step, c.t_in, c.ref) : -1;
     steps_cross(part, steps, (double)job.u * sm.total, sm);
     return sm.step >= 0 ? step_locate<T>(job, mode, V, sm.step, sm.t_in, sm.ref) : -1;
 }
@@ -188,8 +213,11 @@ template <typename T, bool kSoftmaxOnly>
 __global__ void __launch_bounds__(kThreads, kSoftmaxOnly ? kDrawCtasSoftmax : kDrawCtasResidual)
 draw_kernel(const DrawParams prm)
 {
+    // live draws in ascending order: those that read two rows (residual draws: twice the bytes
+    // and more than twice the arithmetic per step) and those that read one
     __shared__ unsigned short s_live[kMaxCompact];
-    __shared__ int s_count[kWarps];
+    __shared__ unsigned short s_light[kSoftmaxOnly ? 1 : kMaxCompact];
+    __shared__ int s_count[2][kWarps];
     __shared__ WarpSmem s_fin[kWarps];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = prm.n, steps = prm.steps;
@@ -198,67 +226,98 @@ draw_kernel(const DrawParams prm)
     pdl_wait();   // the kernel before this one may still be writing first_reject / accepted_len
     if (tid == 0) SPR_DSTAMP(1);
 
-    // ---- which draws are live?  Every CTA builds the same list (ascending draw index).
+    // ---- which draws are live?  Every CTA builds the same lists.
     const bool compact = n <= kMaxCompact;
-    int nlive = n;
+    int nheavy = n, nlight = 0;
     if (compact) {
         // Rounds of 1024 draws: warp w looks at draws w*128 .. w*128+127 of the round, four per
         // lane with their loads in flight together, so a round costs one trip to memory.
-        nlive = 0;
+        nheavy = 0;
         for (int base = 0; base < n; base += kWarps * 128) {
-            bool live[4];
-            unsigned mask[4];
-            int mine = 0;
+            bool heavy[4], light[4];
+            unsigned mh[4], ml[4];
+            int mine_h = 0, mine_l = 0;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int i = base + warp * 128 + j * 32 + lane;
-                live[j] = i < n && draw_is_live(prm, i);
-            }
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int i = base + warp * 128 + j * 32 + lane;
-                if (i < n && !live[j] && blockIdx.x == 0) {
+                const bool live = i < n && draw_is_live(prm, i);
+                // a correction draw from the residual reads the p row and the q row
+                heavy[j] = live;
+                light[j] = false;
+                if constexpr (!kSoftmaxOnly) {
+                    heavy[j] = live && (prm.kind != DRAW_SD || prm.accepted_len[i] < prm.K);
+                    light[j] = live && !heavy[j];
+                }
+                if (i < n && !live && blockIdx.x == 0) {
                     prm.tokens[i] = -1;
                     if (prm.residual_mass) prm.residual_mass[i] = 0.f;
                 }
-                mask[j] = __ballot_sync(0xffffffffu, live[j]);
-                mine += __popc(mask[j]);
-            }
-            if (lane == 0) s_count[warp] = mine;
-            __syncthreads();
-            int before = nlive, all = nlive;
-#pragma unroll
-            for (int w = 0; w < kWarps; ++w) {
-                if (w < warp) before += s_count[w];
-                all += s_count[w];
             }
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                if (live[j])
-                    s_live[before + __popc(mask[j] & ((1u << lane) - 1u))] =
-                        (unsigned short)(base + warp * 128 + j * 32 + lane);
-                before += __popc(mask[j]);
+                mh[j] = __ballot_sync(0xffffffffu, heavy[j]);
+                ml[j] = kSoftmaxOnly ? 0u : __ballot_sync(0xffffffffu, light[j]);
+                mine_h += __popc(mh[j]);
+                mine_l += __popc(ml[j]);
             }
-            nlive = all;
+            if (lane == 0) {
+                s_count[0][warp] = mine_h;
+                s_count[1][warp] = mine_l;
+            }
+            __syncthreads();
+            int before_h = nheavy, all_h = nheavy, before_l = nlight, all_l = nlight;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                if (w < warp) {
+                    before_h += s_count[0][w];
+                    before_l += s_count[1][w];
+                }
+                all_h += s_count[0][w];
+                all_l += s_count[1][w];
+            }
+            const unsigned below = (1u << lane) - 1u;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const unsigned short i = (unsigned short)(base + warp * 128 + j * 32 + lane);
+                if (heavy[j]) s_live[before_h + __popc(mh[j] & below)] = i;
+                if (!kSoftmaxOnly && light[j]) s_light[before_l + __popc(ml[j] & below)] = i;
+                before_h += __popc(mh[j]);
+                before_l += __popc(ml[j]);
+            }
+            nheavy = all_h;
+            nlight = all_l;
             __syncthreads();
         }
     }
 
     if (tid == 0) SPR_DSTAMP(2);
-    // ---- this warp's run of the live draws' steps
-    const int64_t total = (int64_t)nlive * steps;
+    // ---- this warp's run of the live draws' steps.  The steps of the two-row draws, then those
+    // of the one-row draws, laid end to end and cut into runs of equal COST, a two-row step
+    // counting twice: a cut at cost x lies at step ceil(x / 2) inside the first part.
+    const int64_t heavy_steps = (int64_t)nheavy * steps, all_steps = heavy_steps + (int64_t)nlight * steps;
+    const int64_t cost = 2 * heavy_steps + (int64_t)nlight * steps;
     const int64_t warps = (int64_t)gridDim.x * kWarps, gw = (int64_t)blockIdx.x * kWarps + warp;
-    int64_t u = total / warps * gw + min(gw, total % warps);          // runs differ by one step at most
-    const int64_t u_end = u + total / warps + (gw < total % warps ? 1 : 0);
+    auto cut = [&](int64_t g) {     // first step of warp g's run
+        if (kSoftmaxOnly) return all_steps / warps * g + min(g, all_steps % warps);   // every step costs the same
+        const int64_t x = cost / warps * g + min(g, cost % warps);
+        return x <= 2 * heavy_steps ? (x + 1) / 2 : x - heavy_steps;
+    };
+    int64_t u = cut(gw);
+    const int64_t u_end = gw + 1 == warps ? all_steps : cut(gw + 1);
     while (u < u_end) {
         int64_t j = u / steps;
         const int s0 = (int)(u - j * steps);
         const int s1 = (int)min((int64_t)steps, s0 + (u_end - u));
         u += s1 - s0;
-        // correction draws go through the sequences last to first: the statistics pass has just
-        // streamed the rows in ascending order, so the highest ones are the ones still in L2
-        if (!kSoftmaxOnly) j = nlive - 1 - j;
-        const int i = compact ? (int)s_live[j] : (int)j;
+        // Each list is gone through last to first: the statistics pass has just streamed the
+        // rows in ascending order, so the highest ones are the ones still in L2.
+        int i;
+        if (j < nheavy) {
+            j = kSoftmaxOnly ? j : nheavy - 1 - j;
+            i = compact ? (int)s_live[j] : (int)j;
+        } else {
+            i = (int)s_light[nlight - 1 - (j - nheavy)];
+        }
         const Job<T> job = resolve_job<T>(prm, i);
         if (job.mode == MODE_NONE) {   // gated off (when no list was built), or a bad row
             if (s0 == 0 && lane == 0) {

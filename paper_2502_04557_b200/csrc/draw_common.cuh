@@ -8,7 +8,17 @@
 
 namespace spr {
 
-enum { MODE_NONE = 0, MODE_SOFTMAX = 1, MODE_RESIDUAL = 2 };
+// MODE_RESIDUAL forms max(0, p - q) in the ratio form below, accurate however close p and q are;
+// MODE_RESIDUAL_FAST as the plain difference of the two probabilities, which costs a third of the
+// instructions and is accurate enough whenever the residual mass is not tiny (see kResidualRedo).
+enum { MODE_NONE = 0, MODE_SOFTMAX = 1, MODE_RESIDUAL = 2, MODE_RESIDUAL_FAST = 3 };
+
+// The plain difference carries an absolute error of about 5e-7 of the probability mass passed
+// (ex2.approx, two per element).  Where the draw falls is decided in units of the residual mass
+// R, so that error counts 5e-7 / R there: two orders under the 1e-4 a decision must keep from
+// its boundary as long as R >= 0.02.  A draw whose plain-difference mass comes out below that is
+// redone in the ratio form by the warp that finishes it.
+constexpr float kResidualRedo = 0.02f;
 
 template <typename T>
 struct Job {
@@ -63,6 +73,50 @@ __device__ __forceinline__ void residual_weights(const uint4 &vp, const uint4 &v
         const float r = D < 0.25f ? qv * em1 : direct;
         w[e] = D > 0.f ? r : 0.f;
     }
+}
+
+// max(0, p_i - q_i) of one vector as the plain difference of the probabilities
+template <typename T>
+__device__ __forceinline__ void residual_weights_fast(const uint4 &vp, const uint4 &vq, const Job<T> &job,
+                                                      float (&w)[Vec<T>::N])
+{
+    constexpr int N = Vec<T>::N;
+    float fp[N], fq[N];
+    Vec<T>::unpack(vp, fp);
+    Vec<T>::unpack(vq, fq);
+    const uint64_t l2 = pack2(kLog2e, kLog2e), cp2 = pack2(-job.cp, -job.cp), cq2 = pack2(-job.cq, -job.cq);
+    const uint64_t sp2 = pack2(job.sp, job.sp), nsq2 = pack2(-job.sq, -job.sq);
+#pragma unroll
+    for (int e = 0; e < N; e += 2) {
+        float a0, a1, b0, b1, d0, d1;
+        unpack2(fma2(pack2(fp[e], fp[e + 1]), l2, cp2), a0, a1);
+        unpack2(fma2(pack2(fq[e], fq[e + 1]), l2, cq2), b0, b1);
+        const uint64_t qs = mul2(pack2(ex2(b0), ex2(b1)), nsq2);          // -q
+        unpack2(fma2(pack2(ex2(a0), ex2(a1)), sp2, qs), d0, d1);          // p - q
+        w[e] = fmaxf(d0, 0.f);                                            // (-inf) - (-inf): both terms are 0
+        w[e + 1] = fmaxf(d1, 0.f);
+    }
+}
+
+// lane-local sum of those weights over one warp step
+template <typename T>
+__device__ __forceinline__ float residual_step_sum_fast(const uint4 (&rp)[kUnroll], const uint4 (&rq)[kUnroll],
+                                                        const Job<T> &job)
+{
+    constexpr int N = Vec<T>::N;
+    uint64_t acc[kUnroll];
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) {
+        float w[N];
+        residual_weights_fast<T>(rp[j], rq[j], job, w);
+        acc[j] = pack2(w[0], w[1]);
+#pragma unroll
+        for (int e = 2; e < N; e += 2) acc[j] = add2(acc[j], pack2(w[e], w[e + 1]));
+    }
+    float a0, a1, b0, b1;
+    unpack2(add2(acc[0], acc[1]), a0, a1);
+    unpack2(add2(acc[2], acc[3]), b0, b1);
+    return (a0 + a1) + (b0 + b1);
 }
 
 // Scratch of whoever finishes a draw (a CTA in the sharded kernels, one warp in draw_kernel);
@@ -193,7 +247,7 @@ __device__ int step_locate(const Job<T> &job, int mode, int V, int step, double 
     const float off = -ref * kLog2e;
     uint4 rp[kUnroll], rq[kUnroll] = {};
     load_step<T>(job.p_row, f0, V, lane, rp);
-    if (mode == MODE_RESIDUAL) load_step_any<T>(job.q_row, f0, V, lane, rq);
+    if (mode != MODE_SOFTMAX) load_step_any<T>(job.q_row, f0, V, lane, rq);
     double run = 0.0;
     int tok = -1, lastpos = -1;
 #pragma unroll
@@ -204,6 +258,8 @@ __device__ int step_locate(const Job<T> &job, int mode, int V, int step, double 
             Vec<T>::unpack(rp[j], f);
 #pragma unroll
             for (int e = 0; e < N; ++e) w[e] = ex2(fmaf(f[e], kLog2e, off));
+        } else if (mode == MODE_RESIDUAL_FAST) {
+            residual_weights_fast<T>(rp[j], rq[j], job, w);
         } else {
             residual_weights<T>(rp[j], rq[j], job, w);
         }
@@ -408,9 +464,18 @@ __device__ __forceinline__ Crossing warp_crossing(const float2 *part, int steps,
     return c;
 }
 
+// the ratio-form weights as a call: rare in warp_locate (only the redo of a draw with a tiny
+// residual mass gets there), so it is kept out of line there
+template <typename T>
+__device__ __noinline__ void residual_weights_call(const uint4 &vp, const uint4 &vq, const Job<T> &job,
+                                                   float (&w)[Vec<T>::N])
+{
+    residual_weights<T>(vp, vq, job, w);
+}
+
 // Inside step `step`: the first element whose running weight exceeds t_in, as step_locate
 // finds it, with the step's 128 vectors dealt to the lanes four in a row.
-template <typename T>
+template <typename T, bool kUnrolled>
 __device__ __forceinline__ int warp_locate(const Job<T> &job, int mode, int V, int step, double t_in, float ref)
 {
     constexpr int N = Vec<T>::N;
@@ -422,24 +487,32 @@ __device__ __forceinline__ int warp_locate(const Job<T> &job, int mode, int V, i
     uint4 rp[4], rq[4] = {};
 #pragma unroll
     for (int j = 0; j < 4; ++j) rp[j] = load_vec<T>(job.p_row, f0 + j * N, V);
-    if (mode == MODE_RESIDUAL) {
+    if (mode != MODE_SOFTMAX) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) rq[j] = load_vec<T>(job.q_row, f0 + j * N, V);
     }
-    // weights of vector j (recomputed where needed rather than kept: registers are scarce here)
+    // The finish of a draw is cold code that one warp runs once; much of what it costs is
+    // fetching its instructions.  Where the weight formulas are long (a kernel that knows the
+    // residual modes: !kUnrolled) the loops over the lane's four vectors are NOT unrolled (one
+    // copy of the formulas each); the vector is picked with selects, since registers cannot be
+    // indexed by a run-time value.
+    auto pick = [](const uint4 (&r)[4], int j) { return j == 0 ? r[0] : j == 1 ? r[1] : j == 2 ? r[2] : r[3]; };
     auto weights = [&](int j, float (&w)[N]) {
+        const uint4 vp = pick(rp, j);
         if (mode == MODE_SOFTMAX) {
             float f[N];
-            Vec<T>::unpack(rp[j], f);
+            Vec<T>::unpack(vp, f);
 #pragma unroll
             for (int e = 0; e < N; ++e) w[e] = ex2(fmaf(f[e], kLog2e, off));
+        } else if (mode == MODE_RESIDUAL_FAST) {
+            residual_weights_fast<T>(vp, pick(rq, j), job, w);
         } else {
-            residual_weights<T>(rp[j], rq[j], job, w);
+            residual_weights_call<T>(vp, pick(rq, j), job, w);
         }
     };
-    double vs[4];      // weight of each of the lane's vectors
+    double vs0 = 0.0, vs1 = 0.0, vs2 = 0.0, vs3 = 0.0;      // weight of each of the lane's vectors
     int lastpos = -1;
-#pragma unroll
+#pragma unroll(kUnrolled ? 4 : 1)
     for (int j = 0; j < 4; ++j) {
         float w[N];
         weights(j, w);
@@ -449,9 +522,12 @@ __device__ __forceinline__ int warp_locate(const Job<T> &job, int mode, int V, i
             ts += (double)w[e];
             if (w[e] > 0.f) lastpos = f0 + j * N + e;
         }
-        vs[j] = ts;
+        vs0 = j == 0 ? ts : vs0;
+        vs1 = j == 1 ? ts : vs1;
+        vs2 = j == 2 ? ts : vs2;
+        vs3 = j == 3 ? ts : vs3;
     }
-    const double mine = (vs[0] + vs[1]) + (vs[2] + vs[3]);
+    const double mine = (vs0 + vs1) + (vs2 + vs3);
     const double incl = warp_scan_f64(mine, lane);
     const unsigned cross = __ballot_sync(0xffffffffu, incl > t_in);
     int tok = -1;
@@ -461,22 +537,21 @@ __device__ __forceinline__ int warp_locate(const Job<T> &job, int mode, int V, i
         if (lane == owner) {
             double r = incl - mine;
             int last_e = -1;       // last element with weight up to and including the crossing vector
+#pragma unroll(kUnrolled ? 4 : 1)
+            for (int j = 0; j < 4 && found == -1; ++j) {
+                const double vsj = j == 0 ? vs0 : j == 1 ? vs1 : j == 2 ? vs2 : vs3;
+                float w[N];
+                weights(j, w);
+                const bool here = r + vsj > t_in;
+                double rr = r;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if (found == -1) {
-                    float w[N];
-                    weights(j, w);
-                    const bool here = r + vs[j] > t_in;
-                    double rr = r;
-#pragma unroll
-                    for (int e = 0; e < N; ++e) {
-                        rr += (double)w[e];
-                        if (w[e] > 0.f) last_e = f0 + j * N + e;
-                        if (here && found < 0 && rr > t_in && w[e] > 0.f) found = f0 + j * N + e;
-                    }
-                    if (here && found < 0) found = last_e >= 0 ? last_e : -2;   // rounding inside the vector
-                    r += vs[j];
+                for (int e = 0; e < N; ++e) {
+                    rr += (double)w[e];
+                    if (w[e] > 0.f) last_e = f0 + j * N + e;
+                    if (here && found < 0 && rr > t_in && w[e] > 0.f) found = f0 + j * N + e;
                 }
+                if (here && found < 0) found = last_e >= 0 ? last_e : -2;   // rounding inside the vector
+                r += vsj;
             }
         }
         tok = __shfl_sync(0xffffffffu, found, owner);
