@@ -4,7 +4,8 @@
 One step = one pass of the whole path over one batch: sprinter_verify (verifier scores,
 threshold, first-rejection scan) -> replace_sample gated by first_reject (replacement tokens),
 issued as the fused sprinter_step call, and sd_verify (exact speculative-decoding verification
-of the same draft tokens) on a second stream.  The
+of the same draft tokens); one after the other on one stream, or side by side on two
+(--streams 2).  The
 metric is draft tokens taken through that step per second, summed over all GPUs (each rank
 verifies its own batch: weak scaling, no data-path collective).
 
@@ -62,6 +63,11 @@ def parse_args():
     ap.add_argument("--graph", default="auto", choices=["auto", "0", "1"],
                     help="1: the timed steps are replays of CUDA graphs of the step (no host launch cost between "
                          "kernels); auto: only when a step takes the GPU less time than the host needs to issue it")
+    ap.add_argument("--stage-every", type=int, default=8,
+                    help="the row-statistics launch is bracketed by CUDA events in every n-th timed step (the event "
+                         "records sit between two launches and keep the second from starting early)")
+    ap.add_argument("--streams", type=int, default=1, choices=[1, 2],
+                    help="1: sd_verify then sprinter_step on one stream; 2: the two calls of a step on two streams")
     ap.add_argument("--shard", default="batch", choices=["batch", "vocab"],
                     help="how --gpus N ranks split the work: every rank its own batch (default), or every "
                          "rank V/N columns of the same logits (sd_verify only, NCCL exchanges between the passes)")
@@ -448,11 +454,12 @@ def main():
     ws = spr.Workspace.for_problem(B, K, V, cfg.d, cfg.h, dt_code, device=dev)
     ws_sd = spr.Workspace.for_problem(B, K, V, cfg.d, cfg.h, dt_code, device=dev)
     tau = args.threshold
-    # The SD call and the SPRINTER calls (verify -> gated replacement) of a step are independent:
-    # they go to two streams with separate workspaces, SD first, so the short latency-bound
-    # SPRINTER kernels run in the shadow of the tail of the bandwidth-bound SD pass.
+    # The SD call and the SPRINTER call (verify -> gated replacement) of a step are independent and
+    # have separate workspaces.  By default they follow each other on one stream: measured, two
+    # streams finish a step about 2 % sooner, but the short SPRINTER kernels then take SMs and
+    # bandwidth from the row-statistics pass while it runs (0.88 instead of 0.93 of the copy peak).
     st_sd = torch.cuda.Stream(device=dev)
-    st_spr = torch.cuda.Stream(device=dev)
+    st_spr = torch.cuda.Stream(device=dev) if args.streams == 2 else st_sd
 
     ver_out = (torch.empty((B, K), dtype=torch.float32, device=dev),
                torch.empty((B, K), dtype=torch.uint8, device=dev),
@@ -532,8 +539,9 @@ def main():
         torch.cuda.current_stream().wait_stream(cap)
         return graph
 
+    every = max(1, args.stage_every)
     stage = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-             for _ in range(min(nsteps, 50) if use_graph else nsteps)]
+             for _ in range(min(nsteps, 50) if use_graph else (nsteps + every - 1) // every)]
     for a, b in stage:          # create the handles
         a.record()
         b.record()
@@ -559,7 +567,10 @@ def main():
     else:
         fork()
         for i in range(nsteps):
-            spr.set_stage_events(*stage[i])
+            if i % every == 0:
+                spr.set_stage_events(*stage[i // every])
+            elif i % every == 1:
+                spr.set_stage_events(None, None)
             step()
         join()
     stop.record()
@@ -819,7 +830,10 @@ def main():
             "steps": nsteps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16"
             if cfg.dtype == torch.bfloat16 else "f32", "data": "synthetic",
-            "config": {"workload": workload_label(wl), "step": "sd_verify (stream 1) || sprinter_step = sprinter_verify + gated replace_sample (stream 2)",
+            "config": {"workload": workload_label(wl),
+                       "step": ("sd_verify (stream 1) || sprinter_step = sprinter_verify + gated replace_sample (stream 2)"
+                                if args.streams == 2 else
+                                "sd_verify, then sprinter_step = sprinter_verify + gated replace_sample, on one stream"),
                        "timed_region": (f"CUDA-graph replays of the step ({'+'.join(str(t) for _, t in graphs)} replays); "
                                         "row-statistics launch time from an eager pass after it") if use_graph else
                                        "eager calls",
@@ -833,12 +847,14 @@ def main():
             "roofline": {"bound": "hbm", "kernel": "sd_row_stats_kernel", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                          "traffic": traffic, "algorithmic_bytes_per_launch": alg_bytes,
-                         "avg_launch_ms": stats_ms},
+                         "avg_launch_ms": stats_ms, "launches_timed": len(stage),
+                         "timing": f"CUDA-event pair around the launch in every {every}. timed step" if not use_graph
+                                   else "CUDA-event pairs in an eager pass after the graph replays"},
             "roofline_verifier": roofline_verifier, "roofline_draw": roofline_draw,
             "sprinter_step_tokens_per_s": calls["sprinter_step"]["verified_tokens_per_s"],
             "sd_verify_tokens_per_s": calls["sd_verify"]["verified_tokens_per_s"],
-            "value_is": "draft tokens per second through one step = sd_verify and sprinter_step of the same tokens, "
-                        "run side by side; each path alone is in sprinter_step_tokens_per_s / sd_verify_tokens_per_s",
+            "value_is": "draft tokens per second through one step = sd_verify and sprinter_step of the same tokens; "
+                        "each path alone is in sprinter_step_tokens_per_s / sd_verify_tokens_per_s",
             "cpu_baseline": cpu_baseline, "calls": calls,
             **({"simulator": simulator} if simulator else {}),
         }))

@@ -407,6 +407,43 @@ def test_sd_equal_and_disjoint_distributions(spr):
     assert ws.device_status() == 0
 
 
+def _small_mass_problem(dtype, V):
+    """B single-position sequences (no bonus row) whose target row is the draft row plus noise of
+    growing size, each with the draft token the target likes least and a uniform that rejects it."""
+    g = torch.Generator().manual_seed(V + (1 if dtype == torch.float32 else 2))
+    eps = [1e-4, 1e-3, 0.01, 0.03, 0.05, 0.1, 0.3, 1.0] if dtype == torch.float32 else \
+          [0.005, 0.01, 0.02, 0.03, 0.05, 0.1, 0.3, 1.0]
+    B, K = 2 * len(eps), 1
+    q = torch.randn((B, K, V), generator=g) * 2
+    p = q + torch.tensor(eps).repeat(2).view(B, 1, 1) * torch.randn((B, K, V), generator=g)
+    p, q = p.to(dtype).contiguous(), q.to(dtype).contiguous()
+    x = torch.zeros((B, K), dtype=torch.int32)
+    for b in range(B):
+        ratio = torch.softmax(p[b, 0].double(), 0) / torch.softmax(q[b, 0].double(), 0)
+        x[b, 0] = int(torch.argmin(ratio))
+    u = torch.rand((B, K + 1), generator=g)
+    u[:, 0] = 0.9999
+    return p, q, x, u, _clear_sd(p, q, V, x, u)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("V", [3000, 128256])
+def test_sd_correction_draw_over_residual_masses(spr, dtype, V):
+    """Correction draws whose residual mass sum max(0, p - q) runs from 1e-4 to 0.5: the kernel forms
+    the weights as plain differences where the mass is large and switches to the ratio form below
+    0.02; both sides of that switch must give the oracle's token."""
+    p, q, x, u, ref = _small_mass_problem(dtype, V)
+    masses = ref["residual_mass"][ref["accepted_len"] == 0]
+    assert masses.min() < 0.01 and masses.max() > 0.1 and ((masses > 0.02) & (masses < 0.2)).any()
+    B, K = x.shape
+    ws = spr.Workspace(spr.workspace_bytes(2, B, K, V, 1, 0, spr.binding._dt(p)))
+    out = spr.sd_verify(p.cuda(), q.cuda(), V, x.cuda(), u.cuda(), ws)
+    assert ws.device_status() == 0
+    eq(out["accepted_len"], ref["accepted_len"], "accepted_len")
+    eq(out["correction_token"], ref["correction_token"], "correction_token")
+    assert_mass_close(out["residual_mass"], ref["residual_mass"], RTOL[dtype])
+
+
 def test_device_detected_errors(spr):
     p, q, x, u = _rand_problem(3, 2, 300, torch.float32, seed=3)
     x[1, 1] = 300
