@@ -31,10 +31,10 @@ if ROOT not in sys.path:
 # capture summarised under profiles/; reported only while the kernel source is unchanged.
 NCU_TRAFFIC = {
     "sources": ("sd_row_stats.cu", "vocab_common.cuh", "common.cuh"),
-    "sha256": "2b0fecb1e12cbf45b8e20129dcea797c15c1934c08bf50e5d56dd7fa7fe3a644",
-    # (262,815,232 read + 3,749,120 written) / 512 tokens in the B = 32 capture; traffic grows
+    "sha256": "a5db8cfa60cd6d7786e2ad5820d27c529a4ec4c543c62295fd53986bd685569d",
+    # (262,768,128 read + 3,324,160 written) / 512 tokens in the B = 32 capture; traffic grows
     # in proportion to the tokens, so a full launch is this times B*K
-    "bytes_per_unit": 520633,   # DRAM bytes per verified token at V = 128256, bf16
+    "bytes_per_unit": 519711,   # DRAM bytes per verified token at V = 128256, bf16
 }
 
 
@@ -104,8 +104,10 @@ def tensor_peak():
 # profiles/ (a counter that only a profiler gives); reported while the kernel source is unchanged
 NCU_VERIFIER = {
     "sources": ("verifier_tensor.cu", "verifier_common.cuh"),
-    "sha256": None,
-    "tensor_pipe_pct_while_active": None,
+    "sha256": "e8e78bed90e119a4d930a87bd94599ee1ef8689384fe7de5078bf5789d2a0403",
+    # full-size llama3 launch (128 x 128 tiles, grid (1, 4, 32)): 29.2 % of the pipe's peak while
+    # active, 20.0 % of elapsed
+    "tensor_pipe_pct_while_active": 29.2,
     "profile": "profiles/draw_kernel_and_verifier_llama3.md",
 }
 

@@ -256,33 +256,38 @@ draw_kernel(const DrawParams prm)
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 mh[j] = __ballot_sync(0xffffffffu, heavy[j]);
-                ml[j] = kSoftmaxOnly ? 0u : __ballot_sync(0xffffffffu, light[j]);
                 mine_h += __popc(mh[j]);
-                mine_l += __popc(ml[j]);
+                ml[j] = 0u;
+                if constexpr (!kSoftmaxOnly) {
+                    ml[j] = __ballot_sync(0xffffffffu, light[j]);
+                    mine_l += __popc(ml[j]);
+                }
             }
             if (lane == 0) {
                 s_count[0][warp] = mine_h;
-                s_count[1][warp] = mine_l;
+                if constexpr (!kSoftmaxOnly) s_count[1][warp] = mine_l;
             }
             __syncthreads();
             int before_h = nheavy, all_h = nheavy, before_l = nlight, all_l = nlight;
 #pragma unroll
             for (int w = 0; w < kWarps; ++w) {
-                if (w < warp) {
-                    before_h += s_count[0][w];
-                    before_l += s_count[1][w];
-                }
+                if (w < warp) before_h += s_count[0][w];
                 all_h += s_count[0][w];
-                all_l += s_count[1][w];
+                if constexpr (!kSoftmaxOnly) {
+                    if (w < warp) before_l += s_count[1][w];
+                    all_l += s_count[1][w];
+                }
             }
             const unsigned below = (1u << lane) - 1u;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const unsigned short i = (unsigned short)(base + warp * 128 + j * 32 + lane);
                 if (heavy[j]) s_live[before_h + __popc(mh[j] & below)] = i;
-                if (!kSoftmaxOnly && light[j]) s_light[before_l + __popc(ml[j] & below)] = i;
                 before_h += __popc(mh[j]);
-                before_l += __popc(ml[j]);
+                if constexpr (!kSoftmaxOnly) {
+                    if (light[j]) s_light[before_l + __popc(ml[j] & below)] = i;
+                    before_l += __popc(ml[j]);
+                }
             }
             nheavy = all_h;
             nlight = all_l;

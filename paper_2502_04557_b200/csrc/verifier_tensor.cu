@@ -1148,7 +1148,11 @@ extern "C" int spr_debug_max_clusters(int cx, int cy)   // co-resident clusters 
 }
 extern "C" int spr_debug_verifier_stamps(long long *host_out)   // [512][64]
 {
-    return (int)cudaMemcpyFromSymbol(host_out, g_stamps, sizeof(long long) * 512 * 64);
+    cudaError_t e = cudaMemcpyFromSymbol(host_out, g_stamps, sizeof(long long) * 512 * 64);   // reads, then clears
+    void *p = nullptr;
+    if (e == cudaSuccess) e = cudaGetSymbolAddress(&p, g_stamps);
+    if (e == cudaSuccess) e = cudaMemset(p, 0, sizeof(long long) * 512 * 64);
+    return (int)e;
 }
 #endif
 
