@@ -104,7 +104,7 @@ def tensor_peak():
 # profiles/ (a counter that only a profiler gives); reported while the kernel source is unchanged
 NCU_VERIFIER = {
     "sources": ("verifier_tensor.cu", "verifier_common.cuh"),
-    "sha256": "e8e78bed90e119a4d930a87bd94599ee1ef8689384fe7de5078bf5789d2a0403",
+    "sha256": "05f682cd9270bb251daa1c243f73ac4a3d85c05fe772cea7c27af85fb4de9c86",
     # full-size llama3 launch (128 x 128 tiles, grid (1, 4, 32)): 29.2 % of the pipe's peak while
     # active, 20.0 % of elapsed
     "tensor_pipe_pct_while_active": 29.2,
