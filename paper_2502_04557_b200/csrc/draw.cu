@@ -101,19 +101,26 @@ __device__ __forceinline__ void warp_steps(const Job<T> &job, int mode, int V, i
     const int lane = threadIdx.x & 31;
     const int pad = row_pad(job.p_row);
     if (kSoftmaxOnly || mode == MODE_SOFTMAX) {
-        // two steps in flight behind the one being summed
+        // two steps in flight behind the one being summed; the three buffers swap roles by
+        // position in an unrolled loop instead of being copied
         uint4 a[kUnroll], b[kUnroll], c[kUnroll];
-        load_step<T>(job.p_row, s0 * kStep - pad, V, lane, a);
-        if (s0 + 1 < s1) load_step<T>(job.p_row, (s0 + 1) * kStep - pad, V, lane, b);
-        for (int s = s0; s < s1; ++s) {
-            if (s + 2 < s1) load_step<T>(job.p_row, (s + 2) * kStep - pad, V, lane, c);
-            const MS v = softmax_step<T>(a);
+        auto fetch = [&](uint4 (&dst)[kUnroll], int s) { load_step<T>(job.p_row, s * kStep - pad, V, lane, dst); };
+        auto emit = [&](const uint4 (&src)[kUnroll], int s) {
+            const MS v = softmax_step<T>(src);
             if (lane == 0) part[s] = make_float2(v.m, v.s);
-#pragma unroll
-            for (int j = 0; j < kUnroll; ++j) {
-                a[j] = b[j];
-                b[j] = c[j];
-            }
+        };
+        fetch(a, s0);
+        if (s0 + 1 < s1) fetch(b, s0 + 1);
+        for (int s = s0;;) {
+            if (s + 2 < s1) fetch(c, s + 2);
+            emit(a, s);
+            if (++s >= s1) break;
+            if (s + 2 < s1) fetch(a, s + 2);
+            emit(b, s);
+            if (++s >= s1) break;
+            if (s + 2 < s1) fetch(b, s + 2);
+            emit(c, s);
+            if (++s >= s1) break;
         }
     } else {
         uint4 rp[kUnroll], rq[kUnroll], np[kUnroll], nq[kUnroll];

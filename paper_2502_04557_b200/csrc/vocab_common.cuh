@@ -109,30 +109,6 @@ __device__ __forceinline__ int row_pad(const T *row)
     return (int)((reinterpret_cast<uintptr_t>(row) & 15) / sizeof(T));
 }
 
-// (max, sum of exp(x - max)) over the kUnroll vectors a thread holds
-template <typename T>
-__device__ __forceinline__ MS thread_ms(const uint4 (&raw)[kUnroll])
-{
-    constexpr int N = Vec<T>::N;
-    float m = Vec<T>::vmax(raw[0]);
-#pragma unroll
-    for (int j = 1; j < kUnroll; ++j) m = fmaxf(m, Vec<T>::vmax(raw[j]));
-    const float ref = (m == neg_inf()) ? 0.f : m;
-    const float off = -ref * kLog2e;
-    float s = 0.f;
-#pragma unroll
-    for (int j = 0; j < kUnroll; ++j) {
-        float f[N];
-        Vec<T>::unpack(raw[j], f);
-#pragma unroll
-        for (int e = 0; e < N; ++e) s += ex2(fmaf(f[e], kLog2e, off));
-    }
-    MS r;
-    r.m = m;
-    r.s = s;
-    return r;
-}
-
 // Two fp32 lanes per instruction (sm_100 packed fp32): halves the issue slots of the multiply-
 // add and of the accumulation, which matter here because the exp pipe and the issue rate are
 // the co-limiters of the streaming kernels.
@@ -163,6 +139,40 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
     uint64_t d;
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
+}
+
+// (max, sum of exp(x - max)) over the kUnroll vectors a thread holds; the multiply-add and the
+// accumulation run on pairs of fp32 lanes (the issue rate is a co-limiter of the streaming loops)
+template <typename T>
+__device__ __forceinline__ MS thread_ms(const uint4 (&raw)[kUnroll])
+{
+    constexpr int N = Vec<T>::N;
+    float m = Vec<T>::vmax(raw[0]);
+#pragma unroll
+    for (int j = 1; j < kUnroll; ++j) m = fmaxf(m, Vec<T>::vmax(raw[j]));
+    const float ref = (m == neg_inf()) ? 0.f : m;
+    const float off = -ref * kLog2e;
+    const uint64_t scale2 = pack2(kLog2e, kLog2e), off2 = pack2(off, off);
+    uint64_t acc[kUnroll];
+#pragma unroll
+    for (int j = 0; j < kUnroll; ++j) {
+        float f[N];
+        Vec<T>::unpack(raw[j], f);
+        acc[j] = pack2(0.f, 0.f);
+#pragma unroll
+        for (int e = 0; e < N; e += 2) {
+            float t0, t1;
+            unpack2(fma2(pack2(f[e], f[e + 1]), scale2, off2), t0, t1);
+            acc[j] = add2(acc[j], pack2(ex2(t0), ex2(t1)));
+        }
+    }
+    float a0, a1, b0, b1;
+    unpack2(add2(acc[0], acc[1]), a0, a1);
+    unpack2(add2(acc[2], acc[3]), b0, b1);
+    MS r;
+    r.m = m;
+    r.s = (a0 + a1) + (b0 + b1);
+    return r;
 }
 
 // Lane-local online softmax statistics: folds kUnroll vectors into a running (max, sum of

@@ -210,3 +210,21 @@ def test_binding_constants_match_the_header():
     L = spr.lib()
     for code in range(8):                      # every status has a text
         assert len(L.spr_status_string(code).decode()) >= 2
+
+
+def test_bench_refuses_to_time_fewer_ranks_than_asked_for():
+    """`bench.py --gpus N` without a launcher starts N ranks itself, one per GPU; on a machine with
+    fewer GPUs it must stop with a clear message instead of timing one rank and printing n_gpus 1."""
+    import subprocess
+    import sys
+    have = torch.cuda.device_count()
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", str(have + 2), "--steps", "1"],
+                       capture_output=True, text=True, timeout=300,
+                       env={k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")})
+    assert r.returncode != 0
+    assert "refusing to time fewer ranks" in (r.stderr + r.stdout)
+    # a launcher whose world size disagrees with --gpus is refused as well
+    env = dict(os.environ, WORLD_SIZE="1", RANK="0", LOCAL_RANK="0")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "1"],
+                       capture_output=True, text=True, timeout=300, env=env)
+    assert r.returncode != 0 and "must agree" in (r.stderr + r.stdout)
