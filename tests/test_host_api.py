@@ -43,6 +43,9 @@ def test_workspace_bytes():
     b = wb(binding.OP_REPLACE_SAMPLE, 1000, 0, 1000, 0, 0, spr.F32)
     assert 0 < a < b and a % 256 == 0
     assert wb(binding.OP_SPRINTER_VERIFY, 32, 8, 0, 768, 256, spr.BF16) > 0
+    # K = 1: one 64-bit word per token in the ticket zone, which is a quarter of the workspace
+    assert wb(binding.OP_SPRINTER_VERIFY, 4096, 1, 0, 4096, 1024, spr.BF16) >= 256 + 4 * 8 * 4096
+    assert wb(binding.OP_SPRINTER_STEP, 4096, 1, 128256, 4096, 1024, spr.BF16) >= 256 + 4 * 8 * 4096
 
 
 def test_argument_validation_happens_on_the_host():
