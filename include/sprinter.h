@@ -145,9 +145,9 @@ int replace_sample(const void *target_logits, int64_t ldv, int V, int64_t R, con
  * (sprinter_verify) followed by the single target call for the position where the
  * verifier stopped (replace_sample on row b*seq_stride + first_reject[b], skipped
  * when every token passed).  Same arguments, results and error behaviour as those
- * two calls made one after the other with first_reject passed along; here the
- * replacement kernel is launched programmatically behind the verifier kernel, so
- * its launch latency hides in the verifier's tail, and one clear serves both.
+ * two calls made one after the other with first_reject passed along, on one
+ * workspace; for small batches the replacement kernel is launched programmatically
+ * behind the verifier kernel, so that its launch latency hides in the verifier's tail.
  *
  * target_logits [B, seq_stride, ldv] dt with seq_stride >= K rows per sequence (K, or
  * K+1 when a bonus row is kept); uniforms [B] f32; tokens [B] int32 (-1 where nothing
