@@ -290,6 +290,10 @@ int verifier_labels(const void *p_logits, const void *q_logits, int64_t ldv, con
  * and v at zero), t >= 1 the step number, loss [1] f32 (device, optional): the loss BEFORE
  * the update.  Every hidden state is read once (N*d*es bytes per step); sums have a fixed
  * order, so a step is reproducible bit for bit.
+ * Errors on the device: the gradient kernel waits for its rows with a poll limit; if a wait
+ * runs out the status word becomes SPR_ERR_TIMEOUT, no step is taken (theta, adam_m, adam_v
+ * unchanged) and *loss is NaN.  While the status word still holds SPR_ERR_TIMEOUT (it is
+ * cleared by spr_device_status) later steps on that workspace are not taken either.
  * Workspace: spr_workspace_bytes(SPR_OP_VERIFIER_TRAIN, 0, 0, 0, d, 0, dt).
  */
 int verifier_train_step(const void *hidden, const uint8_t *labels, int64_t N, int d, int dt, float *theta,
@@ -406,6 +410,20 @@ int spr_test_sprinter_verify(const void *hidden, const void *W1, const float *b1
                              float *scores, uint8_t *accept, int32_t *first_reject, void *ws, size_t ws_bytes,
                              void *cuda_stream, int bm, int bn, int splits, int cluster_n, int flags,
                              unsigned spin_limit);
+
+/*
+ * spr_test_verifier_train_step - test hook, not part of the stable interface.
+ *
+ * The paper has no counterpart.  verifier_train_step with flags bit 0 set: the gradient
+ * kernel fetches no row, so the first bounded wait of every team of warps runs out after
+ * spin_limit polls (0 = the library's limit).  The call returns SPR_OK, the status word reads
+ * SPR_ERR_TIMEOUT, theta / adam_m / adam_v are left as they were, *loss is NaN, nothing is left
+ * in flight and the workspace stays usable.  flags = 0 is verifier_train_step with that limit.
+ */
+int spr_test_verifier_train_step(const void *hidden, const uint8_t *labels, int64_t N, int d, int dt,
+                                 float *theta, float *adam_m, float *adam_v, int t, float lr, float beta1,
+                                 float beta2, float eps, float *loss, void *ws, size_t ws_bytes,
+                                 void *cuda_stream, int flags, unsigned spin_limit);
 
 /* Synchronises the stream, returns the sticky device status word of `ws`
  * (SPR_OK if nothing was detected) and clears it. */

@@ -25,7 +25,7 @@ EXPORTS = [
     "spr_host_arena_bytes", "sprinter_verify_host", "replace_sample_host", "sd_verify_host",
     "spr_set_stage_events", "replace_sample_static", "sprinter_step", "sprinter_simulate",
     "sd_shard_stats", "sd_shard_decide", "sd_shard_weights", "sd_shard_draw", "sd_shard_decide_weights",
-    "verifier_labels", "verifier_train_step", "spr_test_sprinter_verify",
+    "verifier_labels", "verifier_train_step", "spr_test_sprinter_verify", "spr_test_verifier_train_step",
 ]
 
 
@@ -92,6 +92,8 @@ def lib():
         L.verifier_labels.argtypes = [vp, vp, i64, vp, i32, i32, i32, i32, i32, vp, i32, vp, vp, vp, sz, vp]
         L.verifier_train_step.restype = i32
         L.verifier_train_step.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, i32, f32, f32, f32, f32, vp, vp, sz, vp]
+        L.spr_test_verifier_train_step.restype = i32
+        L.spr_test_verifier_train_step.argtypes = L.verifier_train_step.argtypes + [i32, C.c_uint]
         L.spr_host_arena_bytes.restype = sz
         L.spr_host_arena_bytes.argtypes = [i32, i32, i32, i32, i64, i32, i32, i32]
         L.sprinter_verify_host.restype = i32
@@ -496,9 +498,11 @@ def verifier_labels(p_logits, q_logits, V: int, draft_tokens, lambdas, ws: Works
 
 
 def verifier_train_step(hidden, labels, theta, adam_m, adam_v, t: int, lr: float, ws: Workspace,
-                        beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8, loss=None):
+                        beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8, loss=None,
+                        test_flags: int = 0, spin_limit: int = 0):
     """One Adam step on the mean BCE loss of sigmoid(b + w.s): hidden [N,d], labels u8 [N], theta /
-    adam_m / adam_v f32 [d+1] (updated in place).  Returns the loss before the step (f32 [1])."""
+    adam_m / adam_v f32 [d+1] (updated in place).  Returns the loss before the step (f32 [1]).
+    test_flags / spin_limit: the test hook spr_test_verifier_train_step instead of the public call."""
     _dev(hidden, name="hidden")
     N, d = hidden.shape
     _dev(labels, torch.uint8, "labels")
@@ -510,9 +514,14 @@ def verifier_train_step(hidden, labels, theta, adam_m, adam_v, t: int, lr: float
         raise ValueError("labels must have one entry per hidden state")
     if loss is None:
         loss = torch.empty((1,), dtype=torch.float32, device=hidden.device)
-    rc = lib().verifier_train_step(_ptr(hidden), _ptr(labels), N, d, _dt(hidden), _ptr(theta), _ptr(adam_m),
-                                   _ptr(adam_v), t, lr, beta1, beta2, eps, _ptr(loss), _ptr(ws.buf), ws.nbytes,
-                                   _stream())
+    if test_flags or spin_limit:
+        rc = lib().spr_test_verifier_train_step(_ptr(hidden), _ptr(labels), N, d, _dt(hidden), _ptr(theta),
+                                                _ptr(adam_m), _ptr(adam_v), t, lr, beta1, beta2, eps, _ptr(loss),
+                                                _ptr(ws.buf), ws.nbytes, _stream(), test_flags, spin_limit)
+    else:
+        rc = lib().verifier_train_step(_ptr(hidden), _ptr(labels), N, d, _dt(hidden), _ptr(theta), _ptr(adam_m),
+                                       _ptr(adam_v), t, lr, beta1, beta2, eps, _ptr(loss), _ptr(ws.buf), ws.nbytes,
+                                       _stream())
     _check("verifier_train_step", rc)
     return loss
 

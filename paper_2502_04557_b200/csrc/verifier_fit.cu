@@ -3,6 +3,8 @@
 // linear-layer + sigmoid verifier on the draft model's hidden states.
 #include <string.h>
 
+#include <type_traits>
+
 #include "host_util.h"
 #include "launch.h"
 #include "vocab_common.cuh"
@@ -60,144 +62,90 @@ struct TrainParams {
     float *loss;             // [1] or null
     float *part;             // [ctas, d+2]: per-CTA sums of the gradient terms, then of the loss
     int ctas;
-    int stages;              // rows a warp keeps in flight (queue variant)
+    int *status;             // the workspace's status word
+    uint32_t spin_limit;     // polls of one mbarrier before the gradient kernel gives up
+    int test_flags;          // TRAIN_TEST_NO_FETCH
 };
+enum { TRAIN_TEST_NO_FETCH = 1 };   // test hook: no row is ever fetched, so the first wait of every team runs out
 
-// Gradient pass (one resident wave of CTAs): one warp per sample, samples dealt to warps in a
-// fixed pattern; a lane keeps
-// its columns of the row in registers, so every hidden state is read from HBM exactly once.
+// Gradient pass (one resident wave of CTAs), every hidden state read from HBM exactly once:
 //   z = b + w.s,  r = sigma(z) - y,  grad_w += r s,  grad_b += r,  loss += ln(1 + e^z) - y z
-// The warps of a CTA add their sums in warp order; the CTA's sums go to part[blockIdx.x].
-template <typename T, int VPL>
-__global__ void __launch_bounds__(kThreads, VPL <= 3 ? 3 : (VPL <= 8 ? 2 : 1)) train_grad_kernel(const TrainParams prm)
+// Rows are dealt to teams of warps in a fixed pattern, the teams of a CTA add their sums in team
+// order and the CTA's sums go to part[blockIdx.x]: the result does not depend on timing.
+// Rows go through shared memory.  A team of WPR warps (one warp, or two for rows
+// of more than 8 vectors per lane) owns a ring of SLOTS row buffers, each filled by ONE
+// bulk copy (a row is contiguous) that signals the slot's mbarrier.  The team works on R rows
+// at a time straight out of the ring - their logits are independent chains (dot product, warp
+// sum, sigmoid), which hides those latencies with few warps on the SM - while the other
+// SLOTS - R rows are on their way.  A lane keeps its columns of the weights and of the
+// gradient sums in registers; with two warps per row each warp has half of the columns and the
+// two halves of a dot product meet in shared memory.  A slot is refilled as soon as both
+// passes over it are done.
+constexpr uint32_t kRingSpin = 1u << 22;      // polls of one mbarrier before the kernel gives up
+
+__device__ __forceinline__ uint32_t ring_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool ring_poll(uint64_t *bar, uint32_t parity)
 {
-    constexpr int N = Vec<T>::N;
-    extern __shared__ float smem[];
-    const int d = prm.d;
-    float *sw = smem;              // [d] weights
-    float *red = smem + d;         // [d + 2] CTA sums
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int nv = d / N;          // vectors per row
-    for (int j = tid; j < d; j += kThreads) sw[j] = prm.theta[j];
-    const float bias = prm.theta[d];
-    __syncthreads();
-
-    uint64_t acc[VPL * N / 2];       // packed pairs of fp32 sums (two columns each)
-#pragma unroll
-    for (int e = 0; e < VPL * N / 2; ++e) acc[e] = pack2(0.f, 0.f);
-    double acc_b = 0.0, acc_loss = 0.0;   // same-signed addends: fp32 sums would drift
-    const T *base = static_cast<const T *>(prm.hidden);
-    constexpr bool kPrefetch = VPL <= 4;   // short rows: keep the next row in flight as well
-    auto load_row = [&](int64_t row, uint4 (&dst)[VPL], float &y) {
-        const uint4 *x = reinterpret_cast<const uint4 *>(base + row * d);
-#pragma unroll
-        for (int j = 0; j < VPL; ++j) {
-            const int vi = j * 32 + lane;
-            dst[j] = vi < nv ? ld_stream(x + vi) : make_uint4(0u, 0u, 0u, 0u);
-        }
-        y = (float)prm.labels[row];
-    };
-    const int64_t stride = (int64_t)gridDim.x * kWarps;
-    int64_t row = (int64_t)blockIdx.x * kWarps + warp;
-    uint4 raw[VPL];
-    float y = 0.f;
-    if (row < prm.N) load_row(row, raw, y);
-    for (; row < prm.N; row += stride) {
-        uint4 nxt[VPL];
-        float y_nxt = 0.f;
-        const bool more = row + stride < prm.N;
-        if (kPrefetch && more) load_row(row + stride, nxt, y_nxt);
-        uint64_t dot2 = pack2(0.f, 0.f);   // even and odd columns apart
-#pragma unroll
-        for (int j = 0; j < VPL; ++j) {
-            const int vi = j * 32 + lane;
-            if (vi < nv) {
-                float f[N];
-                Vec<T>::unpack(raw[j], f);
-#pragma unroll
-                for (int e = 0; e < N; e += 2)
-                    dot2 = fma2(pack2(f[e], f[e + 1]), *reinterpret_cast<const uint64_t *>(&sw[vi * N + e]), dot2);
-            }
-        }
-        float d_even, d_odd;
-        unpack2(dot2, d_even, d_odd);
-        const float z = warp_sum(d_even + d_odd) + bias;
-        const float r = 1.f / (1.f + expf(-z)) - y;
-        const uint64_t r2 = pack2(r, r);
-#pragma unroll
-        for (int j = 0; j < VPL; ++j) {
-            float f[N];
-            Vec<T>::unpack(raw[j], f);     // zero beyond the row
-#pragma unroll
-            for (int e = 0; e < N; e += 2)
-                acc[(j * N + e) / 2] = fma2(r2, pack2(f[e], f[e + 1]), acc[(j * N + e) / 2]);
-        }
-        acc_b += (double)r;
-        acc_loss += (double)(fmaxf(z, 0.f) + log1pf(expf(-fabsf(z))) - y * z);
-        if (kPrefetch) {
-#pragma unroll
-            for (int j = 0; j < VPL; ++j) raw[j] = nxt[j];
-            y = y_nxt;
-        } else if (more) {
-            load_row(row + stride, raw, y);
-        }
-    }
-
-    for (int w = 0; w < kWarps; ++w) {     // fixed order: warp 0 stores, the others add
-        if (warp == w) {
-#pragma unroll
-            for (int j = 0; j < VPL; ++j) {
-                const int vi = j * 32 + lane;
-                if (vi < nv) {
-#pragma unroll
-                    for (int e = 0; e < N; e += 2) {
-                        float lo, hi;
-                        unpack2(acc[(j * N + e) / 2], lo, hi);
-                        float *dst = red + vi * N + e;
-                        dst[0] = w == 0 ? lo : dst[0] + lo;
-                        dst[1] = w == 0 ? hi : dst[1] + hi;
-                    }
-                }
-            }
-            if (lane == 0) {
-                red[d] = w == 0 ? (float)acc_b : red[d] + (float)acc_b;
-                red[d + 1] = w == 0 ? (float)acc_loss : red[d + 1] + (float)acc_loss;
-            }
-        }
-        __syncthreads();
-    }
-    float *out = prm.part + (int64_t)blockIdx.x * (d + 2);
-    for (int j = tid; j < d + 2; j += kThreads) out[j] = red[j];
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(ring_addr(bar)), "r"(parity)
+        : "memory");
+    return done != 0u;
 }
-
-// Short rows (at most 4 vectors per lane, d <= 1024 bf16): the same pass, but a warp's next
-// `depth` rows are already on their way into shared memory (cp.async, 16 bytes per lane per
-// copy) while it works on the current one, and the weights stay in registers.  A lane reads back
-// only what it copied itself, so the queue needs no barrier: cp.async.wait_group orders a lane's
-// own copies.  With 16 warps and 8 rows each an SM has ~190 KB of hidden states in flight.
-__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
+__device__ __forceinline__ bool ring_wait(uint64_t *bar, uint32_t parity, uint32_t limit)
 {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
-                 "l"(gmem_src)
+    for (uint32_t n = 0; n < limit; ++n)
+        if (ring_poll(bar, parity)) return true;
+    return false;
+}
+// one row: global -> shared, completion counted in bytes on the slot's mbarrier (one lane calls)
+__device__ __forceinline__ void ring_fetch(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(ring_addr(bar)), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     ring_addr(dst)),
+                 "l"(src), "r"(bytes), "r"(ring_addr(bar))
                  : "memory");
 }
+__device__ __forceinline__ bool feeder_team_has_copies(const TrainParams &prm) { return !(prm.test_flags & TRAIN_TEST_NO_FETCH); }
+// the warps of one team meet (a warp alone: its lanes)
+template <int WPR>
+__device__ __forceinline__ void team_sync(int team)
+{
+    if (WPR == 1) __syncwarp();
+    else asm volatile("bar.sync %0, %1;" ::"r"(team + 1), "r"(WPR * 32) : "memory");
+}
 
-template <typename T, int VPL>
-__global__ void __launch_bounds__(kThreads, 2) train_grad_queue_kernel(const TrainParams prm)
+__host__ __device__ constexpr int ring_ctas_per_sm(int vpl, int wpr) { return wpr == 1 && vpl <= 4 ? 2 : 1; }
+
+template <typename T, int VPL, int WPR, int R, int SLOTS>
+__global__ void __launch_bounds__(kThreads, ring_ctas_per_sm(VPL, WPR)) train_grad_ring_kernel(const TrainParams prm)
 {
     constexpr int N = Vec<T>::N;
-    extern __shared__ __align__(16) unsigned char qsmem[];
-    const int d = prm.d, depth = prm.stages;
+    constexpr int kTeams = kWarps / WPR;
+    constexpr int kSlotVecs = VPL * WPR * 32;
+    extern __shared__ __align__(128) unsigned char rsmem[];
+    __shared__ __align__(8) uint64_t bars[kTeams][SLOTS];
+    __shared__ float halves[kTeams][R][2];    // WPR = 2: the two warps' parts of the R dot products
+    __shared__ int team_fail[kTeams];         // WPR = 2: a wait of one of the team's warps ran out
+    const int d = prm.d;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int nv = d / N;                     // vectors per row
-    const int slot_vecs = VPL * 32;           // vectors per queue slot
-    uint4 *queue = reinterpret_cast<uint4 *>(qsmem) + (size_t)warp * depth * slot_vecs;
-    float *red = reinterpret_cast<float *>(qsmem + (size_t)kWarps * depth * slot_vecs * 16);   // [d + 2] CTA sums
+    const int team = warp / WPR, half = warp % WPR;
+    const int nv = d / N;
+    const uint32_t row_bytes = (uint32_t)d * (uint32_t)sizeof(T);   // a multiple of 16: d is a multiple of N
+    uint4 *ring = reinterpret_cast<uint4 *>(rsmem) + (size_t)team * SLOTS * kSlotVecs;
+    float *red = reinterpret_cast<float *>(rsmem + (size_t)kTeams * SLOTS * kSlotVecs * 16);   // [d + 2]
+    uint64_t *bar = bars[team];
+    const int v0 = half * VPL * 32 + lane;    // this lane's vectors of a row: v0 + 32 j
 
     uint64_t w2[VPL * N / 2];                 // this lane's columns of the weight vector
 #pragma unroll
     for (int j = 0; j < VPL; ++j) {
-        const int vi = j * 32 + lane;
+        const int vi = v0 + j * 32;
 #pragma unroll
         for (int e = 0; e < N; e += 2)
             w2[(j * N + e) / 2] = vi < nv ? pack2(prm.theta[vi * N + e], prm.theta[vi * N + e + 1]) : pack2(0.f, 0.f);
@@ -206,87 +154,185 @@ __global__ void __launch_bounds__(kThreads, 2) train_grad_queue_kernel(const Tra
     uint64_t acc[VPL * N / 2];
 #pragma unroll
     for (int e = 0; e < VPL * N / 2; ++e) acc[e] = pack2(0.f, 0.f);
-    double acc_b = 0.0, acc_loss = 0.0;
+    double acc_b = 0.0, acc_loss = 0.0;       // per lane: see the note on z_keep below
+    float z_keep = 0.f, y_keep = 0.f, r_keep = 0.f;
+    int kept = 0;
 
     const T *base = static_cast<const T *>(prm.hidden);
-    const int64_t stride = (int64_t)gridDim.x * kWarps;
-    const int64_t first = (int64_t)blockIdx.x * kWarps + warp;
-    const int64_t n = first < prm.N ? (prm.N - first + stride - 1) / stride : 0;   // this warp's rows
-    auto enqueue = [&](int64_t i, int slot) {       // row i of this warp -> queue slot (one commit group)
-        if (i < n) {
-            const uint4 *x = reinterpret_cast<const uint4 *>(base + (first + i * stride) * d);
+    const int64_t stride = (int64_t)gridDim.x * kTeams;
+    const int64_t first = (int64_t)blockIdx.x * kTeams + team;
+    const int n = first < prm.N ? (int)((prm.N - first + stride - 1) / stride) : 0;   // this team's rows
+    const bool feeder = half == 0 && lane == 0 && !(prm.test_flags & TRAIN_TEST_NO_FETCH);
+    const uint32_t limit = prm.spin_limit;
+    if (half == 0 && lane == 0) {
+        team_fail[team] = 0;
+        for (int s = 0; s < SLOTS; ++s)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(ring_addr(&bar[s])) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (int i = 0; feeder && i < SLOTS && i < n; ++i)
+            ring_fetch(ring + i * kSlotVecs, base + (first + i * stride) * d, row_bytes, &bar[i]);
+    }
+    team_sync<WPR>(team);
+
+    // Labels: lane l holds the label of row (32 b + l) of this team, the batch after it is on its
+    // way - a label fetched next to its row would cost a full trip to memory per group of rows.
+    auto label_batch = [&](int i0) { return i0 + lane < n ? (float)prm.labels[first + (int64_t)(i0 + lane) * stride] : 0.f; };
+    float y_batch = label_batch(0), y_batch_next = label_batch(32);
+    int slot = 0;                             // ring slot of row i
+    uint32_t parity = 0;                      // of that slot's current fill
+    bool ok = true;
+    int fail_at = 0;                          // first row of the group whose wait ran out
+
+    // rows [i, i + RR) of this team, RR <= R
+    auto group = [&](auto rr_tag, int i) {
+        constexpr int RR = decltype(rr_tag)::value;
+        int s[RR];
+        float y[RR];
+#pragma unroll
+        for (int r = 0; r < RR; ++r) {
+            s[r] = slot + r >= SLOTS ? slot + r - SLOTS : slot + r;
+            const int idx = i + r;
+            if ((idx & 31) == 0 && idx > 0) {
+                y_batch = y_batch_next;
+                y_batch_next = label_batch(idx + 32);
+            }
+            y[r] = __shfl_sync(0xffffffffu, y_batch, idx & 31);
+        }
+#pragma unroll
+        for (int r = 0; r < RR; ++r) ok = ok && ring_wait(&bar[s[r]], slot + r >= SLOTS ? parity ^ 1u : parity, limit);
+        if (WPR > 1) {
+            // a team leaves together: the barriers below need both of its warps
+            if (lane == 0 && !ok) team_fail[team] = 1;
+        }
+        if (WPR == 1 && !ok) {
+            fail_at = i;
+            return;
+        }
+        uint64_t dot[RR][2];
+#pragma unroll
+        for (int r = 0; r < RR; ++r) dot[r][0] = dot[r][1] = pack2(0.f, 0.f);
+        if (ok) {
 #pragma unroll
             for (int j = 0; j < VPL; ++j) {
-                const int vi = j * 32 + lane;
-                if (vi < nv) cp_async16(queue + slot * slot_vecs + vi, x + vi);
+                const int vi = v0 + j * 32;
+#pragma unroll
+                for (int r = 0; r < RR; ++r) {
+                    const uint4 x = vi < nv ? ring[s[r] * kSlotVecs + vi] : make_uint4(0u, 0u, 0u, 0u);
+                    float f[N];
+                    Vec<T>::unpack(x, f);
+#pragma unroll
+                    for (int e = 0; e < N; e += 2)
+                        dot[r][j & 1] = fma2(pack2(f[e], f[e + 1]), w2[(j * N + e) / 2], dot[r][j & 1]);
+                }
             }
         }
-        asm volatile("cp.async.commit_group;" ::: "memory");
+        float zs[RR];
+#pragma unroll
+        for (int r = 0; r < RR; ++r) {
+            float a0, a1, b0, b1;
+            unpack2(dot[r][0], a0, a1);
+            unpack2(dot[r][1], b0, b1);
+            zs[r] = warp_sum((a0 + a1) + (b0 + b1));
+        }
+        if (WPR > 1) {
+            if (lane == 0 && ok) {
+#pragma unroll
+                for (int r = 0; r < RR; ++r) halves[team][r][half] = zs[r];
+            }
+            team_sync<WPR>(team);
+#pragma unroll
+            for (int r = 0; r < RR; ++r) zs[r] = halves[team][r][0] + halves[team][r][1];
+            if (team_fail[team] != 0) ok = false;
+            if (!ok) {
+                fail_at = i;
+                return;
+            }
+        }
+        uint64_t res2[RR];
+#pragma unroll
+        for (int r = 0; r < RR; ++r) {
+            const float z = zs[r] + bias;
+            const float res = 1.f / (1.f + expf(-z)) - y[r];
+            res2[r] = pack2(res, res);
+            // The bias-gradient and loss terms of a row are one lane's business: lane (row count
+            // mod 32) keeps z and y, and every 32 rows each lane works off the row it kept.
+            if (lane == (kept & 31)) {
+                z_keep = z;
+                y_keep = y[r];
+                r_keep = res;
+            }
+            if ((++kept & 31) == 0) {
+                acc_b += (double)r_keep;
+                acc_loss += (double)(fmaxf(z_keep, 0.f) + log1pf(expf(-fabsf(z_keep))) - y_keep * z_keep);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) {
+            const int vi = v0 + j * 32;
+#pragma unroll
+            for (int r = 0; r < RR; ++r) {
+                const uint4 x = vi < nv ? ring[s[r] * kSlotVecs + vi] : make_uint4(0u, 0u, 0u, 0u);
+                float f[N];
+                Vec<T>::unpack(x, f);
+#pragma unroll
+                for (int e = 0; e < N; e += 2)
+                    acc[(j * N + e) / 2] = fma2(res2[r], pack2(f[e], f[e + 1]), acc[(j * N + e) / 2]);
+            }
+        }
+        team_sync<WPR>(team);                  // the whole team is done with the slots: refill them
+        if (feeder) {
+#pragma unroll
+            for (int r = 0; r < RR; ++r) {
+                const int nx = i + r + SLOTS;
+                if (nx < n) ring_fetch(ring + s[r] * kSlotVecs, base + (first + nx * stride) * d, row_bytes, &bar[s[r]]);
+            }
+        }
+        slot += RR;
+        if (slot >= SLOTS) {
+            slot -= SLOTS;
+            parity ^= 1u;
+        }
     };
-    for (int s = 0; s < depth; ++s) enqueue(s, s);
-    float y = n > 0 ? (float)prm.labels[first] : 0.f;
-    int slot = 0;
-    for (int64_t i = 0; i < n; ++i) {
-        const float y_next = i + 1 < n ? (float)prm.labels[first + (i + 1) * stride] : 0.f;
-        // all but the newest depth-1 groups are complete: row i has landed
-        if (depth == 8) asm volatile("cp.async.wait_group 7;" ::: "memory");
-        else if (depth == 4) asm volatile("cp.async.wait_group 3;" ::: "memory");
-        else asm volatile("cp.async.wait_group 0;" ::: "memory");
-        uint4 raw[VPL];
-#pragma unroll
-        for (int j = 0; j < VPL; ++j) {
-            const int vi = j * 32 + lane;
-            raw[j] = vi < nv ? queue[slot * slot_vecs + vi] : make_uint4(0u, 0u, 0u, 0u);
-        }
-        enqueue(i + depth, slot);               // the slot is free again: its values are in registers
-        uint64_t dot2 = pack2(0.f, 0.f);
-#pragma unroll
-        for (int j = 0; j < VPL; ++j) {
-            float f[N];
-            Vec<T>::unpack(raw[j], f);
-#pragma unroll
-            for (int e = 0; e < N; e += 2) dot2 = fma2(pack2(f[e], f[e + 1]), w2[(j * N + e) / 2], dot2);
-        }
-        float d_even, d_odd;
-        unpack2(dot2, d_even, d_odd);
-        const float z = warp_sum(d_even + d_odd) + bias;
-        const float r = 1.f / (1.f + expf(-z)) - y;
-        const uint64_t r2 = pack2(r, r);
-#pragma unroll
-        for (int j = 0; j < VPL; ++j) {
-            float f[N];
-            Vec<T>::unpack(raw[j], f);
-#pragma unroll
-            for (int e = 0; e < N; e += 2)
-                acc[(j * N + e) / 2] = fma2(r2, pack2(f[e], f[e + 1]), acc[(j * N + e) / 2]);
-        }
-        acc_b += (double)r;
-        acc_loss += (double)(fmaxf(z, 0.f) + log1pf(expf(-fabsf(z))) - y * z);
-        y = y_next;
-        if (++slot == depth) slot = 0;
+    int i = 0;
+    for (; ok && i + R <= n; i += R) group(std::integral_constant<int, R>{}, i);
+    for (; ok && i < n; ++i) group(std::integral_constant<int, 1>{}, i);
+    if (!ok) {
+        // A wait ran out: report it, then give the copies still on their way the same bounded
+        // time to land before the CTA's shared memory goes away: rows fail_at .. fail_at + slots.
+        if (lane == 0) raise_status(prm.status, SPR_ERR_TIMEOUT);
+        for (int k = fail_at; feeder_team_has_copies(prm) && k < n && k < fail_at + SLOTS; ++k)
+            ring_wait(&bar[k % SLOTS], (uint32_t)(k / SLOTS) & 1u, limit);
     }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    __syncthreads();
 
-    for (int w = 0; w < kWarps; ++w) {     // fixed order: warp 0 stores, the others add
-        if (warp == w) {
+    if (lane < (kept & 31)) {      // rows kept since the last full round of 32
+        acc_b += (double)r_keep;
+        acc_loss += (double)(fmaxf(z_keep, 0.f) + log1pf(expf(-fabsf(z_keep))) - y_keep * z_keep);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {   // lanes in a fixed (butterfly) order
+        acc_b += __shfl_xor_sync(0xffffffffu, acc_b, o);
+        acc_loss += __shfl_xor_sync(0xffffffffu, acc_loss, o);
+    }
+    __syncthreads();
+    for (int t = 0; t < kTeams; ++t) {     // fixed order: team 0 stores, the others add
+        if (team == t) {
 #pragma unroll
             for (int j = 0; j < VPL; ++j) {
-                const int vi = j * 32 + lane;
+                const int vi = v0 + j * 32;
                 if (vi < nv) {
 #pragma unroll
                     for (int e = 0; e < N; e += 2) {
                         float lo, hi;
                         unpack2(acc[(j * N + e) / 2], lo, hi);
                         float *dst = red + vi * N + e;
-                        dst[0] = w == 0 ? lo : dst[0] + lo;
-                        dst[1] = w == 0 ? hi : dst[1] + hi;
+                        dst[0] = t == 0 ? lo : dst[0] + lo;
+                        dst[1] = t == 0 ? hi : dst[1] + hi;
                     }
                 }
             }
-            if (lane == 0) {
-                red[d] = w == 0 ? (float)acc_b : red[d] + (float)acc_b;
-                red[d + 1] = w == 0 ? (float)acc_loss : red[d + 1] + (float)acc_loss;
+            if (half == 0 && lane == 0) {
+                red[d] = t == 0 ? (float)acc_b : red[d] + (float)acc_b;
+                red[d + 1] = t == 0 ? (float)acc_loss : red[d + 1] + (float)acc_loss;
             }
         }
         __syncthreads();
@@ -302,6 +348,11 @@ __global__ void __launch_bounds__(256) train_adam_kernel(const TrainParams prm)
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     const int d = prm.d;
     if (j > d + 1) return;
+    if (*reinterpret_cast<volatile int *>(prm.status) == SPR_ERR_TIMEOUT) {
+        // the gradient pass gave up: no step is taken, the loss reads NaN
+        if (j == d + 1 && prm.loss) *prm.loss = __int_as_float(0x7fc00000);
+        return;
+    }
     double sum = 0.0;
     for (int c = 0; c < prm.ctas; ++c) sum += (double)prm.part[(int64_t)c * (d + 2) + j];
     sum /= (double)prm.N;
@@ -319,46 +370,24 @@ __global__ void __launch_bounds__(256) train_adam_kernel(const TrainParams prm)
     prm.theta[j] = (float)((double)prm.theta[j] - (double)prm.lr * m_hat / (sqrt(v_hat) + (double)prm.eps));
 }
 
-template <typename T, int VPL>
-cudaError_t launch_grad(const TrainParams &tp, cudaStream_t st)
-{
-    const size_t smem = sizeof(float) * (2 * (size_t)tp.d + 2);
-    cudaError_t e = cudaFuncSetAttribute(train_grad_kernel<T, VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
-    if (e != cudaSuccess) return e;
-    // one full wave: as many CTAs as are resident at once, so that all of them finish together
-    int per_sm = 0, dev = 0, sms = 0;
-    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, train_grad_kernel<T, VPL>, kThreads, smem)) !=
-            cudaSuccess ||
-        (e = cudaGetDevice(&dev)) != cudaSuccess ||
-        (e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
-        return e;
-    TrainParams p = tp;
-    p.ctas = (int)max((int64_t)1, min((int64_t)min(kTrainMaxCtas, per_sm * sms), (tp.N + kWarps - 1) / kWarps));
-    train_grad_kernel<T, VPL><<<p.ctas, kThreads, smem, st>>>(p);
-    train_adam_kernel<<<(tp.d + 2 + 255) / 256, 256, 0, st>>>(p);
-    return cudaGetLastError();
-}
-
-template <typename T, int VPL>
-cudaError_t launch_grad_queue(const TrainParams &tp, cudaStream_t st)
+template <typename T, int VPL, int WPR, int R, int SLOTS>
+cudaError_t launch_grad_ring(const TrainParams &tp, cudaStream_t st)
 {
     TrainParams p = tp;
-    const size_t slot_bytes = (size_t)kWarps * VPL * 32 * 16;       // one queue slot of every warp
-    p.stages = slot_bytes * 8 <= 96 * 1024 ? 8 : 4;
-    const size_t smem = slot_bytes * p.stages + sizeof(float) * ((size_t)tp.d + 2);
-    cudaError_t e = cudaFuncSetAttribute(train_grad_queue_kernel<T, VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
+    constexpr int kTeams = kWarps / WPR;
+    const size_t smem = (size_t)kTeams * SLOTS * VPL * WPR * 32 * 16 + sizeof(float) * ((size_t)tp.d + 2);
+    auto kernel = train_grad_ring_kernel<T, VPL, WPR, R, SLOTS>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     int per_sm = 0, dev = 0, sms = 0;
     if (e != cudaSuccess ||
-        (e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, train_grad_queue_kernel<T, VPL>, kThreads, smem)) !=
-            cudaSuccess ||
+        (e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, smem)) != cudaSuccess ||
         (e = cudaGetDevice(&dev)) != cudaSuccess ||
         (e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
         return e;
     if (per_sm < 1) return cudaErrorInvalidConfiguration;
-    p.ctas = (int)max((int64_t)1, min((int64_t)min(kTrainMaxCtas, per_sm * sms), (tp.N + kWarps - 1) / kWarps));
-    train_grad_queue_kernel<T, VPL><<<p.ctas, kThreads, smem, st>>>(p);
+    // one full wave: as many CTAs as are resident at once, so that all of them finish together
+    p.ctas = (int)max((int64_t)1, min((int64_t)min(kTrainMaxCtas, per_sm * sms), (tp.N + kTeams - 1) / kTeams));
+    kernel<<<p.ctas, kThreads, smem, st>>>(p);
     train_adam_kernel<<<(tp.d + 2 + 255) / 256, 256, 0, st>>>(p);
     return cudaGetLastError();
 }
@@ -367,12 +396,15 @@ template <typename T>
 cudaError_t launch_grad_any(const TrainParams &tp, cudaStream_t st)
 {
     const int vpl = (tp.d / Vec<T>::N + 31) / 32;
-    if (vpl <= 1) return launch_grad_queue<T, 1>(tp, st);
-    if (vpl <= 2) return launch_grad_queue<T, 2>(tp, st);
-    if (vpl <= 3) return launch_grad_queue<T, 3>(tp, st);
-    if (vpl <= 4) return launch_grad_queue<T, 4>(tp, st);
-    if (vpl <= 8) return launch_grad<T, 8>(tp, st);
-    return launch_grad<T, 16>(tp, st);
+    // rows per group and ring slots: about 190 KB of ring per SM (two CTAs share it up to 4 vectors per lane)
+    if (vpl <= 1) return launch_grad_ring<T, 1, 1, 4, 12>(tp, st);
+    if (vpl <= 2) return launch_grad_ring<T, 2, 1, 4, 12>(tp, st);
+    if (vpl <= 3) return launch_grad_ring<T, 3, 1, 4, 8>(tp, st);
+    if (vpl <= 4) return launch_grad_ring<T, 4, 1, 3, 6>(tp, st);
+    if (vpl <= 6) return launch_grad_ring<T, 6, 1, 2, 8>(tp, st);
+    if (vpl <= 8) return launch_grad_ring<T, 8, 1, 2, 6>(tp, st);
+    if (vpl <= 12) return launch_grad_ring<T, 6, 2, 2, 8>(tp, st);
+    return launch_grad_ring<T, 8, 2, 2, 6>(tp, st);
 }
 
 
@@ -440,9 +472,9 @@ int verifier_labels(const void *p_logits, const void *q_logits, int64_t ldv, con
     return finish(e);
 }
 
-int verifier_train_step(const void *hidden, const uint8_t *labels, int64_t N, int d, int dt, float *theta,
-                        float *adam_m, float *adam_v, int t, float lr, float beta1, float beta2, float eps,
-                        float *loss, void *ws, size_t ws_bytes, void *cuda_stream)
+static int train_step(const void *hidden, const uint8_t *labels, int64_t N, int d, int dt, float *theta,
+                      float *adam_m, float *adam_v, int t, float lr, float beta1, float beta2, float eps,
+                      float *loss, void *ws, size_t ws_bytes, void *cuda_stream, int flags, unsigned spin_limit)
 {
     if (!dtype_ok(dt)) return SPR_ERR_UNSUPPORTED;
     if (N < 0 || d <= 0 || t < 1 || !(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) ||
@@ -477,8 +509,29 @@ int verifier_train_step(const void *hidden, const uint8_t *labels, int64_t N, in
     tp.eps = eps;
     tp.loss = loss;
     tp.part = at<float>(ws, part_off);
+    tp.status = at<int>(ws, 0);
+    tp.spin_limit = spin_limit ? spin_limit : kRingSpin;
+    tp.test_flags = flags;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     return finish(dt == SPR_F32 ? launch_grad_any<float>(tp, st) : launch_grad_any<__nv_bfloat16>(tp, st));
+}
+
+int verifier_train_step(const void *hidden, const uint8_t *labels, int64_t N, int d, int dt, float *theta,
+                        float *adam_m, float *adam_v, int t, float lr, float beta1, float beta2, float eps,
+                        float *loss, void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    return train_step(hidden, labels, N, d, dt, theta, adam_m, adam_v, t, lr, beta1, beta2, eps, loss, ws, ws_bytes,
+                      cuda_stream, 0, 0u);
+}
+
+int spr_test_verifier_train_step(const void *hidden, const uint8_t *labels, int64_t N, int d, int dt, float *theta,
+                                 float *adam_m, float *adam_v, int t, float lr, float beta1, float beta2, float eps,
+                                 float *loss, void *ws, size_t ws_bytes, void *cuda_stream, int flags,
+                                 unsigned spin_limit)
+{
+    if (flags & ~TRAIN_TEST_NO_FETCH) return SPR_ERR_INVALID_ARG;
+    return train_step(hidden, labels, N, d, dt, theta, adam_m, adam_v, t, lr, beta1, beta2, eps, loss, ws, ws_bytes,
+                      cuda_stream, flags, spin_limit);
 }
 
 }  // extern "C"

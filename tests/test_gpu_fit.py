@@ -110,6 +110,11 @@ def run_steps(spr, S, y, steps, lr, theta0=None, **hyper):
     (5000, 768, torch.bfloat16), (1, 768, torch.bfloat16), (7, 64, torch.bfloat16), (20000, 256, torch.bfloat16),
     (3000, 2048, torch.bfloat16), (2000, 4096, torch.bfloat16), (4001, 1000, torch.bfloat16),
     (3000, 100, torch.float32), (1500, 2048, torch.float32), (999, 4, torch.float32),
+    # many rows per team of warps: the shared-memory rings go round several times
+    (60000, 768, torch.bfloat16), (40000, 1024, torch.bfloat16), (30000, 1536, torch.bfloat16),
+    (24000, 2048, torch.bfloat16), (16000, 4096, torch.bfloat16), (12000, 2560, torch.bfloat16),
+    (14001, 3072, torch.bfloat16), (70000, 128, torch.bfloat16), (20000, 1024, torch.float32),
+    (9000, 2048, torch.float32), (11000, 1240, torch.float32),
 ], ids=lambda v: str(v).replace("torch.", ""))
 def test_train_steps_match_the_oracle(spr, N, d, dtype):
     """fp32 sums on the GPU against float64: the loss agrees to 2e-5 relative, and since an Adam
@@ -155,6 +160,37 @@ def test_train_is_reproducible_and_rejects_unsupported_widths(spr):
                                         torch.zeros(4, dtype=torch.uint8, device="cuda"), z, z.clone(), z.clone(), 1,
                                         0.01, ws)
         assert e.value.status == 2
+
+
+@pytest.mark.parametrize("N,d,dtype", [(5000, 768, torch.bfloat16), (3000, 2048, torch.bfloat16),
+                                       (2000, 4096, torch.bfloat16), (9, 64, torch.float32)],
+                         ids=lambda v: str(v).replace("torch.", ""))
+def test_train_bounded_wait_runs_out_and_nothing_is_stepped(spr, N, d, dtype):
+    """No row is ever fetched (test flag): every team's first wait expires after a few thousand
+    polls, the launch ends by itself, reports SPR_ERR_TIMEOUT and takes no step; the next call on
+    the same workspace is a normal step."""
+    S, y = teacher_problem(N, d, dtype, seed=21)
+    ws = spr.Workspace(spr.workspace_bytes(bd(spr).OP_VERIFIER_TRAIN, 0, 0, 0, d, 0, bd(spr)._dt(S)))
+    Sg, yg = S.cuda(), y.cuda()
+    g = torch.Generator().manual_seed(22)
+    theta = (0.05 * torch.randn(d + 1, generator=g)).cuda()
+    m, v = torch.rand(d + 1, generator=g).cuda() * 1e-3, torch.rand(d + 1, generator=g).cuda() * 1e-6
+    ref = [x.clone() for x in (theta, m, v)]
+    want = [x.clone() for x in ref]
+    loss_ok = bd(spr).verifier_train_step(Sg, yg, *want, 3, 0.01, ws)       # warm: module load, attributes
+    assert ws.device_status() == 0
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    loss = bd(spr).verifier_train_step(Sg, yg, theta, m, v, 3, 0.01, ws, test_flags=1, spin_limit=4000)
+    b.record()
+    assert ws.device_status() == 5                                          # SPR_ERR_TIMEOUT
+    assert ws.device_status() == 0                                          # reading the status clears it
+    assert torch.isnan(loss).all()
+    assert all(torch.equal(x, r) for x, r in zip((theta, m, v), ref)), "a failed pass must not take a step"
+    assert a.elapsed_time(b) < 50.0, "the failing launch must end quickly"
+    loss = bd(spr).verifier_train_step(Sg, yg, theta, m, v, 3, 0.01, ws)
+    assert ws.device_status() == 0
+    assert torch.equal(loss, loss_ok) and all(torch.equal(x, w) for x, w in zip((theta, m, v), want))
 
 
 def test_labels_then_training_then_the_verifier_call(spr):
