@@ -34,19 +34,7 @@ __global__ void __launch_bounds__(kThreads, 4) sd_row_stats_kernel(const SdParam
     const int V = prm.V;
 
     MS mp{neg_inf(), 0.f}, mq{neg_inf(), 0.f};
-    uint4 rp[kUnroll], rq[kUnroll];
-    load_step<T>(prow, first_p, V, lane, rp);
-    load_step<T>(qrow, first_q, V, lane, rq);
-#pragma unroll
-    for (int it = 0; it < ITERS; ++it) {
-        const int nxt = (it + 1) * kWarps * kStep;
-        const bool more = it + 1 < ITERS && min(first_p, first_q) + nxt < V;   // warp-uniform
-        online_update<T>(rp, mp.m, mp.s);
-        if (more) load_step<T>(prow, first_p + nxt, V, lane, rp);
-        online_update<T>(rq, mq.m, mq.s);
-        if (more) load_step<T>(qrow, first_q + nxt, V, lane, rq);
-        if (!more) break;
-    }
+    stream_segment<T, ITERS, true>(prow, qrow, first_p, first_q, V, lane, mp, mq);
     pdl_trigger();                       // the correction draw may be scheduled behind this grid
     mp = warp_ms(mp);
     mq = warp_ms(mq);

@@ -27,21 +27,7 @@ __device__ __forceinline__ void shard_segment(const T *prow, const T *qrow, int 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int first_p = c * kSegment + warp * kStep - row_pad(prow);
     const int first_q = HAS_Q ? c * kSegment + warp * kStep - row_pad(qrow) : first_p;
-    uint4 rp[kUnroll], rq[kUnroll];
-    load_step<T>(prow, first_p, V, lane, rp);
-    if (HAS_Q) load_step<T>(qrow, first_q, V, lane, rq);
-#pragma unroll
-    for (int it = 0; it < ITERS; ++it) {
-        const int nxt = (it + 1) * kWarps * kStep;
-        const bool more = it + 1 < ITERS && min(first_p, first_q) + nxt < V;   // warp-uniform
-        online_update<T>(rp, mp.m, mp.s);
-        if (more) load_step<T>(prow, first_p + nxt, V, lane, rp);
-        if (HAS_Q) {
-            online_update<T>(rq, mq.m, mq.s);
-            if (more) load_step<T>(qrow, first_q + nxt, V, lane, rq);
-        }
-        if (!more) break;
-    }
+    stream_segment<T, ITERS, HAS_Q>(prow, qrow, first_p, first_q, V, lane, mp, mq);
 }
 
 template <typename T>

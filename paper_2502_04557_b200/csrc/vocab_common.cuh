@@ -228,4 +228,61 @@ __device__ __forceinline__ void load_step(const T *__restrict__ row, int first, 
     }
 }
 
+// One warp's share of a row segment: its ITERS steps (warp steps are kWarps steps apart),
+// starting at element first_p of the p row and first_q of the q row (HAS_Q), folded into the
+// lane-local statistics.  The loads of a warp's next step are issued before the current one is
+// consumed.  When every step is made of whole aligned vectors inside the row(s) - warp-uniform,
+// and true for all but the warps at a row's ends - the loop carries no condition at all, which
+// the compiler unrolls and schedules freely (4 % of the row-statistics pass); same arithmetic in
+// the same order either way.
+template <typename T, int ITERS, bool HAS_Q>
+__device__ __forceinline__ void stream_segment(const T *__restrict__ prow, const T *__restrict__ qrow, int first_p,
+                                               int first_q, int V, int lane, MS &mp, MS &mq)
+{
+    constexpr int N = Vec<T>::N;
+    constexpr int kStep = 32 * kUnroll * N;
+    constexpr int kLast = (ITERS - 1) * kWarps * kStep;
+    uint4 rp[kUnroll], rq[kUnroll];
+    if (first_p >= 0 && first_q >= 0 && first_p + kLast + kStep <= V && first_q + kLast + kStep <= V) {
+        const uint4 *pp = reinterpret_cast<const uint4 *>(prow + first_p) + lane;
+        const uint4 *qq = reinterpret_cast<const uint4 *>(qrow + first_q) + lane;
+        constexpr int kNext = kWarps * kStep / N;     // vectors from one step of a warp to its next
+#pragma unroll
+        for (int j = 0; j < kUnroll; ++j) {
+            rp[j] = ld_stream(pp + j * 32);
+            if (HAS_Q) rq[j] = ld_stream(qq + j * 32);
+        }
+#pragma unroll
+        for (int it = 0; it < ITERS; ++it) {
+            online_update<T>(rp, mp.m, mp.s);
+            if (it + 1 < ITERS) {
+#pragma unroll
+                for (int j = 0; j < kUnroll; ++j) rp[j] = ld_stream(pp + (it + 1) * kNext + j * 32);
+            }
+            if (HAS_Q) {
+                online_update<T>(rq, mq.m, mq.s);
+                if (it + 1 < ITERS) {
+#pragma unroll
+                    for (int j = 0; j < kUnroll; ++j) rq[j] = ld_stream(qq + (it + 1) * kNext + j * 32);
+                }
+            }
+        }
+        return;
+    }
+    load_step<T>(prow, first_p, V, lane, rp);
+    if (HAS_Q) load_step<T>(qrow, first_q, V, lane, rq);
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) {
+        const int nxt = (it + 1) * kWarps * kStep;
+        const bool more = it + 1 < ITERS && min(first_p, first_q) + nxt < V;   // warp-uniform
+        online_update<T>(rp, mp.m, mp.s);
+        if (more) load_step<T>(prow, first_p + nxt, V, lane, rp);
+        if (HAS_Q) {
+            online_update<T>(rq, mq.m, mq.s);
+            if (more) load_step<T>(qrow, first_q + nxt, V, lane, rq);
+        }
+        if (!more) break;
+    }
+}
+
 }  // namespace spr
