@@ -845,7 +845,7 @@ def main():
                               "in all; the L2 holds 126 MB)" if n_copies > 1 else "one copy of the inputs: L2-warm"),
                        "inputs_sha256": inputs_sha,
                        "threshold": tau, "mean_sd_accepted_len": acc_len, "mean_first_reject": fr_mean},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": 4 * nsteps,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": (bd.sd_verify_launches(B, K, V, dt_code) + 2) * nsteps,
             "roofline": {"bound": "hbm", "kernel": "sd_row_stats_kernel", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                          "traffic": traffic, "algorithmic_bytes_per_launch": alg_bytes,

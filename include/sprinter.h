@@ -433,6 +433,11 @@ int spr_device_status(void *ws, void *cuda_stream);
 const char *spr_status_string(int status);
 const char *spr_last_cuda_error(void);
 
+/* Kernels one sd_verify call launches for this shape (2, or 3 when the row-statistics pass is
+ * followed by a separate finish grid; 0 for arguments sd_verify rejects).  The paper has no
+ * counterpart: bookkeeping for callers that count launches. */
+int spr_sd_verify_launches(int B, int K, int V, int dt);
+
 /* Library version: major * 10000 + minor * 100 + patch. */
 int spr_version(void);
 

@@ -21,7 +21,7 @@ PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
 
 EXPORTS = [
     "spr_workspace_bytes", "spr_workspace_init", "sprinter_verify", "replace_sample", "sd_verify",
-    "spr_device_status", "spr_status_string", "spr_last_cuda_error", "spr_version",
+    "spr_device_status", "spr_status_string", "spr_last_cuda_error", "spr_version", "spr_sd_verify_launches",
     "spr_host_arena_bytes", "sprinter_verify_host", "replace_sample_host", "sd_verify_host",
     "spr_set_stage_events", "replace_sample_static", "sprinter_step", "sprinter_simulate",
     "sd_shard_stats", "sd_shard_decide", "sd_shard_weights", "sd_shard_draw", "sd_shard_decide_weights",
@@ -117,6 +117,8 @@ def lib():
         L.spr_last_cuda_error.argtypes = []
         L.spr_version.restype = i32
         L.spr_version.argtypes = []
+        L.spr_sd_verify_launches.restype = i32
+        L.spr_sd_verify_launches.argtypes = [i32, i32, i32, i32]
         _lib = L
     return _lib
 
@@ -163,6 +165,11 @@ def _selectors(rows, first_reject, n: int):
         if t.numel() != n:
             raise ValueError(f"{name} must have one entry per draw ({n}), got {t.numel()}")
         _dev(t, torch.int32, name)
+
+
+def sd_verify_launches(B: int, K: int, V: int, dt: int = BF16) -> int:
+    """Kernels one sd_verify call launches for this shape."""
+    return int(lib().spr_sd_verify_launches(B, K, V, dt))
 
 
 def workspace_bytes(op: int, B: int, K: int = 1, V: int = 1, d: int = 1, h: int = 0, dt: int = BF16) -> int:

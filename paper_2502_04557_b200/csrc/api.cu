@@ -451,6 +451,14 @@ void spr_set_stage_events(void *before, void *after)
     set_stage_events(static_cast<cudaEvent_t>(before), static_cast<cudaEvent_t>(after));
 }
 
+int spr_sd_verify_launches(int B, int K, int V, int dt)
+{
+    if (!dtype_ok(dt) || B <= 0 || K <= 0 || V <= 0 || (int64_t)B * K > 0x7fffffff) return 0;
+    int C, iters;
+    draw_geometry(B * K, stat_steps_per_row(V, dt), &C, &iters);
+    return sd_row_stats_launches(B, K, C, iters) + 1;   // + the correction draw
+}
+
 int spr_version(void) { return 100; }
 
 }  // extern "C"

@@ -156,6 +156,8 @@ struct SimParams {
 cudaError_t launch_simulate(const SimParams &sp, cudaStream_t st);
 
 cudaError_t launch_sd_row_stats(const SdParams &sp, int B, int K, int dt, cudaStream_t st);
+// kernels that launch_sd_row_stats starts for this shape: 1, or 2 (statistics grid + finish grid)
+int sd_row_stats_launches(int B, int K, int chunks, int iters);
 int report_cuda_error(cudaError_t e);  // records the text, returns SPR_ERR_CUDA
 int device_supported();                // SPR_OK on a compute-capability-10 device
 void set_stage_events(cudaEvent_t before, cudaEvent_t after);

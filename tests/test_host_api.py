@@ -31,6 +31,11 @@ def test_library_exports_every_declared_symbol():
         assert hasattr(L, n), f"{n} declared in include/ but not exported"
     assert set(binding.EXPORTS) <= set(names)
     assert L.spr_version() >= 100
+    # launches per sd_verify call: the finish grid exists only behind several waves of four-step CTAs
+    assert L.spr_sd_verify_launches(256, 16, 128256, 1) == 3
+    assert L.spr_sd_verify_launches(4, 4, 1000, 1) == 2
+    assert L.spr_sd_verify_launches(128, 8, 32000, 1) == 2      # one segment per row: nothing to merge
+    assert L.spr_sd_verify_launches(0, 4, 1000, 1) == 0
 
 
 def test_workspace_bytes():
