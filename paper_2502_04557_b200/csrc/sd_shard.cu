@@ -37,11 +37,35 @@ __device__ __forceinline__ float logit_at(const T *row, int x)
     return __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(row)[x]);
 }
 
+// the record of row (b, k): merged statistics and, if the draft token falls into this shard, its two logits
+template <typename T>
+__device__ __forceinline__ void write_record(const ShardStatsParams &prm, int64_t row, int b, int k, bool has_q,
+                                             const T *prow, const T *qrow, float m_p, double z_p, float m_q, double z_q)
+{
+    float lpx = neg_inf(), lqx = neg_inf();
+    if (has_q) {
+        const int x = prm.draft_tokens[(int64_t)b * prm.K + k] - prm.v0;   // index inside the shard
+        if (x >= 0 && x < prm.V) {
+            lpx = logit_at<T>(prow, x);
+            lqx = logit_at<T>(qrow, x);
+        }
+    }
+    float *rec = prm.stats + row * kStatRecord;
+    rec[0] = m_p;
+    rec[1] = (float)z_p;
+    rec[2] = m_q;
+    rec[3] = (float)z_q;
+    rec[4] = lpx;
+    rec[5] = lqx;
+}
+
 // One CTA per (row, segment); row r = b*Kr + k (the first Kr <= Kp positions of every
 // sequence) reads p row b*Kp + k and, when k < K, q row b*K + k (the bonus row k = K has no q
 // row).  The CTA that finishes a row last merges its segments in segment order and writes
 // the row's record.
-template <typename T, int ITERS>
+// kSplit (many waves of CTAs): the CTA writes its segment's partial and leaves, the records
+// are formed by shard_finish_kernel behind this grid (see sd_row_stats_kernel for why).
+template <typename T, int ITERS, bool kSplit>
 __global__ void __launch_bounds__(kThreads, 4) shard_stats_kernel(const ShardStatsParams prm)
 {
     __shared__ float4 s_part[kWarps];
@@ -58,6 +82,7 @@ __global__ void __launch_bounds__(kThreads, 4) shard_stats_kernel(const ShardSta
     MS mp{neg_inf(), 0.f}, mq{neg_inf(), 0.f};
     if (has_q) shard_segment<T, ITERS, true>(prow, qrow, prm.V, c, mp, mq);
     else shard_segment<T, ITERS, false>(prow, qrow, prm.V, c, mp, mq);
+    if (kSplit) pdl_trigger();           // the finish grid may be scheduled behind this one
     mp = warp_ms(mp);
     mq = warp_ms(mq);
     if (lane == 0) s_part[warp] = make_float4(mp.m, mp.s, mq.m, mq.s);
@@ -67,6 +92,10 @@ __global__ void __launch_bounds__(kThreads, 4) shard_stats_kernel(const ShardSta
         const float4 v = lane < kWarps ? s_part[lane] : make_float4(neg_inf(), 0.f, neg_inf(), 0.f);
         mp = warp_ms(MS{v.x, v.y});
         mq = warp_ms(MS{v.z, v.w});
+    }
+    if (kSplit) {
+        if (lane == 0) prm.part[row * C + c] = make_float4(mp.m, mp.s, mq.m, mq.s);
+        return;
     }
     float m_p = mp.m, m_q = mq.m;
     double z_p = mp.s, z_q = mq.s;
@@ -107,23 +136,36 @@ __global__ void __launch_bounds__(kThreads, 4) shard_stats_kernel(const ShardSta
         z_q += bq;
     }
     }
-    if (lane == 0) {
-        float lpx = neg_inf(), lqx = neg_inf();
-        if (has_q) {
-            const int x = prm.draft_tokens[(int64_t)b * prm.K + k] - prm.v0;   // index inside the shard
-            if (x >= 0 && x < prm.V) {
-                lpx = logit_at<T>(prow, x);
-                lqx = logit_at<T>(qrow, x);
-            }
-        }
-        float *rec = prm.stats + row * kStatRecord;
-        rec[0] = m_p;
-        rec[1] = (float)z_p;
-        rec[2] = m_q;
-        rec[3] = (float)z_q;
-        rec[4] = lpx;
-        rec[5] = lqx;
+    if (lane == 0) write_record<T>(prm, row, b, k, has_q, prow, qrow, m_p, z_p, m_q, z_q);
+}
+
+// Behind a kSplit statistics grid: one thread per row merges the row's segment partials in
+// segment order and writes the record.
+template <typename T>
+__global__ void __launch_bounds__(kThreads) shard_finish_kernel(const ShardStatsParams prm, int64_t rows)
+{
+    pdl_wait();                          // every partial of the statistics grid is written
+    const int64_t row = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (row >= rows) return;
+    const int C = prm.chunks;
+    const int b = (int)(row / prm.Kr), k = (int)(row % prm.Kr);
+    const bool has_q = k < prm.K;
+    const T *prow = static_cast<const T *>(prm.p) + ((int64_t)b * prm.Kp + k) * prm.ldv;
+    const T *qrow = has_q ? static_cast<const T *>(prm.q) + ((int64_t)b * prm.K + k) * prm.ldv : prow;
+    const float4 *part = prm.part + row * C;
+    float m_p = neg_inf(), m_q = neg_inf();
+    for (int cc = 0; cc < C; ++cc) {
+        const float4 v = __ldcg(&part[cc]);
+        m_p = fmaxf(m_p, v.x);
+        m_q = fmaxf(m_q, v.z);
     }
+    double z_p = 0.0, z_q = 0.0;
+    for (int cc = 0; cc < C; ++cc) {
+        const float4 v = __ldcg(&part[cc]);
+        z_p += v.y > 0.f ? (double)v.y * exp((double)v.x - (double)m_p) : 0.0;
+        z_q += v.w > 0.f ? (double)v.w * exp((double)v.z - (double)m_q) : 0.0;
+    }
+    write_record<T>(prm, row, b, k, has_q, prow, qrow, m_p, z_p, m_q, z_q);
 }
 
 cudaError_t launch_shard_stats(const ShardStatsParams &sp, int64_t rows, int dt, cudaStream_t st)
@@ -131,7 +173,26 @@ cudaError_t launch_shard_stats(const ShardStatsParams &sp, int64_t rows, int dt,
     const int64_t grid = rows * sp.chunks;
     if (grid > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     if (grid == 0) return cudaSuccess;
-#define SPR_SHARD(T_, I_) shard_stats_kernel<T_, I_><<<(unsigned)grid, kThreads, 0, st>>>(sp)
+#define SPR_SHARD(T_, I_) shard_stats_kernel<T_, I_, false><<<(unsigned)grid, kThreads, 0, st>>>(sp)
+    // several waves of four-step CTAs with more than one segment per row: partials only, then the finish grid
+    const bool split = sp.iters == 4 && sp.chunks > 1 && grid >= 4 * 4 * 148;
+    if (split) {
+        if (dt == SPR_F32) shard_stats_kernel<float, 4, true><<<(unsigned)grid, kThreads, 0, st>>>(sp);
+        else shard_stats_kernel<__nv_bfloat16, 4, true><<<(unsigned)grid, kThreads, 0, st>>>(sp);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)((rows + kThreads - 1) / kThreads));
+        cfg.blockDim = dim3(kThreads);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // scheduled while the statistics grid drains
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return dt == SPR_F32 ? cudaLaunchKernelEx(&cfg, shard_finish_kernel<float>, sp, rows)
+                             : cudaLaunchKernelEx(&cfg, shard_finish_kernel<__nv_bfloat16>, sp, rows);
+    }
     if (dt == SPR_F32) {
         if (sp.iters == 4) SPR_SHARD(float, 4);
         else if (sp.iters == 2) SPR_SHARD(float, 2);
