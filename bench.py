@@ -31,10 +31,11 @@ if ROOT not in sys.path:
 # capture summarised under profiles/; reported only while the kernel source is unchanged.
 NCU_TRAFFIC = {
     "sources": ("sd_row_stats.cu", "vocab_common.cuh", "common.cuh"),
-    "sha256": "92bd41e1748015eae3d0c94b81657c6047c4a0e3192ff0d1087ab2b6b6a18342",
-    # (262,768,128 read + 3,310,848 written) / 512 tokens in the B = 32 capture; traffic grows
-    # in proportion to the tokens, so a full launch is this times B*K
-    "bytes_per_unit": 519685,   # DRAM bytes per verified token at V = 128256, bf16
+    "sha256": "92f757294d7190decb7184a5f36af6e55a97fcbc066b770e53c7166cfdb6104c",
+    # (394,077,184 read + 3,215,360 written) / 768 tokens in the B = 48 capture (the smallest batch that
+    # takes the same kernel variant as the full launch); traffic grows in proportion to the tokens, so a
+    # full launch is this times B*K
+    "bytes_per_unit": 517308,   # DRAM bytes per verified token at V = 128256, bf16
 }
 
 
@@ -605,7 +606,8 @@ def main():
     achieved = alg_bytes / (stats_ms * 1e-3) / 1e9
     peak, peak_kind = peaks()
     traffic = None
-    if NCU_TRAFFIC["sha256"] == kernel_sources_sha() and V == 128256 and es == 2:
+    if (NCU_TRAFFIC["sha256"] == kernel_sources_sha() and V == 128256 and es == 2
+            and bd.sd_verify_launches(B, K, V, dt_code) == 3):   # the kernel variant that was captured
         traffic = NCU_TRAFFIC["bytes_per_unit"] * M
 
     # end to end: host (pinned) tensors through the host-buffer C ABI, copies inside the timing
