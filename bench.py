@@ -436,6 +436,7 @@ def main():
     import torch.distributed as dist
 
     import paper_2502_04557_b200 as spr
+    from paper_2502_04557_b200 import binding as bd
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -734,7 +735,7 @@ def main():
     # vocabulary-sharded sd_verify: what one of G GPUs would run on its V/G columns (the two
     # all-gathers between the passes, 24 B per row and 16 B per sequence per GPU, are not timed)
     if args.vocab_shards > 0:
-        from paper_2502_04557_b200 import binding as bd, sharded
+        from paper_2502_04557_b200 import sharded
         G = args.vocab_shards
         shards = sharded.vocab_shards(V, G, es)
         views = [(wl.p_logits[:, :, v0:v0 + vs], wl.q_logits[:, :, v0:v0 + vs]) for v0, vs in shards]
@@ -763,7 +764,6 @@ def main():
 
     # preparing and fitting the verifier (Section 3.2): labels from the same logits, one optimiser step of
     # the single-layer verifier on N = 2^20 hidden states of the draft model's width
-    from paper_2502_04557_b200 import binding as bd
     ws_fit = spr.Workspace(max(spr.workspace_bytes(bd.OP_VERIFIER_LABELS, B, K, V, 0, 0, dt_code),
                                spr.workspace_bytes(bd.OP_VERIFIER_TRAIN, 0, 0, 0, cfg.d, 0, dt_code)), device=dev)
     t_lab = time_call(lambda: bd.verifier_labels(wl.p_logits, wl.q_logits, V, wl.draft_tokens, [1.0, 1.2, 1.5], ws_fit,

@@ -104,23 +104,35 @@ __device__ __forceinline__ void warp_steps(const Job<T> &job, int mode, int V, i
         // two steps in flight behind the one being summed; the three buffers swap roles by
         // position in an unrolled loop instead of being copied
         uint4 a[kUnroll], b[kUnroll], c[kUnroll];
-        auto fetch = [&](uint4 (&dst)[kUnroll], int s) { load_step<T>(job.p_row, s * kStep - pad, V, lane, dst); };
         auto emit = [&](const uint4 (&src)[kUnroll], int s) {
             const MS v = softmax_step<T>(src);
             if (lane == 0) part[s] = make_float2(v.m, v.s);
         };
-        fetch(a, s0);
-        if (s0 + 1 < s1) fetch(b, s0 + 1);
-        for (int s = s0;;) {
-            if (s + 2 < s1) fetch(c, s + 2);
-            emit(a, s);
-            if (++s >= s1) break;
-            if (s + 2 < s1) fetch(a, s + 2);
-            emit(b, s);
-            if (++s >= s1) break;
-            if (s + 2 < s1) fetch(b, s + 2);
-            emit(c, s);
-            if (++s >= s1) break;
+        auto run = [&](auto fetch) {
+            fetch(a, s0);
+            if (s0 + 1 < s1) fetch(b, s0 + 1);
+            for (int s = s0;;) {
+                if (s + 2 < s1) fetch(c, s + 2);
+                emit(a, s);
+                if (++s >= s1) break;
+                if (s + 2 < s1) fetch(a, s + 2);
+                emit(b, s);
+                if (++s >= s1) break;
+                if (s + 2 < s1) fetch(b, s + 2);
+                emit(c, s);
+                if (++s >= s1) break;
+            }
+        };
+        const int64_t f0 = (int64_t)s0 * kStep - pad;
+        if (f0 >= 0 && (int64_t)s1 * kStep - pad <= V) {
+            // every step of the run is whole aligned vectors inside the row: loads without checks
+            const uint4 *pp = reinterpret_cast<const uint4 *>(job.p_row + f0) + lane;
+            run([&](uint4 (&dst)[kUnroll], int s) {
+#pragma unroll
+                for (int j = 0; j < kUnroll; ++j) dst[j] = ld_stream(pp + (s - s0) * (kStep / N) + j * 32);
+            });
+        } else {
+            run([&](uint4 (&dst)[kUnroll], int s) { load_step<T>(job.p_row, s * kStep - pad, V, lane, dst); });
         }
     } else {
         uint4 rp[kUnroll], rq[kUnroll], np[kUnroll], nq[kUnroll];
