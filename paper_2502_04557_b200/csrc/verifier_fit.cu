@@ -120,7 +120,7 @@ __device__ __forceinline__ void team_sync(int team)
     else asm volatile("bar.sync %0, %1;" ::"r"(team + 1), "r"(WPR * 32) : "memory");
 }
 
-__host__ __device__ constexpr int ring_ctas_per_sm(int vpl, int wpr) { return wpr == 1 && vpl <= 4 ? 2 : 1; }
+__host__ __device__ constexpr int ring_ctas_per_sm(int vpl, int wpr) { return wpr == 1 && vpl <= 2 ? 3 : (wpr == 1 && vpl <= 4 ? 2 : 1); }
 
 template <typename T, int VPL, int WPR, int R, int SLOTS>
 __global__ void __launch_bounds__(kThreads, ring_ctas_per_sm(VPL, WPR)) train_grad_ring_kernel(const TrainParams prm)
@@ -401,9 +401,9 @@ cudaError_t launch_grad_any(const TrainParams &tp, cudaStream_t st)
     if (vpl <= 2) return launch_grad_ring<T, 2, 1, 4, 12>(tp, st);
     if (vpl <= 3) return launch_grad_ring<T, 3, 1, 4, 8>(tp, st);
     if (vpl <= 4) return launch_grad_ring<T, 4, 1, 3, 6>(tp, st);
-    if (vpl <= 6) return launch_grad_ring<T, 6, 1, 2, 8>(tp, st);
+    if (vpl <= 6) return launch_grad_ring<T, 6, 1, 3, 8>(tp, st);
     if (vpl <= 8) return launch_grad_ring<T, 8, 1, 2, 6>(tp, st);
-    if (vpl <= 12) return launch_grad_ring<T, 6, 2, 2, 8>(tp, st);
+    if (vpl <= 12) return launch_grad_ring<T, 6, 2, 3, 8>(tp, st);
     return launch_grad_ring<T, 8, 2, 2, 6>(tp, st);
 }
 
