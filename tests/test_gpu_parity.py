@@ -444,6 +444,41 @@ def test_sd_correction_draw_over_residual_masses(spr, dtype, V):
     assert_mass_close(out["residual_mass"], ref["residual_mass"], RTOL[dtype])
 
 
+@pytest.mark.parametrize("dtype,B,K,V,ldv", [(torch.float32, 37, 33, 20000, 20001), (torch.bfloat16, 74, 16, 33000, None),
+                                             (torch.bfloat16, 40, 30, 40001, 40003)], ids=["f32", "bf16", "bf16-odd"])
+def test_sd_many_waves_of_short_rows(spr, dtype, B, K, V, ldv):
+    """More than four waves of statistics CTAs with two segments per row: the launch shape in which
+    the merge, the accept test and the scan run in their own grid.  Rows at every alignment
+    (odd leading dimension), more than 32 positions per sequence, and - after the clean
+    comparison - sequences with an invalid draft token."""
+    assert spr.binding.sd_verify_launches(B, K, V, spr.binding._dt(torch.empty(0, dtype=dtype))) == 3
+    p, q, x, u = _rand_problem(B, K, V, dtype, seed=B + K + V, ldv=ldv)
+    ref = _clear_sd(p, q, V, x, u)
+    ws = spr.Workspace(spr.workspace_bytes(2, B, K, V, 1, 0, spr.binding._dt(p)))
+    pg, qg, ug = p.cuda(), q.cuda(), u.cuda()
+    out = spr.sd_verify(pg, qg, V, x.cuda(), ug, ws)
+    assert ws.device_status() == 0
+    eq(out["accept"], ref["accept"], "accept")
+    eq(out["accepted_len"], ref["accepted_len"], "accepted_len")
+    eq(out["correction_token"], ref["correction_token"], "correction_token")
+    assert_close_rel(out["p_tok"], ref["p_tok"], RTOL[dtype], "p_tok")
+    assert_close_rel(out["q_tok"], ref["q_tok"], RTOL[dtype], "q_tok")
+    assert_mass_close(out["residual_mass"], ref["residual_mass"], RTOL[dtype])
+    bad = {1: (0, -1), 5: (K - 1, V), B - 1: (K // 2, V + 7)}
+    for b, (k, tok) in bad.items():
+        x[b, k] = tok
+    out = spr.sd_verify(pg, qg, V, x.cuda(), ug, ws)
+    assert ws.device_status() == 6          # SPR_ERR_BAD_TOKEN
+    ref2, rc = oracle.sd_verify(to_np(p), to_np(q), V, to_np(x), to_np(u), return_status=True)
+    assert rc == oracle.ERR_TOKEN
+    eq(out["accepted_len"], ref2["accepted_len"], "accepted_len with invalid tokens")
+    eq(out["correction_token"], ref2["correction_token"], "correction_token with invalid tokens")
+    for b in bad:
+        assert int(out["accepted_len"][b]) == -1 and int(out["accept"][b].sum()) == 0
+    clean = [b for b in range(B) if b not in bad]
+    eq(out["accept"][clean], ref["accept"][clean], "accept of the clean sequences")
+
+
 def test_device_detected_errors(spr):
     p, q, x, u = _rand_problem(3, 2, 300, torch.float32, seed=3)
     x[1, 1] = 300
