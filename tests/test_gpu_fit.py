@@ -49,6 +49,7 @@ def check_labels(spr, p, q, V, x, lambdas, dtype):
 @pytest.mark.parametrize("B,K,V,ldv,Kp", [
     (3, 1, 2, None, 2), (5, 2, 7, None, 2), (4, 3, 1000, None, 4), (2, 33, 129, 131, 34),
     (3, 4, 8191, None, 4), (2, 2, 8193, 8200, 3), (2, 5, 32769, None, 6), (1, 40, 50257, None, 40),
+    (38, 33, 33001, 33003, 34),      # more than four waves of two-segment rows: records written by the finish grid
 ])
 def test_labels_ragged_shapes(spr, dtype, B, K, V, ldv, Kp):
     p, q, x, _ = _rand_problem(B, K, V, dtype, seed=3 + B * 1000 + K * 10 + V, ldv=ldv, Kp=Kp)
