@@ -120,14 +120,18 @@ __device__ __forceinline__ void team_sync(int team)
     else asm volatile("bar.sync %0, %1;" ::"r"(team + 1), "r"(WPR * 32) : "memory");
 }
 
-__host__ __device__ constexpr int ring_ctas_per_sm(int vpl, int wpr) { return wpr == 1 && vpl <= 2 ? 3 : (wpr == 1 && vpl <= 4 ? 2 : 1); }
+__host__ __device__ constexpr int ring_ctas_per_sm(int vpl, int wpr, int g) { return g > 1 ? 2 : (wpr == 1 && vpl <= 4 ? 2 : 1); }
 
-template <typename T, int VPL, int WPR, int R, int SLOTS>
-__global__ void __launch_bounds__(kThreads, ring_ctas_per_sm(VPL, WPR)) train_grad_ring_kernel(const TrainParams prm)
+// G: consecutive rows per slot and per bulk copy (short rows: a copy of 4 KB instead of 512 bytes);
+// a team then takes blocks of G rows, and R divides G so that the rows a team works on together
+// lie in one slot.
+template <typename T, int VPL, int WPR, int R, int SLOTS, int G>
+__global__ void __launch_bounds__(kThreads, ring_ctas_per_sm(VPL, WPR, G)) train_grad_ring_kernel(const TrainParams prm)
 {
+    static_assert(G == 1 || (G % R == 0 && WPR == 1), "the rows of a group share a slot");
     constexpr int N = Vec<T>::N;
     constexpr int kTeams = kWarps / WPR;
-    constexpr int kSlotVecs = VPL * WPR * 32;
+    constexpr int kSlotVecs = VPL * WPR * 32 * G;
     extern __shared__ __align__(128) unsigned char rsmem[];
     __shared__ __align__(8) uint64_t bars[kTeams][SLOTS];
     __shared__ float halves[kTeams][R][2];    // WPR = 2: the two warps' parts of the R dot products
@@ -158,39 +162,50 @@ __global__ void __launch_bounds__(kThreads, ring_ctas_per_sm(VPL, WPR)) train_gr
     float z_keep = 0.f, y_keep = 0.f, r_keep = 0.f;
     int kept = 0;
 
+    // Blocks of G consecutive rows are dealt to the teams in a fixed pattern; block k of this team
+    // is block first + k * stride of the data, goes to slot k % SLOTS and is its (k / SLOTS)-th fill.
     const T *base = static_cast<const T *>(prm.hidden);
+    const int64_t blocks = (prm.N + G - 1) / G;
     const int64_t stride = (int64_t)gridDim.x * kTeams;
     const int64_t first = (int64_t)blockIdx.x * kTeams + team;
-    const int n = first < prm.N ? (int)((prm.N - first + stride - 1) / stride) : 0;   // this team's rows
+    const int nb = first < blocks ? (int)((blocks - first + stride - 1) / stride) : 0;   // this team's blocks
+    // only the last block of the data can be short, and it is the last of its team
+    const int rows_last = nb > 0 ? (int)min((int64_t)G, prm.N - (first + (int64_t)(nb - 1) * stride) * G) : 0;
+    const int n = nb > 0 ? (nb - 1) * G + rows_last : 0;                                 // this team's rows
+    auto rows_in = [&](int k) { return k == nb - 1 ? rows_last : G; };
+    auto row_of = [&](int i) { return (first + (int64_t)(i / G) * stride) * G + i % G; };   // row i of this team
     const bool feeder = half == 0 && lane == 0 && !(prm.test_flags & TRAIN_TEST_NO_FETCH);
+    auto fetch_block = [&](int k) {
+        ring_fetch(ring + (k % SLOTS) * kSlotVecs, base + (first + (int64_t)k * stride) * G * d,
+                   (uint32_t)rows_in(k) * row_bytes, &bar[k % SLOTS]);
+    };
     const uint32_t limit = prm.spin_limit;
     if (half == 0 && lane == 0) {
         team_fail[team] = 0;
         for (int s = 0; s < SLOTS; ++s)
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(ring_addr(&bar[s])) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        for (int i = 0; feeder && i < SLOTS && i < n; ++i)
-            ring_fetch(ring + i * kSlotVecs, base + (first + i * stride) * d, row_bytes, &bar[i]);
+        for (int k = 0; feeder && k < SLOTS && k < nb; ++k) fetch_block(k);
     }
     team_sync<WPR>(team);
 
     // Labels: lane l holds the label of row (32 b + l) of this team, the batch after it is on its
     // way - a label fetched next to its row would cost a full trip to memory per group of rows.
-    auto label_batch = [&](int i0) { return i0 + lane < n ? (float)prm.labels[first + (int64_t)(i0 + lane) * stride] : 0.f; };
+    auto label_batch = [&](int i0) { return i0 + lane < n ? (float)prm.labels[row_of(i0 + lane)] : 0.f; };
     float y_batch = label_batch(0), y_batch_next = label_batch(32);
-    int slot = 0;                             // ring slot of row i
-    uint32_t parity = 0;                      // of that slot's current fill
     bool ok = true;
     int fail_at = 0;                          // first row of the group whose wait ran out
 
     // rows [i, i + RR) of this team, RR <= R
     auto group = [&](auto rr_tag, int i) {
         constexpr int RR = decltype(rr_tag)::value;
-        int s[RR];
+        int s[RR];                             // where row i + r starts in the ring, in vectors
+        int blk[RR];
         float y[RR];
 #pragma unroll
         for (int r = 0; r < RR; ++r) {
-            s[r] = slot + r >= SLOTS ? slot + r - SLOTS : slot + r;
+            blk[r] = (i + r) / G;
+            s[r] = (blk[r] % SLOTS) * kSlotVecs + ((i + r) % G) * (G > 1 ? nv : 0);
             const int idx = i + r;
             if ((idx & 31) == 0 && idx > 0) {
                 y_batch = y_batch_next;
@@ -199,7 +214,8 @@ __global__ void __launch_bounds__(kThreads, ring_ctas_per_sm(VPL, WPR)) train_gr
             y[r] = __shfl_sync(0xffffffffu, y_batch, idx & 31);
         }
 #pragma unroll
-        for (int r = 0; r < RR; ++r) ok = ok && ring_wait(&bar[s[r]], slot + r >= SLOTS ? parity ^ 1u : parity, limit);
+        for (int r = 0; r < RR; ++r)
+            if (G == 1 || r == 0) ok = ok && ring_wait(&bar[blk[r] % SLOTS], (uint32_t)(blk[r] / SLOTS) & 1u, limit);
         if (WPR > 1) {
             // a team leaves together: the barriers below need both of its warps
             if (lane == 0 && !ok) team_fail[team] = 1;
@@ -217,7 +233,7 @@ __global__ void __launch_bounds__(kThreads, ring_ctas_per_sm(VPL, WPR)) train_gr
                 const int vi = v0 + j * 32;
 #pragma unroll
                 for (int r = 0; r < RR; ++r) {
-                    const uint4 x = vi < nv ? ring[s[r] * kSlotVecs + vi] : make_uint4(0u, 0u, 0u, 0u);
+                    const uint4 x = vi < nv ? ring[s[r] + vi] : make_uint4(0u, 0u, 0u, 0u);
                     float f[N];
                     Vec<T>::unpack(x, f);
 #pragma unroll
@@ -271,7 +287,7 @@ __global__ void __launch_bounds__(kThreads, ring_ctas_per_sm(VPL, WPR)) train_gr
             const int vi = v0 + j * 32;
 #pragma unroll
             for (int r = 0; r < RR; ++r) {
-                const uint4 x = vi < nv ? ring[s[r] * kSlotVecs + vi] : make_uint4(0u, 0u, 0u, 0u);
+                const uint4 x = vi < nv ? ring[s[r] + vi] : make_uint4(0u, 0u, 0u, 0u);
                 float f[N];
                 Vec<T>::unpack(x, f);
 #pragma unroll
@@ -282,15 +298,9 @@ __global__ void __launch_bounds__(kThreads, ring_ctas_per_sm(VPL, WPR)) train_gr
         team_sync<WPR>(team);                  // the whole team is done with the slots: refill them
         if (feeder) {
 #pragma unroll
-            for (int r = 0; r < RR; ++r) {
-                const int nx = i + r + SLOTS;
-                if (nx < n) ring_fetch(ring + s[r] * kSlotVecs, base + (first + nx * stride) * d, row_bytes, &bar[s[r]]);
+            for (int r = 0; r < RR; ++r) {     // a block whose last row was just used makes room for block + SLOTS
+                if ((i + r) % G == rows_in(blk[r]) - 1 && blk[r] + SLOTS < nb) fetch_block(blk[r] + SLOTS);
             }
-        }
-        slot += RR;
-        if (slot >= SLOTS) {
-            slot -= SLOTS;
-            parity ^= 1u;
         }
     };
     int i = 0;
@@ -298,9 +308,9 @@ __global__ void __launch_bounds__(kThreads, ring_ctas_per_sm(VPL, WPR)) train_gr
     for (; ok && i < n; ++i) group(std::integral_constant<int, 1>{}, i);
     if (!ok) {
         // A wait ran out: report it, then give the copies still on their way the same bounded
-        // time to land before the CTA's shared memory goes away: rows fail_at .. fail_at + slots.
+        // time to land before the CTA's shared memory goes away: the blocks from fail_at's on.
         if (lane == 0) raise_status(prm.status, SPR_ERR_TIMEOUT);
-        for (int k = fail_at; feeder_team_has_copies(prm) && k < n && k < fail_at + SLOTS; ++k)
+        for (int k = fail_at / G; feeder_team_has_copies(prm) && k < nb && k < fail_at / G + SLOTS; ++k)
             ring_wait(&bar[k % SLOTS], (uint32_t)(k / SLOTS) & 1u, limit);
     }
 
@@ -370,13 +380,13 @@ __global__ void __launch_bounds__(256) train_adam_kernel(const TrainParams prm)
     prm.theta[j] = (float)((double)prm.theta[j] - (double)prm.lr * m_hat / (sqrt(v_hat) + (double)prm.eps));
 }
 
-template <typename T, int VPL, int WPR, int R, int SLOTS>
+template <typename T, int VPL, int WPR, int R, int SLOTS, int G = 1>
 cudaError_t launch_grad_ring(const TrainParams &tp, cudaStream_t st)
 {
     TrainParams p = tp;
     constexpr int kTeams = kWarps / WPR;
-    const size_t smem = (size_t)kTeams * SLOTS * VPL * WPR * 32 * 16 + sizeof(float) * ((size_t)tp.d + 2);
-    auto kernel = train_grad_ring_kernel<T, VPL, WPR, R, SLOTS>;
+    const size_t smem = (size_t)kTeams * SLOTS * VPL * WPR * 32 * G * 16 + sizeof(float) * ((size_t)tp.d + 2);
+    auto kernel = train_grad_ring_kernel<T, VPL, WPR, R, SLOTS, G>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     int per_sm = 0, dev = 0, sms = 0;
     if (e != cudaSuccess ||
@@ -386,7 +396,8 @@ cudaError_t launch_grad_ring(const TrainParams &tp, cudaStream_t st)
         return e;
     if (per_sm < 1) return cudaErrorInvalidConfiguration;
     // one full wave: as many CTAs as are resident at once, so that all of them finish together
-    p.ctas = (int)max((int64_t)1, min((int64_t)min(kTrainMaxCtas, per_sm * sms), (tp.N + kTeams - 1) / kTeams));
+    const int64_t blocks = (tp.N + G - 1) / G;
+    p.ctas = (int)max((int64_t)1, min((int64_t)min(kTrainMaxCtas, per_sm * sms), (blocks + kTeams - 1) / kTeams));
     kernel<<<p.ctas, kThreads, smem, st>>>(p);
     train_adam_kernel<<<(tp.d + 2 + 255) / 256, 256, 0, st>>>(p);
     return cudaGetLastError();
@@ -397,8 +408,8 @@ cudaError_t launch_grad_any(const TrainParams &tp, cudaStream_t st)
 {
     const int vpl = (tp.d / Vec<T>::N + 31) / 32;
     // rows per group and ring slots: about 190 KB of ring per SM (two CTAs share it up to 4 vectors per lane)
-    if (vpl <= 1) return launch_grad_ring<T, 1, 1, 4, 12>(tp, st);
-    if (vpl <= 2) return launch_grad_ring<T, 2, 1, 4, 12>(tp, st);
+    if (vpl <= 1) return launch_grad_ring<T, 1, 1, 4, 3, 8>(tp, st);     // eight rows (4 KB) per copy
+    if (vpl <= 2) return launch_grad_ring<T, 2, 1, 4, 3, 4>(tp, st);     // four rows per copy
     if (vpl <= 3) return launch_grad_ring<T, 3, 1, 4, 8>(tp, st);
     if (vpl <= 4) return launch_grad_ring<T, 4, 1, 3, 6>(tp, st);
     if (vpl <= 6) return launch_grad_ring<T, 6, 1, 3, 8>(tp, st);
