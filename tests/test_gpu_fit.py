@@ -116,6 +116,8 @@ def run_steps(spr, S, y, steps, lr, theta0=None, **hyper):
     (24000, 2048, torch.bfloat16), (16000, 4096, torch.bfloat16), (12000, 2560, torch.bfloat16),
     (14001, 3072, torch.bfloat16), (70000, 128, torch.bfloat16), (20000, 1024, torch.float32),
     (9000, 2048, torch.float32), (11000, 1240, torch.float32),
+    # short rows travel several to a slot: rings that go round, and a last block that is not full
+    (70001, 128, torch.bfloat16), (50003, 512, torch.bfloat16), (40002, 200, torch.float32),
 ], ids=lambda v: str(v).replace("torch.", ""))
 def test_train_steps_match_the_oracle(spr, N, d, dtype):
     """fp32 sums on the GPU against float64: the loss agrees to 2e-5 relative, and since an Adam
@@ -164,7 +166,8 @@ def test_train_is_reproducible_and_rejects_unsupported_widths(spr):
 
 
 @pytest.mark.parametrize("N,d,dtype", [(5000, 768, torch.bfloat16), (3000, 2048, torch.bfloat16),
-                                       (2000, 4096, torch.bfloat16), (9, 64, torch.float32)],
+                                       (2000, 4096, torch.bfloat16), (9, 64, torch.float32),
+                                       (30001, 256, torch.bfloat16)],
                          ids=lambda v: str(v).replace("torch.", ""))
 def test_train_bounded_wait_runs_out_and_nothing_is_stepped(spr, N, d, dtype):
     """No row is ever fetched (test flag): every team's first wait expires after a few thousand
