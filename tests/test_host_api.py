@@ -236,3 +236,10 @@ def test_bench_refuses_to_time_fewer_ranks_than_asked_for():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "1"],
                        capture_output=True, text=True, timeout=300, env=env)
     assert r.returncode != 0 and "must agree" in (r.stderr + r.stdout)
+
+
+def test_stream_probes_compile():
+    """The two stand-alone measurement programs build for sm_100a (no GPU needed to compile)."""
+    from paper_2502_04557_b200 import stream_probes
+    for exe in stream_probes.build():
+        assert os.path.exists(exe) and os.access(exe, os.X_OK)
